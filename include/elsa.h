@@ -1,0 +1,175 @@
+/*
+ * elsa.h -- C ABI of the B200 (sm_100a) N:M sparse-linear library.
+ *
+ * The calls follow the problem statement of ELSA (arXiv 2409.09708): a ViT's
+ * linear modules (qkv, proj, fc1, fc2; Sec. 3, L = 4B) each carry a sparsity
+ * level N:M; the weight of a module is projected onto that level by keeping
+ * the N largest-magnitude values of every group of M consecutive weights
+ * (Sec. 3.1, Eq. 1), stored as the kept values plus one log2(M)-bit index each
+ * (Sec. 1; Sec. 2, Fig. 2 top), and multiplied with dense activations so that
+ * the result is the exact product with the pruned matrix (Sec. 2, Fig. 2
+ * bottom).
+ *
+ * Conventions for every call unless stated otherwise
+ *   - Tensor pointers are DEVICE pointers owned by the caller.  Matrices are
+ *     row-major and contiguous.  W is [out][in] as in nn.Linear: Y = X W^T + b.
+ *     Groups of M run along `in` (the reduction dimension), aligned at
+ *     multiples of M.
+ *   - 16-bit floats (fp16 or bf16, chosen by elsa_dtype) for X, W, values,
+ *     bias and Y; accumulation in fp32; one round-to-nearest-even at the end.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).
+ *     Calls enqueue work and return; they never synchronise and never
+ *     allocate or free device memory.
+ *   - Arguments are validated on the host before anything is launched.  A bad
+ *     argument returns a status; nothing aborts, throws or prints.
+ *     elsa_last_error() gives a thread-local message for the last failure.
+ *   - Pointers must be 16-byte aligned and `in`, `out` multiples of 8 (row
+ *     pitches are then multiples of 16 bytes), else ELSA_ERR_ALIGN.
+ *   - Supported levels: M in {4, 8, 16}, 1 <= N <= M, in % M == 0.
+ *   - The library requires a compute-capability 10.x device (ELSA_ERR_ARCH).
+ *
+ * Packed format (what elsa_nm_compress writes and the other calls read)
+ *   vals: [out][in/M*N] 16-bit, the kept values of each group in ascending
+ *         in-group position, bit patterns unchanged.
+ *   idx : [out][words_per_row] uint32.  The position (0..M-1) of kept value t
+ *         of group g is the b = log2(M)-bit field at bit offset (g*N + t)*b of
+ *         the row's bitstream, least-significant bit first inside
+ *         little-endian words; rows start on a word boundary,
+ *         words_per_row = ceil(in/M*N*b / 32); pad bits are zero.
+ *         N == M stores no indices: idx may be NULL and vals equals W.
+ */
+#ifndef ELSA_H
+#define ELSA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    ELSA_OK = 0,
+    ELSA_ERR_NULL = 1,      /* a required pointer is NULL */
+    ELSA_ERR_SHAPE = 2,     /* non-positive dimension, or in % M != 0 */
+    ELSA_ERR_NM = 3,        /* M not in {4, 8, 16}, N < 1 or N > M */
+    ELSA_ERR_DTYPE = 4,
+    ELSA_ERR_ALIGN = 5,     /* pointer not 16-byte aligned, or in/out not a multiple of 8 */
+    ELSA_ERR_WORKSPACE = 6, /* workspace NULL or smaller than elsa_workspace_bytes() */
+    ELSA_ERR_CUDA = 7,      /* a CUDA runtime/driver call failed; see elsa_last_error() */
+    ELSA_ERR_TIMEOUT = 8,   /* reported through dev_status: a bounded device-side wait gave up */
+    ELSA_ERR_ARCH = 9       /* current device is not compute capability 10.x */
+} elsa_status;
+
+typedef enum { ELSA_F16 = 0, ELSA_BF16 = 1 } elsa_dtype;
+
+/* Which kernel elsa_nm_linear uses.  AUTO is the product path; the others exist so that
+ * tests can force every variant over the same input and require agreement. */
+typedef enum {
+    ELSA_VARIANT_AUTO = 0,
+    ELSA_VARIANT_SIMT = 1,    /* CUDA-core kernel reading the packed form directly (slow; checks) */
+    ELSA_VARIANT_TC_DENSE = 2 /* expand to a dense tile image, tcgen05 dense MMA */
+} elsa_variant;
+
+/* Sizes of the packed form (host-only arithmetic; 0 on invalid arguments). */
+size_t elsa_nm_values_bytes(int out, int in, int N, int M, elsa_dtype dtype);
+size_t elsa_nm_index_bytes(int out, int in, int N, int M); /* 0 when N == M */
+
+/* Bytes of device scratch elsa_nm_linear needs for this problem (host-only arithmetic). */
+size_t elsa_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype dtype);
+
+/*
+ * Sec. 3.1, Eq. 1 with magnitude saliency, then the compressed form of Sec. 1 / Sec. 2.
+ * In every group of M consecutive weights of a row keep the N of largest |w|; |w| is compared
+ * exactly on the 15 magnitude bits (so +0 == -0), and among equals the lowest position wins,
+ * so exactly N positions are kept and the result is unique.
+ *   W    in : [out][in] dense weight
+ *   vals out: [out][in/M*N]
+ *   idx  out: [out][words_per_row], may be NULL iff N == M
+ */
+elsa_status elsa_nm_compress(const void* W, int out, int in, int N, int M, elsa_dtype dtype,
+                             void* vals, uint32_t* idx, void* stream);
+
+/*
+ * Inverse of the compressed form: W_masked [out][in] with +0.0 at pruned positions and the kept
+ * values, bit for bit, at theirs (Sec. 2, Fig. 2: the indices give each value's original position).
+ */
+elsa_status elsa_nm_unpack(const void* vals, const uint32_t* idx, int out, int in, int N, int M,
+                           elsa_dtype dtype, void* W_masked, void* stream);
+
+/*
+ * Sec. 2, Fig. 2 bottom: Y[rows][out] = X[rows][in] * W_masked^T + bias, computed from the packed
+ * weight; only kept weights contribute.  fp32 accumulation, one rounding to the 16-bit output.
+ *   bias       : [out] 16-bit, or NULL
+ *   workspace  : device scratch of at least elsa_workspace_bytes(...) bytes, 256-byte aligned;
+ *                its contents are overwritten; calls that share it must be stream-ordered
+ *   dev_status : optional device word.  The caller zeroes it; if a bounded wait inside the
+ *                kernel ever gives up, the kernel stores ELSA_ERR_TIMEOUT | (site << 8) there and
+ *                all its threads return without trapping.  Read it after synchronising.
+ */
+elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint32_t* idx,
+                           const void* bias, int out, int in, int N, int M, elsa_dtype dtype,
+                           void* Y, void* workspace, size_t workspace_bytes,
+                           uint32_t* dev_status, void* stream);
+
+/* One linear module of the per-layer table (Sec. 3: configuration alpha = (s^1 .. s^L)). */
+typedef struct {
+    const void* X;       /* [rows][in]  device */
+    void* Y;             /* [rows][out] device */
+    const void* vals;    /* packed values, device */
+    const uint32_t* idx; /* packed indices, device; NULL iff N == M */
+    const void* bias;    /* [out] device or NULL */
+    int rows, in, out, N, M;
+} elsa_layer;
+
+/* Largest elsa_workspace_bytes over the table (host-only arithmetic). */
+size_t elsa_vit_workspace_bytes(const elsa_layer* cfg, int n_layers, elsa_dtype dtype);
+
+/*
+ * Runs every layer of the table, in order, on one stream, each under its own level N:M
+ * (Sec. 3, layer-wise configuration alpha).  `cfg` is a HOST array.  The table is validated as a
+ * whole before the first launch; on an error nothing has been enqueued and elsa_last_error()
+ * names the layer.
+ */
+elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dtype,
+                             void* workspace, size_t workspace_bytes, uint32_t* dev_status,
+                             void* stream);
+
+/* One layer of the host-memory variant: every tensor pointer is a HOST pointer. */
+typedef struct {
+    const void* X;    /* [rows][in]  host */
+    void* Y;          /* [rows][out] host, written */
+    const void* W;    /* [out][in]   host, dense weight */
+    const void* bias; /* [out] host or NULL */
+    int rows, in, out, N, M;
+} elsa_host_layer;
+
+/* Bytes of device memory elsa_vit_linears_host needs for this table (host-only arithmetic). */
+size_t elsa_vit_host_device_bytes(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype);
+
+/*
+ * The whole path from host memory (Sec. 3.1 projection, then Sec. 2 product, per layer of the
+ * table): for each layer copy W, bias and X to the device, compress W to its level, multiply,
+ * and copy Y back.  `device_mem` is caller-owned device memory of at least
+ * elsa_vit_host_device_bytes(...) bytes, 256-byte aligned.  Copies are cudaMemcpyAsync on
+ * `stream`: with pinned host memory the call returns after enqueue and Y is valid once the
+ * stream has been synchronised.
+ */
+elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype,
+                                  void* device_mem, size_t device_bytes, uint32_t* dev_status,
+                                  void* stream);
+
+/* Test aid: force the kernel variant used by elsa_nm_linear / elsa_vit_linears (process-wide). */
+elsa_status elsa_set_linear_variant(elsa_variant v);
+elsa_variant elsa_get_linear_variant(void);
+
+/* Number of kernels the library has launched from this process so far. */
+unsigned long long elsa_launch_count(void);
+
+/* Message describing the calling thread's last non-OK status ("" if none). */
+const char* elsa_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ELSA_H */

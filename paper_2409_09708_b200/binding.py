@@ -1,0 +1,213 @@
+"""Thin ctypes binding of ``libelsa.so`` (the C ABI declared in ``include/elsa.h``).
+
+Argument marshalling only: every step of the path runs in the library's CUDA
+kernels.  torch supplies device memory and streams.  There is no fallback: if
+the library has not been built this module raises at import.
+
+Functions carry the names of the C entry points.  Tensors must be CUDA,
+contiguous, fp16 or bf16 (index words are int32 tensors holding the uint32
+bit patterns).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libelsa.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        "libelsa.so is missing: build it with `python -m paper_2409_09708_b200.build` "
+        "(there is no CPU or PyTorch fallback for the sparse-linear path)")
+
+_lib = ctypes.CDLL(LIB_PATH)
+
+OK = 0
+ERR_NAMES = {0: "ELSA_OK", 1: "ELSA_ERR_NULL", 2: "ELSA_ERR_SHAPE", 3: "ELSA_ERR_NM", 4: "ELSA_ERR_DTYPE",
+             5: "ELSA_ERR_ALIGN", 6: "ELSA_ERR_WORKSPACE", 7: "ELSA_ERR_CUDA", 8: "ELSA_ERR_TIMEOUT",
+             9: "ELSA_ERR_ARCH"}
+F16, BF16 = 0, 1
+VARIANT_AUTO, VARIANT_SIMT, VARIANT_TC_DENSE = 0, 1, 2
+
+_vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+
+
+class ElsaLayer(ctypes.Structure):
+    _fields_ = [("X", _vp), ("Y", _vp), ("vals", _vp), ("idx", _vp), ("bias", _vp),
+                ("rows", _i), ("in_", _i), ("out", _i), ("N", _i), ("M", _i)]
+
+
+class ElsaHostLayer(ctypes.Structure):
+    _fields_ = [("X", _vp), ("Y", _vp), ("W", _vp), ("bias", _vp),
+                ("rows", _i), ("in_", _i), ("out", _i), ("N", _i), ("M", _i)]
+
+
+def _sig(name, restype, argtypes):
+    fn = getattr(_lib, name)
+    fn.restype = restype
+    fn.argtypes = argtypes
+    return fn
+
+
+_values_bytes = _sig("elsa_nm_values_bytes", _sz, [_i, _i, _i, _i, _i])
+_index_bytes = _sig("elsa_nm_index_bytes", _sz, [_i, _i, _i, _i])
+_workspace_bytes = _sig("elsa_workspace_bytes", _sz, [_i, _i, _i, _i, _i, _i])
+_compress = _sig("elsa_nm_compress", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
+_unpack = _sig("elsa_nm_unpack", _i, [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp])
+_linear = _sig("elsa_nm_linear", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
+_vit_ws = _sig("elsa_vit_workspace_bytes", _sz, [ctypes.POINTER(ElsaLayer), _i, _i])
+_vit = _sig("elsa_vit_linears", _i, [ctypes.POINTER(ElsaLayer), _i, _i, _vp, _sz, _vp, _vp])
+_vit_host_bytes = _sig("elsa_vit_host_device_bytes", _sz, [ctypes.POINTER(ElsaHostLayer), _i, _i])
+_vit_host = _sig("elsa_vit_linears_host", _i, [ctypes.POINTER(ElsaHostLayer), _i, _i, _vp, _sz, _vp, _vp])
+_set_variant = _sig("elsa_set_linear_variant", _i, [_i])
+_get_variant = _sig("elsa_get_linear_variant", _i, [])
+_launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
+_last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
+
+
+class ElsaError(RuntimeError):
+    def __init__(self, status: int):
+        self.status = status
+        super().__init__("%s: %s" % (ERR_NAMES.get(status, status), elsa_last_error()))
+
+
+def _check(status: int):
+    if status != OK:
+        raise ElsaError(status)
+
+
+def elsa_last_error() -> str:
+    return (_last_error() or b"").decode()
+
+
+def elsa_launch_count() -> int:
+    return int(_launch_count())
+
+
+def elsa_set_linear_variant(v: int):
+    _check(_set_variant(v))
+
+
+def elsa_get_linear_variant() -> int:
+    return int(_get_variant())
+
+
+def dtype_code(dtype: torch.dtype) -> int:
+    if dtype == torch.float16:
+        return F16
+    if dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("fp16 or bf16 expected, got %s" % dtype)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("contiguous tensor expected")
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def elsa_nm_values_bytes(out, in_, N, M, dtype=F16) -> int:
+    return int(_values_bytes(out, in_, N, M, dtype))
+
+
+def elsa_nm_index_bytes(out, in_, N, M) -> int:
+    return int(_index_bytes(out, in_, N, M))
+
+
+def elsa_workspace_bytes(rows, in_, out, N, M, dtype=F16) -> int:
+    return int(_workspace_bytes(rows, in_, out, N, M, dtype))
+
+
+def alloc_packed(out, in_, N, M, dtype: torch.dtype, device="cuda"):
+    """Uninitialised (vals, idx) tensors of the packed form; idx is None when N == M."""
+    vals = torch.empty((out, in_ // M * N), dtype=dtype, device=device)
+    words = elsa_nm_index_bytes(out, in_, N, M) // 4 // out
+    idx = torch.empty((out, words), dtype=torch.int32, device=device) if words else None
+    return vals, idx
+
+
+def elsa_nm_compress(W: torch.Tensor, N: int, M: int, vals=None, idx=None, stream=None):
+    """Packed (vals, idx) of W [out, in] at level N:M."""
+    out, in_ = W.shape
+    if vals is None:
+        if elsa_nm_values_bytes(out, in_, N, M, dtype_code(W.dtype)) == 0:
+            _check(_compress(_ptr(W), out, in_, N, M, dtype_code(W.dtype), None, None, _stream(stream)))
+        vals, idx = alloc_packed(out, in_, N, M, W.dtype, W.device)
+    _check(_compress(_ptr(W), out, in_, N, M, dtype_code(W.dtype), _ptr(vals), _ptr(idx), _stream(stream)))
+    return vals, idx
+
+
+def elsa_nm_unpack(vals: torch.Tensor, idx, out: int, in_: int, N: int, M: int, W_masked=None, stream=None):
+    if W_masked is None:
+        W_masked = torch.empty((out, in_), dtype=vals.dtype, device=vals.device)
+    _check(_unpack(_ptr(vals), _ptr(idx), out, in_, N, M, dtype_code(vals.dtype), _ptr(W_masked), _stream(stream)))
+    return W_masked
+
+
+def alloc_workspace(nbytes: int, device="cuda"):
+    return torch.empty((max(nbytes, 256),), dtype=torch.uint8, device=device)
+
+
+def elsa_nm_linear(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_: int, N: int, M: int,
+                   Y=None, workspace=None, dev_status=None, stream=None):
+    """Y [rows, out] = X [rows, in] . W_masked^T + bias from the packed weight."""
+    rows = X.shape[0]
+    code = dtype_code(X.dtype)
+    if Y is None:
+        Y = torch.empty((rows, out), dtype=X.dtype, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(elsa_workspace_bytes(rows, in_, out, N, M, code), X.device)
+    _check(_linear(_ptr(X), rows, _ptr(vals), _ptr(idx), _ptr(bias), out, in_, N, M, code, _ptr(Y),
+                   _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
+    return Y
+
+
+def make_layer_table(layers):
+    """ctypes array of elsa_layer from dicts / objects with X, Y, vals, idx, bias, N, M tensors."""
+    arr = (ElsaLayer * len(layers))()
+    for a, l in zip(arr, layers):
+        X, Y = l["X"], l["Y"]
+        a.X, a.Y = _ptr(X), _ptr(Y)
+        a.vals, a.idx, a.bias = _ptr(l["vals"]), _ptr(l.get("idx")), _ptr(l.get("bias"))
+        a.rows, a.in_, a.out = X.shape[0], X.shape[1], Y.shape[1]
+        a.N, a.M = l["N"], l["M"]
+    return arr
+
+
+def elsa_vit_workspace_bytes(table, dtype_c: int) -> int:
+    return int(_vit_ws(table, len(table), dtype_c))
+
+
+def elsa_vit_linears(table, dtype_c: int, workspace, dev_status=None, stream=None):
+    _check(_vit(table, len(table), dtype_c, _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
+
+
+def make_host_layer_table(layers):
+    """ctypes array of elsa_host_layer from dicts of HOST tensors X, Y, W, bias and N, M."""
+    arr = (ElsaHostLayer * len(layers))()
+    for a, l in zip(arr, layers):
+        X, Y, W = l["X"], l["Y"], l["W"]
+        a.X, a.Y, a.W, a.bias = _ptr(X), _ptr(Y), _ptr(W), _ptr(l.get("bias"))
+        a.rows, a.in_, a.out = X.shape[0], X.shape[1], W.shape[0]
+        a.N, a.M = l["N"], l["M"]
+    return arr
+
+
+def elsa_vit_host_device_bytes(table, dtype_c: int) -> int:
+    return int(_vit_host_bytes(table, len(table), dtype_c))
+
+
+def elsa_vit_linears_host(table, dtype_c: int, device_mem, dev_status=None, stream=None):
+    _check(_vit_host(table, len(table), dtype_c, _ptr(device_mem), device_mem.numel(), _ptr(dev_status),
+                     _stream(stream)))

@@ -1,0 +1,337 @@
+// C ABI of libelsa: host-side validation, dispatch and error reporting.  No kernel lives here.
+
+#include <stdarg.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <atomic>
+
+#include "elsa_internal.h"
+
+namespace elsa {
+
+static thread_local char g_error[512] = "";
+static std::atomic<unsigned long long> g_launches{0};
+static std::atomic<int> g_variant{(int)ELSA_VARIANT_AUTO};
+
+elsa_status fail(elsa_status st, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_error, sizeof g_error, fmt, ap);
+    va_end(ap);
+    return st;
+}
+
+elsa_status launched(const char* what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "launch of %s failed: %s", what, cudaGetErrorString(e));
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    return ELSA_OK;
+}
+
+elsa_status device_info(DeviceInfo* info)
+{
+    static DeviceInfo cache[64];
+    static std::atomic<bool> have[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaError_t e = cudaGetLastError();
+        return fail(ELSA_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    }
+    const int slot = dev & 63;
+    if (!have[slot].load(std::memory_order_acquire)) {
+        DeviceInfo d;
+        d.device = dev;
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) goto bad;
+        d.sm_count = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) goto bad;
+        d.cc_major = v;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) goto bad;
+        d.smem_optin = (size_t)v;
+        cache[slot] = d;
+        have[slot].store(true, std::memory_order_release);
+    }
+    *info = cache[slot];
+    if (info->cc_major != 10)
+        return fail(ELSA_ERR_ARCH, "device %d has compute capability %d.x; this library is built for 10.x only",
+                    dev, info->cc_major);
+    return ELSA_OK;
+bad:
+    cudaError_t e = cudaGetLastError();
+    return fail(ELSA_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+}
+
+namespace {
+
+bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
+
+elsa_status check_level(int out, int in, int N, int M, int dtype)
+{
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return fail(ELSA_ERR_DTYPE, "dtype %d is neither ELSA_F16 nor ELSA_BF16", dtype);
+    if (out <= 0 || in <= 0) return fail(ELSA_ERR_SHAPE, "non-positive dimension (out=%d, in=%d)", out, in);
+    if (index_bits(M) < 0 || N < 1 || N > M) return fail(ELSA_ERR_NM, "unsupported level %d:%d (M in {4, 8, 16}, 1 <= N <= M)", N, M);
+    if (in % M != 0) return fail(ELSA_ERR_SHAPE, "in=%d is not a multiple of M=%d", in, M);
+    if (in % 8 != 0 || out % 8 != 0) return fail(ELSA_ERR_ALIGN, "in=%d and out=%d must be multiples of 8 (16-byte row pitch)", in, out);
+    return ELSA_OK;
+}
+
+elsa_status check_linear(const void* X, int rows, const void* vals, const uint32_t* idx, const void* bias,
+                         int out, int in, int N, int M, int dtype, const void* Y, const void* workspace,
+                         size_t workspace_bytes)
+{
+    if (!X || !vals || !Y) return fail(ELSA_ERR_NULL, "X, vals and Y must not be NULL");
+    elsa_status st = check_level(out, in, N, M, dtype);
+    if (st != ELSA_OK) return st;
+    if (rows <= 0) return fail(ELSA_ERR_SHAPE, "non-positive rows=%d", rows);
+    if (N != M && !idx) return fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+    if (!aligned16(X) || !aligned16(vals) || !aligned16(Y) || (idx && !aligned16(idx)) ||
+        (bias && !aligned16(bias)))
+        return fail(ELSA_ERR_ALIGN, "X, vals, idx, bias and Y must be 16-byte aligned");
+    const size_t need = elsa_workspace_bytes(rows, in, out, N, M, (elsa_dtype)dtype);
+    if (need) {
+        if (!workspace || workspace_bytes < need)
+            return fail(ELSA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, workspace ? workspace_bytes : (size_t)0);
+        if (((uintptr_t)workspace & 255u) != 0) return fail(ELSA_ERR_ALIGN, "workspace must be 256-byte aligned");
+    }
+    return ELSA_OK;
+}
+
+// After validation: enqueue one layer.
+elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t* idx, const void* bias, int out,
+                       int in, int N, int M, elsa_dtype dtype, void* Y, void* workspace, uint32_t* dev_status,
+                       cudaStream_t stream)
+{
+    const int variant = g_variant.load(std::memory_order_relaxed);
+    if (variant == ELSA_VARIANT_SIMT)
+        return launch_linear_simt((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
+                                  in, N, M, dtype, (uint16_t*)Y, stream);
+    // Tensor-core path.  The dense level multiplies the stored values as they are; every other
+    // level first rebuilds the weight image the MMA reads, in the caller's scratch.
+    const uint16_t* Wd = (const uint16_t*)vals;
+    if (N != M) {
+        elsa_status st = launch_unpack((const uint16_t*)vals, idx, out, in, N, M, (uint16_t*)workspace, stream);
+        if (st != ELSA_OK) return st;
+        Wd = (const uint16_t*)workspace;
+    }
+    return launch_linear_tc_dense((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype,
+                                  (uint16_t*)Y, dev_status, stream);
+}
+
+}  // namespace
+}  // namespace elsa
+
+using namespace elsa;
+
+extern "C" {
+
+size_t elsa_nm_values_bytes(int out, int in, int N, int M, elsa_dtype dtype)
+{
+    if (out <= 0 || in <= 0 || index_bits(M) < 0 || N < 1 || N > M || in % M != 0) return 0;
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return 0;
+    return (size_t)out * values_per_row(in, N, M) * 2;
+}
+
+size_t elsa_nm_index_bytes(int out, int in, int N, int M)
+{
+    if (out <= 0 || in <= 0 || index_bits(M) < 0 || N < 1 || N > M || in % M != 0) return 0;
+    return (size_t)out * index_words_per_row(in, N, M) * 4;
+}
+
+size_t elsa_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype dtype)
+{
+    (void)rows;
+    if (out <= 0 || in <= 0 || index_bits(M) < 0 || N < 1 || N > M || in % M != 0) return 0;
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return 0;
+    if (N == M) return 0;                              // the dense level needs no weight image
+    return round_up((size_t)out * (size_t)in * 2, 256);  // dense image of the masked weight
+}
+
+elsa_status elsa_nm_compress(const void* W, int out, int in, int N, int M, elsa_dtype dtype, void* vals,
+                             uint32_t* idx, void* stream)
+{
+    if (!W || !vals) return fail(ELSA_ERR_NULL, "W and vals must not be NULL");
+    elsa_status st = check_level(out, in, N, M, dtype);
+    if (st != ELSA_OK) return st;
+    if (N != M && !idx) return fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+    if (!aligned16(W) || !aligned16(vals) || (idx && !aligned16(idx)))
+        return fail(ELSA_ERR_ALIGN, "W, vals and idx must be 16-byte aligned");
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != ELSA_OK) return st;
+    return launch_compress((const uint16_t*)W, out, in, N, M, (uint16_t*)vals, N == M ? nullptr : idx,
+                           (cudaStream_t)stream);
+}
+
+elsa_status elsa_nm_unpack(const void* vals, const uint32_t* idx, int out, int in, int N, int M, elsa_dtype dtype,
+                           void* W_masked, void* stream)
+{
+    if (!vals || !W_masked) return fail(ELSA_ERR_NULL, "vals and W_masked must not be NULL");
+    elsa_status st = check_level(out, in, N, M, dtype);
+    if (st != ELSA_OK) return st;
+    if (N != M && !idx) return fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+    if (!aligned16(vals) || !aligned16(W_masked) || (idx && !aligned16(idx)))
+        return fail(ELSA_ERR_ALIGN, "vals, idx and W_masked must be 16-byte aligned");
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != ELSA_OK) return st;
+    return launch_unpack((const uint16_t*)vals, N == M ? nullptr : idx, out, in, N, M, (uint16_t*)W_masked,
+                         (cudaStream_t)stream);
+}
+
+elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint32_t* idx, const void* bias,
+                           int out, int in, int N, int M, elsa_dtype dtype, void* Y, void* workspace,
+                           size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    elsa_status st = check_linear(X, rows, vals, idx, bias, out, in, N, M, dtype, Y, workspace, workspace_bytes);
+    if (st != ELSA_OK) return st;
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != ELSA_OK) return st;
+    return run_linear(X, rows, vals, N == M ? nullptr : idx, bias, out, in, N, M, dtype, Y, workspace, dev_status,
+                      (cudaStream_t)stream);
+}
+
+size_t elsa_vit_workspace_bytes(const elsa_layer* cfg, int n_layers, elsa_dtype dtype)
+{
+    size_t need = 0;
+    if (!cfg) return 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const size_t b = elsa_workspace_bytes(cfg[l].rows, cfg[l].in, cfg[l].out, cfg[l].N, cfg[l].M, dtype);
+        if (b > need) need = b;
+    }
+    return need;
+}
+
+elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dtype, void* workspace,
+                             size_t workspace_bytes, uint32_t* dev_status, void* stream)
+{
+    if (!cfg) return fail(ELSA_ERR_NULL, "cfg must not be NULL");
+    if (n_layers <= 0) return fail(ELSA_ERR_SHAPE, "non-positive n_layers=%d", n_layers);
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_layer& c = cfg[l];
+        elsa_status st = check_linear(c.X, c.rows, c.vals, c.idx, c.bias, c.out, c.in, c.N, c.M, dtype, c.Y,
+                                      workspace, workspace_bytes);
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "layer %d: %s", l, msg);
+        }
+    }
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_layer& c = cfg[l];
+        st = run_linear(c.X, c.rows, c.vals, c.N == c.M ? nullptr : c.idx, c.bias, c.out, c.in, c.N, c.M, dtype,
+                        c.Y, workspace, dev_status, (cudaStream_t)stream);
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "layer %d: %s", l, msg);
+        }
+    }
+    return ELSA_OK;
+}
+
+// Device memory plan of the host-memory variant: regions reused by every layer, each sized for
+// the largest layer: X | Y | W | bias | vals | idx | linear workspace.
+namespace {
+struct HostPlan {
+    size_t x, y, w, bias, vals, idx, ws, total;
+};
+bool host_plan(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype, HostPlan* plan)
+{
+    size_t mx = 0, my = 0, mw = 0, mb = 0, mv = 0, mi = 0, ms = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_host_layer& c = cfg[l];
+        if (c.rows <= 0 || c.in <= 0 || c.out <= 0) return false;
+        auto up = [](size_t& m, size_t v) { if (v > m) m = v; };
+        up(mx, (size_t)c.rows * c.in * 2);
+        up(my, (size_t)c.rows * c.out * 2);
+        up(mw, (size_t)c.out * c.in * 2);
+        up(mb, (size_t)c.out * 2);
+        up(mv, elsa_nm_values_bytes(c.out, c.in, c.N, c.M, dtype));
+        up(mi, elsa_nm_index_bytes(c.out, c.in, c.N, c.M));
+        up(ms, elsa_workspace_bytes(c.rows, c.in, c.out, c.N, c.M, dtype));
+    }
+    size_t off = 0;
+    plan->x = off; off += round_up(mx, 256);
+    plan->y = off; off += round_up(my, 256);
+    plan->w = off; off += round_up(mw, 256);
+    plan->bias = off; off += round_up(mb, 256);
+    plan->vals = off; off += round_up(mv, 256);
+    plan->idx = off; off += round_up(mi, 256);
+    plan->ws = off; off += round_up(ms, 256);
+    plan->total = off;
+    return true;
+}
+}  // namespace
+
+size_t elsa_vit_host_device_bytes(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype)
+{
+    HostPlan plan;
+    if (!cfg || n_layers <= 0 || !host_plan(cfg, n_layers, dtype, &plan)) return 0;
+    return plan.total;
+}
+
+elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype, void* device_mem,
+                                  size_t device_bytes, uint32_t* dev_status, void* stream_)
+{
+    if (!cfg) return fail(ELSA_ERR_NULL, "cfg must not be NULL");
+    if (n_layers <= 0) return fail(ELSA_ERR_SHAPE, "non-positive n_layers=%d", n_layers);
+    HostPlan plan;
+    if (!host_plan(cfg, n_layers, dtype, &plan)) return fail(ELSA_ERR_SHAPE, "a layer has a non-positive dimension");
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_host_layer& c = cfg[l];
+        if (!c.X || !c.Y || !c.W) return fail(ELSA_ERR_NULL, "layer %d: X, Y and W must not be NULL", l);
+        elsa_status st = check_level(c.out, c.in, c.N, c.M, dtype);
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "layer %d: %s", l, msg);
+        }
+    }
+    if (!device_mem || device_bytes < plan.total)
+        return fail(ELSA_ERR_WORKSPACE, "device memory of %zu bytes needed, %zu given", plan.total,
+                    device_mem ? device_bytes : (size_t)0);
+    if (((uintptr_t)device_mem & 255u) != 0) return fail(ELSA_ERR_ALIGN, "device_mem must be 256-byte aligned");
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+
+    cudaStream_t stream = (cudaStream_t)stream_;
+    uint8_t* base = (uint8_t*)device_mem;
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_host_layer& c = cfg[l];
+        void* dX = base + plan.x; void* dY = base + plan.y; void* dW = base + plan.w;
+        void* dB = c.bias ? base + plan.bias : nullptr;
+        void* dV = base + plan.vals; uint32_t* dI = c.N == c.M ? nullptr : (uint32_t*)(base + plan.idx);
+        cudaError_t e = cudaMemcpyAsync(dW, c.W, (size_t)c.out * c.in * 2, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess && c.bias) e = cudaMemcpyAsync(dB, c.bias, (size_t)c.out * 2, cudaMemcpyHostToDevice, stream);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dX, c.X, (size_t)c.rows * c.in * 2, cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "layer %d: host-to-device copy: %s", l, cudaGetErrorString(e));
+        if ((st = launch_compress((const uint16_t*)dW, c.out, c.in, c.N, c.M, (uint16_t*)dV, dI, stream)) != ELSA_OK) return st;
+        if ((st = run_linear(dX, c.rows, dV, dI, dB, c.out, c.in, c.N, c.M, dtype, dY, base + plan.ws, dev_status,
+                             stream)) != ELSA_OK)
+            return st;
+        e = cudaMemcpyAsync(c.Y, dY, (size_t)c.rows * c.out * 2, cudaMemcpyDeviceToHost, stream);
+        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "layer %d: device-to-host copy: %s", l, cudaGetErrorString(e));
+    }
+    return ELSA_OK;
+}
+
+elsa_status elsa_set_linear_variant(elsa_variant v)
+{
+    if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE)
+        return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
+    g_variant.store((int)v, std::memory_order_relaxed);
+    return ELSA_OK;
+}
+
+elsa_variant elsa_get_linear_variant(void) { return (elsa_variant)g_variant.load(std::memory_order_relaxed); }
+
+unsigned long long elsa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* elsa_last_error(void) { return g_error; }
+
+}  // extern "C"

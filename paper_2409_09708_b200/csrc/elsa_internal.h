@@ -1,0 +1,49 @@
+// Internal declarations shared by the translation units of libelsa (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "elsa.h"
+
+namespace elsa {
+
+// log2(M) for the supported group sizes, -1 otherwise.
+inline int index_bits(int M) { return M == 4 ? 2 : M == 8 ? 3 : M == 16 ? 4 : -1; }
+inline size_t values_per_row(int in, int N, int M) { return (size_t)(in / M) * (size_t)N; }
+inline size_t index_words_per_row(int in, int N, int M)
+{
+    if (N == M) return 0;
+    return ((size_t)(in / M) * (size_t)N * (size_t)index_bits(M) + 31) / 32;
+}
+inline size_t round_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Records a message for elsa_last_error() and returns `st`.
+elsa_status fail(elsa_status st, const char* fmt, ...);
+// Counts one kernel launch and converts the launch's cudaError_t.
+elsa_status launched(const char* what);
+
+struct DeviceInfo {
+    int device;
+    int sm_count;
+    int cc_major;
+    size_t smem_optin;
+};
+// Properties of the current device (cached per device).
+elsa_status device_info(DeviceInfo* info);
+
+// --- kernels (each enqueues on `stream` and returns the launch status) ---
+elsa_status launch_compress(const uint16_t* W, int out, int in, int N, int M, uint16_t* vals,
+                            uint32_t* idx, cudaStream_t stream);
+elsa_status launch_unpack(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
+                          uint16_t* Wm, cudaStream_t stream);
+elsa_status launch_linear_simt(const uint16_t* X, int rows, const uint16_t* vals,
+                               const uint32_t* idx, const uint16_t* bias, int out, int in, int N,
+                               int M, elsa_dtype dtype, uint16_t* Y, cudaStream_t stream);
+// Dense tensor-core GEMM Y = X Wd^T + bias with Wd a dense [out][in] image (tcgen05 / TMEM / TMA).
+elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* Wd,
+                                   const uint16_t* bias, int out, int in, elsa_dtype dtype,
+                                   uint16_t* Y, uint32_t* dev_status, cudaStream_t stream);
+
+}  // namespace elsa

@@ -1,0 +1,264 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded bytes.  Masks, packed values and index words must match bit for bit; linear outputs must
+stay within relative Frobenius error 5e-3 and |err| <= 1e-2 * (|ref| + 1) of the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import elsa_oracle as eo
+from paper_2409_09708_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+REL_FRO_TOL = 5e-3
+ELEM_TOL = 1e-2
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2409_09708_b200 import build
+    build.build()
+    from paper_2409_09708_b200 import binding
+    return binding
+
+
+def ocode(dtype):
+    return eo.F16 if dtype == torch.float16 else eo.BF16
+
+
+def idx_bits(idx):
+    return idx.cpu().numpy().view(np.uint32) if idx is not None else np.zeros((0, 0), np.uint32)
+
+
+def check_close(Y_gpu, ref):
+    got = Y_gpu.detach().to(torch.float64).cpu().numpy()
+    assert np.isfinite(got).all()
+    err = got - ref
+    rel = np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30)
+    worst = np.max(np.abs(err) / (np.abs(ref) + 1.0))
+    assert rel <= REL_FRO_TOL, "relative Frobenius error %g" % rel
+    assert worst <= ELEM_TOL, "per-element error %g" % worst
+    return rel, worst
+
+
+def oracle_linear(X, W, bias, N, M, dtype):
+    vals, idx, _ = eo.nm_compress(synth.bits(W), N, M)
+    return eo.nm_linear_f64(synth.bits(X), vals, idx, None if bias is None else synth.bits(bias),
+                            W.shape[0], W.shape[1], N, M, ocode(dtype))
+
+
+# ------------------------------------------------------------------ compress / unpack
+
+COMPRESS_SHAPES = [(768, 768), (16, 64), (40, 1008), (24, 16 * 23), (8, 4096)]
+LEVELS = [(1, 4), (2, 4), (3, 4), (4, 4), (1, 8), (2, 8), (3, 8), (4, 8), (7, 8), (8, 8),
+          (1, 16), (2, 16), (4, 16), (8, 16), (15, 16), (16, 16)]
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("shape", COMPRESS_SHAPES)
+def test_compress_and_unpack_match_oracle_bit_for_bit(lib, shape, dtype):
+    out, in_ = shape
+    W = synth.randn((out, in_), 900 + out + in_, synth.W_STD, dtype)
+    Wb = synth.bits(W).copy()
+    Wb[0, :8] = [0x8000, 0, 0x8000, 0, 0, 0, 0, 0x8000]           # signed zeros
+    Wb[1, :16] = Wb[1, 0]                                           # an all-equal stretch
+    W = synth.from_bits(Wb, dtype)
+    Wd = W.cuda()
+    for N, M in LEVELS:
+        if in_ % M:
+            continue
+        vals, idx = lib.elsa_nm_compress(Wd, N, M)
+        torch.cuda.synchronize()
+        ovals, oidx, omask = eo.nm_compress(Wb, N, M)
+        assert (synth.bits(vals) == ovals).all(), (N, M)
+        assert (idx_bits(idx) == oidx).all(), (N, M)
+        Wm = lib.elsa_nm_unpack(vals, idx, out, in_, N, M)
+        torch.cuda.synchronize()
+        assert (synth.bits(Wm) == eo.nm_unpack(ovals, oidx, out, in_, N, M)).all(), (N, M)
+        assert (synth.bits(Wm) == np.where(omask == 1, Wb, 0)).all()
+
+
+def test_compress_weight_shapes_of_the_workloads(lib):
+    """Every distinct weight shape and level of the DeiT-B and Swin-B tables, checked in full."""
+    seen = set()
+    for name in ("deit_b_block_b64", "deit_b_stack_b256", "swin_b_stack_b128"):
+        layers, dt = synth.workload(name)
+        dtype = synth.torch_dtype(dt)
+        for l in layers:
+            key = (l.out, l.in_, l.N, l.M, dt)
+            if key in seen:
+                continue
+            seen.add(key)
+            W = synth.randn((l.out, l.in_), l.seed_w, synth.W_STD, dtype)
+            vals, idx = lib.elsa_nm_compress(W.cuda(), l.N, l.M)
+            ovals, oidx, _ = eo.nm_compress(synth.bits(W), l.N, l.M)
+            assert (synth.bits(vals) == ovals).all(), key
+            assert (idx_bits(idx) == oidx).all(), key
+    assert len(seen) > 20
+
+
+# ------------------------------------------------------------------ linear
+
+def run_linear(lib, X, W, bias, N, M, variant):
+    lib.elsa_set_linear_variant(variant)
+    try:
+        Wd = W.cuda()
+        vals, idx = lib.elsa_nm_compress(Wd, N, M)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        Y = lib.elsa_nm_linear(X.cuda(), vals, idx, None if bias is None else bias.cuda(),
+                               W.shape[0], W.shape[1], N, M, dev_status=status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0, "device status %#x" % int(status.item())
+        return Y
+    finally:
+        lib.elsa_set_linear_variant(lib.VARIANT_AUTO)
+
+
+VARIANTS = ["simt", "tc_dense"]
+
+
+def variant_code(lib, name):
+    return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "auto": lib.VARIANT_AUTO}[name]
+
+
+LINEAR_CASES = [
+    # rows, in, out, N, M   (ragged row tiles, several K blocks, feature tiles of every width)
+    (197, 768, 768, 4, 8),
+    (130, 64, 128, 2, 4),
+    (1, 128, 64, 1, 4),
+    (300, 200, 384, 3, 8),      # K not a multiple of 64, 192-wide feature tile
+    (257, 1024, 136, 8, 8),     # dense level, out not a multiple of the chunk width
+    (515, 512, 1000, 2, 16),
+    (1024, 3072, 768, 1, 8),
+    (700, 256, 2304, 4, 16),
+]
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("case", LINEAR_CASES)
+def test_linear_matches_oracle(lib, case, dtype, variant):
+    rows, in_, out, N, M = case
+    X = synth.randn((rows, in_), 11 * rows + in_, synth.X_STD, dtype)
+    W = synth.randn((out, in_), 13 * out + in_, synth.W_STD, dtype)
+    bias = synth.randn((out,), 17 * out, synth.B_STD, dtype)
+    Y = run_linear(lib, X, W, bias, N, M, variant_code(lib, variant))
+    check_close(Y, oracle_linear(X, W, bias, N, M, dtype))
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_identity_activations_give_the_masked_weight_exactly(lib, variant):
+    """X = I: Y must be W_masked^T + bias rounded once -- no tolerance, pins indexing and layout."""
+    dtype = torch.float16
+    in_, out = 256, 320
+    W = synth.randn((out, in_), 5, synth.W_STD, dtype)
+    bias = synth.randn((out,), 6, synth.B_STD, dtype)
+    X = torch.eye(in_, dtype=dtype)
+    for N, M in [(2, 8), (1, 4), (3, 8), (8, 8)]:
+        Y = run_linear(lib, X, W, bias, N, M, variant_code(lib, variant))
+        ref = oracle_linear(X, W, bias, N, M, dtype)
+        expect = torch.from_numpy(ref).to(dtype)            # one rounding of the exact value
+        assert torch.equal(Y.cpu(), expect), (N, M)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_integer_inputs_are_exact(lib, variant):
+    """Small integers: every product and partial sum is exact in fp32, so is the result."""
+    rng = np.random.default_rng(3)
+    rows, in_, out = 200, 192, 96
+    X = torch.from_numpy(rng.integers(-4, 5, (rows, in_))).to(torch.bfloat16)
+    W = torch.from_numpy(rng.integers(-8, 9, (out, in_))).to(torch.bfloat16)
+    for N, M in [(4, 8), (2, 4), (1, 16)]:
+        Y = run_linear(lib, X, W, None, N, M, variant_code(lib, variant))
+        ref = oracle_linear(X, W, None, N, M, torch.bfloat16)
+        # the exact integer result, rounded once to bf16 (integers up to 256 are unchanged)
+        assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
+
+
+def test_no_bias_and_zero_rows_of_padding(lib):
+    dtype = torch.bfloat16
+    X = synth.randn((129, 128), 1, 1.0, dtype)
+    W = synth.randn((64, 128), 2, synth.W_STD, dtype)
+    Yc = torch.full((129 + 8, 64), 7.0, dtype=dtype, device="cuda")      # guard rows after Y
+    Wd = W.cuda()
+    vals, idx = lib.elsa_nm_compress(Wd, 2, 4)
+    lib.elsa_nm_linear(X.cuda(), vals, idx, None, 64, 128, 2, 4, Y=Yc[:129])
+    torch.cuda.synchronize()
+    check_close(Yc[:129], oracle_linear(X, W, None, 2, 4, dtype))
+    assert (Yc[129:] == 7.0).all()                                       # nothing written past the last row
+
+
+def test_single_layer_config(lib):
+    """197 x 768 activations, 768 x 768 weight at 4:8, fp16, seed 0: checked in full."""
+    (layer,), dt = synth.workload("single_layer")
+    dtype = synth.torch_dtype(dt)
+    X, W, b = synth.layer_tensors(layer, dtype)
+    ref = oracle_linear(X, W, b, layer.N, layer.M, dtype)
+    for v in ("auto", "simt", "tc_dense"):
+        check_close(run_linear(lib, X, W, b, layer.N, layer.M, variant_code(lib, v)), ref)
+
+
+def stack_check(lib, layers, dtype, rows_sampled, seed):
+    """Run a table through elsa_vit_linears and check sampled rows of every layer against the oracle."""
+    code = lib.dtype_code(dtype)
+    dev = []
+    for l in layers:
+        X, W, b = synth.layer_tensors(l, dtype, device="cuda")
+        vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+        Y = torch.empty((l.rows, l.out), dtype=dtype, device="cuda")
+        dev.append(dict(X=X, Y=Y, W=W, vals=vals, idx=idx, bias=b, N=l.N, M=l.M))
+    table = lib.make_layer_table(dev)
+    ws = lib.alloc_workspace(lib.elsa_vit_workspace_bytes(table, code))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lib.elsa_vit_linears(table, code, ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    for i, (l, d) in enumerate(zip(layers, dev)):
+        pick = synth.sample_rows(l.rows, rows_sampled, seed + i)
+        sel = torch.from_numpy(pick).cuda()
+        Xs = d["X"][sel].cpu()
+        ovals, oidx, _ = eo.nm_compress(synth.bits(d["W"]), l.N, l.M)
+        assert (synth.bits(d["vals"]) == ovals).all() and (idx_bits(d["idx"]) == oidx).all(), l.name
+        ref = eo.nm_linear_f64(synth.bits(Xs), ovals, oidx, synth.bits(d["bias"]), l.out, l.in_, l.N, l.M,
+                               ocode(dtype))
+        check_close(d["Y"][sel], ref)
+        del d["X"], d["Y"]
+
+
+def test_deit_b_block_layers_sampled_rows(lib):
+    """One DeiT-B block at batch 64 (qkv 4:8, proj 2:8, fc1 2:8, fc2 1:8), full size on the GPU,
+    sampled rows against the oracle, weights compared in full."""
+    layers, dt = synth.workload("deit_b_block_b64")
+    stack_check(lib, layers, synth.torch_dtype(dt), 160, 21)
+
+
+def test_deit_b_stack_full_size_sampled_rows(lib):
+    """All 48 DeiT-B linears at batch 256, the configuration the benchmark times."""
+    layers, dt = synth.workload("deit_b_stack_b256")
+    dtype = synth.torch_dtype(dt)
+    # run the whole table in one call, a few layers' worth of memory at a time is not needed: 15 GB fits
+    stack_check(lib, layers, dtype, 24, 31)
+
+
+def test_swin_b_stack_full_size_sampled_rows(lib):
+    layers, dt = synth.workload("swin_b_stack_b128")
+    stack_check(lib, layers, synth.torch_dtype(dt), 24, 41)
+
+
+def test_host_memory_entry_point_matches_device_entry_point(lib):
+    dtype = torch.float16
+    layers = [synth.Layer("a", 300, 256, 384, 2, 8, 1, 2, 3), synth.Layer("b", 300, 384, 128, 4, 4, 4, 5, 6),
+              synth.Layer("c", 77, 128, 256, 1, 16, 7, 8, 9)]
+    host, dev_out = [], []
+    for l in layers:
+        X, W, b = synth.layer_tensors(l, dtype)
+        Y = torch.empty((l.rows, l.out), dtype=dtype).pin_memory()
+        host.append(dict(X=X.pin_memory(), Y=Y, W=W.pin_memory(), bias=b.pin_memory(), N=l.N, M=l.M))
+        dev_out.append(run_linear(lib, X, W, b, l.N, l.M, lib.VARIANT_AUTO).cpu())
+    table = lib.make_host_layer_table(host)
+    code = lib.dtype_code(dtype)
+    mem = lib.alloc_workspace(lib.elsa_vit_host_device_bytes(table, code))
+    lib.elsa_vit_linears_host(table, code, mem)
+    torch.cuda.synchronize()
+    for h, y in zip(host, dev_out):
+        assert torch.equal(h["Y"], y)
