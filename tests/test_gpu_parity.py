@@ -26,8 +26,10 @@ def ocode(dtype):
     return eo.F16 if dtype == torch.float16 else eo.BF16
 
 
-def idx_bits(idx):
-    return idx.cpu().numpy().view(np.uint32) if idx is not None else np.zeros((0, 0), np.uint32)
+def idx_bits(idx, like=None):
+    if idx is None:          # the dense level stores no indices
+        return np.zeros(like.shape if like is not None else (0, 0), np.uint32)
+    return idx.cpu().numpy().view(np.uint32)
 
 
 def check_close(Y_gpu, ref):
@@ -71,7 +73,7 @@ def test_compress_and_unpack_match_oracle_bit_for_bit(lib, shape, dtype):
         torch.cuda.synchronize()
         ovals, oidx, omask = eo.nm_compress(Wb, N, M)
         assert (synth.bits(vals) == ovals).all(), (N, M)
-        assert (idx_bits(idx) == oidx).all(), (N, M)
+        assert (idx_bits(idx, oidx) == oidx).all(), (N, M)
         Wm = lib.elsa_nm_unpack(vals, idx, out, in_, N, M)
         torch.cuda.synchronize()
         assert (synth.bits(Wm) == eo.nm_unpack(ovals, oidx, out, in_, N, M)).all(), (N, M)
@@ -93,7 +95,7 @@ def test_compress_weight_shapes_of_the_workloads(lib):
             vals, idx = lib.elsa_nm_compress(W.cuda(), l.N, l.M)
             ovals, oidx, _ = eo.nm_compress(synth.bits(W), l.N, l.M)
             assert (synth.bits(vals) == ovals).all(), key
-            assert (idx_bits(idx) == oidx).all(), key
+            assert (idx_bits(idx, oidx) == oidx).all(), key
     assert len(seen) > 20
 
 
@@ -218,7 +220,7 @@ def stack_check(lib, layers, dtype, rows_sampled, seed):
         sel = torch.from_numpy(pick).cuda()
         Xs = d["X"][sel].cpu()
         ovals, oidx, _ = eo.nm_compress(synth.bits(d["W"]), l.N, l.M)
-        assert (synth.bits(d["vals"]) == ovals).all() and (idx_bits(d["idx"]) == oidx).all(), l.name
+        assert (synth.bits(d["vals"]) == ovals).all() and (idx_bits(d["idx"], oidx) == oidx).all(), l.name
         ref = eo.nm_linear_f64(synth.bits(Xs), ovals, oidx, synth.bits(d["bias"]), l.out, l.in_, l.N, l.M,
                                ocode(dtype))
         check_close(d["Y"][sel], ref)
