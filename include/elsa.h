@@ -163,6 +163,29 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 elsa_status elsa_set_linear_variant(elsa_variant v);
 elsa_variant elsa_get_linear_variant(void);
 
+/*
+ * Per-launch kernel timing, off by default.  Between elsa_profile_start and elsa_profile_stop every
+ * kernel the library launches is bracketed by a pair of CUDA events on the stream it is launched
+ * on.  elsa_profile_stop synchronises on the recorded events, writes up to `capacity` records in
+ * launch order and returns how many launches were recorded (which may exceed `capacity`).
+ * Both calls are for single-threaded measurement harnesses.
+ */
+typedef enum {
+    ELSA_KERNEL_COMPRESS = 0,
+    ELSA_KERNEL_UNPACK = 1,
+    ELSA_KERNEL_LINEAR_SIMT = 2,
+    ELSA_KERNEL_LINEAR_TC_DENSE = 3
+} elsa_kernel_id;
+
+typedef struct {
+    int kernel; /* elsa_kernel_id */
+    int layer;  /* index into the table of elsa_vit_linears / _host, -1 for single calls */
+    float ms;   /* device time between the two events */
+} elsa_kernel_time;
+
+elsa_status elsa_profile_start(void);
+int elsa_profile_stop(elsa_kernel_time* records, int capacity);
+
 /* Number of kernels the library has launched from this process so far. */
 unsigned long long elsa_launch_count(void);
 

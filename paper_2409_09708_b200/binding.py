@@ -68,6 +68,15 @@ _launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
 _last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
 
 
+class ElsaKernelTime(ctypes.Structure):
+    _fields_ = [("kernel", _i), ("layer", _i), ("ms", ctypes.c_float)]
+
+
+KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense"}
+_profile_start = _sig("elsa_profile_start", _i, [])
+_profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
+
+
 class ElsaError(RuntimeError):
     def __init__(self, status: int):
         self.status = status
@@ -85,6 +94,17 @@ def elsa_last_error() -> str:
 
 def elsa_launch_count() -> int:
     return int(_launch_count())
+
+
+def elsa_profile_start():
+    _check(_profile_start())
+
+
+def elsa_profile_stop(capacity: int = 1 << 16):
+    """List of (kernel name, layer index, ms) for every launch since elsa_profile_start."""
+    buf = (ElsaKernelTime * capacity)()
+    n = min(int(_profile_stop(buf, capacity)), capacity)
+    return [(KERNEL_NAMES.get(buf[i].kernel, str(buf[i].kernel)), buf[i].layer, float(buf[i].ms)) for i in range(n)]
 
 
 def elsa_set_linear_variant(v: int):

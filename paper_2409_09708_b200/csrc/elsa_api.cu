@@ -5,6 +5,8 @@
 #include <string.h>
 
 #include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "elsa_internal.h"
 
@@ -13,6 +15,40 @@ namespace elsa {
 static thread_local char g_error[512] = "";
 static std::atomic<unsigned long long> g_launches{0};
 static std::atomic<int> g_variant{(int)ELSA_VARIANT_AUTO};
+
+namespace {
+struct ProfileRecord {
+    int kernel, layer;
+    cudaEvent_t start, stop;
+};
+std::atomic<bool> g_profile_on{false};
+std::mutex g_profile_mutex;
+std::vector<ProfileRecord> g_profile;
+thread_local int g_profile_layer = -1;
+}  // namespace
+
+void set_profile_layer(int layer) { g_profile_layer = layer; }
+
+ProfileScope::ProfileScope(int kernel, cudaStream_t stream) : slot_(-1), stream_(stream)
+{
+    if (!g_profile_on.load(std::memory_order_relaxed)) return;
+    ProfileRecord r;
+    r.kernel = kernel;
+    r.layer = g_profile_layer;
+    if (cudaEventCreate(&r.start) != cudaSuccess) { cudaGetLastError(); return; }
+    if (cudaEventCreate(&r.stop) != cudaSuccess) { cudaGetLastError(); cudaEventDestroy(r.start); return; }
+    cudaEventRecord(r.start, stream);
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    g_profile.push_back(r);
+    slot_ = (int)g_profile.size() - 1;
+}
+
+ProfileScope::~ProfileScope()
+{
+    if (slot_ < 0) return;
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    if (slot_ < (int)g_profile.size()) cudaEventRecord(g_profile[slot_].stop, stream_);
+}
 
 elsa_status fail(elsa_status st, const char* fmt, ...)
 {
@@ -222,14 +258,17 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
     if (st != ELSA_OK) return st;
     for (int l = 0; l < n_layers; ++l) {
         const elsa_layer& c = cfg[l];
+        set_profile_layer(l);
         st = run_linear(c.X, c.rows, c.vals, c.N == c.M ? nullptr : c.idx, c.bias, c.out, c.in, c.N, c.M, dtype,
                         c.Y, workspace, dev_status, (cudaStream_t)stream);
         if (st != ELSA_OK) {
+            set_profile_layer(-1);
             char msg[400];
             snprintf(msg, sizeof msg, "%s", elsa_last_error());
             return fail(st, "layer %d: %s", l, msg);
         }
     }
+    set_profile_layer(-1);
     return ELSA_OK;
 }
 
@@ -303,6 +342,7 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
     uint8_t* base = (uint8_t*)device_mem;
     for (int l = 0; l < n_layers; ++l) {
         const elsa_host_layer& c = cfg[l];
+        set_profile_layer(l);
         void* dX = base + plan.x; void* dY = base + plan.y; void* dW = base + plan.w;
         void* dB = c.bias ? base + plan.bias : nullptr;
         void* dV = base + plan.vals; uint32_t* dI = c.N == c.M ? nullptr : (uint32_t*)(base + plan.idx);
@@ -317,6 +357,7 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
         e = cudaMemcpyAsync(c.Y, dY, (size_t)c.rows * c.out * 2, cudaMemcpyDeviceToHost, stream);
         if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "layer %d: device-to-host copy: %s", l, cudaGetErrorString(e));
     }
+    set_profile_layer(-1);
     return ELSA_OK;
 }
 
@@ -329,6 +370,39 @@ elsa_status elsa_set_linear_variant(elsa_variant v)
 }
 
 elsa_variant elsa_get_linear_variant(void) { return (elsa_variant)g_variant.load(std::memory_order_relaxed); }
+
+elsa_status elsa_profile_start(void)
+{
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    for (auto& r : g_profile) { cudaEventDestroy(r.start); cudaEventDestroy(r.stop); }
+    g_profile.clear();
+    g_profile_on.store(true, std::memory_order_relaxed);
+    return ELSA_OK;
+}
+
+int elsa_profile_stop(elsa_kernel_time* records, int capacity)
+{
+    g_profile_on.store(false, std::memory_order_relaxed);
+    std::lock_guard<std::mutex> lock(g_profile_mutex);
+    const int n = (int)g_profile.size();
+    for (int i = 0; i < n; ++i) {
+        ProfileRecord& r = g_profile[i];
+        float ms = -1.f;
+        if (cudaEventSynchronize(r.stop) != cudaSuccess || cudaEventElapsedTime(&ms, r.start, r.stop) != cudaSuccess) {
+            cudaGetLastError();
+            ms = -1.f;
+        }
+        if (records && i < capacity) {
+            records[i].kernel = r.kernel;
+            records[i].layer = r.layer;
+            records[i].ms = ms;
+        }
+        cudaEventDestroy(r.start);
+        cudaEventDestroy(r.stop);
+    }
+    g_profile.clear();
+    return n;
+}
 
 unsigned long long elsa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -184,6 +184,7 @@ elsa_status launch_compress(const uint16_t* W, int out, int in, int N, int M, ui
     const long long total = (long long)out * segs_per_row;
     const unsigned grid = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
     const dim3 block(kWarpsPerBlock * 32);
+    ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
     if (M == 4)
         nm_compress_kernel<4><<<grid, block, 0, stream>>>(W, out, in, N, vals, idx, segs_per_row, wpr);
     else if (M == 8)
@@ -199,6 +200,7 @@ elsa_status launch_unpack(const uint16_t* vals, const uint32_t* idx, int out, in
     const long long total = (long long)out * (in / M);
     const unsigned grid = (unsigned)((total + 255) / 256);
     const int wpr = (int)index_words_per_row(in, N, M);
+    ProfileScope scope(ELSA_KERNEL_UNPACK, stream);
     if (M == 4)
         nm_unpack_kernel<4><<<grid, 256, 0, stream>>>(vals, idx, out, in, N, Wm, wpr);
     else if (M == 8)

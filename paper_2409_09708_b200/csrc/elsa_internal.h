@@ -24,6 +24,18 @@ elsa_status fail(elsa_status st, const char* fmt, ...);
 // Counts one kernel launch and converts the launch's cudaError_t.
 elsa_status launched(const char* what);
 
+// Brackets one kernel launch with CUDA events while profiling is on (see elsa_profile_start).
+class ProfileScope {
+public:
+    ProfileScope(int kernel, cudaStream_t stream);
+    ~ProfileScope();
+private:
+    int slot_;
+    cudaStream_t stream_;
+};
+// Layer index attached to the records of the calling thread (-1 outside a table).
+void set_profile_layer(int layer);
+
 struct DeviceInfo {
     int device;
     int sm_count;

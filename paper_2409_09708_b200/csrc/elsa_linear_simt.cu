@@ -72,6 +72,7 @@ elsa_status launch_linear_simt(const uint16_t* X, int rows, const uint16_t* vals
     const int B = index_bits(M);
     const int wpr = (int)index_words_per_row(in, N, M);
     if (grid.y > 65535u) return fail(ELSA_ERR_SHAPE, "SIMT variant supports at most 524280 rows");
+    ProfileScope scope(ELSA_KERNEL_LINEAR_SIMT, stream);
     if (dtype == ELSA_BF16)
         linear_simt_kernel<true><<<grid, block, 0, stream>>>(X, rows, vals, idx, bias, out, in, N, M,
                                                              B, wpr, Y);

@@ -538,6 +538,7 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
         attr_set[slot][fmt] = true;
     }
     const int grid = p.num_tiles < dev.sm_count ? p.num_tiles : dev.sm_count;
+    ProfileScope scope(ELSA_KERNEL_LINEAR_TC_DENSE, stream);
     kernel<<<grid, kThreads, smem, stream>>>(map_x, map_w, map_y, p);
     return launched("linear_tc_dense");
 }
