@@ -387,7 +387,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="deit_b_stack_b256",
                     choices=["single_layer", "deit_b_block_b64", "deit_b_stack_b256", "swin_b_stack_b128"])
-    ap.add_argument("--oracle-rows", type=int, default=128, help="rows per layer of the CPU-oracle sample")
+    ap.add_argument("--oracle-rows", type=int, default=1024, help="rows per layer of the CPU-oracle sample")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
