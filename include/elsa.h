@@ -159,6 +159,38 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
                                   void* device_mem, size_t device_bytes, uint32_t* dev_status,
                                   void* stream);
 
+/*
+ * elsa_nm_linear for callers that have no device memory to hand over as workspace.  (The paper
+ * has no counterpart: this is a packaging variant of the call above, not a step of the method.)
+ *
+ * Who needs it: code that runs where allocating is forbidden or would stall the GPU -- the enqueue
+ * hook of an inference-runtime plugin, a serving loop whose framework has already reserved all
+ * of the device's memory for its own pool (so cudaMalloc fails), or a latency-critical loop that
+ * cannot afford the device-wide synchronisation an allocation implies.  Such callers own X, the
+ * packed weight, bias and Y, but cannot produce one more scratch buffer.
+ *
+ * What it does: the same kernels as elsa_nm_linear (tensor-core variant), with the weight image
+ * rebuilt in a fixed scratch array that lives inside the library, ELSA_STATIC_SCRATCH_BYTES long.
+ * Every GPU on which the library is loaded holds that array until the process exits.  The call
+ * itself performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *
+ * Limits and rules
+ *   - out * in * 2 must not exceed ELSA_STATIC_SCRATCH_BYTES when N < M (ELSA_ERR_WORKSPACE, with
+ *     a message naming both numbers, otherwise).  The dense level N == M needs no scratch and has
+ *     no size limit.
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call before starting any stream capture.
+ *   - All calls on a device share the one array.  It keeps whatever the previous call left in
+ *     it; that is harmless because every call rewrites the whole image it is about to read, so
+ *     nothing in it needs clearing.  Two calls whose kernels can overlap on the GPU (different
+ *     streams without an ordering between them) race on it: keep them stream-ordered.
+ *   - Arguments otherwise as for elsa_nm_linear; the process-wide variant switch is ignored.
+ */
+#define ELSA_STATIC_SCRATCH_BYTES (8u << 20) /* 8 MiB: up to a 1024 x 4096 16-bit weight */
+elsa_status elsa_nm_linear_static(const void* X, int rows, const void* vals, const uint32_t* idx,
+                                  const void* bias, int out, int in, int N, int M,
+                                  elsa_dtype dtype, void* Y, uint32_t* dev_status, void* stream);
+
 /* Test aid: force the kernel variant used by elsa_nm_linear / elsa_vit_linears (process-wide). */
 elsa_status elsa_set_linear_variant(elsa_variant v);
 elsa_variant elsa_get_linear_variant(void);

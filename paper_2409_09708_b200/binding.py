@@ -58,6 +58,8 @@ _workspace_bytes = _sig("elsa_workspace_bytes", _sz, [_i, _i, _i, _i, _i, _i])
 _compress = _sig("elsa_nm_compress", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 _unpack = _sig("elsa_nm_unpack", _i, [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp])
 _linear = _sig("elsa_nm_linear", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
+_linear_static = _sig("elsa_nm_linear_static", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
+STATIC_SCRATCH_BYTES = 8 << 20
 _vit_ws = _sig("elsa_vit_workspace_bytes", _sz, [ctypes.POINTER(ElsaLayer), _i, _i])
 _vit = _sig("elsa_vit_linears", _i, [ctypes.POINTER(ElsaLayer), _i, _i, _vp, _sz, _vp, _vp])
 _vit_host_bytes = _sig("elsa_vit_host_device_bytes", _sz, [ctypes.POINTER(ElsaHostLayer), _i, _i])
@@ -190,6 +192,16 @@ def elsa_nm_linear(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_
         workspace = alloc_workspace(elsa_workspace_bytes(rows, in_, out, N, M, code), X.device)
     _check(_linear(_ptr(X), rows, _ptr(vals), _ptr(idx), _ptr(bias), out, in_, N, M, code, _ptr(Y),
                    _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
+    return Y
+
+
+def elsa_nm_linear_static(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_: int, N: int, M: int,
+                          Y: torch.Tensor, dev_status=None, stream=None):
+    """elsa_nm_linear without a workspace argument, for callers that cannot allocate: the weight
+    image is rebuilt in the library's built-in scratch array (out * in * 2 <= STATIC_SCRATCH_BYTES).
+    Y must be supplied by the caller; nothing is allocated here or in the library."""
+    _check(_linear_static(_ptr(X), X.shape[0], _ptr(vals), _ptr(idx), _ptr(bias), out, in_, N, M,
+                          dtype_code(X.dtype), _ptr(Y), _ptr(dev_status), _stream(stream)))
     return Y
 
 

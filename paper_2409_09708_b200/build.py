@@ -10,7 +10,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libelsa.so")
-SOURCES = ["elsa_api.cu", "elsa_compress.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu"]
+SOURCES = ["elsa_api.cu", "elsa_compress.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu",
+           "elsa_no_alloc.cu"]
 
 
 def nvcc_path() -> str:
