@@ -33,6 +33,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
+GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair")   # one-CTA and CTA-pair forms of the tcgen05 GEMM
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -258,7 +259,7 @@ def run_ours(args):
         k = per_kernel.setdefault(name, [0, 0.0])
         k[0] += 1
         k[1] += ms
-        if name == "linear_tc_dense" and layer >= 0:
+        if name in GEMM_KERNELS and layer >= 0:
             gemm_ms[layer] += ms / args.steps
         if name == "nm_unpack" and layer >= 0:
             unpack_ms[layer] += ms / args.steps
@@ -271,8 +272,10 @@ def run_ours(args):
     bound = "tensor" if share["tensor"] >= share["hbm"] else "hbm"
     frac = sum_roof / sum_gemm if sum_gemm > 0 else None
     peak = peaks["bf16_tflops"] if bound == "tensor" else peaks["hbm_gbs"]
+    gemm_launches = sum(per_kernel.get(k, [0, 0.0])[0] for k in GEMM_KERNELS)
+    gemm_total_ms = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS)
     roofline = {
-        "kernel": "linear_tc_dense", "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
+        "kernel": max(GEMM_KERNELS, key=lambda k: per_kernel.get(k, [0, 0.0])[1]), "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
         "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": frac, "traffic": None,
         "peaks": peaks_kind,
         "definition": "per layer max(kept FLOPs / tensor peak, algorithmic bytes / HBM peak), summed over the "
@@ -281,8 +284,8 @@ def run_ours(args):
         "kept_tflops": kept_flops / sum_gemm / 1e12 if sum_gemm else None,
         "algorithmic_gbs": sum(algorithmic_bytes(l) for l in layers) / sum_gemm / 1e9 if sum_gemm else None,
         "frac_vs_sustained_peak": sum(r[0] for r in roof_sus) / sum_gemm if sum_gemm else None,
-        "launches": per_kernel.get("linear_tc_dense", [0, 0.0])[0],
-        "avg_launch_ms": per_kernel.get("linear_tc_dense", [0, 1.0])[1] / max(per_kernel.get("linear_tc_dense", [1, 0.0])[0], 1),
+        "launches": gemm_launches,
+        "avg_launch_ms": gemm_total_ms / max(gemm_launches, 1),
         "roofline_time_share": {k: v / sum_roof for k, v in share.items()},
     }
     stack_frac = sum_roof / (ms_per_step * 1e-3)

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libelsa.so")
-SOURCES = ["elsa_api.cu", "elsa_compress.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu",
+SOURCES = ["elsa_api.cu", "elsa_compress.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu", "elsa_linear_tc2.cu",
            "elsa_no_alloc.cu"]
 
 
@@ -29,7 +29,7 @@ def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = sources() + [os.path.join(CSRC, "elsa_internal.h"), os.path.join(ROOT, "include", "elsa.h")]
+    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(ROOT, "include", "elsa.h")]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

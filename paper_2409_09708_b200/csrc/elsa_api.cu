@@ -152,6 +152,16 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
         if (st != ELSA_OK) return st;
         Wd = (const uint16_t*)workspace;
     }
+    bool pair = variant == ELSA_VARIANT_TC_PAIR;
+    if (variant == ELSA_VARIANT_AUTO) {
+        DeviceInfo dev;
+        elsa_status st = device_info(&dev);
+        if (st != ELSA_OK) return st;
+        pair = linear_tc_pair_suits(rows, out, dev.sm_count);
+    }
+    if (pair)
+        return launch_linear_tc_pair((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype,
+                                     (uint16_t*)Y, dev_status, stream);
     return launch_linear_tc_dense((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype,
                                   (uint16_t*)Y, dev_status, stream);
 }
@@ -363,7 +373,7 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
-    if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE)
+    if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR)
         return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;

@@ -58,4 +58,11 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
                                    const uint16_t* bias, int out, int in, elsa_dtype dtype,
                                    uint16_t* Y, uint32_t* dev_status, cudaStream_t stream);
 
+// The same GEMM on CTA pairs (cluster of two, tcgen05 cta_group::2); for large row counts.
+elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias,
+                                  int out, int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status,
+                                  cudaStream_t stream);
+// Whether the problem has enough 256-row tiles to occupy every SM pair.
+bool linear_tc_pair_suits(int rows, int out, int sm_count);
+
 }  // namespace elsa

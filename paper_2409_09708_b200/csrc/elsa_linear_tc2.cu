@@ -1,0 +1,368 @@
+// Tensor-core linear for sm_100a on CTA pairs: Y[rows][out] = X[rows][in] * Wd[out][in]^T + bias.
+//
+// Same contraction as elsa_linear_tc.cu (the product step of Sec. 2, Fig. 2 bottom of the ELSA paper,
+// on the weight image the MMA reads), restructured around the limit that kernel ran into: a
+// single-CTA 128 x 256 x 16 MMA reads 12 KB of operands from shared memory in 128 cycles and TMA
+// writes as much, 192 B/clk against the SM's 128 B/clk.  Here two CTAs on neighbouring SMs form a
+// cluster and share one tile of 256 rows x BN features: each CTA stages its own 128 rows of X and
+// only half of the W rows, and one tcgen05.mma.cta_group::2 (M = 256) issued by the leader CTA
+// drives both tensor cores, so each SM moves 2/3 of the bytes per MMA.
+//
+// Per CTA (320 threads):
+//   warp 0      TMA producer for this CTA's operand halves; completion bytes of both CTAs are
+//               credited to the leader's stage barrier
+//   warp 1      allocates tensor memory (pair-wide); in the leader one lane issues the MMAs and
+//               commits, by multicast, onto both CTAs' stage and accumulator barriers
+//   warps 2-9   epilogue, two warps per TMEM lane quarter (alternating 32-column chunks):
+//               tcgen05.ld (next chunk in flight while the current one is converted), + bias in
+//               fp32, round to 16 bit, swizzled staging, TMA store
+// Two TMEM accumulators let the MMAs of tile i+1 overlap the epilogue of tile i.  Every wait is
+// bounded; on expiry ELSA_ERR_TIMEOUT is recorded and all roles of the CTA leave; a cluster barrier
+// before tensor memory is released keeps either CTA from leaving while its partner may still read
+// its shared memory.
+
+#include "elsa_tc_common.cuh"
+
+namespace elsa {
+namespace {
+
+constexpr int kRowsPerCta = 128;   // rows of X per CTA = TMEM lanes
+constexpr int kPairRows = 256;     // MMA M over the pair
+constexpr int kBlockK = 64;
+constexpr int kUmmaK = 16;
+constexpr int kMaxBlockN = 256;
+constexpr int kNumAccum = 2;
+constexpr int kTmemCols = kNumAccum * kMaxBlockN;
+constexpr int kMaxStages = 8;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kEpiCols = 32;
+constexpr int kATileBytes = kRowsPerCta * kBlockK * 2;
+constexpr int kStagingBytes = 32 * kEpiCols * 2;
+constexpr int kStagingTotal = kEpiWarps * 2 * kStagingBytes;
+constexpr int kBiasBytes = kEpiWarps * kMaxBlockN * 4;
+constexpr int kBarrierBytes = 256;
+
+struct PairParams {
+    int rows, in, out;
+    int bn;            // features per pair tile (MMA N)
+    int tiles_n;
+    int num_tiles;     // pair tiles
+    int num_k_blocks;
+    int stages;
+    uint32_t idesc;
+    const uint16_t* bias;
+    uint32_t* dev_status;
+};
+
+template <bool kBf16>
+__global__ void __launch_bounds__(kThreads, 1)
+linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
+                      const __grid_constant__ CUtensorMap map_y, const PairParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = cluster_ctarank();       // 0 = leader of the pair
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+    const int half_bn = p.bn >> 1;
+    const int b_tile_bytes = half_bn * kBlockK * 2;
+    const int stage_bytes = kATileBytes + b_tile_bytes;
+
+    const uint32_t staging_base = smem_base + (uint32_t)(p.stages * stage_bytes);
+    const uint32_t bias_off = (uint32_t)(p.stages * stage_bytes) + kStagingTotal;
+    const uint32_t bar_base = smem_base + bias_off + kBiasBytes;
+    const uint32_t full_bar = bar_base;                       // used in the leader only
+    const uint32_t empty_bar = bar_base + 8 * kMaxStages;     // per CTA
+    const uint32_t tmem_full_bar = bar_base + 16 * kMaxStages;                 // per CTA
+    const uint32_t tmem_empty_bar = tmem_full_bar + 8 * kNumAccum;             // used in the leader only
+    const uint32_t holder_off = bias_off + kBiasBytes + 16 * kMaxStages + 16 * kNumAccum;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off + 4);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int a = 0; a < kNumAccum; ++a) {
+            mbar_init(tmem_full_bar + 8 * a, 1);
+            mbar_init(tmem_empty_bar + 8 * a, 2 * kEpiWarps);   // every epilogue warp of both CTAs
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_base + holder_off, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    // both CTAs' barriers exist and both allocations are done before either CTA signals the other
+    cluster_arrive();
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+                const int m0 = (tile / p.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
+                const int n0 = (tile % p.tiles_n) * p.bn + (int)cta_rank * half_bn;
+                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                    ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
+                    if (!ok) break;
+                    const uint32_t a_dst = smem_base + (uint32_t)(stage * stage_bytes);
+                    // the leader's stage barrier collects the bytes of both CTAs
+                    if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, (uint32_t)(2 * stage_bytes));
+                    const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
+                    tma_load_2d_pair(a_dst, &map_x, bar, kb * kBlockK, m0);
+                    tma_load_2d_pair(a_dst + kATileBytes, &map_w, bar, kb * kBlockK, n0);
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && cta_rank == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+                ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kMaxBlockN);
+                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                    ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_base + (uint32_t)(stage * stage_bytes);
+                    const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
+                    const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
+#pragma unroll
+                    for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                        umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
+                                      (uint32_t)((kb | k) != 0));
+                    }
+                    umma_commit_pair(empty_bar + 8 * stage, 3);   // frees this stage in both CTAs
+                    if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit_pair(tmem_full_bar + 8 * acc, 3);     // accumulator complete in both CTAs
+                if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ epilogue (warps 2..9)
+        const int q = warp & 3;                 // TMEM lane quarter this warp may read
+        const int ew = warp - 2;                // private staging / bias slot
+        const int half = ew >> 2;               // which of the two warps of the quarter: even or odd chunks
+        const uint32_t stage_buf = staging_base + (uint32_t)(ew * 2 * kStagingBytes);
+        float* bias_s = reinterpret_cast<float*>(smem_gen + bias_off) + ew * kMaxBlockN;
+        const uint32_t empty_remote = mapa_shared(tmem_empty_bar, 0);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        uint32_t chunk_counter = 0;
+        const int chunks = p.bn / kEpiCols;
+        const int my_chunks = (chunks - half + 1) / 2;
+
+        for (int tile = pair; tile < p.num_tiles; tile += num_pairs) {
+            const int m0 = (tile / p.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
+            const int n0 = (tile % p.tiles_n) * p.bn;
+            for (int j = lane; j < p.bn; j += 32) {
+                const int o = n0 + j;
+                bias_s[j] = (p.bias != nullptr && o < p.out) ? bias_to_float<kBf16>(p.bias[o]) : 0.f;
+            }
+            __syncwarp();
+            bool ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * kMaxBlockN);
+            const int row0 = m0 + q * 32;
+
+            // converts, stages and stores one 32 x 32 chunk
+            auto emit = [&](const uint32_t (&r)[32], int c) {
+                uint32_t packed[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) {
+                    const float2 b = *reinterpret_cast<const float2*>(bias_s + c * kEpiCols + 2 * j);
+                    packed[j] = pack2<kBf16>(__uint_as_float(r[2 * j]) + b.x, __uint_as_float(r[2 * j + 1]) + b.y);
+                }
+                const uint32_t buf = stage_buf + (chunk_counter & 1u) * kStagingBytes;
+                if (lane == 0) bulk_wait_group_read<1>();   // the store two chunks ago has drained this buffer
+                __syncwarp();
+                const uint32_t row_addr = buf + (uint32_t)(lane * 64);
+                const uint32_t sw = (uint32_t)((lane >> 1) & 3);   // 64-byte swizzle of the staging rows
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + (((uint32_t)j ^ sw) << 4)),
+                                 "r"(packed[4 * j]), "r"(packed[4 * j + 1]), "r"(packed[4 * j + 2]),
+                                 "r"(packed[4 * j + 3])
+                                 : "memory");
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    const int col0 = n0 + c * kEpiCols;
+                    if (row0 < p.rows && col0 < p.out) tma_store_2d(&map_y, buf, col0, row0);
+                    bulk_commit_group();
+                }
+                ++chunk_counter;
+            };
+            // hands the accumulator back once this warp's last load of it has completed
+            auto release = [&]() {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(empty_remote + 8 * acc);
+            };
+
+            uint32_t ra[32], rb[32];
+            tmem_ld_32x32b_x32(t_row + (uint32_t)(half * kEpiCols), ra);
+            for (int i = 0; i < my_chunks; i += 2) {
+                tmem_wait_ld();
+                if (i + 1 < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * (i + 1)) * kEpiCols), rb);
+                else release();
+                emit(ra, half + 2 * i);
+                if (i + 1 < my_chunks) {
+                    tmem_wait_ld();
+                    if (i + 2 < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * (i + 2)) * kEpiCols), ra);
+                    else release();
+                    emit(rb, half + 2 * (i + 1));
+                }
+            }
+            if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (lane == 0) bulk_wait_group_all();
+        __syncwarp();
+    }
+
+    // ------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait gave up: let copies and MMAs that may still be in flight land first
+        for (int i = 0; i < 200; ++i) __nanosleep(10000);
+    }
+    // neither CTA leaves, or frees tensor memory, while its partner may still use its shared memory
+    cluster_arrive();
+    cluster_wait();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+int pick_pair_block_n(int out)
+{
+    int best = 64, best_waste = 1 << 30;
+    const int cand[4] = {256, 192, 128, 64};
+    for (int i = 0; i < 4; ++i) {
+        const int bn = cand[i];
+        const int waste = (out + bn - 1) / bn * bn - out;
+        if (waste < best_waste) { best = bn; best_waste = waste; }
+    }
+    return best;
+}
+
+}  // namespace
+
+bool linear_tc_pair_suits(int rows, int out, int sm_count)
+{
+    // worth pairing CTAs only when there are enough 256-row tiles to occupy every SM pair
+    const int bn = pick_pair_block_n(out);
+    const long long tiles = (long long)((rows + kPairRows - 1) / kPairRows) * ((out + bn - 1) / bn);
+    return tiles >= sm_count / 2;
+}
+
+elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias, int out,
+                                  int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status, cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+
+    PairParams p;
+    p.rows = rows; p.in = in; p.out = out;
+    p.bn = pick_pair_block_n(out);
+    p.tiles_n = (out + p.bn - 1) / p.bn;
+    p.num_tiles = ((rows + kPairRows - 1) / kPairRows) * p.tiles_n;
+    p.num_k_blocks = (in + kBlockK - 1) / kBlockK;
+    p.bias = bias;
+    p.dev_status = dev_status;
+    const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
+    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+
+    const int stage_bytes = kATileBytes + (p.bn / 2) * kBlockK * 2;
+    const int fixed = kStagingTotal + kBiasBytes + kBarrierBytes + 1024;
+    int stages = (int)((dev.smem_optin - fixed) / stage_bytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
+    p.stages = stages;
+    const size_t smem = (size_t)stages * stage_bytes + fixed;
+
+    CUtensorMap map_x, map_w, map_y;
+    if ((st = make_map_2d(&map_x, X, (uint64_t)in, (uint64_t)rows, kBlockK, kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B,
+                          "X")) != ELSA_OK)
+        return st;
+    if ((st = make_map_2d(&map_w, Wd, (uint64_t)in, (uint64_t)out, kBlockK, (uint32_t)(p.bn / 2),
+                          CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
+        return st;
+    if ((st = make_map_2d(&map_y, Y, (uint64_t)out, (uint64_t)rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B, "Y")) !=
+        ELSA_OK)
+        return st;
+
+    auto kernel = dtype == ELSA_BF16 ? linear_tc_pair_kernel<true> : linear_tc_pair_kernel<false>;
+    static int max_pairs[64][2] = {};
+    const int slot = dev.device & 63;
+
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+
+    if (max_pairs[slot][fmt] == 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
+            cudaSuccess) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        }
+        // how many CTA pairs the device can hold at once: the persistent schedule assumes all run together
+        cfg.gridDim = dim3((unsigned)dev.sm_count);
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
+        }
+        max_pairs[slot][fmt] = n;
+    }
+    const int pairs = p.num_tiles < max_pairs[slot][fmt] ? p.num_tiles : max_pairs[slot][fmt];
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+    ProfileScope scope(ELSA_KERNEL_LINEAR_TC_PAIR, stream);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, map_x, map_w, map_y, p);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ELSA_ERR_CUDA, "launch of linear_tc_pair failed: %s", cudaGetErrorString(e));
+    }
+    return launched("linear_tc_pair");
+}
+
+}  // namespace elsa

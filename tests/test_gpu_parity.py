@@ -116,11 +116,12 @@ def run_linear(lib, X, W, bias, N, M, variant):
         lib.elsa_set_linear_variant(lib.VARIANT_AUTO)
 
 
-VARIANTS = ["simt", "tc_dense"]
+VARIANTS = ["simt", "tc_dense", "tc_pair"]
 
 
 def variant_code(lib, name):
-    return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "auto": lib.VARIANT_AUTO}[name]
+    return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
+            "auto": lib.VARIANT_AUTO}[name]
 
 
 LINEAR_CASES = [
@@ -196,7 +197,7 @@ def test_single_layer_config(lib):
     dtype = synth.torch_dtype(dt)
     X, W, b = synth.layer_tensors(layer, dtype)
     ref = oracle_linear(X, W, b, layer.N, layer.M, dtype)
-    for v in ("auto", "simt", "tc_dense"):
+    for v in ("auto", "simt", "tc_dense", "tc_pair"):
         check_close(run_linear(lib, X, W, b, layer.N, layer.M, variant_code(lib, v)), ref)
 
 
