@@ -46,6 +46,8 @@ nm_compress_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint1
     const int warp = threadIdx.x >> 5;
     const long long seg_id = (long long)blockIdx.x * kWarpsPerBlock + warp;
     const long long total = (long long)out * segs_per_row;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
     if (seg_id >= total) return;  // whole warps leave together; no block-wide barrier is used
 
     const int o = (int)(seg_id / segs_per_row);
@@ -123,6 +125,8 @@ nm_unpack_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__
     constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
     const int groups_per_row = in / M;
     const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
     if (gid >= (long long)out * groups_per_row) return;
     const int o = (int)(gid / groups_per_row);
     const int g = (int)(gid % groups_per_row);
@@ -186,11 +190,11 @@ elsa_status launch_compress(const uint16_t* W, int out, int in, int N, int M, ui
     const dim3 block(kWarpsPerBlock * 32);
     ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
     if (M == 4)
-        nm_compress_kernel<4><<<grid, block, 0, stream>>>(W, out, in, N, vals, idx, segs_per_row, wpr);
+        launch_pdl(nm_compress_kernel<4>, dim3(grid), block, 0, stream, 1, W, out, in, N, vals, idx, segs_per_row, wpr);
     else if (M == 8)
-        nm_compress_kernel<8><<<grid, block, 0, stream>>>(W, out, in, N, vals, idx, segs_per_row, wpr);
+        launch_pdl(nm_compress_kernel<8>, dim3(grid), block, 0, stream, 1, W, out, in, N, vals, idx, segs_per_row, wpr);
     else
-        nm_compress_kernel<16><<<grid, block, 0, stream>>>(W, out, in, N, vals, idx, segs_per_row, wpr);
+        launch_pdl(nm_compress_kernel<16>, dim3(grid), block, 0, stream, 1, W, out, in, N, vals, idx, segs_per_row, wpr);
     return launched("nm_compress");
 }
 
@@ -202,11 +206,11 @@ elsa_status launch_unpack(const uint16_t* vals, const uint32_t* idx, int out, in
     const int wpr = (int)index_words_per_row(in, N, M);
     ProfileScope scope(ELSA_KERNEL_UNPACK, stream);
     if (M == 4)
-        nm_unpack_kernel<4><<<grid, 256, 0, stream>>>(vals, idx, out, in, N, Wm, wpr);
+        launch_pdl(nm_unpack_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, Wm, wpr);
     else if (M == 8)
-        nm_unpack_kernel<8><<<grid, 256, 0, stream>>>(vals, idx, out, in, N, Wm, wpr);
+        launch_pdl(nm_unpack_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, Wm, wpr);
     else
-        nm_unpack_kernel<16><<<grid, 256, 0, stream>>>(vals, idx, out, in, N, Wm, wpr);
+        launch_pdl(nm_unpack_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, Wm, wpr);
     return launched("nm_unpack");
 }
 

@@ -36,6 +36,42 @@ private:
 // Layer index attached to the records of the calling thread (-1 outside a table).
 void set_profile_layer(int layer);
 
+#ifdef __CUDACC__
+// Programmatic dependent launch.  Every kernel of the library is launched with the attribute that
+// lets it start while its predecessor on the stream is still draining; in exchange each kernel calls
+// pdl_wait_for_predecessors() before its first access to global memory (it returns once the
+// predecessor grid has completed and its writes are visible) and pdl_release_successors() as soon as
+// its own successor may begin its set-up.  With a predecessor launched the ordinary way both are no-ops.
+__device__ __forceinline__ void pdl_wait_for_predecessors() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release_successors() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                       unsigned cluster_x, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    int n = 0;
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+    if (cluster_x > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = cluster_x;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = 1;
+        ++n;
+    }
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = (unsigned)n;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args&&>(args)...);
+}
+#endif
+
 struct DeviceInfo {
     int device;
     int sm_count;

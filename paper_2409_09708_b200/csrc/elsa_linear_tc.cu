@@ -95,6 +95,9 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    // set-up above touched no global memory; from here on the predecessor's writes are needed
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
@@ -313,7 +316,7 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
     }
     const int grid = p.num_tiles < dev.sm_count ? p.num_tiles : dev.sm_count;
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_DENSE, stream);
-    kernel<<<grid, kThreads, smem, stream>>>(map_x, map_w, map_y, p);
+    launch_pdl(kernel, dim3(grid), dim3(kThreads), smem, stream, 1, map_x, map_w, map_y, p);
     return launched("linear_tc_dense");
 }
 

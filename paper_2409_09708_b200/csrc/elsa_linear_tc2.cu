@@ -105,6 +105,9 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     cluster_wait();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    // set-up above touched no global memory; from here on the predecessor's writes are needed
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (both CTAs)
@@ -355,9 +358,8 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
         max_pairs[slot][fmt] = n;
     }
     const int pairs = p.num_tiles < max_pairs[slot][fmt] ? p.num_tiles : max_pairs[slot][fmt];
-    cfg.gridDim = dim3((unsigned)(2 * pairs));
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_PAIR, stream);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, map_x, map_w, map_y, p);
+    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, map_x, map_w, map_y, p);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(ELSA_ERR_CUDA, "launch of linear_tc_pair failed: %s", cudaGetErrorString(e));
