@@ -1,0 +1,102 @@
+"""Shape / sparsity sweep of elsa_nm_linear and elsa_nm_compress on one GPU.
+
+    python -m paper_2409_09708_b200.sweep [--out gpurun_out/sweep.json] [--reps 5] [--quick]
+
+rows in {4096, 16384, 65536} x (K, O) in {(768,768), (768,3072), (3072,768), (1024,4096), (4096,1024)}
+x level in {1:4, 2:4, 1:8, 2:8, 4:8, 1:16, 2:16, 4:16, 8:16} x {fp16, bf16}: per point the median
+CUDA-event time of elsa_nm_linear (weight-image rebuild + GEMM) with L2 flushed between repetitions
+(small points are otherwise L2-resident), dense-equivalent and kept TFLOP/s, algorithmic GB/s and
+the fraction of the layer's roofline; per weight shape, level and dtype the time and GB/s (bytes
+read + written) of elsa_nm_compress.  Writes a JSON list and prints a short table.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+
+import torch
+
+from . import binding as lib
+from . import synth
+
+
+def load_peaks():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def timed(fn, reps, flush):
+    out = []
+    for _ in range(reps):
+        flush.fill_(1)                       # 512 MB written: evicts the 126 MB L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        out.append(e0.elapsed_time(e1))
+    return statistics.median(out), min(out)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default="gpurun_out/sweep.json")
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--quick", action="store_true", help="rows = 4096 only")
+    args = ap.parse_args()
+    hbm, tf, kind = load_peaks()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    results = []
+    for dt in ("f16", "bf16"):
+        dtype = synth.torch_dtype(dt)
+        code = lib.dtype_code(dtype)
+        cache = {}
+        for l in synth.sweep():
+            if args.quick and l.rows != synth.SWEEP_ROWS[0]:
+                continue
+            wkey = (l.in_, l.out, l.N, l.M)
+            if wkey not in cache:
+                W = synth.randn((l.out, l.in_), l.seed_w, synth.W_STD, dtype, "cuda")
+                vals, idx = lib.alloc_packed(l.out, l.in_, l.N, l.M, dtype)
+                lib.elsa_nm_compress(W, l.N, l.M, vals=vals, idx=idx)
+                ms, best = timed(lambda: lib.elsa_nm_compress(W, l.N, l.M, vals=vals, idx=idx), args.reps, flush)
+                nbytes = W.numel() * 2 + vals.numel() * 2 + (idx.numel() * 4 if idx is not None else 0)
+                results.append({"op": "compress", "dtype": dt, "in": l.in_, "out": l.out, "level": "%d:%d" % (l.N, l.M),
+                                "ms": ms, "ms_min": best, "bytes": nbytes, "gbs": nbytes / ms / 1e6})
+                cache[wkey] = (vals, idx)
+            vals, idx = cache[wkey]
+            X = synth.randn((l.rows, l.in_), l.seed_x, synth.X_STD, dtype, "cuda")
+            b = synth.randn((l.out,), l.seed_b, synth.B_STD, dtype, "cuda")
+            Y = torch.empty((l.rows, l.out), dtype=dtype, device="cuda")
+            ws = lib.alloc_workspace(lib.elsa_workspace_bytes(l.rows, l.in_, l.out, l.N, l.M, code))
+            run = lambda: lib.elsa_nm_linear(X, vals, idx, b, l.out, l.in_, l.N, l.M, Y=Y, workspace=ws, dev_status=status)
+            run(); run()
+            ms, best = timed(run, args.reps, flush)
+            alg = X.numel() * 2 + Y.numel() * 2 + vals.numel() * 2 + (idx.numel() * 4 if idx is not None else 0) + l.out * 2
+            roof = max(l.kept_flops / (tf * 1e12), alg / (hbm * 1e9)) * 1e3
+            results.append({"op": "linear", "dtype": dt, "rows": l.rows, "in": l.in_, "out": l.out,
+                            "level": "%d:%d" % (l.N, l.M), "ms": ms, "ms_min": best,
+                            "dense_equiv_tflops": l.dense_equiv_flops / ms / 1e9, "kept_tflops": l.kept_flops / ms / 1e9,
+                            "algorithmic_gbs": alg / ms / 1e6, "roofline_ms": roof, "roofline_frac": roof / ms,
+                            "bound": "tensor" if l.kept_flops / (tf * 1e12) >= alg / (hbm * 1e9) else "hbm"})
+            del X, Y
+    assert int(status.item()) == 0
+    os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
+    json.dump({"peaks": {"hbm_gbs": hbm, "bf16_tflops": tf, "kind": kind}, "results": results}, open(args.out, "w"), indent=0)
+    lin = [r for r in results if r["op"] == "linear"]
+    cmp_ = [r for r in results if r["op"] == "compress"]
+    print("linear points: %d, median roofline fraction %.3f, min %.3f, max %.3f" % (
+        len(lin), statistics.median(r["roofline_frac"] for r in lin), min(r["roofline_frac"] for r in lin),
+        max(r["roofline_frac"] for r in lin)))
+    print("compress points: %d, median GB/s %.0f, max %.0f" % (
+        len(cmp_), statistics.median(r["gbs"] for r in cmp_), max(r["gbs"] for r in cmp_)))
+
+
+if __name__ == "__main__":
+    main()

@@ -265,3 +265,28 @@ def test_host_memory_entry_point_matches_device_entry_point(lib):
     torch.cuda.synchronize()
     for h, y in zip(host, dev_out):
         assert torch.equal(h["Y"], y)
+
+
+@pytest.mark.parametrize("dt", ["f16", "bf16"])
+def test_sweep_points_sampled_rows(lib, dt):
+    """Every (rows, K, O, level) point of the shape / sparsity sweep at full size: packed weight
+    compared in full once per weight, 12 sampled rows of Y per point against the oracle."""
+    dtype = synth.torch_dtype(dt)
+    packed = {}
+    for i, l in enumerate(synth.sweep()):
+        key = (l.in_, l.out, l.N, l.M)
+        if key not in packed:
+            W = synth.randn((l.out, l.in_), 7000 + len(packed), synth.W_STD, dtype, "cuda")
+            vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+            ovals, oidx, _ = eo.nm_compress(synth.bits(W), l.N, l.M)
+            assert (synth.bits(vals) == ovals).all() and (idx_bits(idx, oidx) == oidx).all(), key
+            packed[key] = (vals, idx, ovals, oidx)
+        vals, idx, ovals, oidx = packed[key]
+        X = synth.randn((l.rows, l.in_), l.seed_x, synth.X_STD, dtype, "cuda")
+        b = synth.randn((l.out,), l.seed_b, synth.B_STD, dtype, "cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        Y = lib.elsa_nm_linear(X, vals, idx, b, l.out, l.in_, l.N, l.M, dev_status=status)
+        pick = torch.from_numpy(synth.sample_rows(l.rows, 12, 900 + i, tile=256)).cuda()
+        ref = eo.nm_linear_f64(synth.bits(X[pick]), ovals, oidx, synth.bits(b), l.out, l.in_, l.N, l.M, ocode(dtype))
+        assert int(status.item()) == 0
+        check_close(Y[pick], ref)
