@@ -144,6 +144,12 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
     if (variant == ELSA_VARIANT_SIMT)
         return launch_linear_simt((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                   in, N, M, dtype, (uint16_t*)Y, stream);
+    if (variant == ELSA_VARIANT_TC_SPARSE) {
+        if (N == M || !linear_tc_sparse_suits(in, N))
+            return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
+        return launch_linear_tc_sparse((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
+                                       in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
+    }
     // Tensor-core path.  The dense level multiplies the stored values as they are; every other
     // level first rebuilds the weight image the MMA reads, in the caller's scratch.
     const uint16_t* Wd = (const uint16_t*)vals;
@@ -192,7 +198,12 @@ size_t elsa_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype 
     if (out <= 0 || in <= 0 || index_bits(M) < 0 || N < 1 || N > M || in % M != 0) return 0;
     if (dtype != ELSA_F16 && dtype != ELSA_BF16) return 0;
     if (N == M) return 0;                              // the dense level needs no weight image
-    return round_up((size_t)out * (size_t)in * 2, 256);  // dense image of the masked weight
+    size_t need = round_up((size_t)out * (size_t)in * 2, 256);  // dense image of the masked weight
+    if (linear_tc_sparse_suits(in, N)) {                          // or its 2-of-4 image + metadata
+        const size_t sp = round_up(linear_tc_sparse_workspace(out, in), 256);
+        if (sp > need) need = sp;
+    }
+    return need;
 }
 
 elsa_status elsa_nm_compress(const void* W, int out, int in, int N, int M, elsa_dtype dtype, void* vals,
@@ -373,7 +384,8 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
-    if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR)
+    if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR &&
+        v != ELSA_VARIANT_TC_SPARSE)
         return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;

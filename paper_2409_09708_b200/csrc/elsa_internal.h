@@ -98,6 +98,13 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
 elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias,
                                   int out, int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status,
                                   cudaStream_t stream);
+// Levels with N <= 2 on the hardware 2:4 sparse MMA: re-encodes the packed weight into `workspace`
+// (2-of-4 values + metadata), then runs the sparse GEMM.
+elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                    const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
+                                    uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
+bool linear_tc_sparse_suits(int in, int N);
+size_t linear_tc_sparse_workspace(int out, int in);
 // Whether the problem has enough 256-row tiles to occupy every SM pair.
 bool linear_tc_pair_suits(int rows, int out, int sm_count);
 

@@ -270,6 +270,66 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar, uint16_t cta_mask
                  : "memory");
 }
 
+// ------------------------------------------------------------------ 2:4-sparse MMA forms
+
+// D[tmem] (+)= A[smem, 2:4-compressed along K] * B[smem]^T.  `tmem_e` is the tensor-memory column
+// holding the metadata of this K step; the column's parity goes into the instruction descriptor's
+// sparsity selector and the even column address into the operand.
+__device__ __forceinline__ void umma_sp_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t tmem_e,
+                                            uint32_t idesc, uint32_t accumulate)
+{
+    const uint32_t idesc_sel = idesc | (tmem_e & 1u);
+    const uint32_t e_addr = tmem_e & ~1u;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "tcgen05.mma.sp.cta_group::1.kind::f16 [%0], %1, %2, [%3], %4, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate)
+        : "memory");
+}
+
+// Copies 128 rows x 16 bytes from shared memory (descriptor) into 4 consecutive columns of the 128
+// lanes of tensor memory.  Ordered with the MMAs issued by the same thread.
+__device__ __forceinline__ void tmem_cp_128x128b(uint32_t taddr, uint64_t s_desc)
+{
+    asm volatile("tcgen05.cp.cta_group::1.128x128b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
+}
+
+// Plain (untiled) bulk copy global -> shared, completion counted on an mbarrier.  Addresses and size
+// are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// K-major tile stored as rows of 64 bytes with the 64-byte swizzle: 8-row groups are 512 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_k_major_sw64(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;   // layout: 64-byte swizzle
+    return d;
+}
+
+// Unswizzled K-major block of 16-byte rows: 8 rows are 128 contiguous bytes, 8-row groups follow
+// each other.
+__device__ __forceinline__ uint64_t smem_desc_rows16_no_swizzle(uint32_t addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)(128 >> 4) << 16;   // leading byte offset (one 16-byte column only: unused)
+    d |= (uint64_t)(128 >> 4) << 32;   // stride between 8-row groups
+    d |= (uint64_t)1 << 46;
+    return d;
+}
+
 // ------------------------------------------------------------------ host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -121,7 +121,7 @@ VARIANTS = ["simt", "tc_dense", "tc_pair"]
 
 def variant_code(lib, name):
     return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
-            "auto": lib.VARIANT_AUTO}[name]
+            "tc_sparse": lib.VARIANT_TC_SPARSE, "auto": lib.VARIANT_AUTO}[name]
 
 
 LINEAR_CASES = [
@@ -176,6 +176,45 @@ def test_integer_inputs_are_exact(lib, variant):
         ref = oracle_linear(X, W, None, N, M, torch.bfloat16)
         # the exact integer result, rounded once to bf16 (integers up to 256 are unchanged)
         assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
+
+
+SPARSE_CASES = [
+    # rows, in, out, N, M: every level the 2:4 sparse MMA can carry, ragged rows and features
+    (197, 768, 768, 2, 8), (500, 128, 384, 1, 4), (225, 64, 128, 2, 4), (1000, 3072, 768, 1, 8),
+    (449, 512, 200, 2, 16), (300, 1024, 136, 1, 16), (7, 48, 8, 2, 4), (2300, 768, 2304, 2, 8),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("case", SPARSE_CASES)
+def test_sparse_mma_variant_matches_oracle(lib, case, dtype):
+    rows, in_, out, N, M = case
+    X = synth.randn((rows, in_), 19 * rows + in_, synth.X_STD, dtype)
+    W = synth.randn((out, in_), 23 * out + in_, synth.W_STD, dtype)
+    bias = synth.randn((out,), 29 * out, synth.B_STD, dtype)
+    Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
+    check_close(Y, oracle_linear(X, W, bias, N, M, dtype))
+
+
+def test_sparse_mma_variant_exact_cases_and_refusals(lib):
+    dtype = torch.float16
+    W = synth.randn((320, 256), 5, synth.W_STD, dtype)
+    bias = synth.randn((320,), 6, synth.B_STD, dtype)
+    X = torch.eye(256, dtype=dtype)
+    for N, M in [(2, 8), (1, 4), (2, 4), (1, 16)]:
+        Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
+        expect = torch.from_numpy(oracle_linear(X, W, bias, N, M, dtype)).to(dtype)
+        assert torch.equal(Y.cpu(), expect), (N, M)
+    rng = np.random.default_rng(5)
+    Xi = torch.from_numpy(rng.integers(-4, 5, (300, 192))).to(torch.bfloat16)
+    Wi = torch.from_numpy(rng.integers(-8, 9, (96, 192))).to(torch.bfloat16)
+    for N, M in [(2, 4), (1, 8), (2, 16)]:
+        Y = run_linear(lib, Xi, Wi, None, N, M, lib.VARIANT_TC_SPARSE)
+        ref = oracle_linear(Xi, Wi, None, N, M, torch.bfloat16)
+        assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
+    for N, M in [(4, 8), (3, 4), (8, 8)]:                      # more than 2 per chunk possible: refused
+        with pytest.raises(lib.ElsaError):
+            run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
 
 
 def test_no_bias_and_zero_rows_of_padding(lib):
