@@ -70,7 +70,8 @@ typedef enum {
     ELSA_VARIANT_SIMT = 1,    /* CUDA-core kernel reading the packed form directly (slow; checks) */
     ELSA_VARIANT_TC_DENSE = 2, /* expand to a dense tile image, tcgen05 dense MMA, one CTA per tile */
     ELSA_VARIANT_TC_PAIR = 3,  /* same, CTA pairs sharing a 256-row tile (tcgen05 cta_group::2) */
-    ELSA_VARIANT_TC_SPARSE = 4 /* N <= 2 only: re-encode as 2-of-4 + metadata, tcgen05 sparse MMA */
+    ELSA_VARIANT_TC_SPARSE = 4, /* N <= 2 only: re-encode as 2-of-4 + metadata, tcgen05 sparse MMA */
+    ELSA_VARIANT_TC_SPARSE_PAIR = 5 /* the same on CTA pairs (256 features x 224 rows per pair) */
 } elsa_variant;
 
 /* Sizes of the packed form (host-only arithmetic; 0 on invalid arguments). */
@@ -211,7 +212,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_DENSE = 3,
     ELSA_KERNEL_LINEAR_TC_PAIR = 4,
     ELSA_KERNEL_NM_TO_SP24 = 5,
-    ELSA_KERNEL_LINEAR_TC_SP24 = 6
+    ELSA_KERNEL_LINEAR_TC_SP24 = 6,
+    ELSA_KERNEL_LINEAR_TC_SP24_PAIR = 7
 } elsa_kernel_id;
 
 typedef struct {

@@ -144,9 +144,13 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
     if (variant == ELSA_VARIANT_SIMT)
         return launch_linear_simt((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                   in, N, M, dtype, (uint16_t*)Y, stream);
-    if (variant == ELSA_VARIANT_TC_SPARSE) {
+    if (variant == ELSA_VARIANT_TC_SPARSE || variant == ELSA_VARIANT_TC_SPARSE_PAIR) {
         if (N == M || !linear_tc_sparse_suits(in, N))
             return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
+        if (variant == ELSA_VARIANT_TC_SPARSE_PAIR)
+            return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx,
+                                                (const uint16_t*)bias, out, in, N, M, dtype, (uint16_t*)Y, workspace,
+                                                dev_status, stream);
         return launch_linear_tc_sparse((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                        in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
     }
@@ -385,7 +389,7 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
     if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR &&
-        v != ELSA_VARIANT_TC_SPARSE)
+        v != ELSA_VARIANT_TC_SPARSE && v != ELSA_VARIANT_TC_SPARSE_PAIR)
         return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;

@@ -103,6 +103,14 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                     const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
                                     uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
+// packed weight -> 2-of-4 image [out][in/2] + metadata blocks of 2 KB per (128 features, block_k of K),
+// block_k = 64 or 128.
+elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
+                              uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
+// The same on CTA pairs (256 features x 224 rows per pair, K blocks of 128).
+elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                         const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
+                                         uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
 size_t linear_tc_sparse_workspace(int out, int in);
 // Whether the problem has enough 256-row tiles to occupy every SM pair.

@@ -58,11 +58,11 @@ template <int M>
 __global__ void __launch_bounds__(256)
 nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx, int out, int in, int N,
                   int words_per_row, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int out_tiles,
-                  int k_blocks)
+                  int k_blocks, int steps_per_block)
 {
     constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
     constexpr int G = 16 / M;                         // groups per 16-k segment
-    const int segs = k_blocks * 4;                    // 16-k segments per (padded) row
+    const int segs = k_blocks * steps_per_block * 2;  // 16-k segments per (padded) row
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
@@ -126,14 +126,15 @@ nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict_
         r.w = sel[6] | ((uint32_t)sel[7] << 16);
         *reinterpret_cast<uint4*>(a_img + (size_t)o * (in / 2) + k0 / 2) = r;
     }
-    // metadata half-word: block (feature tile, k block) -> lane -> 4 words (K step 0, K step 1, unused x2)
+    // metadata half-word: block (feature tile, k block) -> lane -> 4 words, one per K step of 32; a
+    // block covers steps_per_block (2 or 4) steps and leaves the other words zero
     const int ftile = o / kFeatTile, m = o % kFeatTile;
-    const int kb = seg / 4, step = (seg / 2) % 2, k1 = seg % 2;
+    const int kb = seg / (2 * steps_per_block), step = (seg / 2) % steps_per_block, k1 = seg % 2;
     const int lane = (m % 8) + 8 * k1 + 16 * (m / 16);
     const int hi = (m / 8) % 2;
     const size_t word = (((size_t)ftile * k_blocks + kb) * 128 + lane) * 4 + step;
     meta16[2 * word + hi] = (uint16_t)nibbles;
-    meta16[2 * (word + 2) + hi] = 0;                  // the lane's two unused words
+    if (steps_per_block == 2) meta16[2 * (word + 2) + hi] = 0;
 }
 
 // ------------------------------------------------------------------ GEMM
@@ -328,6 +329,28 @@ linear_tc_sp24_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 
 }  // namespace
 
+elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
+                              uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
+{
+    const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
+    const int k_blocks = (in + block_k - 1) / block_k;
+    const int steps = block_k / kSpUmmaK;
+    const long long threads = (long long)tiles_f * kFeatTile * k_blocks * steps * 2;
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+    const int wpr = (int)index_words_per_row(in, N, M);
+    ProfileScope scope(ELSA_KERNEL_NM_TO_SP24, stream);
+    if (M == 4)
+        launch_pdl(nm_to_sp24_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
+                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+    else if (M == 8)
+        launch_pdl(nm_to_sp24_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
+                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+    else
+        launch_pdl(nm_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
+                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+    return launched("nm_to_sp24");
+}
+
 bool linear_tc_sparse_suits(int in, int N)
 {
     // the 2:4 image needs at most 2 kept weights per aligned 4-chunk (guaranteed for N <= 2) and
@@ -357,24 +380,7 @@ elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t*
     uint16_t* a_img = (uint16_t*)workspace;
     uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
 
-    {   // re-encode the packed weight
-        const long long threads = (long long)tiles_f * kFeatTile * k_blocks * 4;
-        const unsigned grid = (unsigned)((threads + 255) / 256);
-        const int wpr = (int)index_words_per_row(in, N, M);
-        ProfileScope scope(ELSA_KERNEL_NM_TO_SP24, stream);
-        cudaError_t e;
-        if (M == 4)
-            e = launch_pdl(nm_to_sp24_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                           (uint16_t*)meta, tiles_f, k_blocks);
-        else if (M == 8)
-            e = launch_pdl(nm_to_sp24_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                           (uint16_t*)meta, tiles_f, k_blocks);
-        else
-            e = launch_pdl(nm_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                           (uint16_t*)meta, tiles_f, k_blocks);
-        (void)e;
-        if ((st = launched("nm_to_sp24")) != ELSA_OK) return st;
-    }
+    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, a_img, meta, stream)) != ELSA_OK) return st;
 
     SpParams p;
     p.rows = rows; p.in = in; p.out = out;

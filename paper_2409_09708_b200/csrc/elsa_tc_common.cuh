@@ -330,6 +330,37 @@ __device__ __forceinline__ uint64_t smem_desc_rows16_no_swizzle(uint32_t addr)
     return d;
 }
 
+// CTA-pair forms of the two above: M = 256 (128 compressed rows of A and their metadata from each
+// CTA), B rows split between the CTAs; the copy runs in both CTAs, each from its own shared memory
+// into its own tensor memory.  Issued by the leader CTA.
+__device__ __forceinline__ void umma_sp_f16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t tmem_e,
+                                                 uint32_t idesc, uint32_t accumulate)
+{
+    const uint32_t idesc_sel = idesc | (tmem_e & 1u);
+    const uint32_t e_addr = tmem_e & ~1u;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], %1, %2, [%3], %4, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_cp_128x128b_pair(uint32_t taddr, uint64_t s_desc)
+{
+    asm volatile("tcgen05.cp.cta_group::2.128x128b [%0], %1;" ::"r"(taddr), "l"(s_desc) : "memory");
+}
+
+// Plain bulk copy whose completion bytes go to an mbarrier that may live in the other CTA of the pair.
+__device__ __forceinline__ void bulk_load_1d_pair(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar_cluster_addr)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar_cluster_addr)
+                 : "memory");
+}
+
 // ------------------------------------------------------------------ host side
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

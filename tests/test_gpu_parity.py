@@ -121,7 +121,8 @@ VARIANTS = ["simt", "tc_dense", "tc_pair"]
 
 def variant_code(lib, name):
     return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
-            "tc_sparse": lib.VARIANT_TC_SPARSE, "auto": lib.VARIANT_AUTO}[name]
+            "tc_sparse": lib.VARIANT_TC_SPARSE, "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR,
+            "auto": lib.VARIANT_AUTO}[name]
 
 
 LINEAR_CASES = [
@@ -185,36 +186,42 @@ SPARSE_CASES = [
 ]
 
 
+SPARSE_VARIANTS = ["tc_sparse", "tc_sparse_pair"]
+
+
+@pytest.mark.parametrize("variant", SPARSE_VARIANTS)
 @pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
 @pytest.mark.parametrize("case", SPARSE_CASES)
-def test_sparse_mma_variant_matches_oracle(lib, case, dtype):
+def test_sparse_mma_variant_matches_oracle(lib, case, dtype, variant):
     rows, in_, out, N, M = case
     X = synth.randn((rows, in_), 19 * rows + in_, synth.X_STD, dtype)
     W = synth.randn((out, in_), 23 * out + in_, synth.W_STD, dtype)
     bias = synth.randn((out,), 29 * out, synth.B_STD, dtype)
-    Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
+    Y = run_linear(lib, X, W, bias, N, M, variant_code(lib, variant))
     check_close(Y, oracle_linear(X, W, bias, N, M, dtype))
 
 
-def test_sparse_mma_variant_exact_cases_and_refusals(lib):
+@pytest.mark.parametrize("variant", SPARSE_VARIANTS)
+def test_sparse_mma_variant_exact_cases_and_refusals(lib, variant):
+    code = variant_code(lib, variant)
     dtype = torch.float16
     W = synth.randn((320, 256), 5, synth.W_STD, dtype)
     bias = synth.randn((320,), 6, synth.B_STD, dtype)
     X = torch.eye(256, dtype=dtype)
     for N, M in [(2, 8), (1, 4), (2, 4), (1, 16)]:
-        Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
+        Y = run_linear(lib, X, W, bias, N, M, code)
         expect = torch.from_numpy(oracle_linear(X, W, bias, N, M, dtype)).to(dtype)
         assert torch.equal(Y.cpu(), expect), (N, M)
     rng = np.random.default_rng(5)
     Xi = torch.from_numpy(rng.integers(-4, 5, (300, 192))).to(torch.bfloat16)
     Wi = torch.from_numpy(rng.integers(-8, 9, (96, 192))).to(torch.bfloat16)
     for N, M in [(2, 4), (1, 8), (2, 16)]:
-        Y = run_linear(lib, Xi, Wi, None, N, M, lib.VARIANT_TC_SPARSE)
+        Y = run_linear(lib, Xi, Wi, None, N, M, code)
         ref = oracle_linear(Xi, Wi, None, N, M, torch.bfloat16)
         assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
     for N, M in [(4, 8), (3, 4), (8, 8)]:                      # more than 2 per chunk possible: refused
         with pytest.raises(lib.ElsaError):
-            run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE)
+            run_linear(lib, X, W, bias, N, M, code)
 
 
 def test_no_bias_and_zero_rows_of_padding(lib):
