@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
-GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair")   # one-CTA and CTA-pair forms of the tcgen05 GEMM
+GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair")   # forms of the tcgen05 GEMM
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -261,7 +261,7 @@ def run_ours(args):
         k[1] += ms
         if name in GEMM_KERNELS and layer >= 0:
             gemm_ms[layer] += ms / args.steps
-        if name == "nm_unpack" and layer >= 0:
+        if name in ("nm_unpack", "nm_to_sp24") and layer >= 0:
             unpack_ms[layer] += ms / args.steps
     kernel_total = sum(v[1] for v in per_kernel.values()) or 1.0
     roof = [roofline_seconds(l, peaks) for l in layers]

@@ -144,6 +144,19 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
     if (variant == ELSA_VARIANT_SIMT)
         return launch_linear_simt((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                   in, N, M, dtype, (uint16_t*)Y, stream);
+    if (variant == ELSA_VARIANT_AUTO && N != M && linear_tc_sparse_suits(in, N) && in >= 768) {
+        // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K
+        // is long enough for the mainloop to outweigh its heavier epilogue (K >= 768) and there are enough
+        // 256 x 224 tiles to fill the CTA pairs; shorter K ties or loses and stays on the dense-rate path.
+        DeviceInfo dev;
+        elsa_status st = device_info(&dev);
+        if (st != ELSA_OK) return st;
+        const long long tiles = (long long)((rows + 223) / 224) * ((out + 255) / 256);
+        if (tiles >= dev.sm_count / 4)
+            return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx,
+                                                (const uint16_t*)bias, out, in, N, M, dtype, (uint16_t*)Y, workspace,
+                                                dev_status, stream);
+    }
     if (variant == ELSA_VARIANT_TC_SPARSE || variant == ELSA_VARIANT_TC_SPARSE_PAIR) {
         if (N == M || !linear_tc_sparse_suits(in, N))
             return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
