@@ -125,14 +125,19 @@ typedef struct {
     int rows, in, out, N, M;
 } elsa_layer;
 
-/* Largest elsa_workspace_bytes over the table (host-only arithmetic). */
+/* Scratch for the table with one region per layer: the sum of elsa_workspace_bytes, each rounded up
+ * to 256 bytes (host-only arithmetic). */
 size_t elsa_vit_workspace_bytes(const elsa_layer* cfg, int n_layers, elsa_dtype dtype);
 
 /*
- * Runs every layer of the table, in order, on one stream, each under its own level N:M
- * (Sec. 3, layer-wise configuration alpha).  `cfg` is a HOST array.  The table is validated as a
- * whole before the first launch; on an error nothing has been enqueued and elsa_last_error()
- * names the layer.
+ * Runs every layer of the table on one stream, each under its own level N:M (Sec. 3, layer-wise
+ * configuration alpha).  `cfg` is a HOST array.  The table is validated as a whole before the
+ * first launch; on an error nothing has been enqueued and elsa_last_error() names the layer.
+ * The layers of a table must be independent of one another (no layer's X is another layer's Y):
+ * given elsa_vit_workspace_bytes(...) of scratch the library builds all weight images first and
+ * lets the layers of each kernel family share persistent launches, so their tiles interleave.
+ * With less scratch -- at least the largest single elsa_workspace_bytes of the table -- the layers
+ * run one after the other through the same region.  Dependent layers go through elsa_nm_linear.
  */
 elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dtype,
                              void* workspace, size_t workspace_bytes, uint32_t* dev_status,
@@ -193,6 +198,11 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 elsa_status elsa_nm_linear_static(const void* X, int rows, const void* vals, const uint32_t* idx,
                                   const void* bias, int out, int in, int N, int M,
                                   elsa_dtype dtype, void* Y, uint32_t* dev_status, void* stream);
+
+/* Measurement aid: turn the sharing of launches inside elsa_vit_linears off (0) or on (non-zero,
+ * the default), process-wide; with it off every layer gets its own launches and its own record
+ * in the per-launch timing below. */
+void elsa_set_grouping(int on);
 
 /* Test aid: force the kernel variant used by elsa_nm_linear / elsa_vit_linears (process-wide). */
 elsa_status elsa_set_linear_variant(elsa_variant v);

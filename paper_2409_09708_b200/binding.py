@@ -65,6 +65,7 @@ _vit = _sig("elsa_vit_linears", _i, [ctypes.POINTER(ElsaLayer), _i, _i, _vp, _sz
 _vit_host_bytes = _sig("elsa_vit_host_device_bytes", _sz, [ctypes.POINTER(ElsaHostLayer), _i, _i])
 _vit_host = _sig("elsa_vit_linears_host", _i, [ctypes.POINTER(ElsaHostLayer), _i, _i, _vp, _sz, _vp, _vp])
 _set_variant = _sig("elsa_set_linear_variant", _i, [_i])
+_set_grouping = _sig("elsa_set_grouping", None, [_i])
 _get_variant = _sig("elsa_get_linear_variant", _i, [])
 _launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
 _last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
@@ -111,6 +112,10 @@ def elsa_profile_stop(capacity: int = 1 << 16):
 
 def elsa_set_linear_variant(v: int):
     _check(_set_variant(v))
+
+
+def elsa_set_grouping(on: bool):
+    _set_grouping(1 if on else 0)
 
 
 def elsa_get_linear_variant() -> int:

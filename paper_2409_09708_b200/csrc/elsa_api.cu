@@ -15,6 +15,7 @@ namespace elsa {
 static thread_local char g_error[512] = "";
 static std::atomic<unsigned long long> g_launches{0};
 static std::atomic<int> g_variant{(int)ELSA_VARIANT_AUTO};
+static std::atomic<bool> g_grouping{true};
 
 namespace {
 struct ProfileRecord {
@@ -135,54 +136,63 @@ elsa_status check_linear(const void* X, int rows, const void* vals, const uint32
     return ELSA_OK;
 }
 
+enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR };
+
+// Which kernel a layer runs on.  AUTO is the product rule; a forced variant is honoured where it applies.
+elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, LinearKind* kind)
+{
+    const int variant = g_variant.load(std::memory_order_relaxed);
+    const bool sparse_ok = N != M && linear_tc_sparse_suits(in, N);
+    switch (variant) {
+    case ELSA_VARIANT_SIMT: *kind = KIND_SIMT; return ELSA_OK;
+    case ELSA_VARIANT_TC_DENSE: *kind = KIND_DENSE_ONE; return ELSA_OK;
+    case ELSA_VARIANT_TC_PAIR: *kind = KIND_DENSE_PAIR; return ELSA_OK;
+    case ELSA_VARIANT_TC_SPARSE:
+    case ELSA_VARIANT_TC_SPARSE_PAIR:
+        if (!sparse_ok)
+            return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
+        *kind = variant == ELSA_VARIANT_TC_SPARSE ? KIND_SPARSE_ONE : KIND_SPARSE_PAIR;
+        return ELSA_OK;
+    default: break;
+    }
+    // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K is
+    // long enough for the mainloop to outweigh its heavier epilogue (K >= 768) and there are enough 256 x 224
+    // tiles to fill the CTA pairs; shorter K ties or loses and stays on the dense-rate path.
+    if (sparse_ok && in >= 768 && (long long)((rows + 223) / 224) * ((out + 255) / 256) >= sm_count / 4)
+        *kind = KIND_SPARSE_PAIR;
+    else
+        *kind = linear_tc_pair_suits(rows, out, sm_count) ? KIND_DENSE_PAIR : KIND_DENSE_ONE;
+    return ELSA_OK;
+}
+
 // After validation: enqueue one layer.
 elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t* idx, const void* bias, int out,
                        int in, int N, int M, elsa_dtype dtype, void* Y, void* workspace, uint32_t* dev_status,
                        cudaStream_t stream)
 {
-    const int variant = g_variant.load(std::memory_order_relaxed);
-    if (variant == ELSA_VARIANT_SIMT)
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    LinearKind kind;
+    if ((st = pick_kind(rows, out, in, N, M, dev.sm_count, &kind)) != ELSA_OK) return st;
+    if (kind == KIND_SIMT)
         return launch_linear_simt((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                   in, N, M, dtype, (uint16_t*)Y, stream);
-    if (variant == ELSA_VARIANT_AUTO && N != M && linear_tc_sparse_suits(in, N) && in >= 768) {
-        // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K
-        // is long enough for the mainloop to outweigh its heavier epilogue (K >= 768) and there are enough
-        // 256 x 224 tiles to fill the CTA pairs; shorter K ties or loses and stays on the dense-rate path.
-        DeviceInfo dev;
-        elsa_status st = device_info(&dev);
-        if (st != ELSA_OK) return st;
-        const long long tiles = (long long)((rows + 223) / 224) * ((out + 255) / 256);
-        if (tiles >= dev.sm_count / 4)
-            return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx,
-                                                (const uint16_t*)bias, out, in, N, M, dtype, (uint16_t*)Y, workspace,
-                                                dev_status, stream);
-    }
-    if (variant == ELSA_VARIANT_TC_SPARSE || variant == ELSA_VARIANT_TC_SPARSE_PAIR) {
-        if (N == M || !linear_tc_sparse_suits(in, N))
-            return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
-        if (variant == ELSA_VARIANT_TC_SPARSE_PAIR)
-            return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx,
-                                                (const uint16_t*)bias, out, in, N, M, dtype, (uint16_t*)Y, workspace,
-                                                dev_status, stream);
+    if (kind == KIND_SPARSE_ONE)
         return launch_linear_tc_sparse((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias, out,
                                        in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
-    }
-    // Tensor-core path.  The dense level multiplies the stored values as they are; every other
-    // level first rebuilds the weight image the MMA reads, in the caller's scratch.
+    if (kind == KIND_SPARSE_PAIR)
+        return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias,
+                                            out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
+    // Dense-rate path.  The dense level multiplies the stored values as they are; every other level first
+    // rebuilds the weight image the MMA reads, in the caller's scratch.
     const uint16_t* Wd = (const uint16_t*)vals;
     if (N != M) {
-        elsa_status st = launch_unpack((const uint16_t*)vals, idx, out, in, N, M, (uint16_t*)workspace, stream);
-        if (st != ELSA_OK) return st;
+        if ((st = launch_unpack((const uint16_t*)vals, idx, out, in, N, M, (uint16_t*)workspace, stream)) != ELSA_OK)
+            return st;
         Wd = (const uint16_t*)workspace;
     }
-    bool pair = variant == ELSA_VARIANT_TC_PAIR;
-    if (variant == ELSA_VARIANT_AUTO) {
-        DeviceInfo dev;
-        elsa_status st = device_info(&dev);
-        if (st != ELSA_OK) return st;
-        pair = linear_tc_pair_suits(rows, out, dev.sm_count);
-    }
-    if (pair)
+    if (kind == KIND_DENSE_PAIR)
         return launch_linear_tc_pair((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype,
                                      (uint16_t*)Y, dev_status, stream);
     return launch_linear_tc_dense((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype,
@@ -267,17 +277,16 @@ elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint
 
 size_t elsa_vit_workspace_bytes(const elsa_layer* cfg, int n_layers, elsa_dtype dtype)
 {
+    // one region per layer, so that every weight image can be built before the grouped launches
     size_t need = 0;
     if (!cfg) return 0;
-    for (int l = 0; l < n_layers; ++l) {
-        const size_t b = elsa_workspace_bytes(cfg[l].rows, cfg[l].in, cfg[l].out, cfg[l].N, cfg[l].M, dtype);
-        if (b > need) need = b;
-    }
+    for (int l = 0; l < n_layers; ++l)
+        need += round_up(elsa_workspace_bytes(cfg[l].rows, cfg[l].in, cfg[l].out, cfg[l].N, cfg[l].M, dtype), 256);
     return need;
 }
 
 elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dtype, void* workspace,
-                             size_t workspace_bytes, uint32_t* dev_status, void* stream)
+                             size_t workspace_bytes, uint32_t* dev_status, void* stream_)
 {
     if (!cfg) return fail(ELSA_ERR_NULL, "cfg must not be NULL");
     if (n_layers <= 0) return fail(ELSA_ERR_SHAPE, "non-positive n_layers=%d", n_layers);
@@ -294,17 +303,100 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    auto layer_fail = [](elsa_status code, int l) {
+        set_profile_layer(-1);
+        char msg[400];
+        snprintf(msg, sizeof msg, "%s", elsa_last_error());
+        return fail(code, "layer %d: %s", l, msg);
+    };
+
+    // With one scratch region per layer (elsa_vit_workspace_bytes) all weight images are built first and the
+    // layers of each kernel family share persistent launches: the layers of a table do not depend on one
+    // another, so their tiles may interleave.  With less scratch (at least the largest layer's, which
+    // validation has checked) the layers run one after the other through the same region.
+    const bool grouped = g_grouping.load(std::memory_order_relaxed) &&
+                         g_variant.load(std::memory_order_relaxed) == ELSA_VARIANT_AUTO &&
+                         workspace_bytes >= elsa_vit_workspace_bytes(cfg, n_layers, dtype);
+    if (!grouped) {
+        for (int l = 0; l < n_layers; ++l) {
+            const elsa_layer& c = cfg[l];
+            set_profile_layer(l);
+            st = run_linear(c.X, c.rows, c.vals, c.N == c.M ? nullptr : c.idx, c.bias, c.out, c.in, c.N, c.M, dtype,
+                            c.Y, workspace, dev_status, stream);
+            if (st != ELSA_OK) return layer_fail(st, l);
+        }
+        set_profile_layer(-1);
+        return ELSA_OK;
+    }
+
+    std::vector<LinearKind> kind(n_layers);
+    std::vector<uint8_t*> region(n_layers);
+    size_t off = 0;
     for (int l = 0; l < n_layers; ++l) {
         const elsa_layer& c = cfg[l];
+        if ((st = pick_kind(c.rows, c.out, c.in, c.N, c.M, dev.sm_count, &kind[l])) != ELSA_OK) return layer_fail(st, l);
+        region[l] = (uint8_t*)workspace + off;
+        off += round_up(elsa_workspace_bytes(c.rows, c.in, c.out, c.N, c.M, dtype), 256);
+    }
+    // weight images
+    for (int l = 0; l < n_layers; ++l) {
+        const elsa_layer& c = cfg[l];
+        if (c.N == c.M) continue;
         set_profile_layer(l);
-        st = run_linear(c.X, c.rows, c.vals, c.N == c.M ? nullptr : c.idx, c.bias, c.out, c.in, c.N, c.M, dtype,
-                        c.Y, workspace, dev_status, (cudaStream_t)stream);
-        if (st != ELSA_OK) {
-            set_profile_layer(-1);
-            char msg[400];
-            snprintf(msg, sizeof msg, "%s", elsa_last_error());
-            return fail(st, "layer %d: %s", l, msg);
+        if (kind[l] == KIND_SPARSE_PAIR)
+            st = launch_linear_tc_sparse_pair_prepare((const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, region[l], stream);
+        else
+            st = launch_unpack((const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, (uint16_t*)region[l], stream);
+        if (st != ELSA_OK) return layer_fail(st, l);
+    }
+    set_profile_layer(-1);
+    // sparse-rate layers, in groups
+    {
+        std::vector<SparseJob> jobs;
+        for (int l = 0; l <= n_layers; ++l) {
+            if (l < n_layers && kind[l] == KIND_SPARSE_PAIR) {
+                const elsa_layer& c = cfg[l];
+                SparseJob j;
+                j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
+                j.workspace = region[l]; j.rows = c.rows; j.in = c.in; j.out = c.out;
+                jobs.push_back(j);
+            }
+            if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_sparse_pair_group_max())) {
+                if ((st = launch_linear_tc_sparse_pair_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
+                    return st;
+                jobs.clear();
+            }
         }
+    }
+    // dense-rate layers on CTA pairs, in groups
+    {
+        std::vector<PairJob> jobs;
+        for (int l = 0; l <= n_layers; ++l) {
+            if (l < n_layers && kind[l] == KIND_DENSE_PAIR) {
+                const elsa_layer& c = cfg[l];
+                PairJob j;
+                j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
+                j.Wd = c.N == c.M ? (const uint16_t*)c.vals : (const uint16_t*)region[l];
+                j.rows = c.rows; j.in = c.in; j.out = c.out;
+                jobs.push_back(j);
+            }
+            if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_pair_group_max())) {
+                if ((st = launch_linear_tc_pair_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
+                    return st;
+                jobs.clear();
+            }
+        }
+    }
+    // small layers: one CTA per tile, one launch each
+    for (int l = 0; l < n_layers; ++l) {
+        if (kind[l] != KIND_DENSE_ONE) continue;
+        const elsa_layer& c = cfg[l];
+        set_profile_layer(l);
+        const uint16_t* Wd = c.N == c.M ? (const uint16_t*)c.vals : (const uint16_t*)region[l];
+        st = launch_linear_tc_dense((const uint16_t*)c.X, c.rows, Wd, (const uint16_t*)c.bias, c.out, c.in, dtype,
+                                    (uint16_t*)c.Y, dev_status, stream);
+        if (st != ELSA_OK) return layer_fail(st, l);
     }
     set_profile_layer(-1);
     return ELSA_OK;
@@ -407,6 +499,8 @@ elsa_status elsa_set_linear_variant(elsa_variant v)
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;
 }
+
+void elsa_set_grouping(int on) { g_grouping.store(on != 0, std::memory_order_relaxed); }
 
 elsa_variant elsa_get_linear_variant(void) { return (elsa_variant)g_variant.load(std::memory_order_relaxed); }
 

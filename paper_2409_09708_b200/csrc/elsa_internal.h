@@ -111,8 +111,34 @@ elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out
 elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                          const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
                                          uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
+// Several N <= 2 layers in one persistent launch of the sparse pair kernel; each job's workspace must
+// already hold its re-encoded weight (launch_linear_tc_sparse_pair_prepare).
+struct SparseJob {
+    const uint16_t* X;
+    const uint16_t* bias;
+    uint16_t* Y;
+    const void* workspace;
+    int rows, in, out;
+};
+int linear_tc_sparse_pair_group_max();
+elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
+                                                 void* workspace, cudaStream_t stream);
+elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                               cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
 size_t linear_tc_sparse_workspace(int out, int in);
+// Several dense-rate layers in one persistent launch of the CTA-pair kernel (at most
+// linear_tc_pair_group_max() of them): their tiles form one sequence.
+struct PairJob {
+    const uint16_t* X;
+    const uint16_t* Wd;     // dense weight image [out][in]
+    const uint16_t* bias;
+    uint16_t* Y;
+    int rows, in, out;
+};
+int linear_tc_pair_group_max();
+elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                        cudaStream_t stream);
 // Whether the problem has enough 256-row tiles to occupy every SM pair.
 bool linear_tc_pair_suits(int rows, int out, int sm_count);
 

@@ -21,6 +21,8 @@
 // before tensor memory is released keeps either CTA from leaving while its partner may still read
 // its shared memory.
 
+#include <mutex>
+
 #include "elsa_tc_common.cuh"
 
 namespace elsa {
@@ -43,22 +45,35 @@ constexpr int kStagingTotal = kEpiWarps * 2 * kStagingBytes;
 constexpr int kBiasBytes = kEpiWarps * kMaxBlockN * 4;
 constexpr int kBarrierBytes = 256;
 
-struct PairParams {
-    int rows, in, out;
+// One layer of a launch.  A launch may carry several layers (a group): the persistent CTA pairs walk the
+// tiles of all of them in one sequence, so the tail of one layer overlaps the head of the next and
+// only one kernel ramp is paid.  All of it lives in kernel-parameter space.
+struct alignas(64) PairLayer {
+    CUtensorMap map_x, map_w, map_y;
+    int rows, out;
     int bn;            // features per pair tile (MMA N)
     int tiles_n;
-    int num_tiles;     // pair tiles
+    int tile_begin;    // index of this layer's first tile in the launch's sequence
     int num_k_blocks;
-    int stages;
     uint32_t idesc;
     const uint16_t* bias;
+};
+
+template <int kMaxLayers>
+struct PairGroup {
+    PairLayer layer[kMaxLayers];
+    int n_layers;
+    int num_tiles;     // over all layers
+    int stages;
     uint32_t* dev_status;
 };
 
-template <bool kBf16>
+constexpr int kStageBytesMax = kATileBytes + (kMaxBlockN / 2) * kBlockK * 2;   // stage slots sized for BN = 256
+constexpr int kGroupMax = 72;   // layers per grouped launch (kernel parameters are limited to 32 KB)
+
+template <bool kBf16, int kMaxLayers>
 __global__ void __launch_bounds__(kThreads, 1)
-linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w,
-                      const __grid_constant__ CUtensorMap map_y, const PairParams p)
+linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -69,9 +84,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
     const uint32_t cta_rank = cluster_ctarank();       // 0 = leader of the pair
     const int pair = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
-    const int half_bn = p.bn >> 1;
-    const int b_tile_bytes = half_bn * kBlockK * 2;
-    const int stage_bytes = kATileBytes + b_tile_bytes;
+    constexpr int stage_bytes = kStageBytesMax;
 
     const uint32_t staging_base = smem_base + (uint32_t)(p.stages * stage_bytes);
     const uint32_t bias_off = (uint32_t)(p.stages * stage_bytes) + kStagingTotal;
@@ -115,18 +128,24 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            int cur = 0;
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
-                const int m0 = (tile / p.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
-                const int n0 = (tile % p.tiles_n) * p.bn + (int)cta_rank * half_bn;
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+                const PairLayer& L = p.layer[cur];
+                const int t = tile - L.tile_begin;
+                const int half_bn = L.bn >> 1;
+                const int m0 = (t / L.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
+                const int n0 = (t % L.tiles_n) * L.bn + (int)cta_rank * half_bn;
+                const uint32_t tx_bytes = (uint32_t)(2 * (kATileBytes + half_bn * kBlockK * 2));
+                for (int kb = 0; kb < L.num_k_blocks; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
                     if (!ok) break;
                     const uint32_t a_dst = smem_base + (uint32_t)(stage * stage_bytes);
                     // the leader's stage barrier collects the bytes of both CTAs
-                    if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, (uint32_t)(2 * stage_bytes));
+                    if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
                     const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
-                    tma_load_2d_pair(a_dst, &map_x, bar, kb * kBlockK, m0);
-                    tma_load_2d_pair(a_dst + kATileBytes, &map_w, bar, kb * kBlockK, n0);
+                    tma_load_2d_pair(a_dst, &L.map_x, bar, kb * kBlockK, m0);
+                    tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * kBlockK, n0);
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -140,12 +159,16 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            int cur = 0;
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+                while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+                const int num_k_blocks = p.layer[cur].num_k_blocks;
+                const uint32_t idesc = p.layer[cur].idesc;
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kMaxBlockN);
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                     if (!ok) break;
                     tc_fence_after();
@@ -154,7 +177,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
                     const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
+                        umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                       (uint32_t)((kb | k) != 0));
                     }
                     umma_commit_pair(empty_bar + 8 * stage, 3);   // frees this stage in both CTAs
@@ -177,15 +200,21 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
         int acc = 0;
         uint32_t acc_phase = 0;
         uint32_t chunk_counter = 0;
-        const int chunks = p.bn / kEpiCols;
-        const int my_chunks = (chunks - half + 1) / 2;
+        int cur = 0;
 
         for (int tile = pair; tile < p.num_tiles; tile += num_pairs) {
-            const int m0 = (tile / p.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
-            const int n0 = (tile % p.tiles_n) * p.bn;
-            for (int j = lane; j < p.bn; j += 32) {
+            while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+            const PairLayer& L = p.layer[cur];
+            const int t = tile - L.tile_begin;
+            const int chunks = L.bn / kEpiCols;
+            const int my_chunks = (chunks - half + 1) / 2;
+            const int m0 = (t / L.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
+            const int n0 = (t % L.tiles_n) * L.bn;
+            const int l_rows = L.rows, l_out = L.out;
+            const uint16_t* l_bias = L.bias;
+            for (int j = lane; j < L.bn; j += 32) {
                 const int o = n0 + j;
-                bias_s[j] = (p.bias != nullptr && o < p.out) ? bias_to_float<kBf16>(p.bias[o]) : 0.f;
+                bias_s[j] = (l_bias != nullptr && o < l_out) ? bias_to_float<kBf16>(l_bias[o]) : 0.f;
             }
             __syncwarp();
             bool ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
@@ -219,7 +248,7 @@ linear_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_co
                 __syncwarp();
                 if (lane == 0) {
                     const int col0 = n0 + c * kEpiCols;
-                    if (row0 < p.rows && col0 < p.out) tma_store_2d(&map_y, buf, col0, row0);
+                    if (row0 < l_rows && col0 < l_out) tma_store_2d(&L.map_y, buf, col0, row0);
                     bulk_commit_group();
                 }
                 ++chunk_counter;
@@ -289,82 +318,113 @@ bool linear_tc_pair_suits(int rows, int out, int sm_count)
     return tiles >= sm_count / 2;
 }
 
-elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias, int out,
-                                  int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status, cudaStream_t stream)
+namespace {
+
+template <bool kBf16, int kMaxLayers>
+elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
+                         const DeviceInfo& dev)
 {
-    DeviceInfo dev;
-    elsa_status st = device_info(&dev);
-    if (st != ELSA_OK) return st;
-
-    PairParams p;
-    p.rows = rows; p.in = in; p.out = out;
-    p.bn = pick_pair_block_n(out);
-    p.tiles_n = (out + p.bn - 1) / p.bn;
-    p.num_tiles = ((rows + kPairRows - 1) / kPairRows) * p.tiles_n;
-    p.num_k_blocks = (in + kBlockK - 1) / kBlockK;
-    p.bias = bias;
-    p.dev_status = dev_status;
+    static PairGroup<kMaxLayers> g;   // host staging of the kernel parameters (single-threaded launch path)
+    static std::mutex g_mutex;
+    std::lock_guard<std::mutex> lock(g_mutex);
     const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
-    p.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+    int tile_begin = 0;
+    for (int i = 0; i < n; ++i) {
+        const PairJob& j = jobs[i];
+        PairLayer& L = g.layer[i];
+        L.rows = j.rows; L.out = j.out;
+        L.bn = pick_pair_block_n(j.out);
+        L.tiles_n = (j.out + L.bn - 1) / L.bn;
+        L.tile_begin = tile_begin;
+        tile_begin += ((j.rows + kPairRows - 1) / kPairRows) * L.tiles_n;
+        L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
+        L.bias = j.bias;
+        L.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+        elsa_status st;
+        if ((st = make_map_2d(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, kBlockK, kRowsPerCta,
+                              CU_TENSOR_MAP_SWIZZLE_128B, "X")) != ELSA_OK)
+            return st;
+        if ((st = make_map_2d(&L.map_w, j.Wd, (uint64_t)j.in, (uint64_t)j.out, kBlockK, (uint32_t)(L.bn / 2),
+                              CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
+            return st;
+        if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B,
+                              "Y")) != ELSA_OK)
+            return st;
+    }
+    g.n_layers = n;
+    g.num_tiles = tile_begin;
+    g.dev_status = dev_status;
 
-    const int stage_bytes = kATileBytes + (p.bn / 2) * kBlockK * 2;
     const int fixed = kStagingTotal + kBiasBytes + kBarrierBytes + 1024;
-    int stages = (int)((dev.smem_optin - fixed) / stage_bytes);
+    int stages = (int)((dev.smem_optin - fixed) / kStageBytesMax);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
-    p.stages = stages;
-    const size_t smem = (size_t)stages * stage_bytes + fixed;
+    g.stages = stages;
+    const size_t smem = (size_t)stages * kStageBytesMax + fixed;
 
-    CUtensorMap map_x, map_w, map_y;
-    if ((st = make_map_2d(&map_x, X, (uint64_t)in, (uint64_t)rows, kBlockK, kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B,
-                          "X")) != ELSA_OK)
-        return st;
-    if ((st = make_map_2d(&map_w, Wd, (uint64_t)in, (uint64_t)out, kBlockK, (uint32_t)(p.bn / 2),
-                          CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
-        return st;
-    if ((st = make_map_2d(&map_y, Y, (uint64_t)out, (uint64_t)rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B, "Y")) !=
-        ELSA_OK)
-        return st;
-
-    auto kernel = dtype == ELSA_BF16 ? linear_tc_pair_kernel<true> : linear_tc_pair_kernel<false>;
-    static int max_pairs[64][2] = {};
+    auto kernel = linear_tc_pair_kernel<kBf16, kMaxLayers>;
+    static int max_pairs[64] = {};
     const int slot = dev.device & 63;
-
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-
-    if (max_pairs[slot][fmt] == 0) {
+    if (max_pairs[slot] == 0) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         }
         // how many CTA pairs the device can hold at once: the persistent schedule assumes all run together
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
         cfg.gridDim = dim3((unsigned)dev.sm_count);
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int m = 0;
+        if (cudaOccupancyMaxActiveClusters(&m, kernel, &cfg) != cudaSuccess || m < 1) {
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
         }
-        max_pairs[slot][fmt] = n;
+        max_pairs[slot] = m;
     }
-    const int pairs = p.num_tiles < max_pairs[slot][fmt] ? p.num_tiles : max_pairs[slot][fmt];
+    const int pairs = g.num_tiles < max_pairs[slot] ? g.num_tiles : max_pairs[slot];
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_PAIR, stream);
-    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, map_x, map_w, map_y, p);
+    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, g);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(ELSA_ERR_CUDA, "launch of linear_tc_pair failed: %s", cudaGetErrorString(e));
     }
     return launched("linear_tc_pair");
+}
+
+}  // namespace
+
+int linear_tc_pair_group_max() { return kGroupMax; }
+
+elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                        cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    if (n == 1)
+        return dtype == ELSA_BF16 ? launch_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+}
+
+elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias, int out,
+                                  int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status, cudaStream_t stream)
+{
+    PairJob job;
+    job.X = X; job.Wd = Wd; job.bias = bias; job.Y = Y;
+    job.rows = rows; job.in = in; job.out = out;
+    return launch_linear_tc_pair_group(&job, 1, dtype, dev_status, stream);
 }
 
 }  // namespace elsa

@@ -14,6 +14,8 @@
 // Per CTA (320 threads): warp 0 TMA producer, warp 1 tensor-memory allocation and (leader) MMA
 // issue, warps 2-9 epilogue.  Waits are bounded as in the other tensor-core kernels.
 
+#include <mutex>
+
 #include "elsa_tc_common.cuh"
 
 namespace elsa {
@@ -44,29 +46,32 @@ constexpr int kBarrierBytes = 256;
 
 static_assert(kStageBytes % 1024 == 0 && kBSubBytes % 1024 == 0, "swizzled tiles stay 1024-byte aligned");
 
-struct SpPairParams {
-    int rows, in, out;
+// One layer of a launch; a launch may carry several (their tiles form one sequence, so one layer's
+// tail overlaps the next one's head).  Lives in kernel-parameter space.
+struct alignas(64) SpPairLayer {
+    CUtensorMap map_a, map_x, map_e, map_y;
+    int rows, out;
     int tiles_f;       // ceil(out / 256)
-    int num_tiles;
+    int tile_begin;    // index of this layer's first tile in the launch's sequence
     int num_k_blocks;  // ceil(in / 128)
+    const uint16_t* bias;
+};
+
+template <int kMaxLayers>
+struct SpPairGroup {
+    SpPairLayer layer[kMaxLayers];
+    int n_layers;
+    int num_tiles;
     int stages;
     uint32_t idesc;
-    const uint16_t* bias;
     uint32_t* dev_status;
 };
 
-template <bool kBf16>
-__device__ __forceinline__ uint32_t to_16(float v)
-{
-    if constexpr (kBf16) return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
-    else return (uint32_t)__half_as_ushort(__float2half_rn(v));
-}
+constexpr int kGroupMax = 56;   // layers per grouped launch (kernel parameters are limited to 32 KB)
 
-template <bool kBf16>
+template <bool kBf16, int kMaxLayers>
 __global__ void __launch_bounds__(kThreads, 1)
-linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_x,
-                           const __grid_constant__ CUtensorMap map_e, const __grid_constant__ CUtensorMap map_y,
-                           const SpPairParams p)
+linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -118,20 +123,24 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
+            int cur = 0;
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
-                const int ft128 = (tile % p.tiles_f) * 2 + (int)cta_rank;   // this CTA's block of 128 features
-                const int r0 = (tile / p.tiles_f) * kRowTile + (int)cta_rank * kRowsPerCta;
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+                const SpPairLayer& L = p.layer[cur];
+                const int t = tile - L.tile_begin;
+                const int ft128 = (t % L.tiles_f) * 2 + (int)cta_rank;   // this CTA's block of 128 features
+                const int r0 = (t / L.tiles_f) * kRowTile + (int)cta_rank * kRowsPerCta;
+                for (int kb = 0; kb < L.num_k_blocks; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
                     if (!ok) break;
                     const uint32_t a_dst = smem_base + (uint32_t)(stage * kStageBytes);
                     if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, (uint32_t)(2 * kStageBytes));
                     const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
-                    tma_load_2d_pair(a_dst, &map_a, bar, kb * (kBlockK / 2), ft128 * kFeatPerCta);
-                    tma_load_2d_pair(a_dst + kATileBytes, &map_x, bar, kb * kBlockK, r0);
-                    tma_load_2d_pair(a_dst + kATileBytes + kBSubBytes, &map_x, bar, kb * kBlockK + 64, r0);
-                    tma_load_2d_pair(a_dst + kATileBytes + kBTileBytes, &map_e, bar, 0,
-                                     (ft128 * p.num_k_blocks + kb) * 128);
+                    tma_load_2d_pair(a_dst, &L.map_a, bar, kb * (kBlockK / 2), ft128 * kFeatPerCta);
+                    tma_load_2d_pair(a_dst + kATileBytes, &L.map_x, bar, kb * kBlockK, r0);
+                    tma_load_2d_pair(a_dst + kATileBytes + kBSubBytes, &L.map_x, bar, kb * kBlockK + 64, r0);
+                    tma_load_2d_pair(a_dst + kATileBytes + kBTileBytes, &L.map_e, bar, 0,
+                                     (ft128 * L.num_k_blocks + kb) * 128);
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -145,12 +154,15 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
             int acc = 0;
             uint32_t acc_phase = 0;
             bool ok = true;
+            int cur = 0;
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+                while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+                const int num_k_blocks = p.layer[cur].num_k_blocks;
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
-                for (int kb = 0; kb < p.num_k_blocks; ++kb) {
+                for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                     if (!ok) break;
                     tc_fence_after();
@@ -198,11 +210,17 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 #pragma unroll
         for (int k = 0; k < 4; ++k) sw_off[k] = (((uint32_t)(lane >> 3)) ^ (uint32_t)k) << 4;
 
+        int cur = 0;
         for (int tile = pair; tile < p.num_tiles; tile += num_pairs) {
-            const int f0 = ((tile % p.tiles_f) * 2 + (int)cta_rank) * kFeatPerCta + q * 32;
-            const int r0 = (tile / p.tiles_f) * kRowTile;
+            while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+            const SpPairLayer& L = p.layer[cur];
+            const int t = tile - L.tile_begin;
+            const int f0 = ((t % L.tiles_f) * 2 + (int)cta_rank) * kFeatPerCta + q * 32;
+            const int r0 = (t / L.tiles_f) * kRowTile;
             const int f = f0 + lane;
-            const float bias_f = (p.bias != nullptr && f < p.out) ? bias_to_float<kBf16>(p.bias[f]) : 0.f;
+            const int l_rows = L.rows, l_out = L.out;
+            const uint16_t* l_bias = L.bias;
+            const float bias_f = (l_bias != nullptr && f < l_out) ? bias_to_float<kBf16>(l_bias[f]) : 0.f;
             bool ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -230,7 +248,7 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
                 __syncwarp();
                 if (lane == 0) {
                     const int row0 = r0 + c * kEpiCols;
-                    if (row0 < p.rows && f0 < p.out) tma_store_2d(&map_y, buf, f0, row0);
+                    if (row0 < l_rows && f0 < l_out) tma_store_2d(&L.map_y, buf, f0, row0);
                     bulk_commit_group();
                 }
                 ++chunk_counter;
@@ -276,59 +294,62 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __gr
 
 }  // namespace
 
-elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
-                                         const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
-                                         uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream)
+namespace {
+
+template <bool kBf16, int kMaxLayers>
+elsa_status launch_sp_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
+                            const DeviceInfo& dev)
 {
-    DeviceInfo dev;
-    elsa_status st = device_info(&dev);
-    if (st != ELSA_OK) return st;
-    if (!linear_tc_sparse_suits(in, N) || N == M)
-        return fail(ELSA_ERR_NM, "level %d:%d with in=%d does not fit the 2:4 sparse MMA path", N, M, in);
-
-    const int tiles_f128 = (out + kFeatPerCta - 1) / kFeatPerCta;
-    const int k_blocks = (in + kBlockK - 1) / kBlockK;
-    uint16_t* a_img = (uint16_t*)workspace;
-    uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
-    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, a_img, meta, stream)) != ELSA_OK) return st;
-
-    SpPairParams p;
-    p.rows = rows; p.in = in; p.out = out;
-    p.tiles_f = (out + kPairFeat - 1) / kPairFeat;
-    p.num_tiles = p.tiles_f * ((rows + kRowTile - 1) / kRowTile);
-    p.num_k_blocks = k_blocks;
-    p.bias = bias;
-    p.dev_status = dev_status;
+    static SpPairGroup<kMaxLayers> g;   // host staging of the kernel parameters
+    static std::mutex g_mutex;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    int tile_begin = 0;
+    for (int i = 0; i < n; ++i) {
+        const SparseJob& j = jobs[i];
+        SpPairLayer& L = g.layer[i];
+        const int tiles_f128 = (j.out + kFeatPerCta - 1) / kFeatPerCta;
+        L.rows = j.rows; L.out = j.out;
+        L.tiles_f = (j.out + kPairFeat - 1) / kPairFeat;
+        L.tile_begin = tile_begin;
+        tile_begin += L.tiles_f * ((j.rows + kRowTile - 1) / kRowTile);
+        L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
+        L.bias = j.bias;
+        const uint16_t* a_img = (const uint16_t*)j.workspace;
+        const uint8_t* meta = (const uint8_t*)j.workspace + round_up((size_t)j.out * (size_t)j.in, 256);
+        elsa_status st;
+        if ((st = make_map_2d(&L.map_a, a_img, (uint64_t)(j.in / 2), (uint64_t)j.out, kBlockK / 2, kFeatPerCta,
+                              CU_TENSOR_MAP_SWIZZLE_128B, "2:4 weight image")) != ELSA_OK)
+            return st;
+        if ((st = make_map_2d(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, 64, kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B,
+                              "X")) != ELSA_OK)
+            return st;
+        // metadata blocks as a matrix of 16-byte rows: 128 rows per (128 features, K block)
+        if ((st = make_map_2d(&L.map_e, meta, 8, (uint64_t)tiles_f128 * L.num_k_blocks * 128, 8, 128,
+                              CU_TENSOR_MAP_SWIZZLE_NONE, "metadata")) != ELSA_OK)
+            return st;
+        if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B,
+                              "Y")) != ELSA_OK)
+            return st;
+    }
+    g.n_layers = n;
+    g.num_tiles = tile_begin;
+    g.dev_status = dev_status;
     const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
-    p.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRowTile >> 3) << 17) |
+    // sparse flag, fp32 accumulate, A and B of type fmt, K-major, N = 224, M = 256 over the pair
+    g.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRowTile >> 3) << 17) |
               ((uint32_t)(kPairFeat >> 4) << 24);
 
     const int fixed = kStagingTotal + kBarrierBytes + 1024;
     int stages = (int)((dev.smem_optin - fixed) / kStageBytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
-    p.stages = stages;
+    g.stages = stages;
     const size_t smem = (size_t)stages * kStageBytes + fixed;
 
-    CUtensorMap map_a, map_x, map_e, map_y;
-    if ((st = make_map_2d(&map_y, Y, (uint64_t)out, (uint64_t)rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B, "Y")) !=
-        ELSA_OK)
-        return st;
-    if ((st = make_map_2d(&map_a, a_img, (uint64_t)(in / 2), (uint64_t)out, kBlockK / 2, kFeatPerCta,
-                          CU_TENSOR_MAP_SWIZZLE_128B, "2:4 weight image")) != ELSA_OK)
-        return st;
-    if ((st = make_map_2d(&map_x, X, (uint64_t)in, (uint64_t)rows, 64, kRowsPerCta, CU_TENSOR_MAP_SWIZZLE_128B, "X")) !=
-        ELSA_OK)
-        return st;
-    // metadata blocks as a matrix of 16-byte rows: 128 rows per (128 features, K block)
-    if ((st = make_map_2d(&map_e, meta, 8, (uint64_t)tiles_f128 * k_blocks * 128, 8, 128, CU_TENSOR_MAP_SWIZZLE_NONE,
-                          "metadata")) != ELSA_OK)
-        return st;
-
-    auto kernel = dtype == ELSA_BF16 ? linear_tc_sp24_pair_kernel<true> : linear_tc_sp24_pair_kernel<false>;
-    static int max_pairs[64][2] = {};
+    auto kernel = linear_tc_sp24_pair_kernel<kBf16, kMaxLayers>;
+    static int max_pairs[64] = {};
     const int slot = dev.device & 63;
-    if (max_pairs[slot][fmt] == 0) {
+    if (max_pairs[slot] == 0) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
@@ -345,21 +366,62 @@ elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint
         cfg.dynamicSmemBytes = smem;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+        int m = 0;
+        if (cudaOccupancyMaxActiveClusters(&m, kernel, &cfg) != cudaSuccess || m < 1) {
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
         }
-        max_pairs[slot][fmt] = n;
+        max_pairs[slot] = m;
     }
-    const int pairs = p.num_tiles < max_pairs[slot][fmt] ? p.num_tiles : max_pairs[slot][fmt];
+    const int pairs = g.num_tiles < max_pairs[slot] ? g.num_tiles : max_pairs[slot];
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_SP24_PAIR, stream);
-    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, map_a, map_x, map_e, map_y, p);
+    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, g);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return fail(ELSA_ERR_CUDA, "launch of linear_tc_sp24_pair failed: %s", cudaGetErrorString(e));
     }
     return launched("linear_tc_sp24_pair");
+}
+
+}  // namespace
+
+int linear_tc_sparse_pair_group_max() { return kGroupMax; }
+
+elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                               cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    if (n == 1)
+        return dtype == ELSA_BF16 ? launch_sp_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_sp_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_sp_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_sp_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+}
+
+elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                         const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
+                                         uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream)
+{
+    if (!linear_tc_sparse_suits(in, N) || N == M)
+        return fail(ELSA_ERR_NM, "level %d:%d with in=%d does not fit the 2:4 sparse MMA path", N, M, in);
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, workspace, stream);
+    if (st != ELSA_OK) return st;
+    SparseJob job;
+    job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;
+    job.rows = rows; job.in = in; job.out = out;
+    return launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
+}
+
+// Re-encodes one packed weight into `workspace` in the form the pair kernel reads (K blocks of 128).
+elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
+                                                 void* workspace, cudaStream_t stream)
+{
+    uint16_t* a_img = (uint16_t*)workspace;
+    uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
+    return launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, a_img, meta, stream);
 }
 
 }  // namespace elsa
