@@ -115,6 +115,22 @@ elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint
                            void* Y, void* workspace, size_t workspace_bytes,
                            uint32_t* dev_status, void* stream);
 
+/* One weight of a table: dense W in, packed form out (as for elsa_nm_compress). */
+typedef struct {
+    const void* W;   /* [out][in] device */
+    void* vals;      /* [out][in/M*N] device, written */
+    uint32_t* idx;   /* index words, device, written; NULL iff N == M */
+    int out, in, N, M;
+} elsa_weight;
+
+/*
+ * elsa_nm_compress for every weight of a table, each to its own level (Sec. 3.1 applied under a
+ * layer-wise configuration alpha, Sec. 3), in one kernel launch per 256 weights.  `w` is a HOST
+ * array; results are bit-identical to per-weight calls.  The table is validated before anything is
+ * launched; elsa_last_error() names the offending entry.
+ */
+elsa_status elsa_vit_compress(const elsa_weight* w, int n_weights, elsa_dtype dtype, void* stream);
+
 /* One linear module of the per-layer table (Sec. 3: configuration alpha = (s^1 .. s^L)). */
 typedef struct {
     const void* X;       /* [rows][in]  device */
@@ -223,7 +239,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_PAIR = 4,
     ELSA_KERNEL_NM_TO_SP24 = 5,
     ELSA_KERNEL_LINEAR_TC_SP24 = 6,
-    ELSA_KERNEL_LINEAR_TC_SP24_PAIR = 7
+    ELSA_KERNEL_LINEAR_TC_SP24_PAIR = 7,
+    ELSA_KERNEL_WEIGHT_IMAGES = 8 /* batched unpack / 2-of-4 re-encoding of a table's weights */
 } elsa_kernel_id;
 
 typedef struct {

@@ -40,6 +40,10 @@ class ElsaLayer(ctypes.Structure):
                 ("rows", _i), ("in_", _i), ("out", _i), ("N", _i), ("M", _i)]
 
 
+class ElsaWeight(ctypes.Structure):
+    _fields_ = [("W", _vp), ("vals", _vp), ("idx", _vp), ("out", _i), ("in_", _i), ("N", _i), ("M", _i)]
+
+
 class ElsaHostLayer(ctypes.Structure):
     _fields_ = [("X", _vp), ("Y", _vp), ("W", _vp), ("bias", _vp),
                 ("rows", _i), ("in_", _i), ("out", _i), ("N", _i), ("M", _i)]
@@ -60,6 +64,7 @@ _unpack = _sig("elsa_nm_unpack", _i, [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp])
 _linear = _sig("elsa_nm_linear", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
 _linear_static = _sig("elsa_nm_linear_static", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 STATIC_SCRATCH_BYTES = 8 << 20
+_vit_compress = _sig("elsa_vit_compress", _i, [ctypes.POINTER(ElsaWeight), _i, _i, _vp])
 _vit_ws = _sig("elsa_vit_workspace_bytes", _sz, [ctypes.POINTER(ElsaLayer), _i, _i])
 _vit = _sig("elsa_vit_linears", _i, [ctypes.POINTER(ElsaLayer), _i, _i, _vp, _sz, _vp, _vp])
 _vit_host_bytes = _sig("elsa_vit_host_device_bytes", _sz, [ctypes.POINTER(ElsaHostLayer), _i, _i])
@@ -75,7 +80,7 @@ class ElsaKernelTime(ctypes.Structure):
     _fields_ = [("kernel", _i), ("layer", _i), ("ms", ctypes.c_float)]
 
 
-KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair"}
+KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 
@@ -220,6 +225,21 @@ def make_layer_table(layers):
         a.rows, a.in_, a.out = X.shape[0], X.shape[1], Y.shape[1]
         a.N, a.M = l["N"], l["M"]
     return arr
+
+
+def make_weight_table(layers):
+    """ctypes array of elsa_weight from dicts with W, vals, idx tensors and N, M."""
+    arr = (ElsaWeight * len(layers))()
+    for a, l in zip(arr, layers):
+        W = l["W"]
+        a.W, a.vals, a.idx = _ptr(W), _ptr(l["vals"]), _ptr(l.get("idx"))
+        a.out, a.in_ = W.shape
+        a.N, a.M = l["N"], l["M"]
+    return arr
+
+
+def elsa_vit_compress(table, dtype_c: int, stream=None):
+    _check(_vit_compress(table, len(table), dtype_c, _stream(stream)))
 
 
 def elsa_vit_workspace_bytes(table, dtype_c: int) -> int:

@@ -275,6 +275,45 @@ elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint
                       (cudaStream_t)stream);
 }
 
+elsa_status elsa_vit_compress(const elsa_weight* w, int n_weights, elsa_dtype dtype, void* stream)
+{
+    if (!w) return fail(ELSA_ERR_NULL, "w must not be NULL");
+    if (n_weights <= 0) return fail(ELSA_ERR_SHAPE, "non-positive n_weights=%d", n_weights);
+    for (int i = 0; i < n_weights; ++i) {
+        const elsa_weight& c = w[i];
+        elsa_status st = ELSA_OK;
+        if (!c.W || !c.vals) st = fail(ELSA_ERR_NULL, "W and vals must not be NULL");
+        else if ((st = check_level(c.out, c.in, c.N, c.M, dtype)) != ELSA_OK) {}
+        else if (c.N != c.M && !c.idx) st = fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+        else if (!aligned16(c.W) || !aligned16(c.vals) || (c.idx && !aligned16(c.idx)))
+            st = fail(ELSA_ERR_ALIGN, "W, vals and idx must be 16-byte aligned");
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "weight %d: %s", i, msg);
+        }
+    }
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    static BatchTable table;              // host staging of the kernel parameters
+    static std::mutex table_mutex;
+    std::lock_guard<std::mutex> lock(table_mutex);
+    table.n = 0;
+    table.total_units = 0;
+    for (int i = 0; i < n_weights; ++i) {
+        const elsa_weight& c = w[i];
+        batch_add_compress(&table, (const uint16_t*)c.W, c.out, c.in, c.N, c.M, (uint16_t*)c.vals,
+                           c.N == c.M ? nullptr : c.idx);
+        if (table.n == kBatchMax || i == n_weights - 1) {
+            if ((st = launch_compress_batch(table, (cudaStream_t)stream)) != ELSA_OK) return st;
+            table.n = 0;
+            table.total_units = 0;
+        }
+    }
+    return ELSA_OK;
+}
+
 size_t elsa_vit_workspace_bytes(const elsa_layer* cfg, int n_layers, elsa_dtype dtype)
 {
     // one region per layer, so that every weight image can be built before the grouped launches
@@ -339,18 +378,31 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
         region[l] = (uint8_t*)workspace + off;
         off += round_up(elsa_workspace_bytes(c.rows, c.in, c.out, c.N, c.M, dtype), 256);
     }
-    // weight images
-    for (int l = 0; l < n_layers; ++l) {
-        const elsa_layer& c = cfg[l];
-        if (c.N == c.M) continue;
-        set_profile_layer(l);
-        if (kind[l] == KIND_SPARSE_PAIR)
-            st = launch_linear_tc_sparse_pair_prepare((const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, region[l], stream);
-        else
-            st = launch_unpack((const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, (uint16_t*)region[l], stream);
-        if (st != ELSA_OK) return layer_fail(st, l);
+    // weight images of all layers, one launch per 256 layers
+    {
+        static BatchTable table;          // host staging of the kernel parameters
+        static std::mutex table_mutex;
+        std::lock_guard<std::mutex> lock(table_mutex);
+        table.n = 0;
+        table.total_units = 0;
+        for (int l = 0; l < n_layers; ++l) {
+            const elsa_layer& c = cfg[l];
+            if (c.N != c.M) {
+                if (kind[l] == KIND_SPARSE_PAIR) {
+                    uint8_t* meta = region[l] + round_up((size_t)c.out * (size_t)c.in, 256);
+                    batch_add_to_sp24(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, 128,
+                                      (uint16_t*)region[l], meta);
+                } else {
+                    batch_add_unpack(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, (uint16_t*)region[l]);
+                }
+            }
+            if (table.n == kBatchMax || (l == n_layers - 1 && table.n > 0)) {
+                if ((st = launch_image_batch(table, stream)) != ELSA_OK) return st;
+                table.n = 0;
+                table.total_units = 0;
+            }
+        }
     }
-    set_profile_layer(-1);
     // sparse-rate layers, in groups
     {
         std::vector<SparseJob> jobs;

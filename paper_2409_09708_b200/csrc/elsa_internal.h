@@ -127,6 +127,30 @@ elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, els
                                                cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
 size_t linear_tc_sparse_workspace(int out, int in);
+// Batched weight-format kernels: one launch over a table of weights (kernel-parameter space).
+enum BatchKind { BATCH_COMPRESS = 0, BATCH_UNPACK = 1, BATCH_TO_SP24 = 2 };
+struct BatchItem {
+    const void* src;
+    const void* src2;
+    void* dst;
+    void* dst2;
+    long long first_unit;   // prefix sum of work units over the table
+    int out, in, N, M, wpr, aux, aux2, kind;
+};
+constexpr int kBatchMax = 256;
+struct BatchTable {
+    BatchItem item[kBatchMax];
+    long long total_units;
+    int n;
+};
+void batch_add_compress(BatchTable* t, const uint16_t* W, int out, int in, int N, int M, uint16_t* vals, uint32_t* idx);
+void batch_add_unpack(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
+                      uint16_t* Wm);
+void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
+                       int block_k, uint16_t* a_img, uint8_t* meta);
+elsa_status launch_compress_batch(const BatchTable& t, cudaStream_t stream);
+elsa_status launch_image_batch(const BatchTable& t, cudaStream_t stream);
+
 // Several dense-rate layers in one persistent launch of the CTA-pair kernel (at most
 // linear_tc_pair_group_max() of them): their tiles form one sequence.
 struct PairJob {

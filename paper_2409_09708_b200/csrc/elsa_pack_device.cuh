@@ -1,0 +1,255 @@
+// Device code of the weight-format kernels, shared by the per-weight launches and the batched ones:
+// N:M projection + packing (Sec. 3.1 / Eq. 1 and the compressed form of Sec. 1 / Sec. 2 of the ELSA
+// paper), its inverse, and the re-encoding of a packed weight as 2-of-4 values + tensor-memory
+// metadata for the sparse MMA.  Each function handles one unit of work given its global index.
+#pragma once
+
+#include "elsa_internal.h"
+
+namespace elsa {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kMaxIndexWordsPerSegment = 64;  // 32 groups x N*b bits, N*b <= 60 for N < M <= 16
+
+template <int M>
+__device__ __forceinline__ void load_group(const uint16_t* p, uint16_t (&w)[M])
+{
+    if constexpr (M == 4) {
+        uint2 v = *reinterpret_cast<const uint2*>(p);
+        w[0] = v.x & 0xFFFF; w[1] = v.x >> 16; w[2] = v.y & 0xFFFF; w[3] = v.y >> 16;
+    } else {
+#pragma unroll
+        for (int q = 0; q < M / 8; ++q) {
+            uint4 v = reinterpret_cast<const uint4*>(p)[q];
+            w[8 * q + 0] = v.x & 0xFFFF; w[8 * q + 1] = v.x >> 16;
+            w[8 * q + 2] = v.y & 0xFFFF; w[8 * q + 3] = v.y >> 16;
+            w[8 * q + 4] = v.z & 0xFFFF; w[8 * q + 5] = v.z >> 16;
+            w[8 * q + 6] = v.w & 0xFFFF; w[8 * q + 7] = v.w >> 16;
+        }
+    }
+}
+
+// One warp compresses 32 consecutive groups of one row, one group per lane.  The 32 groups own
+// exactly N*b whole index words of the row's bitstream, so each warp assembles its words in shared
+// memory and writes them with one coalesced store.
+template <int M>
+__device__ __forceinline__ void compress_segment(const uint16_t* __restrict__ W, int in, int N,
+                                                 uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                 int segs_per_row, int words_per_row, long long seg_id,
+                                                 uint32_t (*words)[kMaxIndexWordsPerSegment])
+{
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+
+    const int o = (int)(seg_id / segs_per_row);
+    const int seg = (int)(seg_id % segs_per_row);
+    const int groups_per_row = in / M;
+    const int g = seg * 32 + lane;
+    const bool valid = g < groups_per_row;
+    const int seg_words = N * B;  // index words this segment owns (when N < M)
+
+    if (words_per_row) {
+        for (int w = lane; w < seg_words; w += 32) words[warp][w] = 0;
+        __syncwarp();
+    }
+
+    if (valid) {
+        uint16_t w[M];
+        load_group<M>(W + (size_t)o * in + (size_t)g * M, w);
+
+        // rank_i = #{j : |w_j| > |w_i|} + #{j < i : |w_j| == |w_i|}; keep iff rank_i < N.
+        // Magnitudes are compared as the 15 low bits of the pattern.
+        uint32_t keep = 0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            const uint32_t ki = w[i] & 0x7FFFu;
+            int rank = 0;
+#pragma unroll
+            for (int j = 0; j < M; ++j) {
+                const uint32_t kj = w[j] & 0x7FFFu;
+                rank += (kj > ki) || (j < i && kj == ki);
+            }
+            keep |= (uint32_t)(rank < N) << i;
+        }
+
+        uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
+        unsigned long long fields = 0;
+        int t = 0;
+#pragma unroll
+        for (int i = 0; i < M; ++i) {
+            if ((keep >> i) & 1u) {
+                v[t] = w[i];
+                fields |= (unsigned long long)i << (t * B);
+                ++t;
+            }
+        }
+
+        if (words_per_row) {
+            const int bit0 = lane * seg_words;  // bit offset of this group's fields in the segment
+            const int w0 = bit0 >> 5, sh = bit0 & 31;
+            // up to 60 bits shifted by up to 31: three words at most
+            const uint32_t lo = (uint32_t)(fields << sh);
+            const uint32_t mid = (uint32_t)(fields >> (32 - sh));
+            const uint32_t hi = sh ? (uint32_t)(fields >> (64 - sh)) : 0u;
+            // a zero part may lie past the segment's last word and is skipped
+            if (lo) atomicOr(&words[warp][w0], lo);
+            if (mid) atomicOr(&words[warp][w0 + 1], mid);
+            if (hi) atomicOr(&words[warp][w0 + 2], hi);
+        }
+    }
+
+    if (words_per_row) {
+        __syncwarp();
+        const int first = seg * seg_words;
+        uint32_t* row = idx + (size_t)o * words_per_row;
+        for (int w = lane; w < seg_words && first + w < words_per_row; w += 32)
+            row[first + w] = words[warp][w];
+    }
+}
+
+// One thread rebuilds one group: N values scattered to their positions, +0.0 elsewhere.
+template <int M>
+__device__ __forceinline__ void unpack_group(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
+                                             int in, int N, uint16_t* __restrict__ Wm, int words_per_row,
+                                             long long gid)
+{
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    const int groups_per_row = in / M;
+    const int o = (int)(gid / groups_per_row);
+    const int g = (int)(gid % groups_per_row);
+
+    const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
+    unsigned long long fields;
+    if (words_per_row) {
+        const uint32_t* row = idx + (size_t)o * words_per_row;
+        const long long bit0 = (long long)g * N * B;
+        const int w0 = (int)(bit0 >> 5), sh = (int)(bit0 & 31);
+        const int nbits = N * B;
+        unsigned long long lo = row[w0];
+        if (sh + nbits > 32) lo |= (unsigned long long)row[w0 + 1] << 32;
+        fields = lo >> sh;
+        if (sh + nbits > 64) fields |= (unsigned long long)row[w0 + 2] << (64 - sh);
+    } else {
+        fields = 0;  // N == M: position t holds value t
+#pragma unroll
+        for (int t = 0; t < M; ++t) fields |= (unsigned long long)t << (t * B);
+    }
+
+    uint16_t w[M];
+#pragma unroll
+    for (int i = 0; i < M; ++i) w[i] = 0;
+    for (int t = 0; t < N; ++t) {
+        const int pos = (int)((fields >> (t * B)) & (M - 1));
+        const uint16_t val = v[t];
+#pragma unroll
+        for (int i = 0; i < M; ++i) w[i] = (i == pos) ? val : w[i];
+    }
+
+    uint16_t* dst = Wm + (size_t)o * in + (size_t)g * M;
+    if constexpr (M == 4) {
+        uint2 r;
+        r.x = w[0] | ((uint32_t)w[1] << 16);
+        r.y = w[2] | ((uint32_t)w[3] << 16);
+        *reinterpret_cast<uint2*>(dst) = r;
+    } else {
+#pragma unroll
+        for (int q = 0; q < M / 8; ++q) {
+            uint4 r;
+            r.x = w[8 * q + 0] | ((uint32_t)w[8 * q + 1] << 16);
+            r.y = w[8 * q + 2] | ((uint32_t)w[8 * q + 3] << 16);
+            r.z = w[8 * q + 4] | ((uint32_t)w[8 * q + 5] << 16);
+            r.w = w[8 * q + 6] | ((uint32_t)w[8 * q + 7] << 16);
+            reinterpret_cast<uint4*>(dst)[q] = r;
+        }
+    }
+}
+
+// One thread per (weight row, 16 consecutive k): rebuilds those 16 positions from the packed form,
+// then emits, per aligned chunk of 4, two values with ascending positions (i0 < i1).  Pruned
+// positions are zero in the rebuilt segment, so a chunk with fewer than two kept weights simply
+// borrows a zero from another position.
+template <int M>
+__device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
+                                                int out, int in, int N, int words_per_row,
+                                                uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
+                                                int k_blocks, int steps_per_block, long long tid)
+{
+    constexpr int kFeatTile = 128;
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    constexpr int G = 16 / M;                         // groups per 16-k segment
+    const int segs = k_blocks * steps_per_block * 2;  // 16-k segments per (padded) row
+    const int o = (int)(tid / segs);                  // padded row index
+    const int seg = (int)(tid % segs);
+    const int k0 = seg * 16;
+
+    uint16_t d[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) d[i] = 0;
+    uint32_t keep = 0;
+    const bool real = o < out && k0 < in;             // in is a multiple of 16 on this path
+    if (real) {
+        const int groups_per_row = in / M;
+        const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N);
+        const uint32_t* row = idx + (size_t)o * words_per_row;
+#pragma unroll
+        for (int gl = 0; gl < G; ++gl) {
+            const int g = k0 / M + gl;
+            for (int t = 0; t < N; ++t) {
+                const long long bit = ((long long)g * N + t) * B;
+                const int w0 = (int)(bit >> 5), sh = (int)(bit & 31);
+                uint32_t f = row[w0] >> sh;
+                if (sh + B > 32) f |= row[w0 + 1] << (32 - sh);
+                const int pos = gl * M + (int)(f & (uint32_t)(M - 1));
+                const uint16_t val = v[(size_t)g * N + t];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) d[i] = (i == pos) ? val : d[i];
+                keep |= 1u << pos;
+            }
+        }
+    }
+
+    uint32_t nibbles = 0;
+    uint16_t sel[8];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t m4 = (keep >> (4 * c)) & 15u;
+        const int cnt = __popc(m4);
+        int i0, i1;
+        if (cnt >= 2) { i0 = __ffs(m4) - 1; i1 = 31 - __clz(m4); }
+        else if (cnt == 1) { const int p = __ffs(m4) - 1; i0 = (p == 3) ? 0 : p; i1 = 3; }
+        else { i0 = 0; i1 = 1; }
+        nibbles |= (uint32_t)(i0 | (i1 << 2)) << (4 * c);
+        uint16_t v0 = d[4 * c], v1 = d[4 * c];
+#pragma unroll
+        for (int i = 1; i < 4; ++i) {
+            v0 = (i == i0) ? d[4 * c + i] : v0;
+            v1 = (i == i1) ? d[4 * c + i] : v1;
+        }
+        sel[2 * c] = v0;
+        sel[2 * c + 1] = v1;
+    }
+
+    if (real) {
+        uint4 r;
+        r.x = sel[0] | ((uint32_t)sel[1] << 16);
+        r.y = sel[2] | ((uint32_t)sel[3] << 16);
+        r.z = sel[4] | ((uint32_t)sel[5] << 16);
+        r.w = sel[6] | ((uint32_t)sel[7] << 16);
+        *reinterpret_cast<uint4*>(a_img + (size_t)o * (in / 2) + k0 / 2) = r;
+    }
+    // metadata half-word: block (feature tile, k block) -> lane -> 4 words, one per K step of 32; a
+    // block covers steps_per_block (2 or 4) steps and leaves the other words zero
+    const int ftile = o / kFeatTile, m = o % kFeatTile;
+    const int kb = seg / (2 * steps_per_block), step = (seg / 2) % steps_per_block, k1 = seg % 2;
+    const int lane = (m % 8) + 8 * k1 + 16 * (m / 16);
+    const int hi = (m / 8) % 2;
+    const size_t word = (((size_t)ftile * k_blocks + kb) * 128 + lane) * 4 + step;
+    meta16[2 * word + hi] = (uint16_t)nibbles;
+    if (steps_per_block == 2) meta16[2 * (word + 2) + hi] = 0;
+}
+
+
+}  // namespace
+}  // namespace elsa

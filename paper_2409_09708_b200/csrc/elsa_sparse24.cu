@@ -21,6 +21,7 @@
 // row m + 8; nibble c of a half-word describes chunk c: position of the first stored value in bits
 // 0-1, of the second in bits 2-3 (first < second).
 
+#include "elsa_pack_device.cuh"
 #include "elsa_tc_common.cuh"
 
 namespace elsa {
@@ -50,91 +51,18 @@ static_assert(kStageBytes % 1024 == 0, "stages keep the 1024-byte alignment of t
 
 // ------------------------------------------------------------------ re-encoding
 
-// One thread per (weight row, 16 consecutive k): rebuilds those 16 positions from the packed form,
-// then emits, per aligned chunk of 4, two values with ascending positions (i0 < i1).  Pruned
-// positions are zero in the rebuilt segment, so a chunk with fewer than two kept weights simply
-// borrows a zero from another position.
+// (the per-segment device code is in elsa_pack_device.cuh)
 template <int M>
 __global__ void __launch_bounds__(256)
 nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx, int out, int in, int N,
                   int words_per_row, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int out_tiles,
                   int k_blocks, int steps_per_block)
 {
-    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
-    constexpr int G = 16 / M;                         // groups per 16-k segment
-    const int segs = k_blocks * steps_per_block * 2;  // 16-k segments per (padded) row
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
-    if (tid >= (long long)out_tiles * kFeatTile * segs) return;
-    const int o = (int)(tid / segs);                  // padded row index
-    const int seg = (int)(tid % segs);
-    const int k0 = seg * 16;
-
-    uint16_t d[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) d[i] = 0;
-    uint32_t keep = 0;
-    const bool real = o < out && k0 < in;             // in is a multiple of 16 on this path
-    if (real) {
-        const int groups_per_row = in / M;
-        const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N);
-        const uint32_t* row = idx + (size_t)o * words_per_row;
-#pragma unroll
-        for (int gl = 0; gl < G; ++gl) {
-            const int g = k0 / M + gl;
-            for (int t = 0; t < N; ++t) {
-                const long long bit = ((long long)g * N + t) * B;
-                const int w0 = (int)(bit >> 5), sh = (int)(bit & 31);
-                uint32_t f = row[w0] >> sh;
-                if (sh + B > 32) f |= row[w0 + 1] << (32 - sh);
-                const int pos = gl * M + (int)(f & (uint32_t)(M - 1));
-                const uint16_t val = v[(size_t)g * N + t];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) d[i] = (i == pos) ? val : d[i];
-                keep |= 1u << pos;
-            }
-        }
-    }
-
-    uint32_t nibbles = 0;
-    uint16_t sel[8];
-#pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        const uint32_t m4 = (keep >> (4 * c)) & 15u;
-        const int cnt = __popc(m4);
-        int i0, i1;
-        if (cnt >= 2) { i0 = __ffs(m4) - 1; i1 = 31 - __clz(m4); }
-        else if (cnt == 1) { const int p = __ffs(m4) - 1; i0 = (p == 3) ? 0 : p; i1 = 3; }
-        else { i0 = 0; i1 = 1; }
-        nibbles |= (uint32_t)(i0 | (i1 << 2)) << (4 * c);
-        uint16_t v0 = d[4 * c], v1 = d[4 * c];
-#pragma unroll
-        for (int i = 1; i < 4; ++i) {
-            v0 = (i == i0) ? d[4 * c + i] : v0;
-            v1 = (i == i1) ? d[4 * c + i] : v1;
-        }
-        sel[2 * c] = v0;
-        sel[2 * c + 1] = v1;
-    }
-
-    if (real) {
-        uint4 r;
-        r.x = sel[0] | ((uint32_t)sel[1] << 16);
-        r.y = sel[2] | ((uint32_t)sel[3] << 16);
-        r.z = sel[4] | ((uint32_t)sel[5] << 16);
-        r.w = sel[6] | ((uint32_t)sel[7] << 16);
-        *reinterpret_cast<uint4*>(a_img + (size_t)o * (in / 2) + k0 / 2) = r;
-    }
-    // metadata half-word: block (feature tile, k block) -> lane -> 4 words, one per K step of 32; a
-    // block covers steps_per_block (2 or 4) steps and leaves the other words zero
-    const int ftile = o / kFeatTile, m = o % kFeatTile;
-    const int kb = seg / (2 * steps_per_block), step = (seg / 2) % steps_per_block, k1 = seg % 2;
-    const int lane = (m % 8) + 8 * k1 + 16 * (m / 16);
-    const int hi = (m / 8) % 2;
-    const size_t word = (((size_t)ftile * k_blocks + kb) * 128 + lane) * 4 + step;
-    meta16[2 * word + hi] = (uint16_t)nibbles;
-    if (steps_per_block == 2) meta16[2 * (word + 2) + hi] = 0;
+    if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
+    to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, tid);
 }
 
 // ------------------------------------------------------------------ GEMM

@@ -248,14 +248,16 @@ def test_single_layer_config(lib):
 
 
 def stack_check(lib, layers, dtype, rows_sampled, seed):
-    """Run a table through elsa_vit_linears and check sampled rows of every layer against the oracle."""
+    """Run a table through elsa_vit_compress + elsa_vit_linears and check the packed weights in full and
+    sampled rows of every layer against the oracle."""
     code = lib.dtype_code(dtype)
     dev = []
     for l in layers:
         X, W, b = synth.layer_tensors(l, dtype, device="cuda")
-        vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+        vals, idx = lib.alloc_packed(l.out, l.in_, l.N, l.M, dtype)
         Y = torch.empty((l.rows, l.out), dtype=dtype, device="cuda")
         dev.append(dict(X=X, Y=Y, W=W, vals=vals, idx=idx, bias=b, N=l.N, M=l.M))
+    lib.elsa_vit_compress(lib.make_weight_table(dev), code)
     table = lib.make_layer_table(dev)
     ws = lib.alloc_workspace(lib.elsa_vit_workspace_bytes(table, code))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
