@@ -14,8 +14,8 @@
 //   warp 1      allocates tensor memory (pair-wide); in the leader one lane issues the MMAs and
 //               commits, by multicast, onto both CTAs' stage and accumulator barriers
 //   warps 2-9   epilogue, two warps per TMEM lane quarter (alternating 32-column chunks):
-//               tcgen05.ld (next chunk in flight while the current one is converted), + bias in
-//               fp32, round to 16 bit, swizzled staging, TMA store
+//               tcgen05.ld of all the warp's chunks, accumulator released, then + bias in fp32,
+//               round to 16 bit, swizzled staging, TMA store
 // Two TMEM accumulators let the MMAs of tile i+1 overlap the epilogue of tile i.  Every wait is
 // bounded; on expiry ELSA_ERR_TIMEOUT is recorded and all roles of the CTA leave; a cluster barrier
 // before tensor memory is released keeps either CTA from leaving while its partner may still read
@@ -39,6 +39,7 @@ constexpr int kMaxStages = 8;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + kEpiWarps * 32;
 constexpr int kEpiCols = 32;
+constexpr int kMaxChunksPerWarp = kMaxBlockN / kEpiCols / 2;   // two warps per TMEM lane quarter share the chunks
 constexpr int kATileBytes = kRowsPerCta * kBlockK * 2;
 constexpr int kStagingBytes = 32 * kEpiCols * 2;
 constexpr int kStagingTotal = kEpiWarps * 2 * kStagingBytes;
@@ -260,20 +261,18 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 if (lane == 0) mbar_arrive_cluster(empty_remote + 8 * acc);
             };
 
-            uint32_t ra[32], rb[32];
-            tmem_ld_32x32b_x32(t_row + (uint32_t)(half * kEpiCols), ra);
-            for (int i = 0; i < my_chunks; i += 2) {
-                tmem_wait_ld();
-                if (i + 1 < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * (i + 1)) * kEpiCols), rb);
-                else release();
-                emit(ra, half + 2 * i);
-                if (i + 1 < my_chunks) {
-                    tmem_wait_ld();
-                    if (i + 2 < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * (i + 2)) * kEpiCols), ra);
-                    else release();
-                    emit(rb, half + 2 * (i + 1));
-                }
-            }
+            // All of this warp's chunks are requested at once and the accumulator is handed back as soon
+            // as they have arrived: a tensor-memory load queues behind the MMAs already issued, so
+            // loads taken one at a time would each pay that wait.
+            uint32_t r[kMaxChunksPerWarp][32];
+#pragma unroll
+            for (int i = 0; i < kMaxChunksPerWarp; ++i)
+                if (i < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * i) * kEpiCols), r[i]);
+            tmem_wait_ld();
+            release();
+#pragma unroll
+            for (int i = 0; i < kMaxChunksPerWarp; ++i)
+                if (i < my_chunks) emit(r[i], half + 2 * i);
             if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait_group_all();
