@@ -114,6 +114,22 @@ class ClockSampler:
                 "samples": len(sm), "power_w_max": max(power)}
 
 
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """The slowest rank's time: what a multi-GPU number is quoted on."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tflops(flops_per_rank: float, world: int, ms: float) -> float:
+    """Replicas only: every rank processes the same table, the job's throughput is the sum over ranks."""
+    return world * flops_per_rank / (ms * 1e-3) / 1e12
+
+
 def dist_env():
     return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
 
@@ -230,11 +246,7 @@ def run_ours(args):
         e1.record()
         barrier()
         recs = lib.elsa_profile_stop() if profile else None
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
+        ms = max_over_ranks(e0.elapsed_time(e1), world)
         return ms, lib.elsa_launch_count() - launches0, recs
 
     for _ in range(args.warmup):
@@ -255,7 +267,7 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     dense_flops = sum(l.dense_equiv_flops for l in layers)
     kept_flops = sum(l.kept_flops for l in layers)
-    value = world * dense_flops / (ms_per_step * 1e-3) / 1e12
+    value = whole_job_tflops(dense_flops, world, ms_per_step)
 
     # ---- per-kernel accounting from the profiled pass
     per_kernel = {}
@@ -379,15 +391,10 @@ def run_e2e(args, lib, synth, layers, dtype, code, dev, world, barrier):
         lib.elsa_vit_linears_host(table, code, mem, dev_status=status)
     e1.record()
     barrier()
-    ms = e0.elapsed_time(e1) / steps
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(e0.elapsed_time(e1) / steps, world)
     assert int(status.item()) == 0
     dense_flops = sum(l.dense_equiv_flops for l in layers)
-    return {"value": world * dense_flops / (ms * 1e-3) / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": whole_job_tflops(dense_flops, world, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
             "api": "elsa_vit_linears_host (pinned host buffers; layers of equal shape share them)"}
 

@@ -48,6 +48,7 @@ def main():
     ap.add_argument("--out", default="gpurun_out/sweep.json")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--quick", action="store_true", help="rows = 4096 only")
+    ap.add_argument("--summary", default=None, help="also write a short markdown summary to this path")
     args = ap.parse_args()
     hbm, tf, kind = load_peaks()
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
@@ -96,6 +97,41 @@ def main():
         max(r["roofline_frac"] for r in lin)))
     print("compress points: %d, median GB/s %.0f, max %.0f" % (
         len(cmp_), statistics.median(r["gbs"] for r in cmp_), max(r["gbs"] for r in cmp_)))
+
+
+    if args.summary:
+        write_summary(args.summary, hbm, tf, kind, lin, cmp_)
+
+
+def write_summary(path, hbm, tf, kind, lin, cmp_):
+    med = statistics.median
+    out = ["# Shape / sparsity sweep (%d linear points, %d compress points) -- summary" % (len(lin), len(cmp_)), "",
+           "Command: `python -m paper_2409_09708_b200.sweep --out gpurun_out/sweep.json --summary <this file>` (B200;",
+           "median of 5 CUDA-event timings per point, 512 MB written between repetitions to flush the 126 MB L2;",
+           "time = weight-image rebuild + GEMM of `elsa_nm_linear` under the automatic dispatch).",
+           "Peaks (%s): %.1f GB/s, %.1f TFLOP/s." % (kind, hbm, tf), "",
+           "Median fraction of the per-point roofline, max(kept FLOPs / tensor peak, algorithmic bytes / HBM peak),",
+           "by level and rows, both dtypes and all five (K, O) shapes:", "",
+           "| level | rows 4096 | rows 16384 | rows 65536 |", "|---|---|---|---|"]
+    for lv in ["%d:%d" % nm for nm in synth.SWEEP_LEVELS]:
+        row = [lv]
+        for R in synth.SWEEP_ROWS:
+            v = [r["roofline_frac"] for r in lin if r["level"] == lv and r["rows"] == R]
+            row.append("%.2f" % med(v) if v else "-")
+        out.append("| " + " | ".join(row) + " |")
+    out += ["", "Dense-equivalent TFLOP/s at rows 65536, median over dtypes, per (K, O) for 2:8 / 4:8:", ""]
+    for K, O in synth.SWEEP_SHAPES:
+        vals = []
+        for lv in ("2:8", "4:8"):
+            v = [r["dense_equiv_tflops"] for r in lin if r["rows"] == 65536 and r["in"] == K and r["out"] == O and r["level"] == lv]
+            vals.append("%.0f" % med(v) if v else "-")
+        out.append("- K=%d, O=%d: %s / %s" % (K, O, vals[0], vals[1]))
+    out += ["", "elsa_nm_compress (bytes read + written / time, cold L2): median %.0f GB/s, best %.0f GB/s; the weights"
+            % (med(r["gbs"] for r in cmp_), max(r["gbs"] for r in cmp_)),
+            "are 1.2-8.4 MB, so a single launch lasts a few microseconds and is latency-bound; tables of weights go",
+            "through `elsa_vit_compress`, one launch for all of them.", ""]
+    with open(path, "w") as f:
+        f.write("\n".join(out))
 
 
 if __name__ == "__main__":

@@ -98,6 +98,21 @@ def test_vit_linears_reports_the_layer(lib):
     assert lib.elsa_vit_workspace_bytes(table, 0) == lib.elsa_workspace_bytes(4, 8, 8, 2, 4)
 
 
+def test_vit_compress_reports_the_weight(lib):
+    table = (lib.ElsaWeight * 3)()
+    for t in table:
+        t.W, t.vals, t.idx = FAKE, FAKE, FAKE
+        t.out, t.in_, t.N, t.M = 8, 16, 2, 8
+    table[2].in_ = 20                                       # not a multiple of M
+    assert lib._vit_compress(table, 3, 0, None) == 2
+    assert lib.elsa_last_error().startswith("weight 2:")
+    table[2].in_ = 16
+    table[1].idx = None
+    assert lib._vit_compress(table, 3, 0, None) == 1 and lib.elsa_last_error().startswith("weight 1:")
+    assert lib._vit_compress(None, 3, 0, None) == 1
+    assert lib._vit_compress(table, 0, 0, None) == 2
+
+
 def test_variant_switch_and_launch_counter(lib):
     assert lib.elsa_get_linear_variant() == lib.VARIANT_AUTO
     lib.elsa_set_linear_variant(lib.VARIANT_SIMT)

@@ -296,6 +296,52 @@ def test_swin_b_stack_full_size_sampled_rows(lib):
     stack_check(lib, layers, synth.torch_dtype(dt), 24, 41)
 
 
+def test_shared_launches_give_the_same_bits_as_one_launch_per_layer(lib):
+    """elsa_vit_linears with per-layer scratch (layers share persistent launches) against the same
+    table run layer by layer, on a table that mixes all three tensor-core families."""
+    dtype = torch.bfloat16
+    code = lib.dtype_code(dtype)
+    layers = [synth.Layer("sparse_a", 9000, 768, 768, 2, 8, 201, 202, 203),
+              synth.Layer("dense_pair_a", 19000, 256, 384, 4, 8, 204, 205, 206),
+              synth.Layer("small", 150, 128, 64, 1, 4, 207, 208, 209),
+              synth.Layer("dense_level", 19000, 512, 256, 8, 8, 210, 211, 212),
+              synth.Layer("sparse_b", 9000, 1024, 512, 1, 16, 213, 214, 215),
+              synth.Layer("dense_pair_b", 20000, 128, 1000, 3, 8, 216, 217, 218)]
+    dev = []
+    for l in layers:
+        X, W, b = synth.layer_tensors(l, dtype, device="cuda")
+        vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+        dev.append(dict(X=X, W=W, vals=vals, idx=idx, bias=b, N=l.N, M=l.M,
+                        Y=torch.empty((l.rows, l.out), dtype=dtype, device="cuda")))
+    table = lib.make_layer_table(dev)
+    ws = lib.alloc_workspace(lib.elsa_vit_workspace_bytes(table, code))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    lib.elsa_vit_linears(table, code, ws, dev_status=status)
+    torch.cuda.synchronize()
+    shared = [d["Y"].clone() for d in dev]
+    for d in dev:
+        d["Y"].zero_()
+    lib.elsa_set_grouping(False)
+    try:
+        lib.elsa_vit_linears(table, code, ws, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        lib.elsa_set_grouping(True)
+    assert int(status.item()) == 0
+    for l, d, y in zip(layers, dev, shared):
+        assert torch.equal(d["Y"], y), l.name
+        pick = torch.from_numpy(synth.sample_rows(l.rows, 40, 77)).cuda()
+        check_close(y[pick], oracle_linear(d["X"][pick].cpu(), d["W"].cpu(), d["bias"].cpu(), l.N, l.M, dtype))
+    # a scratch of only the largest layer's size still works: the layers then run one after the other
+    small_ws = lib.alloc_workspace(max(lib.elsa_workspace_bytes(l.rows, l.in_, l.out, l.N, l.M, code) for l in layers))
+    for d in dev:
+        d["Y"].zero_()
+    lib.elsa_vit_linears(table, code, small_ws, dev_status=status)
+    torch.cuda.synchronize()
+    for d, y in zip(dev, shared):
+        assert torch.equal(d["Y"], y)
+
+
 def test_host_memory_entry_point_matches_device_entry_point(lib):
     dtype = torch.float16
     layers = [synth.Layer("a", 300, 256, 384, 2, 8, 1, 2, 3), synth.Layer("b", 300, 384, 128, 4, 4, 4, 5, 6),
