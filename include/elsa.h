@@ -175,9 +175,12 @@ size_t elsa_vit_host_device_bytes(const elsa_host_layer* cfg, int n_layers, elsa
  * The whole path from host memory (Sec. 3.1 projection, then Sec. 2 product, per layer of the
  * table): for each layer copy W, bias and X to the device, compress W to its level, multiply,
  * and copy Y back.  `device_mem` is caller-owned device memory of at least
- * elsa_vit_host_device_bytes(...) bytes, 256-byte aligned.  Copies are cudaMemcpyAsync on
- * `stream`: with pinned host memory the call returns after enqueue and Y is valid once the
- * stream has been synchronised.
+ * elsa_vit_host_device_bytes(...) bytes (two slots, so that one layer's copies overlap its
+ * neighbours' kernels), 256-byte aligned.  Copies in and out run on two streams the library creates
+ * once per device (no device memory is allocated) and are ordered against the kernels on `stream`
+ * by events; `stream` itself waits for the last copy out, so with pinned host memory the call
+ * returns after enqueue and every Y is valid once `stream` has been synchronised.  One call at a
+ * time per device.
  */
 elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype,
                                   void* device_mem, size_t device_bytes, uint32_t* dev_status,

@@ -454,12 +454,44 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
     return ELSA_OK;
 }
 
-// Device memory plan of the host-memory variant: regions reused by every layer, each sized for
-// the largest layer: X | Y | W | bias | vals | idx | linear workspace.
+// Device memory plan of the host-memory variant: two slots, used by alternate layers so that the
+// copies of one layer overlap the kernels of its neighbours; each slot holds regions sized for the
+// largest layer: X | Y | W | bias | vals | idx | linear workspace.
 namespace {
 struct HostPlan {
-    size_t x, y, w, bias, vals, idx, ws, total;
+    size_t x, y, w, bias, vals, idx, ws, slot, total;
 };
+
+// Copy streams and ordering events of the host-memory variant, created once per device.
+struct HostPipe {
+    cudaStream_t in, out;
+    cudaEvent_t start, in_done[2], compute_done[2], out_done[2];
+    bool ready;
+};
+HostPipe g_pipe[64];
+std::mutex g_pipe_mutex;
+
+elsa_status host_pipe(int device, HostPipe** pipe)
+{
+    std::lock_guard<std::mutex> lock(g_pipe_mutex);
+    HostPipe& p = g_pipe[device & 63];
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.in, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.out, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < 2; ++i)
+            ok = cudaEventCreateWithFlags(&p.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.compute_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.out_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "creating the copy streams: %s", cudaGetErrorString(e));
+        }
+        p.ready = true;
+    }
+    *pipe = &p;
+    return ELSA_OK;
+}
 bool host_plan(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype, HostPlan* plan)
 {
     size_t mx = 0, my = 0, mw = 0, mb = 0, mv = 0, mi = 0, ms = 0;
@@ -483,7 +515,8 @@ bool host_plan(const elsa_host_layer* cfg, int n_layers, elsa_dtype dtype, HostP
     plan->vals = off; off += round_up(mv, 256);
     plan->idx = off; off += round_up(mi, 256);
     plan->ws = off; off += round_up(ms, 256);
-    plan->total = off;
+    plan->slot = off;
+    plan->total = 2 * off;
     return true;
 }
 }  // namespace
@@ -521,25 +554,56 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
     if (st != ELSA_OK) return st;
 
     cudaStream_t stream = (cudaStream_t)stream_;
-    uint8_t* base = (uint8_t*)device_mem;
+    HostPipe* pipe = nullptr;
+    if ((st = host_pipe(dev.device, &pipe)) != ELSA_OK) return st;
+    // Three queues: host-to-device copies, kernels (the caller's stream), device-to-host copies.  Layer l
+    // uses slot l % 2; events order a slot's copy-in after the kernels that last read it, its kernels after
+    // its copy-in and after the copy-out that last read its Y, and its copy-out after its kernels.
+    auto cuda_fail = [](cudaError_t e, int l, const char* what) {
+        cudaGetLastError();
+        set_profile_layer(-1);
+        return fail(ELSA_ERR_CUDA, "layer %d: %s: %s", l, what, cudaGetErrorString(e));
+    };
+    cudaError_t e = cudaEventRecord(pipe->start, stream);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->in, pipe->start, 0);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->out, pipe->start, 0);
+    if (e != cudaSuccess) return cuda_fail(e, 0, "ordering the copy streams");
     for (int l = 0; l < n_layers; ++l) {
         const elsa_host_layer& c = cfg[l];
+        const int slot = l & 1;
+        uint8_t* base = (uint8_t*)device_mem + (size_t)slot * plan.slot;
         set_profile_layer(l);
         void* dX = base + plan.x; void* dY = base + plan.y; void* dW = base + plan.w;
         void* dB = c.bias ? base + plan.bias : nullptr;
         void* dV = base + plan.vals; uint32_t* dI = c.N == c.M ? nullptr : (uint32_t*)(base + plan.idx);
-        cudaError_t e = cudaMemcpyAsync(dW, c.W, (size_t)c.out * c.in * 2, cudaMemcpyHostToDevice, stream);
-        if (e == cudaSuccess && c.bias) e = cudaMemcpyAsync(dB, c.bias, (size_t)c.out * 2, cudaMemcpyHostToDevice, stream);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(dX, c.X, (size_t)c.rows * c.in * 2, cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "layer %d: host-to-device copy: %s", l, cudaGetErrorString(e));
+        // copy-in
+        e = cudaSuccess;
+        if (l >= 2) e = cudaStreamWaitEvent(pipe->in, pipe->compute_done[slot], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dW, c.W, (size_t)c.out * c.in * 2, cudaMemcpyHostToDevice, pipe->in);
+        if (e == cudaSuccess && c.bias) e = cudaMemcpyAsync(dB, c.bias, (size_t)c.out * 2, cudaMemcpyHostToDevice, pipe->in);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dX, c.X, (size_t)c.rows * c.in * 2, cudaMemcpyHostToDevice, pipe->in);
+        if (e == cudaSuccess) e = cudaEventRecord(pipe->in_done[slot], pipe->in);
+        if (e != cudaSuccess) return cuda_fail(e, l, "host-to-device copy");
+        // kernels
+        e = cudaStreamWaitEvent(stream, pipe->in_done[slot], 0);
+        if (e == cudaSuccess && l >= 2) e = cudaStreamWaitEvent(stream, pipe->out_done[slot], 0);
+        if (e != cudaSuccess) return cuda_fail(e, l, "ordering the kernels");
         if ((st = launch_compress((const uint16_t*)dW, c.out, c.in, c.N, c.M, (uint16_t*)dV, dI, stream)) != ELSA_OK) return st;
         if ((st = run_linear(dX, c.rows, dV, dI, dB, c.out, c.in, c.N, c.M, dtype, dY, base + plan.ws, dev_status,
                              stream)) != ELSA_OK)
             return st;
-        e = cudaMemcpyAsync(c.Y, dY, (size_t)c.rows * c.out * 2, cudaMemcpyDeviceToHost, stream);
-        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "layer %d: device-to-host copy: %s", l, cudaGetErrorString(e));
+        e = cudaEventRecord(pipe->compute_done[slot], stream);
+        // copy-out
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(pipe->out, pipe->compute_done[slot], 0);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(c.Y, dY, (size_t)c.rows * c.out * 2, cudaMemcpyDeviceToHost, pipe->out);
+        if (e == cudaSuccess) e = cudaEventRecord(pipe->out_done[slot], pipe->out);
+        if (e != cudaSuccess) return cuda_fail(e, l, "device-to-host copy");
     }
     set_profile_layer(-1);
+    // the caller's stream is complete only when the last copies out are
+    e = cudaStreamWaitEvent(stream, pipe->out_done[(n_layers - 1) & 1], 0);
+    if (e == cudaSuccess && n_layers >= 2) e = cudaStreamWaitEvent(stream, pipe->out_done[n_layers & 1], 0);
+    if (e != cudaSuccess) return cuda_fail(e, n_layers - 1, "joining the copy streams");
     return ELSA_OK;
 }
 
