@@ -42,7 +42,8 @@ constexpr int kEpiCols = 32;
 constexpr int kMaxChunksPerWarp = kMaxBlockN / kEpiCols / 2;   // two warps per TMEM lane quarter share the chunks
 constexpr int kATileBytes = kRowsPerCta * kBlockK * 2;
 constexpr int kStagingBytes = 32 * kEpiCols * 2;
-constexpr int kStagingTotal = kEpiWarps * 2 * kStagingBytes;
+constexpr int kStagingBufs = 1;     // one staging buffer per epilogue warp: the shared memory goes to a sixth pipeline stage instead
+constexpr int kStagingTotal = kEpiWarps * kStagingBufs * kStagingBytes;
 constexpr int kBiasBytes = kEpiWarps * kMaxBlockN * 4;
 constexpr int kBarrierBytes = 256;
 
@@ -195,7 +196,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int ew = warp - 2;                // private staging / bias slot
         const int half = ew >> 2;               // which of the two warps of the quarter: even or odd chunks
-        const uint32_t stage_buf = staging_base + (uint32_t)(ew * 2 * kStagingBytes);
+        const uint32_t stage_buf = staging_base + (uint32_t)(ew * kStagingBufs * kStagingBytes);
         float* bias_s = reinterpret_cast<float*>(smem_gen + bias_off) + ew * kMaxBlockN;
         const uint32_t empty_remote = mapa_shared(tmem_empty_bar, 0);
         int acc = 0;
@@ -233,8 +234,8 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     const float2 b = *reinterpret_cast<const float2*>(bias_s + c * kEpiCols + 2 * j);
                     packed[j] = pack2<kBf16>(__uint_as_float(r[2 * j]) + b.x, __uint_as_float(r[2 * j + 1]) + b.y);
                 }
-                const uint32_t buf = stage_buf + (chunk_counter & 1u) * kStagingBytes;
-                if (lane == 0) bulk_wait_group_read<1>();   // the store two chunks ago has drained this buffer
+                const uint32_t buf = stage_buf + (chunk_counter % kStagingBufs) * kStagingBytes;
+                if (lane == 0) bulk_wait_group_read<kStagingBufs - 1>();   // the store that last used this buffer has drained it
                 __syncwarp();
                 const uint32_t row_addr = buf + (uint32_t)(lane * 64);
                 const uint32_t sw = (uint32_t)((lane >> 1) & 3);   // 64-byte swizzle of the staging rows
