@@ -131,6 +131,28 @@ typedef struct {
  */
 elsa_status elsa_vit_compress(const elsa_weight* w, int n_weights, elsa_dtype dtype, void* stream);
 
+/*
+ * Sec. 3.1, subset-superset relation: all levels N:M of a supernet layer share one weight, and the
+ * magnitude ranks inside a group do not depend on N.  This call reads W once and writes the packed
+ * form of every requested level N_list[l]:M (same M), each bit-identical to what elsa_nm_compress
+ * writes for that level.  `N_list`, `vals` and `idx` are HOST arrays of n_levels entries holding
+ * device pointers (idx[l] may be NULL iff N_list[l] == M); n_levels <= 16.
+ */
+elsa_status elsa_nm_compress_levels(const void* W, int out, int in, int M, const int* N_list, int n_levels,
+                                    elsa_dtype dtype, void* const* vals, uint32_t* const* idx, void* stream);
+
+/*
+ * Sec. 3.1 "dynamic masking" as the supernet's forward uses it (Alg. 2: the shared weight is
+ * projected to the sampled level on every step): Y = X * (W_sup projected onto N:M)^T + bias
+ * straight from the dense shared weight W_sup [out][in], with no packed copy.  The projection is
+ * the one elsa_nm_compress defines, so the result equals elsa_nm_linear on the packed form of
+ * W_sup at that level (bit for bit when both take the same kernel family).  `workspace` as for
+ * elsa_nm_linear (elsa_workspace_bytes of the same shape and level).
+ */
+elsa_status elsa_nm_linear_masked(const void* X, int rows, const void* W_sup, const void* bias, int out, int in,
+                                  int N, int M, elsa_dtype dtype, void* Y, void* workspace,
+                                  size_t workspace_bytes, uint32_t* dev_status, void* stream);
+
 /* One linear module of the per-layer table (Sec. 3: configuration alpha = (s^1 .. s^L)). */
 typedef struct {
     const void* X;       /* [rows][in]  device */

@@ -64,6 +64,9 @@ _unpack = _sig("elsa_nm_unpack", _i, [_vp, _vp, _i, _i, _i, _i, _i, _vp, _vp])
 _linear = _sig("elsa_nm_linear", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
 _linear_static = _sig("elsa_nm_linear_static", _i, [_vp, _i, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 STATIC_SCRATCH_BYTES = 8 << 20
+_compress_levels = _sig("elsa_nm_compress_levels", _i, [_vp, _i, _i, _i, ctypes.POINTER(_i), _i, _i,
+                                                        ctypes.POINTER(_vp), ctypes.POINTER(_vp), _vp])
+_linear_masked = _sig("elsa_nm_linear_masked", _i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
 _vit_compress = _sig("elsa_vit_compress", _i, [ctypes.POINTER(ElsaWeight), _i, _i, _vp])
 _vit_ws = _sig("elsa_vit_workspace_bytes", _sz, [ctypes.POINTER(ElsaLayer), _i, _i])
 _vit = _sig("elsa_vit_linears", _i, [ctypes.POINTER(ElsaLayer), _i, _i, _vp, _sz, _vp, _vp])
@@ -178,6 +181,33 @@ def elsa_nm_compress(W: torch.Tensor, N: int, M: int, vals=None, idx=None, strea
         vals, idx = alloc_packed(out, in_, N, M, W.dtype, W.device)
     _check(_compress(_ptr(W), out, in_, N, M, dtype_code(W.dtype), _ptr(vals), _ptr(idx), _stream(stream)))
     return vals, idx
+
+
+def elsa_nm_compress_levels(W: torch.Tensor, N_list, M: int, stream=None):
+    """Packed (vals, idx) of W at every level N:M of N_list, from one read of W."""
+    out, in_ = W.shape
+    packed = [alloc_packed(out, in_, N, M, W.dtype, W.device) for N in N_list]
+    n = len(N_list)
+    Ns = (_i * n)(*N_list)
+    vals = (_vp * n)(*[_ptr(v) for v, _ in packed])
+    idx = (_vp * n)(*[_ptr(i) for _, i in packed])
+    _check(_compress_levels(_ptr(W), out, in_, M, Ns, n, dtype_code(W.dtype), vals, idx, _stream(stream)))
+    return packed
+
+
+def elsa_nm_linear_masked(X: torch.Tensor, W_sup: torch.Tensor, bias, N: int, M: int, Y=None, workspace=None,
+                          dev_status=None, stream=None):
+    """Y = X . (W_sup projected onto N:M)^T + bias straight from the dense shared weight."""
+    rows, in_ = X.shape
+    out = W_sup.shape[0]
+    code = dtype_code(X.dtype)
+    if Y is None:
+        Y = torch.empty((rows, out), dtype=X.dtype, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(elsa_workspace_bytes(rows, in_, out, N, M, code), X.device)
+    _check(_linear_masked(_ptr(X), rows, _ptr(W_sup), _ptr(bias), out, in_, N, M, code, _ptr(Y), _ptr(workspace),
+                          workspace.numel(), _ptr(dev_status), _stream(stream)))
+    return Y
 
 
 def elsa_nm_unpack(vals: torch.Tensor, idx, out: int, in_: int, N: int, M: int, W_masked=None, stream=None):

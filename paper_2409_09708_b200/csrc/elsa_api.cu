@@ -275,6 +275,72 @@ elsa_status elsa_nm_linear(const void* X, int rows, const void* vals, const uint
                       (cudaStream_t)stream);
 }
 
+elsa_status elsa_nm_compress_levels(const void* W, int out, int in, int M, const int* N_list, int n_levels,
+                                    elsa_dtype dtype, void* const* vals, uint32_t* const* idx, void* stream)
+{
+    if (!W || !N_list || !vals || !idx) return fail(ELSA_ERR_NULL, "W, N_list, vals and idx must not be NULL");
+    if (n_levels < 1 || n_levels > kMaxLevels)
+        return fail(ELSA_ERR_SHAPE, "n_levels=%d is outside 1..%d", n_levels, kMaxLevels);
+    if (!aligned16(W)) return fail(ELSA_ERR_ALIGN, "W must be 16-byte aligned");
+    LevelTable t;
+    t.n = n_levels;
+    for (int l = 0; l < n_levels; ++l) {
+        elsa_status st = check_level(out, in, N_list[l], M, dtype);
+        if (st == ELSA_OK && !vals[l]) st = fail(ELSA_ERR_NULL, "vals must not be NULL");
+        if (st == ELSA_OK && N_list[l] != M && !idx[l]) st = fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+        if (st == ELSA_OK && (!aligned16(vals[l]) || (idx[l] && !aligned16(idx[l]))))
+            st = fail(ELSA_ERR_ALIGN, "vals and idx must be 16-byte aligned");
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "level %d: %s", l, msg);
+        }
+        t.N[l] = N_list[l];
+        t.vals[l] = (uint16_t*)vals[l];
+        t.idx[l] = N_list[l] == M ? nullptr : idx[l];
+    }
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    return launch_compress_levels((const uint16_t*)W, out, in, M, t, (cudaStream_t)stream);
+}
+
+elsa_status elsa_nm_linear_masked(const void* X, int rows, const void* W_sup, const void* bias, int out, int in,
+                                  int N, int M, elsa_dtype dtype, void* Y, void* workspace, size_t workspace_bytes,
+                                  uint32_t* dev_status, void* stream_)
+{
+    // the dense weight takes the place of vals in the checks (same alignment rules), no index words
+    uint32_t* no_idx = N == M ? nullptr : (uint32_t*)W_sup;
+    elsa_status st = check_linear(X, rows, W_sup, no_idx, bias, out, in, N, M, dtype, Y, workspace, workspace_bytes);
+    if (st != ELSA_OK) return st;
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != ELSA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    LinearKind kind;
+    if ((st = pick_kind(rows, out, in, N, M, dev.sm_count, &kind)) != ELSA_OK) return st;
+    if (kind == KIND_SIMT || kind == KIND_SPARSE_ONE)
+        return fail(ELSA_ERR_NM, "the forced variant has no mask-on-load form");
+    if (kind == KIND_SPARSE_PAIR) {
+        uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
+        if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, (uint16_t*)workspace, meta, stream)) != ELSA_OK)
+            return st;
+        SparseJob job;
+        job.X = (const uint16_t*)X; job.bias = (const uint16_t*)bias; job.Y = (uint16_t*)Y; job.workspace = workspace;
+        job.rows = rows; job.in = in; job.out = out;
+        return launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
+    }
+    const uint16_t* Wd = (const uint16_t*)W_sup;     // the dense level multiplies the shared weight as it is
+    if (N != M) {
+        if ((st = launch_mask((const uint16_t*)W_sup, out, in, N, M, (uint16_t*)workspace, stream)) != ELSA_OK) return st;
+        Wd = (const uint16_t*)workspace;
+    }
+    if (kind == KIND_DENSE_PAIR)
+        return launch_linear_tc_pair((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype, (uint16_t*)Y,
+                                     dev_status, stream);
+    return launch_linear_tc_dense((const uint16_t*)X, rows, Wd, (const uint16_t*)bias, out, in, dtype, (uint16_t*)Y,
+                                  dev_status, stream);
+}
+
 elsa_status elsa_vit_compress(const elsa_weight* w, int n_weights, elsa_dtype dtype, void* stream)
 {
     if (!w) return fail(ELSA_ERR_NULL, "w must not be NULL");

@@ -35,6 +35,31 @@ nm_unpack_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__
     unpack_group<M>(vals, idx, in, N, Wm, words_per_row, gid);
 }
 
+// All requested levels N:M of one weight from a single read of it (the ranks do not depend on N).
+template <int M>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+nm_compress_levels_kernel(const uint16_t* __restrict__ W, int out, int in, const LevelTable t, int segs_per_row)
+{
+    __shared__ uint32_t words[kWarpsPerBlock][kMaxIndexWordsPerSegment];
+    const long long seg_id = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    if (seg_id >= (long long)out * segs_per_row) return;
+    compress_segment_levels<M>(W, in, t.n, t.N, t.vals, t.idx, segs_per_row, seg_id, words);
+}
+
+// Dense weight projected onto level N:M, still dense (pruned positions +0.0).
+template <int M>
+__global__ void __launch_bounds__(256)
+nm_mask_kernel(const uint16_t* __restrict__ W, long long groups, int N, uint16_t* __restrict__ Wm)
+{
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    if (gid >= groups) return;
+    mask_group<M>(W, N, Wm, gid);
+}
+
 // ---- batched forms: one launch over a table of weights.  A unit is a warp segment (compress) or a
 // thread (weight-image kernels); every block looks its first unit up in the table's prefix sums.
 
@@ -127,6 +152,30 @@ elsa_status launch_unpack(const uint16_t* vals, const uint32_t* idx, int out, in
     else
         launch_pdl(nm_unpack_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, Wm, wpr);
     return launched("nm_unpack");
+}
+
+elsa_status launch_compress_levels(const uint16_t* W, int out, int in, int M, const LevelTable& t, cudaStream_t stream)
+{
+    const int segs_per_row = (in / M + 31) / 32;
+    const long long total = (long long)out * segs_per_row;
+    const unsigned grid = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    const dim3 block(kWarpsPerBlock * 32);
+    ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
+    if (M == 4) launch_pdl(nm_compress_levels_kernel<4>, dim3(grid), block, 0, stream, 1, W, out, in, t, segs_per_row);
+    else if (M == 8) launch_pdl(nm_compress_levels_kernel<8>, dim3(grid), block, 0, stream, 1, W, out, in, t, segs_per_row);
+    else launch_pdl(nm_compress_levels_kernel<16>, dim3(grid), block, 0, stream, 1, W, out, in, t, segs_per_row);
+    return launched("nm_compress (levels)");
+}
+
+elsa_status launch_mask(const uint16_t* W, int out, int in, int N, int M, uint16_t* Wm, cudaStream_t stream)
+{
+    const long long groups = (long long)out * (in / M);
+    const unsigned grid = (unsigned)((groups + 255) / 256);
+    ProfileScope scope(ELSA_KERNEL_WEIGHT_IMAGES, stream);
+    if (M == 4) launch_pdl(nm_mask_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, W, groups, N, Wm);
+    else if (M == 8) launch_pdl(nm_mask_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, W, groups, N, Wm);
+    else launch_pdl(nm_mask_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, W, groups, N, Wm);
+    return launched("nm_mask");
 }
 
 // ---- batched launchers

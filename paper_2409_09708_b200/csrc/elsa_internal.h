@@ -127,6 +127,19 @@ elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, els
                                                cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
 size_t linear_tc_sparse_workspace(int out, int in);
+// Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
+constexpr int kMaxLevels = 16;
+struct LevelTable {
+    int n;
+    int N[kMaxLevels];
+    uint16_t* vals[kMaxLevels];
+    uint32_t* idx[kMaxLevels];
+};
+elsa_status launch_compress_levels(const uint16_t* W, int out, int in, int M, const LevelTable& t, cudaStream_t stream);
+elsa_status launch_mask(const uint16_t* W, int out, int in, int N, int M, uint16_t* Wm, cudaStream_t stream);
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, uint16_t* a_img,
+                                 uint8_t* meta, cudaStream_t stream);
+
 // Batched weight-format kernels: one launch over a table of weights (kernel-parameter space).
 enum BatchKind { BATCH_COMPRESS = 0, BATCH_UNPACK = 1, BATCH_TO_SP24 = 2 };
 struct BatchItem {

@@ -33,11 +33,45 @@ __device__ __forceinline__ void load_group(const uint16_t* p, uint16_t (&w)[M])
 // One warp compresses 32 consecutive groups of one row, one group per lane.  The 32 groups own
 // exactly N*b whole index words of the row's bitstream, so each warp assembles its words in shared
 // memory and writes them with one coalesced store.
+// Ranks of the M magnitudes of one group, 4 bits each: rank_i = #{j : |w_j| > |w_i|} + #{j < i : |w_j| == |w_i|}
+// (larger magnitude first, lower position first among equals).  Magnitudes are compared as the 15 low
+// bits of the pattern.  The level N keeps exactly the elements with rank < N, for every N at once.
 template <int M>
-__device__ __forceinline__ void compress_segment(const uint16_t* __restrict__ W, int in, int N,
-                                                 uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
-                                                 int segs_per_row, int words_per_row, long long seg_id,
-                                                 uint32_t (*words)[kMaxIndexWordsPerSegment])
+__device__ __forceinline__ unsigned long long group_ranks(const uint16_t (&w)[M])
+{
+    unsigned long long ranks = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        const uint32_t ki = w[i] & 0x7FFFu;
+        int rank = 0;
+#pragma unroll
+        for (int j = 0; j < M; ++j) {
+            const uint32_t kj = w[j] & 0x7FFFu;
+            rank += (kj > ki) || (j < i && kj == ki);
+        }
+        ranks |= (unsigned long long)rank << (4 * i);
+    }
+    return ranks;
+}
+
+template <int M>
+__device__ __forceinline__ uint32_t keep_mask(unsigned long long ranks, int N)
+{
+    uint32_t keep = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) keep |= (uint32_t)((int)((ranks >> (4 * i)) & 15ull) < N) << i;
+    return keep;
+}
+
+// One warp compresses 32 consecutive groups of one row, one group per lane, to each of `n_levels`
+// levels N_list[l]:M (one read of W, ranks computed once).  The 32 groups own exactly N*b whole index
+// words of the row's bitstream, so the warp assembles its words in shared memory and writes them with
+// one coalesced store.
+template <int M>
+__device__ __forceinline__ void compress_segment_levels(const uint16_t* __restrict__ W, int in, int n_levels,
+                                                        const int* N_list, uint16_t* const* vals_list,
+                                                        uint32_t* const* idx_list, int segs_per_row, long long seg_id,
+                                                        uint32_t (*words)[kMaxIndexWordsPerSegment])
 {
     constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
     const int lane = threadIdx.x & 31;
@@ -48,64 +82,99 @@ __device__ __forceinline__ void compress_segment(const uint16_t* __restrict__ W,
     const int groups_per_row = in / M;
     const int g = seg * 32 + lane;
     const bool valid = g < groups_per_row;
-    const int seg_words = N * B;  // index words this segment owns (when N < M)
 
-    if (words_per_row) {
-        for (int w = lane; w < seg_words; w += 32) words[warp][w] = 0;
-        __syncwarp();
+    uint16_t w[M];
+    unsigned long long ranks = 0;
+    if (valid) {
+        load_group<M>(W + (size_t)o * in + (size_t)g * M, w);
+        ranks = group_ranks<M>(w);
     }
 
-    if (valid) {
-        uint16_t w[M];
-        load_group<M>(W + (size_t)o * in + (size_t)g * M, w);
-
-        // rank_i = #{j : |w_j| > |w_i|} + #{j < i : |w_j| == |w_i|}; keep iff rank_i < N.
-        // Magnitudes are compared as the 15 low bits of the pattern.
-        uint32_t keep = 0;
-#pragma unroll
-        for (int i = 0; i < M; ++i) {
-            const uint32_t ki = w[i] & 0x7FFFu;
-            int rank = 0;
-#pragma unroll
-            for (int j = 0; j < M; ++j) {
-                const uint32_t kj = w[j] & 0x7FFFu;
-                rank += (kj > ki) || (j < i && kj == ki);
-            }
-            keep |= (uint32_t)(rank < N) << i;
-        }
-
-        uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
-        unsigned long long fields = 0;
-        int t = 0;
-#pragma unroll
-        for (int i = 0; i < M; ++i) {
-            if ((keep >> i) & 1u) {
-                v[t] = w[i];
-                fields |= (unsigned long long)i << (t * B);
-                ++t;
-            }
-        }
+    for (int l = 0; l < n_levels; ++l) {
+        const int N = N_list[l];
+        uint16_t* vals = vals_list[l];
+        uint32_t* idx = idx_list[l];
+        const int words_per_row = (N == M) ? 0 : (groups_per_row * N * B + 31) / 32;
+        const int seg_words = N * B;  // index words this segment owns (when N < M)
 
         if (words_per_row) {
-            const int bit0 = lane * seg_words;  // bit offset of this group's fields in the segment
-            const int w0 = bit0 >> 5, sh = bit0 & 31;
-            // up to 60 bits shifted by up to 31: three words at most
-            const uint32_t lo = (uint32_t)(fields << sh);
-            const uint32_t mid = (uint32_t)(fields >> (32 - sh));
-            const uint32_t hi = sh ? (uint32_t)(fields >> (64 - sh)) : 0u;
-            // a zero part may lie past the segment's last word and is skipped
-            if (lo) atomicOr(&words[warp][w0], lo);
-            if (mid) atomicOr(&words[warp][w0 + 1], mid);
-            if (hi) atomicOr(&words[warp][w0 + 2], hi);
+            for (int k = lane; k < seg_words; k += 32) words[warp][k] = 0;
+            __syncwarp();
+        }
+        if (valid) {
+            const uint32_t keep = keep_mask<M>(ranks, N);
+            uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
+            unsigned long long fields = 0;
+            int t = 0;
+#pragma unroll
+            for (int i = 0; i < M; ++i) {
+                if ((keep >> i) & 1u) {
+                    v[t] = w[i];
+                    fields |= (unsigned long long)i << (t * B);
+                    ++t;
+                }
+            }
+            if (words_per_row) {
+                const int bit0 = lane * seg_words;  // bit offset of this group's fields in the segment
+                const int w0 = bit0 >> 5, sh = bit0 & 31;
+                // up to 60 bits shifted by up to 31: three words at most
+                const uint32_t lo = (uint32_t)(fields << sh);
+                const uint32_t mid = (uint32_t)(fields >> (32 - sh));
+                const uint32_t hi = sh ? (uint32_t)(fields >> (64 - sh)) : 0u;
+                // a zero part may lie past the segment's last word and is skipped
+                if (lo) atomicOr(&words[warp][w0], lo);
+                if (mid) atomicOr(&words[warp][w0 + 1], mid);
+                if (hi) atomicOr(&words[warp][w0 + 2], hi);
+            }
+        }
+        if (words_per_row) {
+            __syncwarp();
+            const int first = seg * seg_words;
+            uint32_t* row = idx + (size_t)o * words_per_row;
+            for (int k = lane; k < seg_words && first + k < words_per_row; k += 32) row[first + k] = words[warp][k];
+            __syncwarp();
         }
     }
+}
 
-    if (words_per_row) {
-        __syncwarp();
-        const int first = seg * seg_words;
-        uint32_t* row = idx + (size_t)o * words_per_row;
-        for (int w = lane; w < seg_words && first + w < words_per_row; w += 32)
-            row[first + w] = words[warp][w];
+// Single level: the form elsa_nm_compress uses.
+template <int M>
+__device__ __forceinline__ void compress_segment(const uint16_t* __restrict__ W, int in, int N,
+                                                 uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                 int segs_per_row, int words_per_row, long long seg_id,
+                                                 uint32_t (*words)[kMaxIndexWordsPerSegment])
+{
+    (void)words_per_row;
+    uint16_t* vals_one = vals;
+    uint32_t* idx_one = idx;
+    compress_segment_levels<M>(W, in, 1, &N, &vals_one, &idx_one, segs_per_row, seg_id, words);
+}
+
+// One thread projects one group of the dense weight onto level N:M: kept values stay, the others
+// become +0.0 (the "dynamic masking" of Sec. 3.1 applied to the shared weight, with no packed form).
+template <int M>
+__device__ __forceinline__ void mask_group(const uint16_t* __restrict__ W, int N, uint16_t* __restrict__ Wm, long long gid)
+{
+    uint16_t w[M];
+    load_group<M>(W + (size_t)gid * M, w);
+    const uint32_t keep = keep_mask<M>(group_ranks<M>(w), N);
+    uint16_t* dst = Wm + (size_t)gid * M;
+    if constexpr (M == 4) {
+        uint2 r;
+        r.x = (keep & 1u ? w[0] : 0u) | ((uint32_t)(keep & 2u ? w[1] : 0u) << 16);
+        r.y = (keep & 4u ? w[2] : 0u) | ((uint32_t)(keep & 8u ? w[3] : 0u) << 16);
+        *reinterpret_cast<uint2*>(dst) = r;
+    } else {
+#pragma unroll
+        for (int q = 0; q < M / 8; ++q) {
+            uint32_t x[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int i = 8 * q + 2 * k;
+                x[k] = ((keep >> i) & 1u ? (uint32_t)w[i] : 0u) | (((keep >> (i + 1)) & 1u ? (uint32_t)w[i + 1] : 0u) << 16);
+            }
+            reinterpret_cast<uint4*>(dst)[q] = make_uint4(x[0], x[1], x[2], x[3]);
+        }
     }
 }
 
@@ -170,46 +239,14 @@ __device__ __forceinline__ void unpack_group(const uint16_t* __restrict__ vals, 
 // then emits, per aligned chunk of 4, two values with ascending positions (i0 < i1).  Pruned
 // positions are zero in the rebuilt segment, so a chunk with fewer than two kept weights simply
 // borrows a zero from another position.
-template <int M>
-__device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
-                                                int out, int in, int N, int words_per_row,
-                                                uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
-                                                int k_blocks, int steps_per_block, long long tid)
+// Second half of the 2-of-4 re-encoding: given 16 consecutive positions of a weight row with the pruned
+// ones already zero (d) and the kept set (keep), emits two values per aligned chunk of 4 (ascending
+// positions, a zero borrowed where fewer than two are kept) and the chunk nibbles as tensor memory wants them.
+__device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep, bool real, int o, int seg, int k0, int in,
+                                          uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int k_blocks,
+                                          int steps_per_block)
 {
     constexpr int kFeatTile = 128;
-    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
-    constexpr int G = 16 / M;                         // groups per 16-k segment
-    const int segs = k_blocks * steps_per_block * 2;  // 16-k segments per (padded) row
-    const int o = (int)(tid / segs);                  // padded row index
-    const int seg = (int)(tid % segs);
-    const int k0 = seg * 16;
-
-    uint16_t d[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) d[i] = 0;
-    uint32_t keep = 0;
-    const bool real = o < out && k0 < in;             // in is a multiple of 16 on this path
-    if (real) {
-        const int groups_per_row = in / M;
-        const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N);
-        const uint32_t* row = idx + (size_t)o * words_per_row;
-#pragma unroll
-        for (int gl = 0; gl < G; ++gl) {
-            const int g = k0 / M + gl;
-            for (int t = 0; t < N; ++t) {
-                const long long bit = ((long long)g * N + t) * B;
-                const int w0 = (int)(bit >> 5), sh = (int)(bit & 31);
-                uint32_t f = row[w0] >> sh;
-                if (sh + B > 32) f |= row[w0 + 1] << (32 - sh);
-                const int pos = gl * M + (int)(f & (uint32_t)(M - 1));
-                const uint16_t val = v[(size_t)g * N + t];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) d[i] = (i == pos) ? val : d[i];
-                keep |= 1u << pos;
-            }
-        }
-    }
-
     uint32_t nibbles = 0;
     uint16_t sel[8];
 #pragma unroll
@@ -250,6 +287,82 @@ __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ val
     if (steps_per_block == 2) meta16[2 * (word + 2) + hi] = 0;
 }
 
+
+
+// One thread per (weight row, 16 consecutive k) of a PACKED weight: rebuilds those 16 positions, then
+// emits their 2-of-4 form.
+template <int M>
+__device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
+                                                int out, int in, int N, int words_per_row,
+                                                uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
+                                                int k_blocks, int steps_per_block, long long tid)
+{
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    constexpr int G = 16 / M;                         // groups per 16-k segment
+    const int segs = k_blocks * steps_per_block * 2;  // 16-k segments per (padded) row
+    const int o = (int)(tid / segs);                  // padded row index
+    const int seg = (int)(tid % segs);
+    const int k0 = seg * 16;
+
+    uint16_t d[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) d[i] = 0;
+    uint32_t keep = 0;
+    const bool real = o < out && k0 < in;             // in is a multiple of 16 on this path
+    if (real) {
+        const int groups_per_row = in / M;
+        const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N);
+        const uint32_t* row = idx + (size_t)o * words_per_row;
+#pragma unroll
+        for (int gl = 0; gl < G; ++gl) {
+            const int g = k0 / M + gl;
+            for (int t = 0; t < N; ++t) {
+                const long long bit = ((long long)g * N + t) * B;
+                const int w0 = (int)(bit >> 5), sh = (int)(bit & 31);
+                uint32_t f = row[w0] >> sh;
+                if (sh + B > 32) f |= row[w0 + 1] << (32 - sh);
+                const int pos = gl * M + (int)(f & (uint32_t)(M - 1));
+                const uint16_t val = v[(size_t)g * N + t];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) d[i] = (i == pos) ? val : d[i];
+                keep |= 1u << pos;
+            }
+        }
+    }
+    sp24_emit(d, keep, real, o, seg, k0, in, a_img, meta16, k_blocks, steps_per_block);
+}
+
+// The same from the DENSE shared weight: the 16 positions are projected onto level N:M on the fly
+// (N <= 2), so the supernet's forward needs no packed copy of the weight.
+template <int M>
+__device__ __forceinline__ void dense_to_sp24_segment(const uint16_t* __restrict__ W, int out, int in, int N,
+                                                      uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
+                                                      int k_blocks, int steps_per_block, long long tid)
+{
+    constexpr int G = 16 / M;
+    const int segs = k_blocks * steps_per_block * 2;
+    const int o = (int)(tid / segs);
+    const int seg = (int)(tid % segs);
+    const int k0 = seg * 16;
+
+    uint16_t d[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) d[i] = 0;
+    uint32_t keep = 0;
+    const bool real = o < out && k0 < in;
+    if (real) {
+#pragma unroll
+        for (int gl = 0; gl < G; ++gl) {
+            uint16_t w[M];
+            load_group<M>(W + (size_t)o * in + k0 + gl * M, w);
+            const uint32_t kg = keep_mask<M>(group_ranks<M>(w), N);
+#pragma unroll
+            for (int i = 0; i < M; ++i) d[gl * M + i] = ((kg >> i) & 1u) ? w[i] : (uint16_t)0;
+            keep |= kg << (gl * M);
+        }
+    }
+    sp24_emit(d, keep, real, o, seg, k0, in, a_img, meta16, k_blocks, steps_per_block);
+}
 
 }  // namespace
 }  // namespace elsa

@@ -65,6 +65,18 @@ nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict_
     to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, tid);
 }
 
+template <int M>
+__global__ void __launch_bounds__(256)
+dense_to_sp24_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint16_t* __restrict__ a_img,
+                     uint16_t* __restrict__ meta16, int out_tiles, int k_blocks, int steps_per_block)
+{
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
+    dense_to_sp24_segment<M>(W, out, in, N, a_img, meta16, k_blocks, steps_per_block, tid);
+}
+
 // ------------------------------------------------------------------ GEMM
 
 struct SpParams {
@@ -277,6 +289,27 @@ elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out
         launch_pdl(nm_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
                    (uint16_t*)meta, tiles_f, k_blocks, steps);
     return launched("nm_to_sp24");
+}
+
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, uint16_t* a_img,
+                                 uint8_t* meta, cudaStream_t stream)
+{
+    const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
+    const int k_blocks = (in + block_k - 1) / block_k;
+    const int steps = block_k / kSpUmmaK;
+    const long long threads = (long long)tiles_f * kFeatTile * k_blocks * steps * 2;
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+    ProfileScope scope(ELSA_KERNEL_NM_TO_SP24, stream);
+    if (M == 4)
+        launch_pdl(dense_to_sp24_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
+                   tiles_f, k_blocks, steps);
+    else if (M == 8)
+        launch_pdl(dense_to_sp24_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
+                   tiles_f, k_blocks, steps);
+    else
+        launch_pdl(dense_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
+                   tiles_f, k_blocks, steps);
+    return launched("dense_to_sp24");
 }
 
 bool linear_tc_sparse_suits(int in, int N)

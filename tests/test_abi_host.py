@@ -113,6 +113,27 @@ def test_vit_compress_reports_the_weight(lib):
     assert lib._vit_compress(table, 0, 0, None) == 2
 
 
+def test_supernet_side_entry_points_validate_their_arguments(lib):
+    import ctypes
+    n = 2
+    Ns = (ctypes.c_int * n)(1, 2)
+    vals = (ctypes.c_void_p * n)(FAKE, FAKE)
+    idx = (ctypes.c_void_p * n)(FAKE, FAKE)
+    f = lib._compress_levels
+    assert f(None, 8, 16, 8, Ns, n, 0, vals, idx, None) == 1
+    assert f(FAKE, 8, 16, 8, Ns, 0, 0, vals, idx, None) == 2
+    assert f(FAKE, 8, 16, 8, Ns, 17, 0, vals, idx, None) == 2
+    assert f(FAKE, 8, 20, 8, Ns, n, 0, vals, idx, None) == 2 and lib.elsa_last_error().startswith("level 0:")
+    bad = (ctypes.c_int * n)(1, 9)
+    assert f(FAKE, 8, 16, 8, bad, n, 0, vals, idx, None) == 3 and lib.elsa_last_error().startswith("level 1:")
+    noidx = (ctypes.c_void_p * n)(FAKE, None)
+    assert f(FAKE, 8, 16, 8, Ns, n, 0, vals, noidx, None) == 1
+    g = lib._linear_masked
+    assert g(FAKE, 4, None, None, 8, 8, 2, 4, 0, FAKE, 0x20000, 1 << 20, None, None) == 1
+    assert g(FAKE, 4, FAKE, None, 8, 8, 5, 4, 0, FAKE, 0x20000, 1 << 20, None, None) == 3
+    assert g(FAKE, 4, FAKE, None, 8, 8, 2, 4, 0, FAKE, None, 0, None, None) == 6
+
+
 def test_variant_switch_and_launch_counter(lib):
     assert lib.elsa_get_linear_variant() == lib.VARIANT_AUTO
     lib.elsa_set_linear_variant(lib.VARIANT_SIMT)

@@ -384,3 +384,52 @@ def test_sweep_points_sampled_rows(lib, dt):
         ref = eo.nm_linear_f64(synth.bits(X[pick]), ovals, oidx, synth.bits(b), l.out, l.in_, l.N, l.M, ocode(dtype))
         assert int(status.item()) == 0
         check_close(Y[pick], ref)
+
+
+# ------------------------------------------------------------------ supernet-side forms (Sec. 3.1)
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("M,N_list", [(4, [1, 2, 3, 4]), (8, [1, 2, 3, 4, 8]), (16, [1, 2, 4, 8, 15, 16])])
+def test_all_levels_in_one_pass_match_the_oracle(lib, M, N_list, dtype):
+    """Shared weight, every level of the search space from one read: each level's packed form is the
+    oracle's, bit for bit (and the kept sets nest, Sec. 3.1)."""
+    W = synth.randn((72, 16 * 23), 300 + M, synth.W_STD, dtype)
+    Wb = synth.bits(W)
+    packed = lib.elsa_nm_compress_levels(W.cuda(), N_list, M)
+    torch.cuda.synchronize()
+    prev = None
+    for N, (vals, idx) in zip(N_list, packed):
+        ovals, oidx, omask = eo.nm_compress(Wb, N, M)
+        assert (synth.bits(vals) == ovals).all(), (N, M)
+        assert (idx_bits(idx, oidx) == oidx).all(), (N, M)
+        if prev is not None:
+            assert (omask >= prev).all()
+        prev = omask
+
+
+MASKED_CASES = [
+    # rows, in, out, N, M -> kernel family the automatic dispatch takes
+    (9000, 768, 512, 2, 8),      # 2:4 sparse MMA on CTA pairs, re-encoded from the dense weight
+    (9000, 1024, 256, 1, 16),    # the same, M = 16
+    (19000, 256, 384, 4, 8),     # dense-rate pair kernel on the masked image
+    (19000, 512, 256, 8, 8),     # dense level: the shared weight as it is
+    (197, 768, 768, 3, 8),       # small: one CTA per tile
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("case", MASKED_CASES)
+def test_mask_on_load_linear_matches_oracle_and_packed_path(lib, case, dtype):
+    rows, in_, out, N, M = case
+    X = synth.randn((rows, in_), 31 * rows + in_, synth.X_STD, dtype, "cuda")
+    W = synth.randn((out, in_), 37 * out + in_, synth.W_STD, dtype, "cuda")
+    bias = synth.randn((out,), 41 * out, synth.B_STD, dtype, "cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Y = lib.elsa_nm_linear_masked(X, W, bias, N, M, dev_status=status)
+    vals, idx = lib.elsa_nm_compress(W, N, M)
+    Y_packed = lib.elsa_nm_linear(X, vals, idx, bias, out, in_, N, M, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.equal(Y, Y_packed)                      # same projection, same kernels
+    pick = torch.from_numpy(synth.sample_rows(rows, 48, 5)).cuda()
+    check_close(Y[pick], oracle_linear(X[pick].cpu(), W.cpu(), bias.cpu(), N, M, dtype))
