@@ -1,9 +1,9 @@
 #!/usr/bin/env python
 """Benchmark of the N:M sparse-linear path on seeded synthetic ViT workloads.
 
-One step = one pass of the whole path over the workload's layer table: elsa_nm_compress of every
-layer's dense weight to its level, then elsa_vit_linears over the table (per layer: rebuild the
-weight image the MMA reads, tcgen05 GEMM with bias).  The default workload is the 48-layer DeiT-B
+One step = one pass of the whole path over the workload's layer table: elsa_vit_compress of every
+layer's dense weight to its level, then elsa_vit_linears over the table (weight images the MMAs
+read, then the tcgen05 GEMMs with bias; layers of a kernel family share persistent launches).  The default workload is the 48-layer DeiT-B
 stack at batch 256 in bf16 with a seeded level per layer from {1:8, 2:8, 4:8, 8:8}.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
