@@ -285,6 +285,8 @@ def run_ours(args):
     kernel_total = sum(v[1] for v in per_kernel.values()) or 1.0
     roof = [roofline_seconds(l, peaks) for l in layers]
     roof_sus = [roofline_seconds(l, peaks, "bf16_tflops_sustained") for l in layers]
+    nominal = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}      # data-sheet figures, for context only
+    roof_nom = [roofline_seconds(l, nominal) for l in layers]
     sum_roof = sum(r[0] for r in roof)
     # GEMM time per step: the shared launches of the profiled pass, as the timed region runs them
     sum_gemm = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS) / args.steps * 1e-3
@@ -305,6 +307,7 @@ def run_ours(args):
         "kept_tflops": kept_flops / sum_gemm / 1e12 if sum_gemm else None,
         "algorithmic_gbs": sum(algorithmic_bytes(l) for l in layers) / sum_gemm / 1e9 if sum_gemm else None,
         "frac_vs_sustained_peak": sum(r[0] for r in roof_sus) / sum_gemm if sum_gemm else None,
+        "frac_vs_nominal_peaks": sum(r[0] for r in roof_nom) / sum_gemm if sum_gemm else None,
         "launches": gemm_launches,
         "avg_launch_ms": gemm_total_ms / max(gemm_launches, 1),
         "roofline_time_share": {k: v / sum_roof for k, v in share.items()},
@@ -328,6 +331,9 @@ def run_ours(args):
         "roofline": roofline,
         "kernels": {k: {"launches": v[0], "ms": v[1], "share": v[1] / kernel_total} for k, v in per_kernel.items()},
         "ms_per_step_profiled": prof_ms / args.steps,
+        "compress_gbs": (sum(l.out * l.in_ * 2 + algorithmic_bytes(l) - 2 * l.rows * (l.in_ + l.out) - l.out * 2
+                             for l in layers) * args.steps / per_kernel["nm_compress"][1] / 1e6)
+                        if per_kernel.get("nm_compress", [0, 0.0])[1] > 0 else None,
         "clocks": clocks,
     }
 
@@ -407,13 +413,16 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="deit_b_stack_b256",
                     choices=["single_layer", "deit_b_block_b64", "deit_b_stack_b256", "swin_b_stack_b128"])
-    ap.add_argument("--oracle-rows", type=int, default=4096, help="rows per layer of the CPU-oracle sample")
+    ap.add_argument("--oracle-rows", type=int, default=None,
+                    help="rows per layer of the CPU-oracle sample (default 4096 for cpu_baseline, 1024 per step of --impl reference)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.oracle_rows is None:
+        args.oracle_rows = 1024 if args.impl == "reference" else 4096
     if args.impl == "reference":
         run_reference(args)
     else:
