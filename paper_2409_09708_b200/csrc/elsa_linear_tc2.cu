@@ -8,7 +8,7 @@
 // only half of the W rows, and one tcgen05.mma.cta_group::2 (M = 256) issued by the leader CTA
 // drives both tensor cores, so each SM moves 2/3 of the bytes per MMA.
 //
-// Per CTA (320 threads):
+// Per CTA (352 threads):
 //   warp 0      TMA producer for this CTA's operand halves; completion bytes of both CTAs are
 //               credited to the leader's stage barrier
 //   warp 1      allocates tensor memory (pair-wide); in the leader one lane issues the MMAs and
@@ -16,6 +16,8 @@
 //   warps 2-9   epilogue, two warps per TMEM lane quarter (alternating 32-column chunks):
 //               tcgen05.ld of all the warp's chunks, accumulator released, then + bias in fp32,
 //               round to 16 bit, swizzled staging, TMA store
+//   warp 10     bias loader: copies the next tile's bias into one of two shared buffers, so the
+//               epilogue warps issue no global loads of their own
 // Two TMEM accumulators let the MMAs of tile i+1 overlap the epilogue of tile i.  Every wait is
 // bounded; on expiry ELSA_ERR_TIMEOUT is recorded and all roles of the CTA leave; a cluster barrier
 // before tensor memory is released keeps either CTA from leaving while its partner may still read
@@ -37,14 +39,16 @@ constexpr int kNumAccum = 2;
 constexpr int kTmemCols = kNumAccum * kMaxBlockN;
 constexpr int kMaxStages = 8;
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kEpiParts = kEpiWarps / 4;   // warps per TMEM lane quarter; they share the quarter's chunks
+constexpr int kBiasWarp = 2 + kEpiWarps;
+constexpr int kThreads = (kBiasWarp + 1) * 32;
 constexpr int kEpiCols = 32;
-constexpr int kMaxChunksPerWarp = kMaxBlockN / kEpiCols / 2;   // two warps per TMEM lane quarter share the chunks
+constexpr int kMaxChunksPerWarp = kMaxBlockN / kEpiCols / kEpiParts;
 constexpr int kATileBytes = kRowsPerCta * kBlockK * 2;
 constexpr int kStagingBytes = 32 * kEpiCols * 2;
 constexpr int kStagingBufs = 1;     // one staging buffer per epilogue warp: the shared memory goes to a sixth pipeline stage instead
 constexpr int kStagingTotal = kEpiWarps * kStagingBufs * kStagingBytes;
-constexpr int kBiasBytes = kEpiWarps * kMaxBlockN * 4;
+constexpr int kBiasBytes = 2 * kMaxBlockN * 2;   // two tiles' bias as stored (16 bit)
 constexpr int kBarrierBytes = 256;
 
 // One layer of a launch.  A launch may carry several layers (a group): the persistent CTA pairs walk the
@@ -95,7 +99,9 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
     const uint32_t empty_bar = bar_base + 8 * kMaxStages;     // per CTA
     const uint32_t tmem_full_bar = bar_base + 16 * kMaxStages;                 // per CTA
     const uint32_t tmem_empty_bar = tmem_full_bar + 8 * kNumAccum;             // used in the leader only
-    const uint32_t holder_off = bias_off + kBiasBytes + 16 * kMaxStages + 16 * kNumAccum;
+    const uint32_t bias_full_bar = tmem_empty_bar + 8 * kNumAccum;             // per CTA
+    const uint32_t bias_empty_bar = bias_full_bar + 16;                        // per CTA
+    const uint32_t holder_off = bias_off + kBiasBytes + 16 * kMaxStages + 16 * kNumAccum + 32;
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off + 4);
 
@@ -107,6 +113,10 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         for (int a = 0; a < kNumAccum; ++a) {
             mbar_init(tmem_full_bar + 8 * a, 1);
             mbar_init(tmem_empty_bar + 8 * a, 2 * kEpiWarps);   // every epilogue warp of both CTAs
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(bias_full_bar + 8 * b, 1);
+            mbar_init(bias_empty_bar + 8 * b, kEpiWarps);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -191,35 +201,56 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             }
         }
         __syncwarp();
+    } else if (warp == kBiasWarp) {
+        // ------------------------------------------------ bias loader: tile i + 1's bias while tile i is stored
+        // (kept out of the epilogue warps: a global load in flight there holds up their proxy fences)
+        int cur = 0;
+        uint32_t it = 0;
+        for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++it) {
+            while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
+            const PairLayer& L = p.layer[cur];
+            const int n0 = ((tile - L.tile_begin) % L.tiles_n) * L.bn;
+            const uint32_t b = it & 1u;
+            bool ok = mbar_wait(bias_empty_bar + 8 * b, ((it >> 1) & 1u) ^ 1u, abort_flag, p.dev_status, 5);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const uint16_t* l_bias = L.bias;
+            for (int j = lane; j < L.bn; j += 32) {
+                const int o = n0 + j;
+                const uint16_t v = (l_bias != nullptr && o < L.out) ? __ldg(l_bias + o) : (uint16_t)0;
+                asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_base + bias_off + b * (kMaxBlockN * 2) + (uint32_t)(j * 2)), "h"(v)
+                             : "memory");
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bias_full_bar + 8 * b);
+        }
+        __syncwarp();
     } else {
         // ------------------------------------------------ epilogue (warps 2..9)
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
-        const int ew = warp - 2;                // private staging / bias slot
-        const int half = ew >> 2;               // which of the two warps of the quarter: even or odd chunks
+        const int ew = warp - 2;                // private staging slot
+        const int part = ew >> 2;               // which of the quarter's warps: chunks part, part + kEpiParts, ...
         const uint32_t stage_buf = staging_base + (uint32_t)(ew * kStagingBufs * kStagingBytes);
-        float* bias_s = reinterpret_cast<float*>(smem_gen + bias_off) + ew * kMaxBlockN;
         const uint32_t empty_remote = mapa_shared(tmem_empty_bar, 0);
         int acc = 0;
         uint32_t acc_phase = 0;
         uint32_t chunk_counter = 0;
         int cur = 0;
+        uint32_t it = 0;
 
-        for (int tile = pair; tile < p.num_tiles; tile += num_pairs) {
+        for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++it) {
             while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
             const PairLayer& L = p.layer[cur];
             const int t = tile - L.tile_begin;
             const int chunks = L.bn / kEpiCols;
-            const int my_chunks = (chunks - half + 1) / 2;
+            const int my_chunks = (chunks - part + kEpiParts - 1) / kEpiParts;
             const int m0 = (t / L.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
             const int n0 = (t % L.tiles_n) * L.bn;
             const int l_rows = L.rows, l_out = L.out;
-            const uint16_t* l_bias = L.bias;
-            for (int j = lane; j < L.bn; j += 32) {
-                const int o = n0 + j;
-                bias_s[j] = (l_bias != nullptr && o < l_out) ? bias_to_float<kBf16>(l_bias[o]) : 0.f;
-            }
-            __syncwarp();
-            bool ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
+            const uint32_t bias_b = it & 1u;
+            const uint32_t bias_cur = smem_base + bias_off + bias_b * (kMaxBlockN * 2);
+            bool ok = mbar_wait(bias_full_bar + 8 * bias_b, (it >> 1) & 1u, abort_flag, p.dev_status, 6);
+            ok = ok && mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after();
@@ -228,23 +259,37 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 
             // converts, stages and stores one 32 x 32 chunk
             auto emit = [&](const uint32_t (&r)[32], int c) {
-                uint32_t packed[16];
+                // 16 columns: + bias (read as stored, eight values per load), rounded to 16 bit
+                auto convert16 = [&](int h, uint32_t (&pk)[8]) {
 #pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const float2 b = *reinterpret_cast<const float2*>(bias_s + c * kEpiCols + 2 * j);
-                    packed[j] = pack2<kBf16>(__uint_as_float(r[2 * j]) + b.x, __uint_as_float(r[2 * j + 1]) + b.y);
-                }
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t bw[4];
+                        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3])
+                                     : "r"(bias_cur + (uint32_t)(c * kEpiCols * 2 + (2 * h + g) * 16)));
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float2 bv = raw2_to_float2<kBf16>(bw[e]);
+                            const int j = 8 * h + 4 * g + e;
+                            pk[4 * g + e] = pack2<kBf16>(__uint_as_float(r[2 * j]) + bv.x, __uint_as_float(r[2 * j + 1]) + bv.y);
+                        }
+                    }
+                };
                 const uint32_t buf = stage_buf + (chunk_counter % kStagingBufs) * kStagingBytes;
-                if (lane == 0) bulk_wait_group_read<kStagingBufs - 1>();   // the store that last used this buffer has drained it
-                __syncwarp();
                 const uint32_t row_addr = buf + (uint32_t)(lane * 64);
                 const uint32_t sw = (uint32_t)((lane >> 1) & 3);   // 64-byte swizzle of the staging rows
+                uint32_t pk[8];
+                convert16(0, pk);
+                if (lane == 0) bulk_wait_group_read<kStagingBufs - 1>();   // the store that last used this buffer has drained it
+                __syncwarp();
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + (((uint32_t)j ^ sw) << 4)),
-                                 "r"(packed[4 * j]), "r"(packed[4 * j + 1]), "r"(packed[4 * j + 2]),
-                                 "r"(packed[4 * j + 3])
-                                 : "memory");
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1) convert16(1, pk);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + (((uint32_t)(2 * h + j) ^ sw) << 4)),
+                                     "r"(pk[4 * j]), "r"(pk[4 * j + 1]), "r"(pk[4 * j + 2]), "r"(pk[4 * j + 3])
+                                     : "memory");
+                    }
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -268,12 +313,15 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             uint32_t r[kMaxChunksPerWarp][32];
 #pragma unroll
             for (int i = 0; i < kMaxChunksPerWarp; ++i)
-                if (i < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((half + 2 * i) * kEpiCols), r[i]);
+                if (i < my_chunks) tmem_ld_32x32b_x32(t_row + (uint32_t)((part + kEpiParts * i) * kEpiCols), r[i]);
             tmem_wait_ld();
             release();
 #pragma unroll
             for (int i = 0; i < kMaxChunksPerWarp; ++i)
-                if (i < my_chunks) emit(r[i], half + 2 * i);
+                if (i < my_chunks) emit(r[i], part + kEpiParts * i);
+            // this warp has read the tile's bias for the last time
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bias_empty_bar + 8 * bias_b);
             if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
         }
         if (lane == 0) bulk_wait_group_all();

@@ -189,6 +189,14 @@ __device__ __forceinline__ uint32_t pack2(float lo, float hi)
     }
 }
 
+// Two 16-bit values packed in a word (low half first) as floats.
+template <bool kBf16>
+__device__ __forceinline__ float2 raw2_to_float2(uint32_t w)
+{
+    if constexpr (kBf16) return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+    else return __half22float2(*reinterpret_cast<const __half2*>(&w));
+}
+
 template <bool kBf16>
 __device__ __forceinline__ float bias_to_float(uint16_t u)
 {
