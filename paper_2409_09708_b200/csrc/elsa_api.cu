@@ -136,7 +136,7 @@ elsa_status check_linear(const void* X, int rows, const void* vals, const uint32
     return ELSA_OK;
 }
 
-enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR };
+enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR, KIND_SPARSE_WS };
 
 // Which kernel a layer runs on.  AUTO is the product rule; a forced variant is honoured where it applies.
 elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, LinearKind* kind)
@@ -152,6 +152,12 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
         if (!sparse_ok)
             return fail(ELSA_ERR_NM, "the sparse-MMA variant needs N <= 2 < M and in %% 16 == 0 (got %d:%d, in=%d)", N, M, in);
         *kind = variant == ELSA_VARIANT_TC_SPARSE ? KIND_SPARSE_ONE : KIND_SPARSE_PAIR;
+        return ELSA_OK;
+    case ELSA_VARIANT_TC_SPARSE_WS:
+        if (N == M || !linear_tc_sparse_ws_suits(in, out, N, sm_count))
+            return fail(ELSA_ERR_NM, "the weight-stationary sparse variant needs N <= 2 < M, in %% 128 == 0 and in <= 1024 "
+                        "(got %d:%d, in=%d)", N, M, in);
+        *kind = KIND_SPARSE_WS;
         return ELSA_OK;
     default: break;
     }
@@ -184,6 +190,9 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
     if (kind == KIND_SPARSE_PAIR)
         return launch_linear_tc_sparse_pair((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias,
                                             out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
+    if (kind == KIND_SPARSE_WS)
+        return launch_linear_tc_sparse_ws((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias,
+                                          out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
     // Dense-rate path.  The dense level multiplies the stored values as they are; every other level first
     // rebuilds the weight image the MMA reads, in the caller's scratch.
     const uint16_t* Wd = (const uint16_t*)vals;
@@ -320,14 +329,15 @@ elsa_status elsa_nm_linear_masked(const void* X, int rows, const void* W_sup, co
     if ((st = pick_kind(rows, out, in, N, M, dev.sm_count, &kind)) != ELSA_OK) return st;
     if (kind == KIND_SIMT || kind == KIND_SPARSE_ONE)
         return fail(ELSA_ERR_NM, "the forced variant has no mask-on-load form");
-    if (kind == KIND_SPARSE_PAIR) {
+    if (kind == KIND_SPARSE_PAIR || kind == KIND_SPARSE_WS) {
         uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
         if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, (uint16_t*)workspace, meta, stream)) != ELSA_OK)
             return st;
         SparseJob job;
         job.X = (const uint16_t*)X; job.bias = (const uint16_t*)bias; job.Y = (uint16_t*)Y; job.workspace = workspace;
         job.rows = rows; job.in = in; job.out = out;
-        return launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
+        return kind == KIND_SPARSE_WS ? launch_linear_tc_sparse_ws_group(&job, 1, dtype, dev_status, stream)
+                                      : launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
     }
     const uint16_t* Wd = (const uint16_t*)W_sup;     // the dense level multiplies the shared weight as it is
     if (N != M) {
@@ -454,7 +464,7 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
         for (int l = 0; l < n_layers; ++l) {
             const elsa_layer& c = cfg[l];
             if (c.N != c.M) {
-                if (kind[l] == KIND_SPARSE_PAIR) {
+                if (kind[l] == KIND_SPARSE_PAIR || kind[l] == KIND_SPARSE_WS) {
                     uint8_t* meta = region[l] + round_up((size_t)c.out * (size_t)c.in, 256);
                     batch_add_to_sp24(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, 128,
                                       (uint16_t*)region[l], meta);
@@ -482,6 +492,24 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
             }
             if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_sparse_pair_group_max())) {
                 if ((st = launch_linear_tc_sparse_pair_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
+                    return st;
+                jobs.clear();
+            }
+        }
+    }
+    // sparse-rate layers whose weight block fits tensor memory, in groups
+    {
+        std::vector<SparseJob> jobs;
+        for (int l = 0; l <= n_layers; ++l) {
+            if (l < n_layers && kind[l] == KIND_SPARSE_WS) {
+                const elsa_layer& c = cfg[l];
+                SparseJob j;
+                j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
+                j.workspace = region[l]; j.rows = c.rows; j.in = c.in; j.out = c.out;
+                jobs.push_back(j);
+            }
+            if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_sparse_ws_group_max())) {
+                if ((st = launch_linear_tc_sparse_ws_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
                     return st;
                 jobs.clear();
             }
@@ -676,7 +704,7 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
     if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR &&
-        v != ELSA_VARIANT_TC_SPARSE && v != ELSA_VARIANT_TC_SPARSE_PAIR)
+        v != ELSA_VARIANT_TC_SPARSE && v != ELSA_VARIANT_TC_SPARSE_PAIR && v != ELSA_VARIANT_TC_SPARSE_WS)
         return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;

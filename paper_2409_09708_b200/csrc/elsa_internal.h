@@ -126,6 +126,15 @@ elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uin
 elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
                                                cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
+// The same product with the 256-feature weight block of each CTA pair resident in tensor memory for a
+// whole layer (in % 128 == 0, in <= 1024); jobs as for the pair kernel, same re-encoded weight.
+int linear_tc_sparse_ws_group_max();
+bool linear_tc_sparse_ws_suits(int in, int out, int N, int sm_count);
+elsa_status launch_linear_tc_sparse_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                             cudaStream_t stream);
+elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                       const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
+                                       void* workspace, uint32_t* dev_status, cudaStream_t stream);
 size_t linear_tc_sparse_workspace(int out, int in);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
 constexpr int kMaxLevels = 16;

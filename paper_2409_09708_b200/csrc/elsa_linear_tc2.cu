@@ -136,7 +136,9 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer (both CTAs)
-        if (lane == 0) {
+        // The whole warp walks the loop and waits; one elected lane issues (see the MMA warp).
+        {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -151,13 +153,17 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 const uint32_t tx_bytes = (uint32_t)(2 * (kATileBytes + half_bn * kBlockK * 2));
                 for (int kb = 0; kb < L.num_k_blocks; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     const uint32_t a_dst = smem_base + (uint32_t)(stage * stage_bytes);
-                    // the leader's stage barrier collects the bytes of both CTAs
-                    if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
                     const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
-                    tma_load_2d_pair(a_dst, &L.map_x, bar, kb * kBlockK, m0);
-                    tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * kBlockK, n0);
+                    if (elected) {
+                        // the leader's stage barrier collects the bytes of both CTAs
+                        if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
+                        tma_load_2d_pair(a_dst, &L.map_x, bar, kb * kBlockK, m0);
+                        tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * kBlockK, n0);
+                    }
+                    __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -165,7 +171,11 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && cta_rank == 0) {
+        // The whole warp walks the loop and waits on the barriers with its operands in uniform
+        // registers; only the MMA and commit instructions are predicated on one elected lane.  A
+        // single thread inside a divergent branch needs about twice as long to issue one MMA.
+        if (cta_rank == 0) {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -177,11 +187,13 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 const int num_k_blocks = p.layer[cur].num_k_blocks;
                 const uint32_t idesc = p.layer[cur].idesc;
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kMaxBlockN);
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + (uint32_t)(stage * stage_bytes);
@@ -189,14 +201,15 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                      (uint32_t)((kb | k) != 0));
+                        if (elected)
+                            umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                          (uint32_t)((kb | k) != 0));
                     }
-                    umma_commit_pair(empty_bar + 8 * stage, 3);   // frees this stage in both CTAs
+                    if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);   // frees this stage in both CTAs
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit_pair(tmem_full_bar + 8 * acc, 3);     // accumulator complete in both CTAs
+                if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);     // accumulator complete in both CTAs
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }

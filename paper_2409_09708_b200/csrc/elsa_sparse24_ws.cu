@@ -1,0 +1,564 @@
+// N:M sparse linear (N <= 2) on the 2:4 sparse MMA with the weight held in tensor memory.
+//
+// Same product as elsa_sparse24_pair.cu (Sec. 2, Fig. 2 bottom of the ELSA paper, on the 2-of-4
+// re-encoding of the packed weight).  That kernel streams the compressed weight tile and its metadata
+// through shared memory again for every tile of token rows, and at the sparse MMA rate the weight and
+// activation bytes together exceed what shared memory can deliver per cycle.  Here the weight does
+// not move: a CTA pair owns one block of 256 output features of a layer for the whole layer.  Its
+// 2-of-4 values (in/4 columns) and metadata (in/32 columns) are written once into the tensor memory
+// of the two CTAs and every tcgen05.mma.sp reads its A operand from there; shared memory carries
+// activations only.  What is left of tensor memory holds one accumulator of `nt` token rows (256 for
+// in <= 768).  The wide tile is deliberate: issuing one MMA costs the issuing warp on the order of a
+// hundred cycles whatever its shape, and a sparse MMA over 256 token rows lasts 128 cycles, so only the
+// widest instruction keeps the tensor pipe fed; the price is that the epilogue's tensor-memory reads and
+// the next tile's MMAs cannot overlap (the conversion and the stores still do).
+//
+// Schedule of a layer over P pairs: F = ceil(out / 256) feature blocks, G = P / F row groups.  Pair p
+// takes feature block p % F and the row tiles g, g + G, g + 2G, ... with g = p / F, so the F pairs
+// of a group read the same activation rows at about the same time (one fetch from HBM, the rest from
+// L2).  Pairs beyond G * F sit the layer out.  A launch may carry several layers; each pair walks
+// them in order, reloading its weight block at every layer.
+//
+// Per CTA: warp 0 TMA producer for this CTA's half of the activation rows; warp 1 tensor-memory
+// allocation and, in the leader, MMA issue; the remaining warps write the weight block into tensor
+// memory at the start of a layer and run the epilogue (lanes are features; see
+// elsa_sparse24_pair.cu for the transposing store).  Waits are bounded as in the other kernels.
+
+#include <mutex>
+
+#include "elsa_tc_common.cuh"
+
+namespace elsa {
+namespace {
+
+constexpr int kFeatPerCta = 128;   // weight rows per CTA = TMEM lanes
+constexpr int kPairFeat = 256;     // MMA M over the pair
+constexpr int kMaxRowTile = 256;   // token rows per pair tile (MMA N), per layer <= this
+constexpr int kBlockK = 128;       // granularity of `in` (one metadata block)
+constexpr int kStageK = 256;       // logical K per pipeline stage: eight MMAs per barrier round trip
+constexpr int kSpUmmaK = 32;
+constexpr int kNumAccum = 1;
+constexpr int kTmemCols = 512;
+constexpr int kMaxIn = 1024;       // in / 4 + in / 32 + nt columns must fit 512
+constexpr int kMaxStages = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kEpiParts = kEpiWarps / 4;   // warps per TMEM lane quarter
+constexpr int kThreads = 64 + kEpiWarps * 32;
+constexpr int kEpiCols = 32;
+constexpr int kBSubBytes = (kMaxRowTile / 2) * 128;   // one 64-wide K slice: up to 128 rows of 128 bytes
+constexpr int kStageBytes = (kStageK / 64) * kBSubBytes;
+constexpr int kStagingBytes = 32 * kEpiCols * 2;      // one buffer per epilogue warp
+constexpr int kStagingTotal = kEpiWarps * kStagingBytes;
+constexpr int kBarrierBytes = 512;
+
+static_assert(kBSubBytes % 1024 == 0, "swizzled tiles stay 1024-byte aligned");
+
+struct alignas(64) WsLayer {
+    CUtensorMap map_x, map_y;
+    const uint16_t* a_img;   // 2-of-4 values [out][in / 2]
+    const uint8_t* meta;     // metadata blocks of 2 KB per (128 features, 128 k)
+    const uint16_t* bias;
+    int rows, out, in;
+    int nt;            // token rows per pair tile
+    int tiles_f;       // F
+    int groups;        // G
+    int row_tiles;     // ceil(rows / nt)
+    int num_k_blocks;  // in / 128 (metadata blocks per 128 features)
+    uint32_t idesc;
+};
+
+constexpr int kGroupMax = 92;   // layers per launch (kernel parameters are limited to 32 KB)
+
+template <int kMaxLayers>
+struct WsGroup {
+    WsLayer layer[kMaxLayers];
+    int n_layers;
+    int stages;
+    uint32_t* dev_status;
+};
+
+// A from tensor memory: lane = weight row, 8 columns per K step of 32 (16 kept values of 16 bits).
+__device__ __forceinline__ void umma_sp_f16_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t tmem_e,
+                                                    uint32_t idesc, uint32_t accumulate)
+{
+    const uint32_t idesc_sel = idesc | (tmem_e & 1u);
+    const uint32_t e_addr = tmem_e & ~1u;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %5, 0;\n"
+        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], [%1], %2, [%3], %4, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate)
+        : "memory");
+}
+
+// Lane i of the warp writes 16 / 4 consecutive columns of TMEM lane (lane base + i).
+__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_st_32x32b_x4(uint32_t taddr, const uint32_t (&r)[4])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3])
+                 : "memory");
+}
+
+// 3-D TMA load into this CTA's shared memory, completion bytes credited to an mbarrier that may live in
+// the other CTA of the pair.
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0,
+                                                 int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+// Row-major 16-bit matrix [rows][in] seen as [in / 64][rows][64]: one box of (64, box_rows, 4) is a K stage
+// of 256 as four 128-byte-swizzled quarters of box_rows rows each.
+elsa_status make_map_x_quarters(CUtensorMap* map, const void* base, uint64_t in, uint64_t rows, uint32_t box_rows)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(ELSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {64, rows, in / 64};
+    cuuint64_t strides[2] = {in * 2, 128};
+    cuuint32_t box[3] = {64, box_rows, kStageK / 64};
+    cuuint32_t elem[3] = {1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(base), dims, strides, box, elem,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for X rejected (CUresult %d)", (int)rc);
+    return ELSA_OK;
+}
+
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Arrival that publishes this CTA's tensor-memory writes to the MMA issuer of the leader CTA.
+__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+template <bool kBf16, int kMaxLayers>
+__global__ void __launch_bounds__(kThreads, 1)
+linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = cluster_ctarank();
+    const int pair = blockIdx.x >> 1;
+
+    const uint32_t staging_base = smem_base + (uint32_t)(p.stages * kStageBytes);
+    const uint32_t bar_off = (uint32_t)(p.stages * kStageBytes) + kStagingTotal;
+    const uint32_t bar_base = smem_base + bar_off;
+    const uint32_t full_bar = bar_base;                       // leader only
+    const uint32_t empty_bar = bar_base + 8 * kMaxStages;     // per CTA
+    const uint32_t tmem_full_bar = bar_base + 16 * kMaxStages;        // per CTA
+    const uint32_t tmem_empty_bar = tmem_full_bar + 8 * kNumAccum;    // leader only
+    const uint32_t w_ready_bar = tmem_empty_bar + 8 * kNumAccum;      // leader only
+    const uint32_t holder_off = bar_off + 16 * kMaxStages + 16 * kNumAccum + 8;
+    volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off + 4);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            mbar_init(full_bar + 8 * s, 1);
+            mbar_init(empty_bar + 8 * s, 1);
+        }
+        for (int a = 0; a < kNumAccum; ++a) {
+            mbar_init(tmem_full_bar + 8 * a, 1);
+            mbar_init(tmem_empty_bar + 8 * a, 2 * kEpiWarps);
+        }
+        mbar_init(w_ready_bar, 2 * kEpiWarps);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async_smem();
+    }
+    if (warp == 1) tmem_alloc_pair(smem_base + holder_off, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    cluster_arrive();
+    cluster_wait();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+
+    if (warp == 0) {
+        // ------------------------------------------------ producer: this CTA's half of the activation rows
+        // (whole warp converged, one elected lane issues: see the MMA warp).  One 3-D copy per stage
+        // brings the four 64-wide K quarters of the stage: [quarter][row][128 bytes]; quarters beyond `in`
+        // (a last stage of 128) arrive as zeros and are not multiplied.
+        {
+            const bool elected = elect_one();
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int li = 0; ok && li < p.n_layers; ++li) {
+                const WsLayer& L = p.layer[li];
+                if (pair >= L.groups * L.tiles_f) continue;
+                const int half_rows = L.nt >> 1;
+                const uint32_t tx_bytes = (uint32_t)(2 * (kStageK / 64) * half_rows * 128);   // both CTAs' boxes, in full
+                const int num_k_stages = (L.in + kStageK - 1) / kStageK;
+                for (int r = pair / L.tiles_f; ok && r < L.row_tiles; r += L.groups) {
+                    const int r0 = r * L.nt + (int)cta_rank * half_rows;
+                    for (int ks = 0; ks < num_k_stages; ++ks) {
+                        ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
+                        if (!ok) break;
+                        const uint32_t dst = smem_base + (uint32_t)(stage * kStageBytes);
+                        const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
+                        if (elected) {
+                            if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
+                            tma_load_3d_pair(dst, &L.map_x, bar, 0, r0, (kStageK / 64) * ks);
+                        }
+                        __syncwarp();
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer (leader CTA only)
+        // The whole warp walks the loop and waits on the barriers; one elected lane issues.  With the
+        // warp converged the descriptors stay in uniform registers, which roughly halves the cost of
+        // issuing one MMA compared with a single thread inside a divergent branch (measured: ~85 -> ~40
+        // cycles), and an MMA of 128 token rows lasts only 64 cycles.
+        if (cta_rank == 0) {
+            const bool elected = elect_one();
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            uint32_t w_phase = 0;
+            bool ok = true;
+            for (int li = 0; ok && li < p.n_layers; ++li) {
+                const WsLayer& L = p.layer[li];
+                if (pair >= L.groups * L.tiles_f) continue;
+                const int g = pair / L.tiles_f;
+                if (g >= L.row_tiles) continue;
+                // the weight block of this layer is in tensor memory (both CTAs)
+                ok = mbar_wait(w_ready_bar, w_phase, abort_flag, p.dev_status, 7);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                w_phase ^= 1u;
+                tc_fence_after();
+                const uint32_t a_col0 = tmem_base + (uint32_t)(kNumAccum * L.nt);
+                const uint32_t e_col0 = a_col0 + (uint32_t)(L.in >> 2);
+                const uint32_t idesc = L.idesc;
+                const int num_k_stages = (L.in + kStageK - 1) / kStageK;
+                const bool half_tail = (L.in % kStageK) != 0;      // the last stage holds 128 of K only
+                const uint32_t quarter = (uint32_t)(L.nt * 64) >> 4;   // descriptor units between K quarters
+                for (int r = g; ok && r < L.row_tiles; r += L.groups) {
+                    ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * L.nt);
+                    for (int ks = 0; ks < num_k_stages; ++ks) {
+                        ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint64_t b_desc0 = smem_desc_k_major_sw128(smem_base + (uint32_t)(stage * kStageBytes));
+                        const uint32_t a_col = a_col0 + (uint32_t)(ks * 8 * (kStageK / kSpUmmaK));
+                        const uint32_t e_col = e_col0 + (uint32_t)(ks * (kStageK / kSpUmmaK));
+                        // operands are computed by the whole warp (they stay uniform); only the instruction
+                        // itself is predicated on the elected lane
+                        if (half_tail && ks == num_k_stages - 1) {
+#pragma unroll
+                            for (int j = 0; j < kStageK / kSpUmmaK / 2; ++j) {
+                                const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)(j >> 1) * quarter + 4u * (uint32_t)(j & 1));
+                                if (elected)
+                                    umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
+                                                        (uint32_t)((ks | j) != 0));
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < kStageK / kSpUmmaK; ++j) {
+                                const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)(j >> 1) * quarter + 4u * (uint32_t)(j & 1));
+                                if (elected)
+                                    umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
+                                                        (uint32_t)((ks | j) != 0));
+                            }
+                        }
+                        if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);
+                        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);
+                    if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ weight loader + epilogue: lanes are features
+        const int q = warp & 3;                 // TMEM lane quarter this warp may touch
+        const int part = (warp - 2) >> 2;       // which of the quarter's warps
+        const uint32_t empty_remote = mapa_shared(tmem_empty_bar, 0);
+        const uint32_t w_ready_remote = mapa_shared(w_ready_bar, 0);
+        const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        const bool odd = (lane & 1) != 0;
+        const uint32_t buf = staging_base + (uint32_t)((warp - 2) * kStagingBytes);
+        // staging address pieces that do not depend on the row pair (see elsa_sparse24_pair.cu)
+        const uint32_t prmt_sel = odd ? 0x7632u : 0x5410u;
+        const uint32_t lane_off = (odd ? 64u : 0u) + (uint32_t)(((lane >> 1) & 3) * 4);
+        uint32_t sw_off[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) sw_off[k] = (((uint32_t)(lane >> 3)) ^ (uint32_t)k) << 4;
+
+        bool ok = true;
+        for (int li = 0; ok && li < p.n_layers; ++li) {
+            const WsLayer& L = p.layer[li];
+            if (pair >= L.groups * L.tiles_f) continue;
+            const int g = pair / L.tiles_f;
+            if (g >= L.row_tiles) continue;
+            const int ft128 = (pair % L.tiles_f) * 2 + (int)cta_rank;
+            const int f0 = ft128 * kFeatPerCta + q * 32;
+            const int f = f0 + lane;
+            const int l_rows = L.rows, l_out = L.out, nt = L.nt;
+            const bool f_ok = f < l_out;
+
+            // ---- this warp's share of the weight block into tensor memory.  Every MMA of the previous
+            // layer has completed: this warp waited for the accumulator of that layer's last tile.
+            {
+                const uint32_t a_col0 = lane_base + (uint32_t)(kNumAccum * nt);
+                const uint32_t e_col0 = a_col0 + (uint32_t)(L.in >> 2);
+                const uint4* a_row = reinterpret_cast<const uint4*>(L.a_img + (size_t)(f_ok ? f : 0) * (size_t)(L.in >> 1));
+                const int a_chunks = L.in >> 6;          // 16 columns (64 bytes) each
+                for (int c = part; c < a_chunks; c += kEpiParts) {
+                    uint32_t v[16];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 t = make_uint4(0u, 0u, 0u, 0u);
+                        if (f_ok) t = __ldg(a_row + 4 * c + i);
+                        v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
+                    }
+                    tmem_st_32x32b_x16(a_col0 + (uint32_t)(16 * c), v);
+                }
+                const bool blk_ok = ft128 * kFeatPerCta < l_out;
+                const uint4* e_blk = reinterpret_cast<const uint4*>(L.meta) +
+                                     (size_t)(blk_ok ? ft128 : 0) * (size_t)L.num_k_blocks * 128 + (size_t)(q * 32 + lane);
+                for (int kb = part; kb < L.num_k_blocks; kb += kEpiParts) {
+                    uint4 t = make_uint4(0u, 0u, 0u, 0u);
+                    if (blk_ok) t = __ldg(e_blk + (size_t)kb * 128);
+                    uint32_t v[4] = {t.x, t.y, t.z, t.w};
+                    tmem_st_32x32b_x4(e_col0 + (uint32_t)(4 * kb), v);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster_release(w_ready_remote);
+            }
+            const float bias_f = (L.bias != nullptr && f_ok) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
+            const int chunks = nt / kEpiCols;
+
+            for (int r = g; r < L.row_tiles; r += L.groups) {
+                const int r0 = r * nt;
+                ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_row = lane_base + (uint32_t)(acc * nt);
+                // this warp's chunks of 32 token rows: part, part + kEpiParts; both are read before the
+                // accumulator goes back to the MMA warp
+                uint32_t rr[2][32];
+                const bool mine0 = part < chunks, mine1 = part + kEpiParts < chunks;
+                if (mine0) tmem_ld_32x32b_x32(t_row + (uint32_t)(part * kEpiCols), rr[0]);
+                if (mine1) tmem_ld_32x32b_x32(t_row + (uint32_t)((part + kEpiParts) * kEpiCols), rr[1]);
+                if (mine0) tmem_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_cluster(empty_remote + 8 * acc);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (!(h == 0 ? mine0 : mine1)) continue;
+                    if (lane == 0) bulk_wait_group_read<0>();   // the previous store has drained the buffer
+                    __syncwarp();
+                    // staging tile [32 token rows][32 features], 64-byte rows with the 64-byte swizzle; this
+                    // lane writes the feature pair (lane & ~1, lane | 1) of one row per row pair
+                    // (all exchanges first, then all stores: interleaved, each store would wait for its shuffle)
+                    uint32_t word[16];
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const uint32_t own = pack2<kBf16>(__uint_as_float(rr[h][2 * j]) + bias_f, __uint_as_float(rr[h][2 * j + 1]) + bias_f);
+                        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, own, 1);
+                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(word[j]) : "r"(odd ? got : own), "r"(odd ? own : got), "r"(prmt_sel));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + lane_off + (uint32_t)(j * 128) + sw_off[j & 3]), "r"(word[j])
+                                     : "memory");
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        const int row0 = r0 + (part + h * kEpiParts) * kEpiCols;
+                        if (row0 < l_rows && f0 < l_out) tma_store_2d(&L.map_y, buf, f0, row0);
+                        bulk_commit_group();
+                    }
+                }
+                if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+        if (lane == 0) bulk_wait_group_all();
+        __syncwarp();
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        for (int i = 0; i < 200; ++i) __nanosleep(10000);
+    }
+    cluster_arrive();
+    cluster_wait();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc_pair(tmem_base, kTmemCols);
+    }
+}
+
+// Token rows per pair tile for a layer of this input width: the largest multiple of 32, at most
+// kMaxRowTile, that leaves room for the weight block and its metadata; 0 if none does.
+int ws_row_tile(int in)
+{
+    const int left = kTmemCols - in / 4 - in / 32;
+    int nt = left / kNumAccum / 32 * 32;
+    static_assert(kNumAccum == 1, "one accumulator: see the head of this file");
+    if (nt > kMaxRowTile) nt = kMaxRowTile;
+    return nt >= 64 ? nt : 0;
+}
+
+template <bool kBf16, int kMaxLayers>
+elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
+                            const DeviceInfo& dev)
+{
+    auto kernel = linear_tc_sp24_ws_kernel<kBf16, kMaxLayers>;
+    const int fixed = kStagingTotal + kBarrierBytes + 1024;
+    int stages = (int)((dev.smem_optin - fixed) / kStageBytes);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
+    const size_t smem = (size_t)stages * kStageBytes + fixed;
+
+    static int max_pairs[64] = {};
+    const int slot = dev.device & 63;
+    if (max_pairs[slot] == 0) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
+            cudaSuccess) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        }
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.gridDim = dim3((unsigned)dev.sm_count);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int m = 0;
+        if (cudaOccupancyMaxActiveClusters(&m, kernel, &cfg) != cudaSuccess || m < 1) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
+        }
+        max_pairs[slot] = m;
+    }
+    const int pairs = max_pairs[slot];
+
+    static WsGroup<kMaxLayers> g;   // host staging of the kernel parameters
+    static std::mutex g_mutex;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
+    int used_pairs = 0;
+    for (int i = 0; i < n; ++i) {
+        const SparseJob& j = jobs[i];
+        WsLayer& L = g.layer[i];
+        L.nt = ws_row_tile(j.in);
+        L.tiles_f = (j.out + kPairFeat - 1) / kPairFeat;
+        if (L.nt == 0 || j.in % kBlockK != 0 || L.tiles_f > pairs)
+            return fail(ELSA_ERR_SHAPE, "in=%d out=%d does not fit the weight-stationary sparse kernel", j.in, j.out);
+        L.rows = j.rows; L.out = j.out; L.in = j.in;
+        L.row_tiles = (j.rows + L.nt - 1) / L.nt;
+        L.groups = pairs / L.tiles_f;
+        if (L.groups > L.row_tiles) L.groups = L.row_tiles;
+        if (L.groups * L.tiles_f > used_pairs) used_pairs = L.groups * L.tiles_f;
+        L.num_k_blocks = j.in / kBlockK;
+        L.bias = j.bias;
+        L.a_img = (const uint16_t*)j.workspace;
+        L.meta = (const uint8_t*)j.workspace + round_up((size_t)j.out * (size_t)j.in, 256);
+        // sparse flag, fp32 accumulate, A and B of type fmt, K-major, N = nt, M = 256 over the pair
+        L.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.nt >> 3) << 17) |
+                  ((uint32_t)(kPairFeat >> 4) << 24);
+        elsa_status st;
+        if ((st = make_map_x_quarters(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, (uint32_t)(L.nt / 2))) != ELSA_OK) return st;
+        if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B,
+                              "Y")) != ELSA_OK)
+            return st;
+    }
+    g.n_layers = n;
+    g.stages = stages;
+    g.dev_status = dev_status;
+
+    ProfileScope scope(ELSA_KERNEL_LINEAR_TC_SP24_WS, stream);
+    cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * used_pairs)), dim3(kThreads), smem, stream, 2, g);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(ELSA_ERR_CUDA, "launch of linear_tc_sp24_ws failed: %s", cudaGetErrorString(e));
+    }
+    return launched("linear_tc_sp24_ws");
+}
+
+}  // namespace
+
+int linear_tc_sparse_ws_group_max() { return kGroupMax; }
+
+bool linear_tc_sparse_ws_suits(int in, int out, int N, int sm_count)
+{
+    return linear_tc_sparse_suits(in, N) && in % kBlockK == 0 && in <= kMaxIn && ws_row_tile(in) != 0 &&
+           (out + kPairFeat - 1) / kPairFeat <= sm_count / 2;
+}
+
+elsa_status launch_linear_tc_sparse_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                             cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    if (n == 1)
+        return dtype == ELSA_BF16 ? launch_ws_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_ws_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_ws_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_ws_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+}
+
+elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                       const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
+                                       void* workspace, uint32_t* dev_status, cudaStream_t stream)
+{
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, workspace, stream);
+    if (st != ELSA_OK) return st;
+    SparseJob job;
+    job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;
+    job.rows = rows; job.in = in; job.out = out;
+    return launch_linear_tc_sparse_ws_group(&job, 1, dtype, dev_status, stream);
+}
+
+}  // namespace elsa

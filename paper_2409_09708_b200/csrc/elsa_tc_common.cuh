@@ -214,6 +214,20 @@ __device__ __forceinline__ uint32_t cluster_ctarank()
     return r;
 }
 
+// True in exactly one lane of the (converged) warp.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t e;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xFFFFFFFF;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(e));
+    return e != 0;
+}
+
 // Address, in the cluster's shared window, of this CTA's shared address `addr` inside CTA `rank`.
 __device__ __forceinline__ uint32_t mapa_shared(uint32_t addr, uint32_t rank)
 {

@@ -25,7 +25,8 @@ def main():
     ap.add_argument("--level", default="2:8")
     ap.add_argument("--dtype", default="bf16", choices=["f16", "bf16"])
     ap.add_argument("--reps", type=int, default=3)
-    ap.add_argument("--variant", default="auto", choices=["auto", "simt", "tc_dense", "tc_pair", "tc_sparse", "tc_sparse_pair"])
+    ap.add_argument("--variant", default="auto", choices=["auto", "simt", "tc_dense", "tc_pair", "tc_sparse", "tc_sparse_pair",
+                                                            "tc_sparse_ws"])
     args = ap.parse_args()
     N, M = (int(v) for v in args.level.split(":"))
     dtype = synth.torch_dtype(args.dtype)
@@ -37,7 +38,8 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     lib.elsa_set_linear_variant({"auto": lib.VARIANT_AUTO, "simt": lib.VARIANT_SIMT,
                                  "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR, "tc_sparse": lib.VARIANT_TC_SPARSE,
-                                 "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR}[args.variant])
+                                 "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR,
+                                 "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS}[args.variant])
     times = []
     for _ in range(args.reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

@@ -122,7 +122,7 @@ VARIANTS = ["simt", "tc_dense", "tc_pair"]
 def variant_code(lib, name):
     return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
             "tc_sparse": lib.VARIANT_TC_SPARSE, "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR,
-            "auto": lib.VARIANT_AUTO}[name]
+            "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS, "auto": lib.VARIANT_AUTO}[name]
 
 
 LINEAR_CASES = [
@@ -222,6 +222,55 @@ def test_sparse_mma_variant_exact_cases_and_refusals(lib, variant):
     for N, M in [(4, 8), (3, 4), (8, 8)]:                      # more than 2 per chunk possible: refused
         with pytest.raises(lib.ElsaError):
             run_linear(lib, X, W, bias, N, M, code)
+
+
+WS_CASES = [
+    # rows, in, out, N, M: weight block resident in tensor memory (in % 128 == 0, in <= 1024); ragged row
+    # tiles, a half-empty feature block, more row tiles than row groups, the narrower tile of in = 1024
+    (197, 768, 768, 2, 8), (500, 128, 384, 1, 4), (449, 512, 200, 2, 16), (300, 1024, 136, 1, 16),
+    (2300, 768, 2304, 2, 8), (40000, 256, 520, 2, 4), (9000, 1024, 1024, 1, 8), (1, 128, 8, 1, 4),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("case", WS_CASES)
+def test_weight_stationary_sparse_variant_matches_oracle(lib, case, dtype):
+    rows, in_, out, N, M = case
+    X = synth.randn((rows, in_), 31 * rows + in_, synth.X_STD, dtype)
+    W = synth.randn((out, in_), 37 * out + in_, synth.W_STD, dtype)
+    bias = synth.randn((out,), 41 * out, synth.B_STD, dtype)
+    Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE_WS)
+    if rows <= 4096:
+        check_close(Y, oracle_linear(X, W, bias, N, M, dtype))
+    else:                                                   # sampled rows: first, last, and a seeded spread
+        pick = torch.from_numpy(synth.sample_rows(rows, 512, 7))
+        check_close(Y.cpu()[pick], oracle_linear(X[pick], W, bias, N, M, dtype))
+
+
+def test_weight_stationary_sparse_variant_exact_cases_and_refusals(lib):
+    code = lib.VARIANT_TC_SPARSE_WS
+    dtype = torch.float16
+    W = synth.randn((320, 256), 5, synth.W_STD, dtype)
+    bias = synth.randn((320,), 6, synth.B_STD, dtype)
+    X = torch.eye(256, dtype=dtype)
+    for N, M in [(2, 8), (1, 4), (2, 4), (1, 16)]:
+        Y = run_linear(lib, X, W, bias, N, M, code)
+        expect = torch.from_numpy(oracle_linear(X, W, bias, N, M, dtype)).to(dtype)
+        assert torch.equal(Y.cpu(), expect), (N, M)
+    rng = np.random.default_rng(5)
+    Xi = torch.from_numpy(rng.integers(-4, 5, (300, 384))).to(torch.bfloat16)
+    Wi = torch.from_numpy(rng.integers(-8, 9, (96, 384))).to(torch.bfloat16)
+    for N, M in [(2, 4), (1, 8), (2, 16)]:
+        Y = run_linear(lib, Xi, Wi, None, N, M, code)
+        ref = oracle_linear(Xi, Wi, None, N, M, torch.bfloat16)
+        assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
+    for N, M in [(4, 8), (3, 4), (8, 8)]:                      # more than 2 per chunk possible: refused
+        with pytest.raises(lib.ElsaError):
+            run_linear(lib, X, W, bias, N, M, code)
+    with pytest.raises(lib.ElsaError):                         # K block of 128 does not divide in
+        run_linear(lib, torch.eye(192, dtype=dtype), synth.randn((64, 192), 7, synth.W_STD, dtype), None, 2, 4, code)
+    with pytest.raises(lib.ElsaError):                         # weight block larger than tensor memory
+        run_linear(lib, torch.zeros((8, 2048), dtype=dtype), synth.randn((64, 2048), 8, synth.W_STD, dtype), None, 2, 4, code)
 
 
 def test_no_bias_and_zero_rows_of_padding(lib):
