@@ -164,8 +164,14 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
     // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K is
     // long enough for the mainloop to outweigh its heavier epilogue (K >= 768) and there are enough 256 x 224
     // tiles to fill the CTA pairs; shorter K ties or loses and stays on the dense-rate path.
-    if (sparse_ok && in >= 768 && (long long)((rows + 223) / 224) * ((out + 255) / 256) >= sm_count / 4)
-        *kind = KIND_SPARSE_PAIR;
+    if (sparse_ok && in >= 768 && (long long)((rows + 223) / 224) * ((out + 255) / 256) >= sm_count / 4) {
+        // With the weight block resident in tensor memory the activations are the only shared-memory
+        // traffic; measured faster than streaming the weight for K around 768 once a layer has at least
+        // four blocks of 256 features (qkv, fc1: 10-15 %), equal or slower elsewhere.
+        const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in >= 640 && in <= 896 && out >= 1024 &&
+                        rows >= 256 * (sm_count / 2) / ((out + 255) / 256);
+        *kind = ws ? KIND_SPARSE_WS : KIND_SPARSE_PAIR;
+    }
     else
         *kind = linear_tc_pair_suits(rows, out, sm_count) ? KIND_DENSE_PAIR : KIND_DENSE_ONE;
     return ELSA_OK;

@@ -101,7 +101,9 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
 
     if (warp == 0) {
         // ------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // whole warp converged, one elected lane issues (see the MMA warp)
+        {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -110,12 +112,16 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                 const int n0 = (tile % p.tiles_n) * p.bn;
                 for (int kb = 0; kb < p.num_k_blocks; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     const uint32_t a_dst = smem_base + (uint32_t)(stage * stage_bytes);
                     const uint32_t bar = full_bar + 8 * stage;
-                    mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
-                    tma_load_2d(a_dst, &map_x, bar, kb * kBlockK, m0);
-                    tma_load_2d(a_dst + kATileBytes, &map_w, bar, kb * kBlockK, n0);
+                    if (elected) {
+                        mbar_arrive_expect_tx(bar, (uint32_t)stage_bytes);
+                        tma_load_2d(a_dst, &map_x, bar, kb * kBlockK, m0);
+                        tma_load_2d(a_dst + kATileBytes, &map_w, bar, kb * kBlockK, n0);
+                    }
+                    __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -123,7 +129,11 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // The whole warp walks the loop with its operands in uniform registers; only the tensor-core
+        // instructions are predicated on one elected lane (a single thread inside a divergent branch
+        // needs about twice as long per MMA).
+        {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -131,11 +141,13 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kMaxBlockN);
                 for (int kb = 0; kb < p.num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + (uint32_t)(stage * stage_bytes);
@@ -145,14 +157,15 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the
                         // 16-byte-unit start address field
-                        umma_f16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
-                                 (uint32_t)((kb | k) != 0));
+                        if (elected)
+                            umma_f16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
+                                     (uint32_t)((kb | k) != 0));
                     }
-                    umma_commit(empty_bar + 8 * stage);  // frees the stage once these MMAs have read it
+                    if (elected) umma_commit(empty_bar + 8 * stage);  // frees the stage once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit(tmem_full_bar + 8 * acc);    // accumulator complete
+                if (elected) umma_commit(tmem_full_bar + 8 * acc);    // accumulator complete
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }

@@ -119,7 +119,9 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
 
     if (warp == 0) {
         // ------------------------------------------------ producer (both CTAs)
-        if (lane == 0) {
+        // whole warp converged, one elected lane issues (see the MMA warp)
+        {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -132,15 +134,19 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                 const int r0 = (t / L.tiles_f) * kRowTile + (int)cta_rank * kRowsPerCta;
                 for (int kb = 0; kb < L.num_k_blocks; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     const uint32_t a_dst = smem_base + (uint32_t)(stage * kStageBytes);
-                    if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, (uint32_t)(2 * kStageBytes));
                     const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
-                    tma_load_2d_pair(a_dst, &L.map_a, bar, kb * (kBlockK / 2), ft128 * kFeatPerCta);
-                    tma_load_2d_pair(a_dst + kATileBytes, &L.map_x, bar, kb * kBlockK, r0);
-                    tma_load_2d_pair(a_dst + kATileBytes + kBSubBytes, &L.map_x, bar, kb * kBlockK + 64, r0);
-                    tma_load_2d_pair(a_dst + kATileBytes + kBTileBytes, &L.map_e, bar, 0,
-                                     (ft128 * L.num_k_blocks + kb) * 128);
+                    if (elected) {
+                        if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, (uint32_t)(2 * kStageBytes));
+                        tma_load_2d_pair(a_dst, &L.map_a, bar, kb * (kBlockK / 2), ft128 * kFeatPerCta);
+                        tma_load_2d_pair(a_dst + kATileBytes, &L.map_x, bar, kb * kBlockK, r0);
+                        tma_load_2d_pair(a_dst + kATileBytes + kBSubBytes, &L.map_x, bar, kb * kBlockK + 64, r0);
+                        tma_load_2d_pair(a_dst + kATileBytes + kBTileBytes, &L.map_e, bar, 0,
+                                         (ft128 * L.num_k_blocks + kb) * 128);
+                    }
+                    __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -148,7 +154,11 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && cta_rank == 0) {
+        // The whole warp walks the loop with its operands in uniform registers; only the tensor-core
+        // instructions are predicated on one elected lane (a single thread inside a divergent branch
+        // needs about twice as long per MMA).
+        if (cta_rank == 0) {
+            const bool elected = elect_one();
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -159,11 +169,13 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                 while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
                 const int num_k_blocks = p.layer[cur].num_k_blocks;
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
+                ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + (uint32_t)(stage * kStageBytes);
@@ -172,19 +184,21 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                     const uint64_t b_desc1 = smem_desc_k_major_sw128(a_addr + kATileBytes + kBSubBytes);
                     const uint32_t e_col = tmem_base + (uint32_t)(kMetaCol0 + 4 * stage);
                     // each CTA's metadata block into its own tensor memory; runs before the MMAs below
-                    tmem_cp_128x128b_pair(e_col, smem_desc_rows16_no_swizzle(a_addr + kATileBytes + kBTileBytes));
+                    const uint64_t e_desc = smem_desc_rows16_no_swizzle(a_addr + kATileBytes + kBTileBytes);
+                    if (elected) tmem_cp_128x128b_pair(e_col, e_desc);
 #pragma unroll
                     for (int j = 0; j < kBlockK / kSpUmmaK; ++j) {
                         // K step of 32: 32 bytes of compressed A, 64 bytes of B in the half that holds it
                         const uint64_t b_desc = (j < 2 ? b_desc0 : b_desc1) + (uint64_t)(4 * (j & 1));
-                        umma_sp_f16_pair(d_tmem, a_desc + (uint64_t)(2 * j), b_desc, e_col + (uint32_t)j, p.idesc,
-                                         (uint32_t)((kb | j) != 0));
+                        if (elected)
+                            umma_sp_f16_pair(d_tmem, a_desc + (uint64_t)(2 * j), b_desc, e_col + (uint32_t)j, p.idesc,
+                                             (uint32_t)((kb | j) != 0));
                     }
-                    umma_commit_pair(empty_bar + 8 * stage, 3);
+                    if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                umma_commit_pair(tmem_full_bar + 8 * acc, 3);
+                if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }
@@ -232,18 +246,21 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                 __syncwarp();
                 // staging tile [32 token rows][32 features], 64-byte rows with the 64-byte swizzle; this lane
                 // writes the feature pair (lane & ~1, lane | 1) of one row per row pair
+                // (all exchanges first, then all stores: interleaved, each store would wait for its shuffle)
+                uint32_t word[16];
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     // own feature, token rows j (low half) and j + 1 (high half), rounded once
                     const uint32_t own = pack2<kBf16>(__uint_as_float(r[j]) + bias_f, __uint_as_float(r[j + 1]) + bias_f);
                     const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, own, 1);
                     // even lane: row j of (own, right neighbour); odd lane: row j + 1 of (left neighbour, own)
-                    uint32_t word;
-                    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(word) : "r"(odd ? got : own), "r"(odd ? own : got), "r"(prmt_sel));
-                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + lane_off + (uint32_t)(j * 64) + sw_off[(j >> 1) & 3]),
-                                 "r"(word)
-                                 : "memory");
+                    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(word[j >> 1]) : "r"(odd ? got : own), "r"(odd ? own : got), "r"(prmt_sel));
                 }
+#pragma unroll
+                for (int j = 0; j < 32; j += 2)
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + lane_off + (uint32_t)(j * 64) + sw_off[(j >> 1) & 3]),
+                                 "r"(word[j >> 1])
+                                 : "memory");
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {

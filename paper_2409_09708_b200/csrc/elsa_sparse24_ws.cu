@@ -239,6 +239,9 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
         // cycles), and an MMA of 128 token rows lasts only 64 cycles.
         if (cta_rank == 0) {
             const bool elected = elect_one();
+            // the base address was read from shared memory into an ordinary register; a warp reduction
+            // returns it in a uniform one, so that every address derived from it stays uniform too
+            const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -256,7 +259,7 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                 if (!ok) break;
                 w_phase ^= 1u;
                 tc_fence_after();
-                const uint32_t a_col0 = tmem_base + (uint32_t)(kNumAccum * L.nt);
+                const uint32_t a_col0 = tmem_u + (uint32_t)(kNumAccum * L.nt);
                 const uint32_t e_col0 = a_col0 + (uint32_t)(L.in >> 2);
                 const uint32_t idesc = L.idesc;
                 const int num_k_stages = (L.in + kStageK - 1) / kStageK;
@@ -267,7 +270,7 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(acc * L.nt);
+                    const uint32_t d_tmem = tmem_u + (uint32_t)(acc * L.nt);
                     for (int ks = 0; ks < num_k_stages; ++ks) {
                         ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                         if (!ok) break;
