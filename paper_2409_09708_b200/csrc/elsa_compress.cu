@@ -77,43 +77,73 @@ __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 nm_compress_batch_kernel(const __grid_constant__ BatchTable t)
 {
     __shared__ uint32_t words[kWarpsPerBlock][kMaxIndexWordsPerSegment];
-    const long long unit = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     pdl_wait_for_predecessors();
     pdl_release_successors();
-    if (unit >= t.total_units) return;
-    const BatchItem& it = t.item[find_item(t, unit)];
-    const long long seg_id = unit - it.first_unit;
-    const uint16_t* W = (const uint16_t*)it.src;
-    uint16_t* vals = (uint16_t*)it.dst;
-    uint32_t* idx = (uint32_t*)it.dst2;
-    if (it.M == 4) compress_segment<4>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
-    else if (it.M == 8) compress_segment<8>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
-    else compress_segment<16>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+    // A block owns a contiguous range of units and its warps walk it side by side; the table is searched
+    // once per block and stepped through afterwards (a search per unit costs several dependent reads of
+    // kernel-parameter memory, more than the unit's own work).
+    const long long per_block = (t.total_units + gridDim.x - 1) / gridDim.x;
+    const long long begin = (long long)blockIdx.x * per_block;
+    const long long end = begin + per_block < t.total_units ? begin + per_block : t.total_units;
+    if (begin >= end) return;
+    int cur = find_item(t, begin);
+    long long cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
+    BatchItem it = t.item[cur];
+    for (long long unit = begin + (threadIdx.x >> 5); unit < end; unit += kWarpsPerBlock) {
+        if (unit >= cur_end) {
+            while (unit >= cur_end) {
+                ++cur;
+                cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
+            }
+            it = t.item[cur];
+        }
+        const long long seg_id = unit - it.first_unit;
+        const uint16_t* W = (const uint16_t*)it.src;
+        uint16_t* vals = (uint16_t*)it.dst;
+        uint32_t* idx = (uint32_t*)it.dst2;
+        if (it.M == 4) compress_segment<4>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+        else if (it.M == 8) compress_segment<8>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+        else compress_segment<16>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+    }
 }
 
 __global__ void __launch_bounds__(256)
 nm_image_batch_kernel(const __grid_constant__ BatchTable t)
 {
-    const long long unit = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
-    if (unit >= t.total_units) return;
-    const BatchItem& it = t.item[find_item(t, unit)];
-    const long long local = unit - it.first_unit;
-    const uint16_t* vals = (const uint16_t*)it.src;
-    const uint32_t* idx = (const uint32_t*)it.src2;
-    if (it.kind == BATCH_UNPACK) {
-        uint16_t* Wm = (uint16_t*)it.dst;
-        if (it.M == 4) unpack_group<4>(vals, idx, it.in, it.N, Wm, it.wpr, local);
-        else if (it.M == 8) unpack_group<8>(vals, idx, it.in, it.N, Wm, it.wpr, local);
-        else unpack_group<16>(vals, idx, it.in, it.N, Wm, it.wpr, local);
-    } else {
-        uint16_t* a_img = (uint16_t*)it.dst;
-        uint16_t* meta16 = (uint16_t*)it.dst2;
-        // aux = K blocks of the metadata layout, aux2 = K steps per block
-        if (it.M == 4) to_sp24_segment<4>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
-        else if (it.M == 8) to_sp24_segment<8>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
-        else to_sp24_segment<16>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
+    // contiguous range of units per block, table searched once per block (see the compress kernel)
+    const long long per_block = (t.total_units + gridDim.x - 1) / gridDim.x;
+    const long long begin = (long long)blockIdx.x * per_block;
+    const long long end = begin + per_block < t.total_units ? begin + per_block : t.total_units;
+    if (begin >= end) return;
+    int cur = find_item(t, begin);
+    long long cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
+    BatchItem it = t.item[cur];
+    for (long long unit = begin + threadIdx.x; unit < end; unit += blockDim.x) {
+        if (unit >= cur_end) {
+            while (unit >= cur_end) {
+                ++cur;
+                cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
+            }
+            it = t.item[cur];
+        }
+        const long long local = unit - it.first_unit;
+        const uint16_t* vals = (const uint16_t*)it.src;
+        const uint32_t* idx = (const uint32_t*)it.src2;
+        if (it.kind == BATCH_UNPACK) {
+            uint16_t* Wm = (uint16_t*)it.dst;
+            if (it.M == 4) unpack_group<4>(vals, idx, it.in, it.N, Wm, it.wpr, local);
+            else if (it.M == 8) unpack_group<8>(vals, idx, it.in, it.N, Wm, it.wpr, local);
+            else unpack_group<16>(vals, idx, it.in, it.N, Wm, it.wpr, local);
+        } else {
+            uint16_t* a_img = (uint16_t*)it.dst;
+            uint16_t* meta16 = (uint16_t*)it.dst2;
+            // aux = K blocks of the metadata layout, aux2 = K steps per block
+            if (it.M == 4) to_sp24_segment<4>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
+            else if (it.M == 8) to_sp24_segment<8>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
+            else to_sp24_segment<16>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, local);
+        }
     }
 }
 
@@ -222,18 +252,28 @@ void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx,
 elsa_status launch_compress_batch(const BatchTable& t, cudaStream_t stream)
 {
     if (t.n == 0) return ELSA_OK;
-    const unsigned grid = (unsigned)((t.total_units + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    long long grid = (t.total_units + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    const long long waves = (long long)dev.sm_count * (2048 / (kWarpsPerBlock * 32)) * 4;   // a few waves of resident blocks
+    if (grid > waves) grid = waves;
     ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
-    launch_pdl(nm_compress_batch_kernel, dim3(grid), dim3(kWarpsPerBlock * 32), 0, stream, 1, t);
+    launch_pdl(nm_compress_batch_kernel, dim3((unsigned)grid), dim3(kWarpsPerBlock * 32), 0, stream, 1, t);
     return launched("nm_compress (batched)");
 }
 
 elsa_status launch_image_batch(const BatchTable& t, cudaStream_t stream)
 {
     if (t.n == 0) return ELSA_OK;
-    const unsigned grid = (unsigned)((t.total_units + 255) / 256);
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    long long grid = (t.total_units + 255) / 256;
+    const long long waves = (long long)dev.sm_count * 8 * 4;
+    if (grid > waves) grid = waves;
     ProfileScope scope(ELSA_KERNEL_WEIGHT_IMAGES, stream);
-    launch_pdl(nm_image_batch_kernel, dim3(grid), dim3(256), 0, stream, 1, t);
+    launch_pdl(nm_image_batch_kernel, dim3((unsigned)grid), dim3(256), 0, stream, 1, t);
     return launched("weight images (batched)");
 }
 
