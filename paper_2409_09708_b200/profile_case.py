@@ -5,6 +5,10 @@
 
 Prints one JSON line with the CUDA-event time of each repetition (compress once, then `reps`
 calls of elsa_nm_linear), the layer's algorithmic bytes and kept FLOPs.
+
+    python -m paper_2409_09708_b200.profile_case --compress-table deit_b_stack_b256 --reps 3
+
+runs elsa_vit_compress over the weights of a workload table instead (weights only, no activations).
 """
 from __future__ import annotations
 
@@ -17,6 +21,31 @@ from . import binding as lib
 from . import synth
 
 
+def compress_table(workload, reps):
+    layers, dt = synth.workload(workload)
+    dtype = synth.torch_dtype(dt)
+    dev = []
+    for l in layers:
+        W = synth.randn((l.out, l.in_), l.seed_w, synth.W_STD, dtype, device="cuda")
+        vals, idx = lib.alloc_packed(l.out, l.in_, l.N, l.M, dtype)
+        dev.append(dict(W=W, vals=vals, idx=idx, N=l.N, M=l.M))
+    table = lib.make_weight_table(dev)
+    code = lib.dtype_code(dtype)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for rep in range(reps):
+        flush.fill_(rep)                          # the weights leave L2 between repetitions
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        lib.elsa_vit_compress(table, code)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    nbytes = sum(l.out * l.in_ * 2 + lib.elsa_nm_values_bytes(l.out, l.in_, l.N, l.M, code) +
+                 lib.elsa_nm_index_bytes(l.out, l.in_, l.N, l.M) for l in layers)
+    print(json.dumps({"workload": workload, "weights": len(layers), "ms": times, "bytes_read_and_written": nbytes}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--rows", type=int, default=50432)
@@ -27,7 +56,10 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--variant", default="auto", choices=["auto", "simt", "tc_dense", "tc_pair", "tc_sparse", "tc_sparse_pair",
                                                             "tc_sparse_ws"])
+    ap.add_argument("--compress-table", default=None, help="workload whose weights go through elsa_vit_compress")
     args = ap.parse_args()
+    if args.compress_table:
+        return compress_table(args.compress_table, args.reps)
     N, M = (int(v) for v in args.level.split(":"))
     dtype = synth.torch_dtype(args.dtype)
     layer = synth.Layer("case", args.rows, args.in_, args.out, N, M, 1, 2, 3)
