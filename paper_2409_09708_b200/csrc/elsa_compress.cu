@@ -16,11 +16,17 @@ nm_compress_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint1
                    uint32_t* __restrict__ idx, int segs_per_row, int words_per_row)
 {
     __shared__ uint32_t words[kWarpsPerBlock][kMaxIndexWordsPerSegment];
+    __shared__ CompactEntry table[M == 16 ? 1 : (1 << M)];
+    if constexpr (M != 16) {
+        build_compact_table<M>(table);
+        __syncthreads();
+    }
     const long long seg_id = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     pdl_wait_for_predecessors();
     pdl_release_successors();
-    if (seg_id >= (long long)out * segs_per_row) return;  // whole warps leave together; no block-wide barrier is used
-    compress_segment<M>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
+    if (seg_id >= (long long)out * segs_per_row) return;  // whole warps leave together; no block-wide barrier follows
+    if constexpr (M == 16) compress_segment<M>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
+    else compress_segment_fast<M>(W, in, N, vals, idx, segs_per_row, seg_id, words, table);
 }
 
 template <int M>
@@ -73,10 +79,24 @@ __device__ __forceinline__ int find_item(const BatchTable& t, long long unit)
     return lo;
 }
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+// Groups of 16 take the general path; kept out of line so that its registers do not count against the
+// fast path of the batched kernel.
+__device__ __noinline__ void compress_segment16_call(const uint16_t* W, int in, int N, uint16_t* vals, uint32_t* idx,
+                                                     int segs_per_row, int words_per_row, long long seg_id,
+                                                     uint32_t (*words)[kMaxIndexWordsPerSegment])
+{
+    compress_segment<16>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
+}
+
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 5)
 nm_compress_batch_kernel(const __grid_constant__ BatchTable t)
 {
     __shared__ uint32_t words[kWarpsPerBlock][kMaxIndexWordsPerSegment];
+    __shared__ CompactEntry table8[256];
+    __shared__ CompactEntry table4[16];
+    build_compact_table<8>(table8);
+    build_compact_table<4>(table4);
+    __syncthreads();
     pdl_wait_for_predecessors();
     pdl_release_successors();
     // A block owns a contiguous range of units and its warps walk it side by side; the table is searched
@@ -88,22 +108,21 @@ nm_compress_batch_kernel(const __grid_constant__ BatchTable t)
     if (begin >= end) return;
     int cur = find_item(t, begin);
     long long cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
-    BatchItem it = t.item[cur];
     for (long long unit = begin + (threadIdx.x >> 5); unit < end; unit += kWarpsPerBlock) {
         if (unit >= cur_end) {
             while (unit >= cur_end) {
                 ++cur;
                 cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
             }
-            it = t.item[cur];
         }
+        const BatchItem& it = t.item[cur];
         const long long seg_id = unit - it.first_unit;
         const uint16_t* W = (const uint16_t*)it.src;
         uint16_t* vals = (uint16_t*)it.dst;
         uint32_t* idx = (uint32_t*)it.dst2;
-        if (it.M == 4) compress_segment<4>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
-        else if (it.M == 8) compress_segment<8>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
-        else compress_segment<16>(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+        if (it.M == 4) compress_segment_fast<4>(W, it.in, it.N, vals, idx, it.aux, seg_id, words, table4);
+        else if (it.M == 8) compress_segment_fast<8>(W, it.in, it.N, vals, idx, it.aux, seg_id, words, table8);
+        else compress_segment16_call(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
     }
 }
 

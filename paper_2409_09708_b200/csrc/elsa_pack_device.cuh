@@ -137,6 +137,162 @@ __device__ __forceinline__ void compress_segment_levels(const uint16_t* __restri
     }
 }
 
+// ---- single-level fast path for M = 4 and M = 8 (the levels of the ViT tables) -------------------
+//
+// Same result as compress_segment_levels with one level, in about a third of the instructions:
+//   * every position gets a unique key (magnitude bits above, M-1-position below), so "the N of largest
+//     magnitude, lowest position first among equals" is "key >= the N-th largest key";
+//   * the N-th largest key comes from a sorting network (5 / 19 compare-exchanges);
+//   * kept values are compacted with byte permutes driven by a small table in shared memory: for each
+//     keep mask, the kept positions in ascending order as 4-bit fields (the permute selectors) and as
+//     log2(M)-bit fields (the index bits to store);
+//   * one vector store per group for the values.
+struct CompactEntry { uint32_t order4; uint32_t fields; };
+
+template <int M>
+__device__ __forceinline__ void build_compact_table(CompactEntry* table)
+{
+    constexpr int B = (M == 4) ? 2 : 3;
+    for (int m = threadIdx.x; m < (1 << M); m += blockDim.x) {
+        uint32_t o4 = 0, f = 0;
+        int t = 0;
+        for (int i = 0; i < M; ++i)
+            if ((m >> i) & 1) { o4 |= (uint32_t)i << (4 * t); f |= (uint32_t)i << (B * t); ++t; }
+        table[m].order4 = o4;
+        table[m].fields = f;
+    }
+}
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t r;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
+    return r;
+}
+
+__device__ __forceinline__ void sort2_desc(uint32_t& a, uint32_t& b)
+{
+    const uint32_t hi = max(a, b), lo = min(a, b);
+    a = hi; b = lo;
+}
+
+// Keep mask of one group: bit i set iff position i is among the N kept.  h[] are the 16-bit patterns.
+template <int M>
+__device__ __forceinline__ uint32_t keep_mask_sorted(const uint32_t (&h)[M], int N)
+{
+    constexpr int S = (M == 4) ? 2 : 3;
+    uint32_t k[M], s[M];
+#pragma unroll
+    for (int i = 0; i < M; ++i) { k[i] = ((h[i] & 0x7FFFu) << S) | (uint32_t)(M - 1 - i); s[i] = k[i]; }
+    if constexpr (M == 4) {
+        sort2_desc(s[0], s[1]); sort2_desc(s[2], s[3]);
+        sort2_desc(s[0], s[2]); sort2_desc(s[1], s[3]);
+        sort2_desc(s[1], s[2]);
+    } else {
+        sort2_desc(s[0], s[1]); sort2_desc(s[2], s[3]); sort2_desc(s[4], s[5]); sort2_desc(s[6], s[7]);
+        sort2_desc(s[0], s[2]); sort2_desc(s[1], s[3]); sort2_desc(s[4], s[6]); sort2_desc(s[5], s[7]);
+        sort2_desc(s[1], s[2]); sort2_desc(s[5], s[6]);
+        sort2_desc(s[0], s[4]); sort2_desc(s[1], s[5]); sort2_desc(s[2], s[6]); sort2_desc(s[3], s[7]);
+        sort2_desc(s[2], s[4]); sort2_desc(s[3], s[5]);
+        sort2_desc(s[1], s[2]); sort2_desc(s[3], s[4]); sort2_desc(s[5], s[6]);
+    }
+    uint32_t thr = s[0];
+#pragma unroll
+    for (int t = 1; t < M; ++t) thr = (N > t) ? s[t] : thr;      // the N-th largest key
+    uint32_t keep = 0;
+#pragma unroll
+    for (int i = 0; i < M; ++i) keep |= (k[i] >= thr ? 1u : 0u) << i;
+    return keep;
+}
+
+template <int M>
+__device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict__ W, int in, int N,
+                                                      uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                      int segs_per_row, long long seg_id,
+                                                      uint32_t (*words)[kMaxIndexWordsPerSegment],
+                                                      const CompactEntry* table)
+{
+    static_assert(M == 4 || M == 8, "fast path for groups of 4 and 8");
+    constexpr int B = (M == 4) ? 2 : 3;
+    constexpr int R = M / 2;                      // 32-bit registers per group
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int o = (int)(seg_id / segs_per_row);
+    const int seg = (int)(seg_id % segs_per_row);
+    const int groups_per_row = in / M;
+    const int g = seg * 32 + lane;
+    const bool valid = g < groups_per_row;
+    const int words_per_row = (N == M) ? 0 : (groups_per_row * N * B + 31) / 32;
+    const int seg_words = N * B;
+
+    uint32_t r[R];
+#pragma unroll
+    for (int q = 0; q < R; ++q) r[q] = 0;
+    if (valid) {
+        const uint16_t* src = W + (size_t)o * in + (size_t)g * M;
+        if constexpr (M == 4) { const uint2 v = *reinterpret_cast<const uint2*>(src); r[0] = v.x; r[1] = v.y; }
+        else { const uint4 v = *reinterpret_cast<const uint4*>(src); r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w; }
+    }
+    uint16_t* dst = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
+    if (N == M) {                                 // dense level: the values are the weight
+        if (valid) {
+            if constexpr (M == 4) *reinterpret_cast<uint2*>(dst) = make_uint2(r[0], r[1]);
+            else *reinterpret_cast<uint4*>(dst) = make_uint4(r[0], r[1], r[2], r[3]);
+        }
+        return;
+    }
+    for (int k = lane; k < seg_words; k += 32) words[warp][k] = 0;
+    __syncwarp();
+    if (valid) {
+        uint32_t h[M];
+#pragma unroll
+        for (int q = 0; q < R; ++q) { h[2 * q] = r[q] & 0xFFFFu; h[2 * q + 1] = r[q] >> 16; }
+        const uint32_t keep = keep_mask_sorted<M>(h, N);
+        const CompactEntry e = table[keep];
+        // low and high bytes of the halfwords as two planes, compacted by the position list, re-interleaved
+        uint32_t w[R];
+        if constexpr (M == 4) {
+            const uint32_t lo = prmt(prmt(r[0], r[1], 0x6420u), 0u, e.order4);
+            const uint32_t hi = prmt(prmt(r[0], r[1], 0x7531u), 0u, e.order4);
+            w[0] = prmt(lo, hi, 0x5140u);
+            w[1] = prmt(lo, hi, 0x7362u);
+        } else {
+            const uint32_t l0 = prmt(r[0], r[1], 0x6420u), l1 = prmt(r[2], r[3], 0x6420u);
+            const uint32_t h0 = prmt(r[0], r[1], 0x7531u), h1 = prmt(r[2], r[3], 0x7531u);
+            const uint32_t lo03 = prmt(l0, l1, e.order4 & 0xFFFFu), lo47 = prmt(l0, l1, e.order4 >> 16);
+            const uint32_t hi03 = prmt(h0, h1, e.order4 & 0xFFFFu), hi47 = prmt(h0, h1, e.order4 >> 16);
+            w[0] = prmt(lo03, hi03, 0x5140u);
+            w[1] = prmt(lo03, hi03, 0x7362u);
+            w[2] = prmt(lo47, hi47, 0x5140u);
+            w[3] = prmt(lo47, hi47, 0x7362u);
+        }
+        // the group's N values are contiguous: the widest store their common alignment allows
+        if ((N & 3) == 0) {
+            *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[1]);          // N = 4 (M = 8)
+        } else if ((N & 1) == 0) {
+#pragma unroll
+            for (int q = 0; q < R; ++q)
+                if (q < (N >> 1)) reinterpret_cast<uint32_t*>(dst)[q] = w[q];
+        } else {
+#pragma unroll
+            for (int t = 0; t < M; ++t)
+                if (t < N) dst[t] = (uint16_t)(w[t >> 1] >> (16 * (t & 1)));
+        }
+        // index bits: at most 21 (M = 8) or 6 (M = 4) bits at bit offset lane * N * B of the segment
+        const int bit0 = lane * seg_words;
+        const int w0 = bit0 >> 5, sh = bit0 & 31;
+        const uint32_t lo = e.fields << sh;
+        const uint32_t hi = sh ? (e.fields >> (32 - sh)) : 0u;
+        if (lo) atomicOr(&words[warp][w0], lo);
+        if (hi) atomicOr(&words[warp][w0 + 1], hi);
+    }
+    __syncwarp();
+    const int first = seg * seg_words;
+    uint32_t* row = idx + (size_t)o * words_per_row;
+    for (int k = lane; k < seg_words && first + k < words_per_row; k += 32) row[first + k] = words[warp][k];
+    __syncwarp();
+}
+
 // Single level: the form elsa_nm_compress uses.
 template <int M>
 __device__ __forceinline__ void compress_segment(const uint16_t* __restrict__ W, int in, int N,
