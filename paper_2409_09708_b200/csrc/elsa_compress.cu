@@ -21,12 +21,15 @@ nm_compress_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint1
         build_compact_table<M>(table);
         __syncthreads();
     }
-    const long long seg_id = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5);
     pdl_wait_for_predecessors();
     pdl_release_successors();
-    if (seg_id >= (long long)out * segs_per_row) return;  // whole warps leave together; no block-wide barrier follows
-    if constexpr (M == 16) compress_segment<M>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
-    else compress_segment_fast<M>(W, in, N, vals, idx, segs_per_row, seg_id, words, table);
+    // warps walk the segments with the stride of the grid (whole warps leave together; no block-wide barrier follows)
+    const long long total = (long long)out * segs_per_row;
+    for (long long seg_id = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); seg_id < total;
+         seg_id += (long long)gridDim.x * kWarpsPerBlock) {
+        if constexpr (M == 16) compress_segment<M>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
+        else compress_segment_fast<M>(W, in, N, vals, idx, segs_per_row, seg_id, words, table);
+    }
 }
 
 template <int M>
@@ -175,7 +178,12 @@ elsa_status launch_compress(const uint16_t* W, int out, int in, int N, int M, ui
     const int segs_per_row = (groups_per_row + 31) / 32;
     const int wpr = (int)index_words_per_row(in, N, M);
     const long long total = (long long)out * segs_per_row;
-    const unsigned grid = (unsigned)((total + kWarpsPerBlock - 1) / kWarpsPerBlock);
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    long long blocks = (total + kWarpsPerBlock - 1) / kWarpsPerBlock;
+    if (blocks > (long long)dev.sm_count * 8) blocks = (long long)dev.sm_count * 8;   // one wave of resident blocks
+    const unsigned grid = (unsigned)blocks;
     const dim3 block(kWarpsPerBlock * 32);
     ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
     if (M == 4)

@@ -176,6 +176,9 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         // single thread inside a divergent branch needs about twice as long to issue one MMA.
         if (cta_rank == 0) {
             const bool elected = elect_one();
+            // the base address came from shared memory in an ordinary register; a warp reduction returns it
+            // in a uniform one, so that the addresses derived from it stay uniform too
+            const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -190,7 +193,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kMaxBlockN);
+                const uint32_t d_tmem = tmem_u + (uint32_t)(acc * kMaxBlockN);
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                     ok = __all_sync(0xFFFFFFFFu, ok);

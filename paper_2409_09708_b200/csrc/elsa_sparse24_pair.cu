@@ -159,6 +159,9 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
         // needs about twice as long per MMA).
         if (cta_rank == 0) {
             const bool elected = elect_one();
+            // the base address came from shared memory in an ordinary register; a warp reduction returns it
+            // in a uniform one, so that the addresses derived from it stay uniform too
+            const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -172,7 +175,7 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kAccStride);
+                const uint32_t d_tmem = tmem_u + (uint32_t)(acc * kAccStride);
                 for (int kb = 0; kb < num_k_blocks; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                     ok = __all_sync(0xFFFFFFFFu, ok);
@@ -182,7 +185,7 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                     const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
                     const uint64_t b_desc0 = smem_desc_k_major_sw128(a_addr + kATileBytes);
                     const uint64_t b_desc1 = smem_desc_k_major_sw128(a_addr + kATileBytes + kBSubBytes);
-                    const uint32_t e_col = tmem_base + (uint32_t)(kMetaCol0 + 4 * stage);
+                    const uint32_t e_col = tmem_u + (uint32_t)(kMetaCol0 + 4 * stage);
                     // each CTA's metadata block into its own tensor memory; runs before the MMAs below
                     const uint64_t e_desc = smem_desc_rows16_no_swizzle(a_addr + kATileBytes + kBTileBytes);
                     if (elected) tmem_cp_128x128b_pair(e_col, e_desc);
