@@ -34,6 +34,14 @@ if ROOT not in sys.path:
 METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
 GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws")   # forms of the tcgen05 GEMM
+
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE grouped launch of each GEMM kernel inside this
+# benchmark's default run, from a one-pass ncu capture of the same command
+# (profiles/bench_deit_b_stack_b256_dram_traffic.md).  Valid for the kernels as captured; set an entry to
+# None when its kernel changes.
+MEASURED_DRAM_TRAFFIC = {
+    "deit_b_stack_b256": {"linear_tc_pair": 8.773e9, "linear_tc_sp24_ws": 4.70e9, "linear_tc_sp24_pair": 3.571e9},
+}
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -277,9 +285,11 @@ def run_ours(args):
         k = per_kernel.setdefault(name, [0, 0.0])
         k[0] += 1
         k[1] += ms
+    layer_kernel = {}                       # which GEMM kernel runs each layer (from the one-launch-per-layer pass)
     for name, layer, ms in recs_layer:
         if name in GEMM_KERNELS and layer >= 0:
             gemm_ms[layer] += ms / layer_steps
+            layer_kernel[layer] = name
         if name in ("nm_unpack", "nm_to_sp24", "weight_images") and layer >= 0:
             unpack_ms[layer] += ms / layer_steps
     kernel_total = sum(v[1] for v in per_kernel.values()) or 1.0
@@ -296,9 +306,16 @@ def run_ours(args):
     peak = peaks["bf16_tflops"] if bound == "tensor" else peaks["hbm_gbs"]
     gemm_launches = sum(per_kernel.get(k, [0, 0.0])[0] for k in GEMM_KERNELS)
     gemm_total_ms = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS)
+    top_kernel = max(GEMM_KERNELS, key=lambda k: per_kernel.get(k, [0, 0.0])[1])
+    top_launches = per_kernel.get(top_kernel, [0, 0.0])[0]
     roofline = {
-        "kernel": max(GEMM_KERNELS, key=lambda k: per_kernel.get(k, [0, 0.0])[1]), "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
-        "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": frac, "traffic": None,
+        "kernel": top_kernel, "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
+        "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": frac,
+        # one launch of `kernel` per step carries all its layers; the capture does not apply otherwise
+        "traffic": MEASURED_DRAM_TRAFFIC.get(args.workload, {}).get(top_kernel) if top_launches == args.steps else None,
+        "traffic_note": "DRAM bytes (read + written) of one launch of `kernel`, which carries all of its layers "
+                        "(ncu, one pass, same command); traffic_algorithmic is the same layers' algorithmic bytes",
+        "traffic_algorithmic": sum(algorithmic_bytes(l) for i, l in enumerate(layers) if layer_kernel.get(i) == top_kernel),
         "peaks": peaks_kind,
         "definition": "per layer max(kept FLOPs / tensor peak, algorithmic bytes / HBM peak), summed over the "
                       "layers, divided by the summed CUDA-event durations of the GEMM launches that ran them "
