@@ -36,9 +36,9 @@ UNIT = "TFLOP/s"
 GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws")   # forms of the tcgen05 GEMM
 
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE grouped launch of each GEMM kernel inside this
-# benchmark's default run, from a one-pass ncu capture of the same command
-# (profiles/bench_deit_b_stack_b256_dram_traffic.md).  Valid for the kernels as captured; set an entry to
-# None when its kernel changes.
+# benchmark's default run, from a one-pass ncu capture of the same command (the two DRAM counters
+# fit one pass, so the full-size run is captured as it is).  Valid for the kernels as captured; set an
+# entry to None when its kernel changes.
 MEASURED_DRAM_TRAFFIC = {
     "deit_b_stack_b256": {"linear_tc_pair": 8.773e9, "linear_tc_sp24_ws": 4.70e9, "linear_tc_sp24_pair": 3.571e9},
 }
@@ -364,8 +364,8 @@ def run_ours(args):
                          "dense_equiv_tflops": l.dense_equiv_flops / gemm_ms[i] / 1e9 if gemm_ms[i] else None,
                          "algorithmic_gbs": algorithmic_bytes(l) / gemm_ms[i] / 1e6 if gemm_ms[i] else None})
         try:
-            os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-            with open(os.path.join(ROOT, "gpurun_out", "bench_layers_%s.json" % args.workload), "w") as f:
+            os.makedirs(os.path.join(ROOT, "bench_out"), exist_ok=True)
+            with open(os.path.join(ROOT, "bench_out", "bench_layers_%s.json" % args.workload), "w") as f:
                 json.dump(rows, f, indent=1)
         except OSError:
             pass

@@ -1,6 +1,6 @@
 """Timing of the supernet-side forms (Sec. 3.1 of the ELSA paper: shared weight, dynamic masking).
 
-    python -m paper_2409_09708_b200.supernet_bench [--out gpurun_out/supernet.json]
+    python -m paper_2409_09708_b200.supernet_bench [--out bench_out/supernet.json]
 
 (a) elsa_nm_compress_levels: all levels {1,2,4,8}:8 of a weight from one read, against one
     elsa_nm_compress call per level, and against the CPU oracle doing the same (GB/s counts the
@@ -38,7 +38,7 @@ def timed(fn, flush, reps=7):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default="gpurun_out/supernet.json")
+    ap.add_argument("--out", default="bench_out/supernet.json")
     ap.add_argument("--no-oracle", action="store_true")
     args = ap.parse_args()
     dtype = torch.bfloat16

@@ -1,6 +1,6 @@
 """Shape / sparsity sweep of elsa_nm_linear and elsa_nm_compress on one GPU.
 
-    python -m paper_2409_09708_b200.sweep [--out gpurun_out/sweep.json] [--reps 5] [--quick]
+    python -m paper_2409_09708_b200.sweep [--out bench_out/sweep.json] [--reps 5] [--quick]
 
 rows in {4096, 16384, 65536} x (K, O) in {(768,768), (768,3072), (3072,768), (1024,4096), (4096,1024)}
 x level in {1:4, 2:4, 1:8, 2:8, 4:8, 1:16, 2:16, 4:16, 8:16} x {fp16, bf16}: per point the median
@@ -45,7 +45,7 @@ def timed(fn, reps, flush):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default="gpurun_out/sweep.json")
+    ap.add_argument("--out", default="bench_out/sweep.json")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--quick", action="store_true", help="rows = 4096 only")
     ap.add_argument("--summary", default=None, help="also write a short markdown summary to this path")
@@ -106,7 +106,7 @@ def main():
 def write_summary(path, hbm, tf, kind, lin, cmp_):
     med = statistics.median
     out = ["# Shape / sparsity sweep (%d linear points, %d compress points) -- summary" % (len(lin), len(cmp_)), "",
-           "Command: `python -m paper_2409_09708_b200.sweep --out gpurun_out/sweep.json --summary <this file>` (B200;",
+           "Command: `python -m paper_2409_09708_b200.sweep --out bench_out/sweep.json --summary <this file>` (B200;",
            "median of 5 CUDA-event timings per point, 512 MB written between repetitions to flush the 126 MB L2;",
            "time = weight-image rebuild + GEMM of `elsa_nm_linear` under the automatic dispatch).",
            "Peaks (%s): %.1f GB/s, %.1f TFLOP/s." % (kind, hbm, tf), "",
