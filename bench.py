@@ -329,7 +329,11 @@ def run_ours(args):
         "avg_launch_ms": gemm_total_ms / max(gemm_launches, 1),
         "roofline_time_share": {k: v / sum_roof for k, v in share.items()},
     }
-    stack_frac = sum_roof / (ms_per_step * 1e-3)
+    # the step also compresses every weight: its own roofline is the bytes it must move (dense W in, packed
+    # values and index words out) at the HBM peak
+    compress_bytes = sum(l.out * l.in_ * 2 + algorithmic_bytes(l) - 2 * l.rows * (l.in_ + l.out) - l.out * 2 for l in layers)
+    compress_roof = compress_bytes / (peaks["hbm_gbs"] * 1e9)
+    stack_frac = (sum_roof + compress_roof) / (ms_per_step * 1e-3)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -344,12 +348,12 @@ def run_ours(args):
         "actual_tflops": world * kept_flops / (ms_per_step * 1e-3) / 1e12,
         "ms_per_stack": ms_per_step,
         "stack_roofline_frac": stack_frac,
+        "stack_roofline_ms": {"linears": sum_roof * 1e3, "compress": compress_roof * 1e3},
         "gpu_launches": launches,
         "roofline": roofline,
         "kernels": {k: {"launches": v[0], "ms": v[1], "share": v[1] / kernel_total} for k, v in per_kernel.items()},
         "ms_per_step_profiled": prof_ms / args.steps,
-        "compress_gbs": (sum(l.out * l.in_ * 2 + algorithmic_bytes(l) - 2 * l.rows * (l.in_ + l.out) - l.out * 2
-                             for l in layers) * args.steps / per_kernel["nm_compress"][1] / 1e6)
+        "compress_gbs": (compress_bytes * args.steps / per_kernel["nm_compress"][1] / 1e6)
                         if per_kernel.get("nm_compress", [0, 0.0])[1] > 0 else None,
         "clocks": clocks,
     }
