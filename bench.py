@@ -35,12 +35,13 @@ METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
 GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws")   # forms of the tcgen05 GEMM
 
-# dram__bytes_read.sum + dram__bytes_write.sum of ONE grouped launch of each GEMM kernel inside this
-# benchmark's default run, from a one-pass ncu capture of the same command (the two DRAM counters
+# dram__bytes_read.sum + dram__bytes_write.sum of each GEMM kernel's launches over ONE step of this
+# benchmark, from a one-pass ncu capture of the same command (the two DRAM counters
 # fit one pass, so the full-size run is captured as it is).  Valid for the kernels as captured; set an
 # entry to None when its kernel changes.
 MEASURED_DRAM_TRAFFIC = {
     "deit_b_stack_b256": {"linear_tc_pair": 8.773e9, "linear_tc_sp24_ws": 4.70e9, "linear_tc_sp24_pair": 3.571e9},
+    "swin_b_stack_b128": {"linear_tc_pair": 10.458e9, "linear_tc_sp24_pair": 2.485e9},
 }
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
@@ -311,11 +312,13 @@ def run_ours(args):
     roofline = {
         "kernel": top_kernel, "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
         "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": frac,
-        # one launch of `kernel` per step carries all its layers; the capture does not apply otherwise
-        "traffic": MEASURED_DRAM_TRAFFIC.get(args.workload, {}).get(top_kernel) if top_launches == args.steps else None,
-        "traffic_note": "DRAM bytes (read + written) of one launch of `kernel`, which carries all of its layers "
-                        "(ncu, one pass, same command); traffic_algorithmic is the same layers' algorithmic bytes",
-        "traffic_algorithmic": sum(algorithmic_bytes(l) for i, l in enumerate(layers) if layer_kernel.get(i) == top_kernel),
+        # per launch, like `achieved`: the step's bytes of `kernel` over its launches per step (layers share launches)
+        "traffic": (MEASURED_DRAM_TRAFFIC[args.workload][top_kernel] * args.steps / top_launches
+                    if top_launches and top_kernel in MEASURED_DRAM_TRAFFIC.get(args.workload, {}) else None),
+        "traffic_note": "DRAM bytes (read + written) per launch of `kernel`, whose launches carry all of its layers "
+                        "(ncu, one pass, same command); traffic_algorithmic is the same layers' algorithmic bytes per launch",
+        "traffic_algorithmic": (sum(algorithmic_bytes(l) for i, l in enumerate(layers) if layer_kernel.get(i) == top_kernel)
+                                * args.steps / top_launches if top_launches else None),
         "peaks": peaks_kind,
         "definition": "per layer max(kept FLOPs / tensor peak, algorithmic bytes / HBM peak), summed over the "
                       "layers, divided by the summed CUDA-event durations of the GEMM launches that ran them "
