@@ -345,6 +345,21 @@ def test_swin_b_stack_full_size_sampled_rows(lib):
     stack_check(lib, layers, synth.torch_dtype(dt), 24, 41)
 
 
+def test_weight_stationary_layers_share_one_launch(lib):
+    """A table whose layers all take the weight-stationary sparse kernel under the automatic rule
+    (N <= 2, in of 768-896, out >= 1024): feature blocks that do not divide the CTA pairs (5 and 10 blocks),
+    a last block of only 8 features, ragged row tiles, two different K; one launch carries them all."""
+    dtype = torch.bfloat16
+    layers = [synth.Layer("a", 6000, 896, 1280, 1, 8, 501, 502, 503),
+              synth.Layer("b", 5001, 768, 1024, 2, 8, 511, 512, 513),
+              synth.Layer("c", 4100, 768, 2312, 2, 4, 521, 522, 523),
+              synth.Layer("d", 7777, 896, 3072, 1, 16, 531, 532, 533)]
+    lib.elsa_profile_start()
+    stack_check(lib, layers, dtype, 96, 51)
+    recs = lib.elsa_profile_stop()
+    assert [k for (k, _, _) in recs if k.startswith("linear")] == ["linear_tc_sp24_ws"], recs
+
+
 def test_shared_launches_give_the_same_bits_as_one_launch_per_layer(lib):
     """elsa_vit_linears with per-layer scratch (layers share persistent launches) against the same
     table run layer by layer, on a table that mixes all three tensor-core families."""
