@@ -346,6 +346,57 @@ __device__ __forceinline__ void unpack_group(const uint16_t* __restrict__ vals, 
     const int g = (int)(gid % groups_per_row);
 
     const uint16_t* v = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
+    if constexpr (M != 16) {
+        // Groups of 4 and 8 with N < M: the kept values are loaded with the widest access their alignment
+        // allows, split into a plane of low bytes and a plane of high bytes, scattered to their positions by
+        // byte permutes (selector nibble of position i = slot holding its value; unused positions point at
+        // slot M-1, which is zero because N < M), and re-interleaved.
+        if (words_per_row) {
+            constexpr int R = M / 2;
+            const uint32_t* row = idx + (size_t)o * words_per_row;
+            const int bit0 = g * N * B;
+            const int w0 = bit0 >> 5, sh = bit0 & 31;
+            const uint32_t lo = row[w0];
+            const uint32_t hi = (sh + N * B > 32) ? row[w0 + 1] : 0u;
+            const uint32_t fields = __funnelshift_r(lo, hi, sh);
+            uint32_t vr[R];
+#pragma unroll
+            for (int q = 0; q < R; ++q) vr[q] = 0;
+            if ((N & 3) == 0) {                                   // N = 4 (M = 8)
+                const uint2 t = *reinterpret_cast<const uint2*>(v);
+                vr[0] = t.x; vr[1] = t.y;
+            } else if ((N & 1) == 0) {
+#pragma unroll
+                for (int q = 0; q < R; ++q)
+                    if (q < (N >> 1)) vr[q] = reinterpret_cast<const uint32_t*>(v)[q];
+            } else {
+#pragma unroll
+                for (int t = 0; t < M; ++t)
+                    if (t < N) vr[t >> 1] |= (uint32_t)v[t] << (16 * (t & 1));
+            }
+            uint32_t inv = (M == 8) ? 0x77777777u : 0x3333u;
+#pragma unroll
+            for (int t = 0; t < M - 1; ++t)
+                if (t < N) {
+                    const uint32_t pos4 = ((fields >> (t * B)) & (uint32_t)(M - 1)) * 4u;
+                    inv = (inv & ~(0xFu << pos4)) | ((uint32_t)t << pos4);
+                }
+            uint16_t* dst = Wm + (size_t)o * in + (size_t)g * M;
+            if constexpr (M == 4) {
+                const uint32_t pl = prmt(prmt(vr[0], vr[1], 0x6420u), 0u, inv);
+                const uint32_t ph = prmt(prmt(vr[0], vr[1], 0x7531u), 0u, inv);
+                *reinterpret_cast<uint2*>(dst) = make_uint2(prmt(pl, ph, 0x5140u), prmt(pl, ph, 0x7362u));
+            } else {
+                const uint32_t l0 = prmt(vr[0], vr[1], 0x6420u), l1 = prmt(vr[2], vr[3], 0x6420u);
+                const uint32_t h0 = prmt(vr[0], vr[1], 0x7531u), h1 = prmt(vr[2], vr[3], 0x7531u);
+                const uint32_t pl03 = prmt(l0, l1, inv & 0xFFFFu), pl47 = prmt(l0, l1, inv >> 16);
+                const uint32_t ph03 = prmt(h0, h1, inv & 0xFFFFu), ph47 = prmt(h0, h1, inv >> 16);
+                *reinterpret_cast<uint4*>(dst) = make_uint4(prmt(pl03, ph03, 0x5140u), prmt(pl03, ph03, 0x7362u),
+                                                            prmt(pl47, ph47, 0x5140u), prmt(pl47, ph47, 0x7362u));
+            }
+            return;
+        }
+    }
     unsigned long long fields;
     if (words_per_row) {
         const uint32_t* row = idx + (size_t)o * words_per_row;
