@@ -168,7 +168,7 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
         // With the weight block resident in tensor memory the activations are the only shared-memory
         // traffic; measured faster than streaming the weight for K around 768 once a layer has at least
         // four blocks of 256 features (qkv, fc1: 10-15 %), equal or slower elsewhere.
-        const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in >= 640 && in <= 896 && out >= 1024 &&
+        const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in <= 896 && out >= 1024 &&
                         rows >= 256 * (sm_count / 2) / ((out + 255) / 256);
         *kind = ws ? KIND_SPARSE_WS : KIND_SPARSE_PAIR;
     }
