@@ -336,8 +336,9 @@ elsa_status elsa_nm_linear_masked(const void* X, int rows, const void* W_sup, co
     if (kind == KIND_SIMT || kind == KIND_SPARSE_ONE)
         return fail(ELSA_ERR_NM, "the forced variant has no mask-on-load form");
     if (kind == KIND_SPARSE_PAIR || kind == KIND_SPARSE_WS) {
-        uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
-        if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, (uint16_t*)workspace, meta, stream)) != ELSA_OK)
+        uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
+        if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, kind == KIND_SPARSE_WS, (uint16_t*)workspace, meta,
+                                       stream)) != ELSA_OK)
             return st;
         SparseJob job;
         job.X = (const uint16_t*)X; job.bias = (const uint16_t*)bias; job.Y = (uint16_t*)Y; job.workspace = workspace;
@@ -471,9 +472,9 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
             const elsa_layer& c = cfg[l];
             if (c.N != c.M) {
                 if (kind[l] == KIND_SPARSE_PAIR || kind[l] == KIND_SPARSE_WS) {
-                    uint8_t* meta = region[l] + round_up((size_t)c.out * (size_t)c.in, 256);
+                    uint8_t* meta = region[l] + sp24_meta_offset(c.out, c.in);
                     batch_add_to_sp24(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, 128,
-                                      (uint16_t*)region[l], meta);
+                                      kind[l] == KIND_SPARSE_WS, (uint16_t*)region[l], meta);
                 } else {
                     batch_add_unpack(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, (uint16_t*)region[l]);
                 }

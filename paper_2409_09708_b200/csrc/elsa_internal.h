@@ -103,10 +103,13 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                     const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
                                     uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
-// packed weight -> 2-of-4 image [out][in/2] + metadata blocks of 2 KB per (128 features, block_k of K),
-// block_k = 64 or 128.
+// packed weight -> 2-of-4 image [out rounded up to 32][in/2] + metadata blocks of 2 KB per (128 features,
+// block_k of K), block_k = 64 or 128.  `permuted`: row r of every block of 32 image rows holds feature
+// 8 * (r % 4) + r / 4 of the block (the lane order of the weight-stationary kernel), else feature r.
 elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
-                              uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
+                              bool permuted, uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
+// Where the metadata blocks start in a layer's scratch: after the image, whose rows are rounded up to 32.
+inline size_t sp24_meta_offset(int out, int in) { return round_up((size_t)((out + 31) / 32 * 32) * (size_t)in, 256); }
 // The same on CTA pairs (256 features x 224 rows per pair, K blocks of 128).
 elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                          const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
@@ -122,7 +125,7 @@ struct SparseJob {
 };
 int linear_tc_sparse_pair_group_max();
 elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                                                 void* workspace, cudaStream_t stream);
+                                                 bool permuted, void* workspace, cudaStream_t stream);
 elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
                                                cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
@@ -146,8 +149,8 @@ struct LevelTable {
 };
 elsa_status launch_compress_levels(const uint16_t* W, int out, int in, int M, const LevelTable& t, cudaStream_t stream);
 elsa_status launch_mask(const uint16_t* W, int out, int in, int N, int M, uint16_t* Wm, cudaStream_t stream);
-elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, uint16_t* a_img,
-                                 uint8_t* meta, cudaStream_t stream);
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, bool permuted,
+                                 uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
 
 // Batched weight-format kernels: one launch over a table of weights (kernel-parameter space).
 enum BatchKind { BATCH_COMPRESS = 0, BATCH_UNPACK = 1, BATCH_TO_SP24 = 2 };
@@ -157,7 +160,7 @@ struct BatchItem {
     void* dst;
     void* dst2;
     long long first_unit;   // prefix sum of work units over the table
-    int out, in, N, M, wpr, aux, aux2, kind;
+    int out, in, N, M, wpr, aux, aux2, aux3, kind;
 };
 constexpr int kBatchMax = 256;
 struct BatchTable {
@@ -169,7 +172,7 @@ void batch_add_compress(BatchTable* t, const uint16_t* W, int out, int in, int N
 void batch_add_unpack(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
                       uint16_t* Wm);
 void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                       int block_k, uint16_t* a_img, uint8_t* meta);
+                       int block_k, bool permuted, uint16_t* a_img, uint8_t* meta);
 elsa_status launch_compress_batch(const BatchTable& t, cudaStream_t stream);
 elsa_status launch_image_batch(const BatchTable& t, cudaStream_t stream);
 

@@ -449,10 +449,15 @@ __device__ __forceinline__ void unpack_group(const uint16_t* __restrict__ vals, 
 // Second half of the 2-of-4 re-encoding: given 16 consecutive positions of a weight row with the pruned
 // ones already zero (d) and the kept set (keep), emits two values per aligned chunk of 4 (ascending
 // positions, a zero borrowed where fewer than two are kept) and the chunk nibbles as tensor memory wants them.
-__device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep, bool real, int o, int seg, int k0, int in,
-                                          uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int k_blocks,
-                                          int steps_per_block)
+// With `permuted`, weight row o lands in image row (o & ~31) | (4 * (o % 8) + (o % 32) / 8), so that row r of a
+// block of 32 holds feature 8 * (r % 4) + r / 4: the order in which the weight-stationary kernel's transposing
+// stores want the features in tensor-memory lanes.  The image has its rows rounded up to 32; rows past `out`
+// are written as zeros.
+__device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep, bool real, int o_src, int seg, int k0, int in,
+                                          int out, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int k_blocks,
+                                          int steps_per_block, bool permuted)
 {
+    const int o = permuted ? ((o_src & ~31) | (4 * (o_src & 7) + ((o_src & 31) >> 3))) : o_src;
     constexpr int kFeatTile = 128;
     uint32_t nibbles = 0;
     uint16_t sel[8];
@@ -475,7 +480,7 @@ __device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep
         sel[2 * c + 1] = v1;
     }
 
-    if (real) {
+    if (k0 < in && o_src < ((out + 31) & ~31)) {      // `d` is all zero where the row or the segment is padding
         uint4 r;
         r.x = sel[0] | ((uint32_t)sel[1] << 16);
         r.y = sel[2] | ((uint32_t)sel[3] << 16);
@@ -502,7 +507,7 @@ template <int M>
 __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
                                                 int out, int in, int N, int words_per_row,
                                                 uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
-                                                int k_blocks, int steps_per_block, long long tid)
+                                                int k_blocks, int steps_per_block, bool permuted, long long tid)
 {
     constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
     constexpr int G = 16 / M;                         // groups per 16-k segment
@@ -536,7 +541,7 @@ __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ val
             }
         }
     }
-    sp24_emit(d, keep, real, o, seg, k0, in, a_img, meta16, k_blocks, steps_per_block);
+    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, permuted);
 }
 
 // The same from the DENSE shared weight: the 16 positions are projected onto level N:M on the fly
@@ -544,7 +549,7 @@ __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ val
 template <int M>
 __device__ __forceinline__ void dense_to_sp24_segment(const uint16_t* __restrict__ W, int out, int in, int N,
                                                       uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
-                                                      int k_blocks, int steps_per_block, long long tid)
+                                                      int k_blocks, int steps_per_block, bool permuted, long long tid)
 {
     constexpr int G = 16 / M;
     const int segs = k_blocks * steps_per_block * 2;
@@ -568,7 +573,7 @@ __device__ __forceinline__ void dense_to_sp24_segment(const uint16_t* __restrict
             keep |= kg << (gl * M);
         }
     }
-    sp24_emit(d, keep, real, o, seg, k0, in, a_img, meta16, k_blocks, steps_per_block);
+    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, permuted);
 }
 
 }  // namespace

@@ -56,25 +56,25 @@ template <int M>
 __global__ void __launch_bounds__(256)
 nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx, int out, int in, int N,
                   int words_per_row, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int out_tiles,
-                  int k_blocks, int steps_per_block)
+                  int k_blocks, int steps_per_block, int permuted)
 {
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
     if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
-    to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, tid);
+    to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, permuted != 0, tid);
 }
 
 template <int M>
 __global__ void __launch_bounds__(256)
 dense_to_sp24_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint16_t* __restrict__ a_img,
-                     uint16_t* __restrict__ meta16, int out_tiles, int k_blocks, int steps_per_block)
+                     uint16_t* __restrict__ meta16, int out_tiles, int k_blocks, int steps_per_block, int permuted)
 {
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
     if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
-    dense_to_sp24_segment<M>(W, out, in, N, a_img, meta16, k_blocks, steps_per_block, tid);
+    dense_to_sp24_segment<M>(W, out, in, N, a_img, meta16, k_blocks, steps_per_block, permuted != 0, tid);
 }
 
 // ------------------------------------------------------------------ GEMM
@@ -270,8 +270,9 @@ linear_tc_sp24_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }  // namespace
 
 elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
-                              uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
+                              bool permuted, uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
 {
+    const int perm = permuted ? 1 : 0;
     const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
     const int k_blocks = (in + block_k - 1) / block_k;
     const int steps = block_k / kSpUmmaK;
@@ -281,19 +282,20 @@ elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out
     ProfileScope scope(ELSA_KERNEL_NM_TO_SP24, stream);
     if (M == 4)
         launch_pdl(nm_to_sp24_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+                   (uint16_t*)meta, tiles_f, k_blocks, steps, perm);
     else if (M == 8)
         launch_pdl(nm_to_sp24_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+                   (uint16_t*)meta, tiles_f, k_blocks, steps, perm);
     else
         launch_pdl(nm_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, vals, idx, out, in, N, wpr, a_img,
-                   (uint16_t*)meta, tiles_f, k_blocks, steps);
+                   (uint16_t*)meta, tiles_f, k_blocks, steps, perm);
     return launched("nm_to_sp24");
 }
 
-elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, uint16_t* a_img,
-                                 uint8_t* meta, cudaStream_t stream)
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, bool permuted,
+                                 uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
 {
+    const int perm = permuted ? 1 : 0;
     const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
     const int k_blocks = (in + block_k - 1) / block_k;
     const int steps = block_k / kSpUmmaK;
@@ -302,13 +304,13 @@ elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int 
     ProfileScope scope(ELSA_KERNEL_NM_TO_SP24, stream);
     if (M == 4)
         launch_pdl(dense_to_sp24_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
-                   tiles_f, k_blocks, steps);
+                   tiles_f, k_blocks, steps, perm);
     else if (M == 8)
         launch_pdl(dense_to_sp24_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
-                   tiles_f, k_blocks, steps);
+                   tiles_f, k_blocks, steps, perm);
     else
         launch_pdl(dense_to_sp24_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, W, out, in, N, a_img, (uint16_t*)meta,
-                   tiles_f, k_blocks, steps);
+                   tiles_f, k_blocks, steps, perm);
     return launched("dense_to_sp24");
 }
 
@@ -323,7 +325,7 @@ size_t linear_tc_sparse_workspace(int out, int in)
 {
     const size_t tiles = (size_t)(out + kFeatTile - 1) / kFeatTile;
     const size_t kbs = (size_t)(in + kBlockK - 1) / kBlockK;
-    return round_up((size_t)out * (size_t)in, 256) + tiles * kbs * kMetaBytes;
+    return sp24_meta_offset(out, in) + tiles * kbs * kMetaBytes;
 }
 
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
@@ -339,9 +341,9 @@ elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t*
     const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
     const int k_blocks = (in + kBlockK - 1) / kBlockK;
     uint16_t* a_img = (uint16_t*)workspace;
-    uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
+    uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
 
-    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, a_img, meta, stream)) != ELSA_OK) return st;
+    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, false, a_img, meta, stream)) != ELSA_OK) return st;
 
     SpParams p;
     p.rows = rows; p.in = in; p.out = out;

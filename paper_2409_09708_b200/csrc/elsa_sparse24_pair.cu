@@ -335,7 +335,7 @@ elsa_status launch_sp_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
         L.bias = j.bias;
         const uint16_t* a_img = (const uint16_t*)j.workspace;
-        const uint8_t* meta = (const uint8_t*)j.workspace + round_up((size_t)j.out * (size_t)j.in, 256);
+        const uint8_t* meta = (const uint8_t*)j.workspace + sp24_meta_offset(j.out, j.in);
         elsa_status st;
         if ((st = make_map_2d(&L.map_a, a_img, (uint64_t)(j.in / 2), (uint64_t)j.out, kBlockK / 2, kFeatPerCta,
                               CU_TENSOR_MAP_SWIZZLE_128B, "2:4 weight image")) != ELSA_OK)
@@ -427,7 +427,7 @@ elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint
 {
     if (!linear_tc_sparse_suits(in, N) || N == M)
         return fail(ELSA_ERR_NM, "level %d:%d with in=%d does not fit the 2:4 sparse MMA path", N, M, in);
-    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, workspace, stream);
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, false, workspace, stream);
     if (st != ELSA_OK) return st;
     SparseJob job;
     job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;
@@ -437,11 +437,11 @@ elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint
 
 // Re-encodes one packed weight into `workspace` in the form the pair kernel reads (K blocks of 128).
 elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                                                 void* workspace, cudaStream_t stream)
+                                                 bool permuted, void* workspace, cudaStream_t stream)
 {
     uint16_t* a_img = (uint16_t*)workspace;
-    uint8_t* meta = (uint8_t*)workspace + round_up((size_t)out * (size_t)in, 256);
-    return launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, a_img, meta, stream);
+    uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
+    return launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, permuted, a_img, meta, stream);
 }
 
 }  // namespace elsa

@@ -7,11 +7,11 @@
 // not move: a CTA pair owns one block of 256 output features of a layer for the whole layer.  Its
 // 2-of-4 values (in/4 columns) and metadata (in/32 columns) are written once into the tensor memory
 // of the two CTAs and every tcgen05.mma.sp reads its A operand from there; shared memory carries
-// activations only.  What is left of tensor memory holds one accumulator of `nt` token rows (256 for
-// in <= 768).  The wide tile is deliberate: issuing one MMA costs the issuing warp on the order of a
-// hundred cycles whatever its shape, and a sparse MMA over 256 token rows lasts 128 cycles, so only the
-// widest instruction keeps the tensor pipe fed; the price is that the epilogue's tensor-memory reads and
-// the next tile's MMAs cannot overlap (the conversion and the stores still do).
+// activations only.  What is left of tensor memory holds TWO accumulators of `nt` token rows each
+// (144 for in = 768), so the epilogue of one tile runs under the MMAs of the next.  Narrow MMAs only
+// pay because the issuing lane is predicated inside the instruction's own asm block: a branch around
+// each tcgen05.mma costs the issuing warp about 80 cycles per instruction, the predicated form under
+// 40, and a sparse MMA over 144 token rows lasts 72.
 //
 // Schedule of a layer over P pairs: F = ceil(out / 256) feature blocks, G = P / F row groups.  Pair p
 // takes feature block p % F and the row tiles g, g + G, g + 2G, ... with g = p / F, so the F pairs
@@ -20,9 +20,14 @@
 // them in order, reloading its weight block at every layer.
 //
 // Per CTA: warp 0 TMA producer for this CTA's half of the activation rows; warp 1 tensor-memory
-// allocation and, in the leader, MMA issue; the remaining warps write the weight block into tensor
-// memory at the start of a layer and run the epilogue (lanes are features; see
-// elsa_sparse24_pair.cu for the transposing store).  Waits are bounded as in the other kernels.
+// allocation and, in the leader, MMA issue; twelve epilogue warps (three per tensor-memory lane
+// quarter, each with its own run of token columns) write the weight block into tensor memory at the
+// start of a layer and run the epilogue.  The accumulator is transposed (lanes are features, columns
+// are token rows) and Y is row-major, so the epilogue has to turn a lane's column pair into a row's
+// feature run.  stmatrix with .trans does that in one instruction per 8 x 32 outputs if lane t of a
+// quarter holds feature 8 * (t % 4) + t / 4 of its 32; the weight image is therefore built with its
+// rows in that order (`permuted` form of nm_to_sp24), and only the bias index and the store address
+// here know about it.  Waits are bounded as in the other kernels.
 
 #include <mutex>
 
@@ -33,33 +38,31 @@ namespace {
 
 constexpr int kFeatPerCta = 128;   // weight rows per CTA = TMEM lanes
 constexpr int kPairFeat = 256;     // MMA M over the pair
-constexpr int kMaxRowTile = 256;   // token rows per pair tile (MMA N), per layer <= this
 constexpr int kBlockK = 128;       // granularity of `in` (one metadata block)
 constexpr int kStageK = 256;       // logical K per pipeline stage: eight MMAs per barrier round trip
 constexpr int kSpUmmaK = 32;
-constexpr int kNumAccum = 1;
+constexpr int kNumAccum = 2;
 constexpr int kTmemCols = 512;
-constexpr int kMaxIn = 1024;       // in / 4 + in / 32 + nt columns must fit 512
+constexpr int kMaxIn = 1024;       // in / 4 + in / 32 + 2 * nt columns must fit 512
 constexpr int kMaxStages = 8;
-constexpr int kEpiWarps = 16;
-constexpr int kEpiParts = kEpiWarps / 4;   // warps per TMEM lane quarter
+constexpr int kEpiParts = 3;       // epilogue warps per TMEM lane quarter
+constexpr int kEpiWarps = 4 * kEpiParts;
 constexpr int kThreads = 64 + kEpiWarps * 32;
-constexpr int kEpiCols = 32;
-constexpr int kBSubBytes = (kMaxRowTile / 2) * 128;   // one 64-wide K slice: up to 128 rows of 128 bytes
-constexpr int kStageBytes = (kStageK / 64) * kBSubBytes;
-constexpr int kStagingBytes = 32 * kEpiCols * 2;      // one buffer per epilogue warp
+constexpr int kStepCols = 16;      // token rows per tcgen05.ld / pair of stmatrix
+constexpr int kMaxSteps = 4;       // steps per epilogue warp and tile
+constexpr int kMaxRowTile = kStepCols * kMaxSteps * kEpiParts;   // 192 token rows per pair tile (MMA N)
+constexpr int kStagingBytes = kMaxSteps * kStepCols * 64;        // per epilogue warp: rows of 32 features
 constexpr int kStagingTotal = kEpiWarps * kStagingBytes;
 constexpr int kBarrierBytes = 512;
 
-static_assert(kBSubBytes % 1024 == 0, "swizzled tiles stay 1024-byte aligned");
-
 struct alignas(64) WsLayer {
     CUtensorMap map_x, map_y;
-    const uint16_t* a_img;   // 2-of-4 values [out][in / 2]
+    const uint16_t* a_img;   // 2-of-4 values [out rounded up to 32][in / 2], rows in the permuted order
     const uint8_t* meta;     // metadata blocks of 2 KB per (128 features, 128 k)
     const uint16_t* bias;
     int rows, out, in;
     int nt;            // token rows per pair tile
+    int steps_per_warp;   // 16-column steps each epilogue warp of a quarter takes
     int tiles_f;       // F
     int groups;        // G
     int row_tiles;     // ceil(rows / nt)
@@ -74,23 +77,62 @@ struct WsGroup {
     WsLayer layer[kMaxLayers];
     int n_layers;
     int stages;
+    int stage_bytes;   // one pipeline stage: kStageK / 64 quarters of (largest nt / 2) rows of 128 bytes
     uint32_t* dev_status;
 };
 
 // A from tensor memory: lane = weight row, 8 columns per K step of 32 (16 kept values of 16 bits).
+// Called by the whole (converged) warp; `issue` is non-zero in the one lane that issues.  The predicate
+// lives inside the asm block so that the compiler cannot turn it into a branch around the instruction.
 __device__ __forceinline__ void umma_sp_f16_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t tmem_e,
-                                                    uint32_t idesc, uint32_t accumulate)
+                                                    uint32_t idesc, uint32_t accumulate, uint32_t issue)
 {
     const uint32_t idesc_sel = idesc | (tmem_e & 1u);
     const uint32_t e_addr = tmem_e & ~1u;
     asm volatile(
         "{\n"
-        ".reg .pred p;\n"
+        ".reg .pred p, q;\n"
         "setp.ne.b32 p, %5, 0;\n"
-        "tcgen05.mma.sp.cta_group::2.kind::f16 [%0], [%1], %2, [%3], %4, p;\n"
+        "setp.ne.b32 q, %6, 0;\n"
+        "@q tcgen05.mma.sp.cta_group::2.kind::f16 [%0], [%1], %2, [%3], %4, p;\n"
         "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate)
+        "r"(a_tmem), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate), "r"(issue)
         : "memory");
+}
+
+// umma_commit_pair, predicated the same way.
+__device__ __forceinline__ void umma_commit_pair_if(uint32_t bar, uint16_t cta_mask, uint32_t issue)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred q;\n"
+        "setp.ne.b32 q, %2, 0;\n"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n"
+        "}\n" ::"r"(bar),
+        "h"(cta_mask), "r"(issue)
+        : "memory");
+}
+
+// Lane i of the warp receives 16 consecutive fp32 columns of TMEM lane (lane base + i).
+__device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Four 8 x 8 matrices of 16-bit values, transposed on the way to shared memory: the two halves of
+// register i of lane t go to column t / 4 of rows 2 * (t % 4) and 2 * (t % 4) + 1 of matrix i, whose
+// eight 16-byte rows are at the addresses given by lanes 8 * i .. 8 * i + 7.
+__device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+{
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r0), "r"(r1),
+                 "r"(r2), "r"(r3)
+                 : "memory");
 }
 
 // Lane i of the warp writes 16 / 4 consecutive columns of TMEM lane (lane base + i).
@@ -160,15 +202,16 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
     const uint32_t cta_rank = cluster_ctarank();
     const int pair = blockIdx.x >> 1;
 
-    const uint32_t staging_base = smem_base + (uint32_t)(p.stages * kStageBytes);
-    const uint32_t bar_off = (uint32_t)(p.stages * kStageBytes) + kStagingTotal;
+    const uint32_t staging_base = smem_base + (uint32_t)(p.stages * p.stage_bytes);
+    const uint32_t bar_off = (uint32_t)(p.stages * p.stage_bytes) + kStagingTotal;
     const uint32_t bar_base = smem_base + bar_off;
     const uint32_t full_bar = bar_base;                       // leader only
     const uint32_t empty_bar = bar_base + 8 * kMaxStages;     // per CTA
     const uint32_t tmem_full_bar = bar_base + 16 * kMaxStages;        // per CTA
     const uint32_t tmem_empty_bar = tmem_full_bar + 8 * kNumAccum;    // leader only
     const uint32_t w_ready_bar = tmem_empty_bar + 8 * kNumAccum;      // leader only
-    const uint32_t holder_off = bar_off + 16 * kMaxStages + 16 * kNumAccum + 8;
+    const uint32_t layer_bar = w_ready_bar + 8;                       // per CTA: epilogue warps between layers
+    const uint32_t holder_off = bar_off + 16 * kMaxStages + 16 * kNumAccum + 16;
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off + 4);
 
@@ -182,6 +225,7 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
             mbar_init(tmem_empty_bar + 8 * a, 2 * kEpiWarps);
         }
         mbar_init(w_ready_bar, 2 * kEpiWarps);
+        mbar_init(layer_bar, kEpiWarps);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async_smem();
@@ -218,7 +262,7 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                         ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
                         ok = __all_sync(0xFFFFFFFFu, ok);
                         if (!ok) break;
-                        const uint32_t dst = smem_base + (uint32_t)(stage * kStageBytes);
+                        const uint32_t dst = smem_base + (uint32_t)(stage * p.stage_bytes);
                         const uint32_t bar = mapa_shared(full_bar + 8 * stage, 0);
                         if (elected) {
                             if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
@@ -233,12 +277,12 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
         __syncwarp();
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer (leader CTA only)
-        // The whole warp walks the loop and waits on the barriers; one elected lane issues.  With the
-        // warp converged the descriptors stay in uniform registers, which roughly halves the cost of
-        // issuing one MMA compared with a single thread inside a divergent branch (measured: ~85 -> ~40
-        // cycles), and an MMA of 128 token rows lasts only 64 cycles.
+        // The whole warp walks the loop and waits on the barriers; one elected lane issues, through a
+        // predicate inside each instruction's asm block.  With the warp converged the descriptors stay in
+        // uniform registers and no branch surrounds the instruction: measured ~36 cycles per MMA, against
+        // ~80 with `if (elected)` around it and more with a single thread inside a divergent branch.
         if (cta_rank == 0) {
-            const bool elected = elect_one();
+            const uint32_t elected = elect_one() ? 1u : 0u;
             // the base address was read from shared memory into an ordinary register; a warp reduction
             // returns it in a uniform one, so that every address derived from it stays uniform too
             const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
@@ -273,9 +317,10 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                     const uint32_t d_tmem = tmem_u + (uint32_t)(acc * L.nt);
                     for (int ks = 0; ks < num_k_stages; ++ks) {
                         ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
+                        ok = __all_sync(0xFFFFFFFFu, ok);
                         if (!ok) break;
                         tc_fence_after();
-                        const uint64_t b_desc0 = smem_desc_k_major_sw128(smem_base + (uint32_t)(stage * kStageBytes));
+                        const uint64_t b_desc0 = smem_desc_k_major_sw128(smem_base + (uint32_t)(stage * p.stage_bytes));
                         const uint32_t a_col = a_col0 + (uint32_t)(ks * 8 * (kStageK / kSpUmmaK));
                         const uint32_t e_col = e_col0 + (uint32_t)(ks * (kStageK / kSpUmmaK));
                         // operands are computed by the whole warp (they stay uniform); only the instruction
@@ -284,24 +329,22 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
 #pragma unroll
                             for (int j = 0; j < kStageK / kSpUmmaK / 2; ++j) {
                                 const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)(j >> 1) * quarter + 4u * (uint32_t)(j & 1));
-                                if (elected)
-                                    umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
-                                                        (uint32_t)((ks | j) != 0));
+                                umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
+                                                    (uint32_t)((ks | j) != 0), elected);
                             }
                         } else {
 #pragma unroll
                             for (int j = 0; j < kStageK / kSpUmmaK; ++j) {
                                 const uint64_t b_desc = b_desc0 + (uint64_t)((uint32_t)(j >> 1) * quarter + 4u * (uint32_t)(j & 1));
-                                if (elected)
-                                    umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
-                                                        (uint32_t)((ks | j) != 0));
+                                umma_sp_f16_pair_ts(d_tmem, a_col + (uint32_t)(8 * j), b_desc, e_col + (uint32_t)j, idesc,
+                                                    (uint32_t)((ks | j) != 0), elected);
                             }
                         }
-                        if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);
+                        umma_commit_pair_if(empty_bar + 8 * stage, 3, elected);
                         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                     }
                     if (!ok) break;
-                    if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);
+                    umma_commit_pair_if(tmem_full_bar + 8 * acc, 3, elected);
                     if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
                 }
             }
@@ -316,16 +359,17 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
         const uint32_t lane_base = tmem_base + ((uint32_t)(q * 32) << 16);
         int acc = 0;
         uint32_t acc_phase = 0;
-        const bool odd = (lane & 1) != 0;
+        uint32_t layer_phase = 0;
         const uint32_t buf = staging_base + (uint32_t)((warp - 2) * kStagingBytes);
-        // staging address pieces that do not depend on the row pair (see elsa_sparse24_pair.cu)
-        const uint32_t prmt_sel = odd ? 0x7632u : 0x5410u;
-        const uint32_t lane_off = (odd ? 64u : 0u) + (uint32_t)(((lane >> 1) & 3) * 4);
-        uint32_t sw_off[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) sw_off[k] = (((uint32_t)(lane >> 3)) ^ (uint32_t)k) << 4;
+        // Lane t holds feature 8 * (t % 4) + t / 4 of the quarter's 32.  The staging buffer is rows of 32
+        // features (64 bytes, no swizzle); one stmatrix.x4.trans writes 8 token rows: lane t gives the
+        // address of (row 2 * (t / 8) + (t & 1), features 8 * ((t % 8) / 2) ...), and the two rows of a
+        // matrix are 128 consecutive bytes, so no two of its addresses share a bank.
+        const int feat_in_quarter = 8 * (lane & 3) + (lane >> 2);
+        const uint32_t st_addr = buf + (uint32_t)((2 * (lane >> 3) + (lane & 1)) * 64 + ((lane & 7) >> 1) * 16);
 
         bool ok = true;
+        bool first_layer = true;
         for (int li = 0; ok && li < p.n_layers; ++li) {
             const WsLayer& L = p.layer[li];
             if (pair >= L.groups * L.tiles_f) continue;
@@ -333,28 +377,43 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
             if (g >= L.row_tiles) continue;
             const int ft128 = (pair % L.tiles_f) * 2 + (int)cta_rank;
             const int f0 = ft128 * kFeatPerCta + q * 32;
-            const int f = f0 + lane;
+            const int f = f0 + feat_in_quarter;
             const int l_rows = L.rows, l_out = L.out, nt = L.nt;
             const bool f_ok = f < l_out;
 
+            // The column ranges of accumulators and weight block depend on the layer, and the warps of a
+            // quarter read different columns of the same lanes: nobody writes the new weight block before
+            // every epilogue warp of this CTA has read its last accumulator of the previous layer.
+            if (!first_layer) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(layer_bar);
+                ok = mbar_wait(layer_bar, layer_phase, abort_flag, p.dev_status, 8);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                layer_phase ^= 1u;
+            }
+            first_layer = false;
+
             // ---- this warp's share of the weight block into tensor memory.  Every MMA of the previous
-            // layer has completed: this warp waited for the accumulator of that layer's last tile.
+            // layer has completed: this warp waited for the accumulator of that layer's last tile.  Image
+            // row (block base + TMEM lane) is already the row of the feature this lane holds.
             {
                 const uint32_t a_col0 = lane_base + (uint32_t)(kNumAccum * nt);
                 const uint32_t e_col0 = a_col0 + (uint32_t)(L.in >> 2);
-                const uint4* a_row = reinterpret_cast<const uint4*>(L.a_img + (size_t)(f_ok ? f : 0) * (size_t)(L.in >> 1));
+                const uint4* a_row = reinterpret_cast<const uint4*>(L.a_img + (size_t)(ft128 * kFeatPerCta + q * 32 + lane) * (size_t)(L.in >> 1));
+                const bool blk_ok = ft128 * kFeatPerCta < l_out;     // rows of a started block of 32 exist (zero beyond out)
+                const bool row_ok = f0 < l_out;
                 const int a_chunks = L.in >> 6;          // 16 columns (64 bytes) each
                 for (int c = part; c < a_chunks; c += kEpiParts) {
                     uint32_t v[16];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint4 t = make_uint4(0u, 0u, 0u, 0u);
-                        if (f_ok) t = __ldg(a_row + 4 * c + i);
+                        if (row_ok) t = __ldg(a_row + 4 * c + i);
                         v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
                     }
                     tmem_st_32x32b_x16(a_col0 + (uint32_t)(16 * c), v);
                 }
-                const bool blk_ok = ft128 * kFeatPerCta < l_out;
                 const uint4* e_blk = reinterpret_cast<const uint4*>(L.meta) +
                                      (size_t)(blk_ok ? ft128 : 0) * (size_t)L.num_k_blocks * 128 + (size_t)(q * 32 + lane);
                 for (int kb = part; kb < L.num_k_blocks; kb += kEpiParts) {
@@ -369,51 +428,54 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                 if (lane == 0) mbar_arrive_cluster_release(w_ready_remote);
             }
             const float bias_f = (L.bias != nullptr && f_ok) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
-            const int chunks = nt / kEpiCols;
+            // this warp's run of token columns: steps of 16, [first_step, first_step + my_steps)
+            const int total_steps = nt / kStepCols;
+            const int first_step = part * L.steps_per_warp;
+            int my_steps = total_steps - first_step;
+            if (my_steps > L.steps_per_warp) my_steps = L.steps_per_warp;
+            if (my_steps < 0) my_steps = 0;
 
             for (int r = g; r < L.row_tiles; r += L.groups) {
-                const int r0 = r * nt;
+                const int row0 = r * nt + first_step * kStepCols;
                 ok = mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t t_row = lane_base + (uint32_t)(acc * nt);
-                // this warp's chunks of 32 token rows: part, part + kEpiParts; both are read before the
-                // accumulator goes back to the MMA warp
-                uint32_t rr[2][32];
-                const bool mine0 = part < chunks, mine1 = part + kEpiParts < chunks;
-                if (mine0) tmem_ld_32x32b_x32(t_row + (uint32_t)(part * kEpiCols), rr[0]);
-                if (mine1) tmem_ld_32x32b_x32(t_row + (uint32_t)((part + kEpiParts) * kEpiCols), rr[1]);
-                if (mine0) tmem_wait_ld();
+                const uint32_t t_col = lane_base + (uint32_t)(acc * nt + first_step * kStepCols);
+                // all of this warp's columns are requested at once and the accumulator goes back to the MMA
+                // warp before anything is converted
+                uint32_t rr[kMaxSteps][16];
+#pragma unroll
+                for (int s = 0; s < kMaxSteps; ++s)
+                    if (s < my_steps) tmem_ld_32x32b_x16(t_col + (uint32_t)(s * kStepCols), rr[s]);
+                if (my_steps > 0) tmem_wait_ld();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive_cluster(empty_remote + 8 * acc);
+                if (lane == 0) {
+                    mbar_arrive_cluster(empty_remote + 8 * acc);
+                    bulk_wait_group_read<0>();   // the stores of the previous tile have drained the buffer
+                }
+                __syncwarp();
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    if (!(h == 0 ? mine0 : mine1)) continue;
-                    if (lane == 0) bulk_wait_group_read<0>();   // the previous store has drained the buffer
-                    __syncwarp();
-                    // staging tile [32 token rows][32 features], 64-byte rows with the 64-byte swizzle; this
-                    // lane writes the feature pair (lane & ~1, lane | 1) of one row per row pair
-                    // (all exchanges first, then all stores: interleaved, each store would wait for its shuffle)
-                    uint32_t word[16];
+                for (int s = 0; s < kMaxSteps; ++s) {
+                    if (s >= my_steps) continue;
+                    uint32_t w[8];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const uint32_t own = pack2<kBf16>(__uint_as_float(rr[h][2 * j]) + bias_f, __uint_as_float(rr[h][2 * j + 1]) + bias_f);
-                        const uint32_t got = __shfl_xor_sync(0xFFFFFFFFu, own, 1);
-                        asm("prmt.b32 %0, %1, %2, %3;" : "=r"(word[j]) : "r"(odd ? got : own), "r"(odd ? own : got), "r"(prmt_sel));
+                    for (int j = 0; j < 8; ++j)
+                        w[j] = pack2<kBf16>(__uint_as_float(rr[s][2 * j]) + bias_f, __uint_as_float(rr[s][2 * j + 1]) + bias_f);
+                    stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64), w[0], w[1], w[2], w[3]);
+                    stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64 + 512), w[4], w[5], w[6], w[7]);
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (f0 < l_out) {
+#pragma unroll
+                        for (int s = 0; s < kMaxSteps; ++s)
+                            if (s < my_steps && row0 + s * kStepCols < l_rows)
+                                tma_store_2d(&L.map_y, buf + (uint32_t)(s * kStepCols * 64), f0, row0 + s * kStepCols);
                     }
-#pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + lane_off + (uint32_t)(j * 128) + sw_off[j & 3]), "r"(word[j])
-                                     : "memory");
-                    fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        const int row0 = r0 + (part + h * kEpiParts) * kEpiCols;
-                        if (row0 < l_rows && f0 < l_out) tma_store_2d(&L.map_y, buf, f0, row0);
-                        bulk_commit_group();
-                    }
+                    bulk_commit_group();
                 }
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
@@ -435,13 +497,12 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
     }
 }
 
-// Token rows per pair tile for a layer of this input width: the largest multiple of 32, at most
-// kMaxRowTile, that leaves room for the weight block and its metadata; 0 if none does.
+// Token rows per pair tile for a layer of this input width: the largest multiple of 16, at most
+// kMaxRowTile, such that two accumulators fit beside the weight block and its metadata; 0 if none does.
 int ws_row_tile(int in)
 {
     const int left = kTmemCols - in / 4 - in / 32;
-    int nt = left / kNumAccum / 32 * 32;
-    static_assert(kNumAccum == 1, "one accumulator: see the head of this file");
+    int nt = left / kNumAccum / kStepCols * kStepCols;
     if (nt > kMaxRowTile) nt = kMaxRowTile;
     return nt >= 64 ? nt : 0;
 }
@@ -452,10 +513,19 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
 {
     auto kernel = linear_tc_sp24_ws_kernel<kBf16, kMaxLayers>;
     const int fixed = kStagingTotal + kBarrierBytes + 1024;
-    int stages = (int)((dev.smem_optin - fixed) / kStageBytes);
+    int max_nt = 0;
+    for (int i = 0; i < n; ++i) {
+        const int nt = ws_row_tile(jobs[i].in);
+        if (nt > max_nt) max_nt = nt;
+    }
+    if (max_nt == 0) return fail(ELSA_ERR_SHAPE, "in=%d does not fit the weight-stationary sparse kernel", jobs[0].in);
+    // a stage slot is sized for the widest row tile of the launch, so that narrow tiles still keep
+    // the same number of activation bytes in flight
+    const int stage_bytes = (kStageK / 64) * (max_nt / 2) * 128;
+    int stages = (int)((dev.smem_optin - fixed) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
-    const size_t smem = (size_t)stages * kStageBytes + fixed;
+    const size_t smem = (size_t)stages * stage_bytes + fixed;
 
     static int max_pairs[64] = {};
     const int slot = dev.device & 63;
@@ -473,7 +543,7 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         attr[0].val.clusterDim.z = 1;
         cfg.gridDim = dim3((unsigned)dev.sm_count);
         cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem;
+        cfg.dynamicSmemBytes = dev.smem_optin;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
         int m = 0;
@@ -498,6 +568,7 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         if (L.nt == 0 || j.in % kBlockK != 0 || L.tiles_f > pairs)
             return fail(ELSA_ERR_SHAPE, "in=%d out=%d does not fit the weight-stationary sparse kernel", j.in, j.out);
         L.rows = j.rows; L.out = j.out; L.in = j.in;
+        L.steps_per_warp = (L.nt / kStepCols + kEpiParts - 1) / kEpiParts;
         L.row_tiles = (j.rows + L.nt - 1) / L.nt;
         L.groups = pairs / L.tiles_f;
         if (L.groups > L.row_tiles) L.groups = L.row_tiles;
@@ -505,18 +576,19 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         L.num_k_blocks = j.in / kBlockK;
         L.bias = j.bias;
         L.a_img = (const uint16_t*)j.workspace;
-        L.meta = (const uint8_t*)j.workspace + round_up((size_t)j.out * (size_t)j.in, 256);
+        L.meta = (const uint8_t*)j.workspace + sp24_meta_offset(j.out, j.in);
         // sparse flag, fp32 accumulate, A and B of type fmt, K-major, N = nt, M = 256 over the pair
         L.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.nt >> 3) << 17) |
                   ((uint32_t)(kPairFeat >> 4) << 24);
         elsa_status st;
         if ((st = make_map_x_quarters(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, (uint32_t)(L.nt / 2))) != ELSA_OK) return st;
-        if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B,
+        if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, 32, kStepCols, CU_TENSOR_MAP_SWIZZLE_NONE,
                               "Y")) != ELSA_OK)
             return st;
     }
     g.n_layers = n;
     g.stages = stages;
+    g.stage_bytes = stage_bytes;
     g.dev_status = dev_status;
 
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_SP24_WS, stream);
@@ -556,7 +628,7 @@ elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16
                                        const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
                                        void* workspace, uint32_t* dev_status, cudaStream_t stream)
 {
-    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, workspace, stream);
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, true, workspace, stream);
     if (st != ELSA_OK) return st;
     SparseJob job;
     job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;
