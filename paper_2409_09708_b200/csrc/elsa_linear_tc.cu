@@ -133,7 +133,7 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         // instructions are predicated on one elected lane (a single thread inside a divergent branch
         // needs about twice as long per MMA).
         {
-            const bool elected = elect_one();
+            const uint32_t elected = elect_one() ? 1u : 0u;
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -157,15 +157,14 @@ linear_tc_dense_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
                         // advancing K by 16 elements = 32 bytes inside the swizzle row: +2 in the
                         // 16-byte-unit start address field
-                        if (elected)
-                            umma_f16(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
-                                     (uint32_t)((kb | k) != 0));
+                        umma_f16_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc,
+                                    (uint32_t)((kb | k) != 0), elected);
                     }
-                    if (elected) umma_commit(empty_bar + 8 * stage);  // frees the stage once these MMAs have read it
+                    umma_commit_if(empty_bar + 8 * stage, elected);  // frees the stage once these MMAs have read it
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (elected) umma_commit(tmem_full_bar + 8 * acc);    // accumulator complete
+                umma_commit_if(tmem_full_bar + 8 * acc, elected);    // accumulator complete
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }

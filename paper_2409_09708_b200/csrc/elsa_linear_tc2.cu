@@ -175,7 +175,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         // registers; only the MMA and commit instructions are predicated on one elected lane.  A
         // single thread inside a divergent branch needs about twice as long to issue one MMA.
         if (cta_rank == 0) {
-            const bool elected = elect_one();
+            const uint32_t elected = elect_one() ? 1u : 0u;
             // the base address came from shared memory in an ordinary register; a warp reduction returns it
             // in a uniform one, so that the addresses derived from it stay uniform too
             const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
@@ -204,15 +204,14 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        if (elected)
-                            umma_f16_pair(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                          (uint32_t)((kb | k) != 0));
+                        umma_f16_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                         (uint32_t)((kb | k) != 0), elected);
                     }
-                    if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);   // frees this stage in both CTAs
+                    umma_commit_pair_if(empty_bar + 8 * stage, 3, elected);   // frees this stage in both CTAs
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);     // accumulator complete in both CTAs
+                umma_commit_pair_if(tmem_full_bar + 8 * acc, 3, elected);     // accumulator complete in both CTAs
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }

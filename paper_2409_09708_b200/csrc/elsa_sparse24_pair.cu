@@ -158,7 +158,7 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
         // instructions are predicated on one elected lane (a single thread inside a divergent branch
         // needs about twice as long per MMA).
         if (cta_rank == 0) {
-            const bool elected = elect_one();
+            const uint32_t elected = elect_one() ? 1u : 0u;
             // the base address came from shared memory in an ordinary register; a warp reduction returns it
             // in a uniform one, so that the addresses derived from it stay uniform too
             const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
@@ -188,20 +188,19 @@ linear_tc_sp24_pair_kernel(const __grid_constant__ SpPairGroup<kMaxLayers> p)
                     const uint32_t e_col = tmem_u + (uint32_t)(kMetaCol0 + 4 * stage);
                     // each CTA's metadata block into its own tensor memory; runs before the MMAs below
                     const uint64_t e_desc = smem_desc_rows16_no_swizzle(a_addr + kATileBytes + kBTileBytes);
-                    if (elected) tmem_cp_128x128b_pair(e_col, e_desc);
+                    tmem_cp_128x128b_pair_if(e_col, e_desc, elected);
 #pragma unroll
                     for (int j = 0; j < kBlockK / kSpUmmaK; ++j) {
                         // K step of 32: 32 bytes of compressed A, 64 bytes of B in the half that holds it
                         const uint64_t b_desc = (j < 2 ? b_desc0 : b_desc1) + (uint64_t)(4 * (j & 1));
-                        if (elected)
-                            umma_sp_f16_pair(d_tmem, a_desc + (uint64_t)(2 * j), b_desc, e_col + (uint32_t)j, p.idesc,
-                                             (uint32_t)((kb | j) != 0));
+                        umma_sp_f16_pair_if(d_tmem, a_desc + (uint64_t)(2 * j), b_desc, e_col + (uint32_t)j, p.idesc,
+                                            (uint32_t)((kb | j) != 0), elected);
                     }
-                    if (elected) umma_commit_pair(empty_bar + 8 * stage, 3);
+                    umma_commit_pair_if(empty_bar + 8 * stage, 3, elected);
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (elected) umma_commit_pair(tmem_full_bar + 8 * acc, 3);
+                umma_commit_pair_if(tmem_full_bar + 8 * acc, 3, elected);
                 if (++acc == kNumAccum) { acc = 0; acc_phase ^= 1u; }
             }
         }

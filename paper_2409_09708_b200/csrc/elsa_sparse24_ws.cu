@@ -100,19 +100,6 @@ __device__ __forceinline__ void umma_sp_f16_pair_ts(uint32_t d_tmem, uint32_t a_
         : "memory");
 }
 
-// umma_commit_pair, predicated the same way.
-__device__ __forceinline__ void umma_commit_pair_if(uint32_t bar, uint16_t cta_mask, uint32_t issue)
-{
-    asm volatile(
-        "{\n"
-        ".reg .pred q;\n"
-        "setp.ne.b32 q, %2, 0;\n"
-        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n"
-        "}\n" ::"r"(bar),
-        "h"(cta_mask), "r"(issue)
-        : "memory");
-}
-
 // Lane i of the warp receives 16 consecutive fp32 columns of TMEM lane (lane base + i).
 __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)[16])
 {
