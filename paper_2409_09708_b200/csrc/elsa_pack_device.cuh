@@ -184,6 +184,33 @@ __device__ __forceinline__ uint32_t keep_mask_sorted(const uint32_t (&h)[M], int
     uint32_t k[M], s[M];
 #pragma unroll
     for (int i = 0; i < M; ++i) { k[i] = ((h[i] & 0x7FFFu) << S) | (uint32_t)(M - 1 - i); s[i] = k[i]; }
+    if constexpr (M == 8) {
+        // The levels of the ViT tables need less than a full sort.  Keys are unique and carry their position
+        // in the low bits, so the one or two largest keys name the kept positions directly; for N = 4 two
+        // sorted halves give the 4th largest without merging them.
+        if (N <= 2) {
+            sort2_desc(s[0], s[1]); sort2_desc(s[2], s[3]); sort2_desc(s[4], s[5]); sort2_desc(s[6], s[7]);
+            // top two of each half from two sorted pairs, then of the whole group
+            const uint32_t a0 = max(s[0], s[2]), a1 = max(min(s[0], s[2]), max(s[1], s[3]));
+            const uint32_t b0 = max(s[4], s[6]), b1 = max(min(s[4], s[6]), max(s[5], s[7]));
+            const uint32_t top = max(a0, b0), second = max(min(a0, b0), max(a1, b1));
+            uint32_t keep = 1u << (7u - (top & 7u));
+            if (N == 2) keep |= 1u << (7u - (second & 7u));
+            return keep;
+        }
+        if (N == 4) {
+            sort2_desc(s[0], s[1]); sort2_desc(s[2], s[3]); sort2_desc(s[4], s[5]); sort2_desc(s[6], s[7]);
+            sort2_desc(s[0], s[2]); sort2_desc(s[1], s[3]); sort2_desc(s[4], s[6]); sort2_desc(s[5], s[7]);
+            sort2_desc(s[1], s[2]); sort2_desc(s[5], s[6]);
+            // i elements of one half and j of the other lie above min(a_i, b_j): with i + j = 2 it is at most the
+            // 4th largest, and so are a_3 and b_3 (a half that supplies all four); the largest candidate is it
+            const uint32_t thr4 = max(max(max(s[3], s[7]), min(s[0], s[6])), max(min(s[1], s[5]), min(s[2], s[4])));
+            uint32_t keep4 = 0;
+#pragma unroll
+            for (int i = 0; i < M; ++i) keep4 |= (k[i] >= thr4 ? 1u : 0u) << i;
+            return keep4;
+        }
+    }
     if constexpr (M == 4) {
         sort2_desc(s[0], s[1]); sort2_desc(s[2], s[3]);
         sort2_desc(s[0], s[2]); sort2_desc(s[1], s[3]);
@@ -205,34 +232,42 @@ __device__ __forceinline__ uint32_t keep_mask_sorted(const uint32_t (&h)[M], int
     return keep;
 }
 
+// Split in two so that a warp can have the loads of several segments in flight before it works on the
+// first: one 16-byte load per lane is too little outstanding memory traffic to cover its own latency.
 template <int M>
-__device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict__ W, int in, int N,
-                                                      uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
-                                                      int segs_per_row, long long seg_id,
-                                                      uint32_t (*words)[kMaxIndexWordsPerSegment],
-                                                      const CompactEntry* table)
+__device__ __forceinline__ void compress_fast_load(const uint16_t* __restrict__ W, int in, int o, int seg,
+                                                   uint32_t (&r)[M / 2])
+{
+    constexpr int R = M / 2;                      // 32-bit registers per group
+    const int lane = threadIdx.x & 31;
+    const int g = seg * 32 + lane;
+#pragma unroll
+    for (int q = 0; q < R; ++q) r[q] = 0;
+    if (g < in / M) {
+        const uint16_t* src = W + (size_t)o * in + (size_t)g * M;
+        if constexpr (M == 4) { const uint2 v = *reinterpret_cast<const uint2*>(src); r[0] = v.x; r[1] = v.y; }
+        else { const uint4 v = *reinterpret_cast<const uint4*>(src); r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w; }
+    }
+}
+
+template <int M>
+__device__ __forceinline__ void compress_fast_emit(const uint32_t (&r)[M / 2], int in, int N,
+                                                   uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                   int o, int seg,
+                                                   uint32_t (*words)[kMaxIndexWordsPerSegment],
+                                                   const CompactEntry* table)
 {
     static_assert(M == 4 || M == 8, "fast path for groups of 4 and 8");
     constexpr int B = (M == 4) ? 2 : 3;
-    constexpr int R = M / 2;                      // 32-bit registers per group
+    constexpr int R = M / 2;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    const int o = (int)(seg_id / segs_per_row);
-    const int seg = (int)(seg_id % segs_per_row);
     const int groups_per_row = in / M;
     const int g = seg * 32 + lane;
     const bool valid = g < groups_per_row;
     const int words_per_row = (N == M) ? 0 : (groups_per_row * N * B + 31) / 32;
     const int seg_words = N * B;
 
-    uint32_t r[R];
-#pragma unroll
-    for (int q = 0; q < R; ++q) r[q] = 0;
-    if (valid) {
-        const uint16_t* src = W + (size_t)o * in + (size_t)g * M;
-        if constexpr (M == 4) { const uint2 v = *reinterpret_cast<const uint2*>(src); r[0] = v.x; r[1] = v.y; }
-        else { const uint4 v = *reinterpret_cast<const uint4*>(src); r[0] = v.x; r[1] = v.y; r[2] = v.z; r[3] = v.w; }
-    }
     uint16_t* dst = vals + (size_t)o * ((size_t)groups_per_row * N) + (size_t)g * N;
     if (N == M) {                                 // dense level: the values are the weight
         if (valid) {
@@ -291,6 +326,21 @@ __device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict
     uint32_t* row = idx + (size_t)o * words_per_row;
     for (int k = lane; k < seg_words && first + k < words_per_row; k += 32) row[first + k] = words[warp][k];
     __syncwarp();
+}
+
+template <int M>
+__device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict__ W, int in, int N,
+                                                      uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                      int segs_per_row, long long seg_id,
+                                                      uint32_t (*words)[kMaxIndexWordsPerSegment],
+                                                      const CompactEntry* table)
+{
+    // a weight has far fewer than 2^32 segments: 32-bit division
+    const uint32_t o = (uint32_t)seg_id / (uint32_t)segs_per_row;
+    const uint32_t seg = (uint32_t)seg_id - o * (uint32_t)segs_per_row;
+    uint32_t r[M / 2];
+    compress_fast_load<M>(W, in, (int)o, (int)seg, r);
+    compress_fast_emit<M>(r, in, N, vals, idx, (int)o, (int)seg, words, table);
 }
 
 // Single level: the form elsa_nm_compress uses.
