@@ -33,7 +33,7 @@ if ROOT not in sys.path:
 
 METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
-GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws")   # forms of the tcgen05 GEMM
+GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws", "linear_tc_sp24_st")   # forms of the tcgen05 GEMM
 
 # dram__bytes_read.sum + dram__bytes_write.sum of each GEMM kernel's launches over ONE step of this
 # benchmark, from a one-pass ncu capture of the same command (the two DRAM counters

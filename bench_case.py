@@ -1,12 +1,12 @@
 """Runs one N:M linear layer a few times through the C ABI: a small, bounded case for profilers.
 
-    python -m paper_2409_09708_b200.profile_case --rows 50432 --in 768 --out 3072 --level 2:8 \
+    python bench_case.py --rows 50432 --in 768 --out 3072 --level 2:8 \
         --dtype bf16 --reps 3
 
 Prints one JSON line with the CUDA-event time of each repetition (compress once, then `reps`
 calls of elsa_nm_linear), the layer's algorithmic bytes and kept FLOPs.
 
-    python -m paper_2409_09708_b200.profile_case --compress-table deit_b_stack_b256 --reps 3
+    python bench_case.py --compress-table deit_b_stack_b256 --reps 3
 
 runs elsa_vit_compress over the weights of a workload table instead (weights only, no activations).
 """
@@ -17,8 +17,15 @@ import json
 
 import torch
 
-from . import binding as lib
-from . import synth
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2409_09708_b200 import binding as lib
+from paper_2409_09708_b200 import synth
 
 
 def compress_table(workload, reps):
@@ -55,7 +62,7 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["f16", "bf16"])
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--variant", default="auto", choices=["auto", "simt", "tc_dense", "tc_pair", "tc_sparse", "tc_sparse_pair",
-                                                            "tc_sparse_ws"])
+                                                            "tc_sparse_ws", "tc_sparse_st"])
     ap.add_argument("--compress-table", default=None, help="workload whose weights go through elsa_vit_compress")
     args = ap.parse_args()
     if args.compress_table:
@@ -71,7 +78,8 @@ def main():
     lib.elsa_set_linear_variant({"auto": lib.VARIANT_AUTO, "simt": lib.VARIANT_SIMT,
                                  "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR, "tc_sparse": lib.VARIANT_TC_SPARSE,
                                  "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR,
-                                 "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS}[args.variant])
+                                 "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS,
+                                 "tc_sparse_st": lib.VARIANT_TC_SPARSE_ST}[args.variant])
     times = []
     for _ in range(args.reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)

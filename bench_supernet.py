@@ -1,10 +1,10 @@
 """Timing of the supernet-side forms (Sec. 3.1 of the ELSA paper: shared weight, dynamic masking).
 
-    python -m paper_2409_09708_b200.supernet_bench [--out bench_out/supernet.json]
+    python bench_supernet.py [--out bench_out/supernet.json]
 
 (a) elsa_nm_compress_levels: all levels {1,2,4,8}:8 of a weight from one read, against one
-    elsa_nm_compress call per level, and against the CPU oracle doing the same (GB/s counts the
-    dense weight once plus every packed form written).
+    elsa_nm_compress call per level (GB/s counts the dense weight once plus every packed form
+    written).
 (b) elsa_nm_linear_masked (dense shared weight + level, no packed copy) against elsa_nm_compress +
     elsa_nm_linear on the DeiT-B layer shapes at batch 256, bf16.
 CUDA-event medians of 7 repetitions, 512 MB written between repetitions to flush L2.
@@ -13,14 +13,19 @@ from __future__ import annotations
 
 import argparse
 import json
-import os
 import statistics
-import time
 
 import torch
 
-from . import binding as lib
-from . import synth
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2409_09708_b200 import binding as lib
+from paper_2409_09708_b200 import synth
 
 
 def timed(fn, flush, reps=7):
@@ -39,7 +44,6 @@ def timed(fn, flush, reps=7):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--out", default="bench_out/supernet.json")
-    ap.add_argument("--no-oracle", action="store_true")
     args = ap.parse_args()
     dtype = torch.bfloat16
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")
@@ -54,14 +58,6 @@ def main():
         nbytes = W.numel() * 2 + sum(v.numel() * 2 + (i.numel() * 4 if i is not None else 0) for v, i in packed)
         rec = {"op": "compress_levels", "out": out, "in": in_, "levels": levels, "ms_one_pass": ms_all,
                "ms_per_level_calls": ms_each, "gbs_one_pass": nbytes / ms_all / 1e6}
-        if not args.no_oracle:
-            from oracle import elsa_oracle as eo
-            Wb = synth.bits(W)
-            t0 = time.perf_counter()
-            for N in levels:
-                eo.nm_compress(Wb, N, 8)
-            rec["oracle_ms"] = (time.perf_counter() - t0) * 1e3
-            rec["oracle_cores"] = eo.omp_threads()
         results.append(rec)
     rows = 256 * 197
     for name, in_, out in [("qkv", 768, 2304), ("proj", 768, 768), ("fc1", 768, 3072), ("fc2", 3072, 768)]:

@@ -1,6 +1,6 @@
 """Shape / sparsity sweep of elsa_nm_linear and elsa_nm_compress on one GPU.
 
-    python -m paper_2409_09708_b200.sweep [--out bench_out/sweep.json] [--reps 5] [--quick]
+    python bench_sweep.py [--out bench_out/sweep.json] [--reps 5] [--quick]
 
 rows in {4096, 16384, 65536} x (K, O) in {(768,768), (768,3072), (3072,768), (1024,4096), (4096,1024)}
 x level in {1:4, 2:4, 1:8, 2:8, 4:8, 1:16, 2:16, 4:16, 8:16} x {fp16, bf16}: per point the median
@@ -13,17 +13,23 @@ from __future__ import annotations
 
 import argparse
 import json
-import os
 import statistics
 
 import torch
 
-from . import binding as lib
-from . import synth
+import os
+import sys
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2409_09708_b200 import binding as lib
+from paper_2409_09708_b200 import synth
 
 
 def load_peaks():
-    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         d = json.load(open(path))
         return float(d["hbm_gbs"]), float(d["bf16_tflops"]), "measured"
@@ -106,7 +112,7 @@ def main():
 def write_summary(path, hbm, tf, kind, lin, cmp_):
     med = statistics.median
     out = ["# Shape / sparsity sweep (%d linear points, %d compress points) -- summary" % (len(lin), len(cmp_)), "",
-           "Command: `python -m paper_2409_09708_b200.sweep --out bench_out/sweep.json --summary <this file>` (B200;",
+           "Command: `python bench_sweep.py --out bench_out/sweep.json --summary <this file>` (B200;",
            "median of 5 CUDA-event timings per point, 512 MB written between repetitions to flush the 126 MB L2;",
            "time = weight-image rebuild + GEMM of `elsa_nm_linear` under the automatic dispatch).",
            "Peaks (%s): %.1f GB/s, %.1f TFLOP/s." % (kind, hbm, tf), "",

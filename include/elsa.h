@@ -72,8 +72,10 @@ typedef enum {
     ELSA_VARIANT_TC_PAIR = 3,  /* same, CTA pairs sharing a 256-row tile (tcgen05 cta_group::2) */
     ELSA_VARIANT_TC_SPARSE = 4, /* N <= 2 only: re-encode as 2-of-4 + metadata, tcgen05 sparse MMA */
     ELSA_VARIANT_TC_SPARSE_PAIR = 5, /* the same on CTA pairs (256 features x 224 rows per pair) */
-    ELSA_VARIANT_TC_SPARSE_WS = 6 /* N <= 2, in % 128 == 0, in <= 1024: CTA pairs that keep their 256-feature
-                                   * weight block and its metadata in tensor memory for a whole layer */
+    ELSA_VARIANT_TC_SPARSE_WS = 6, /* N <= 2, in % 128 == 0, in <= 1024: CTA pairs that keep their 256-feature
+                                    * weight block and its metadata in tensor memory for a whole layer */
+    ELSA_VARIANT_TC_SPARSE_ST = 7  /* N <= 2, in % 128 == 0, any length: the weight block streams through
+                                    * tensor memory in K chunks of 256, shared memory carries activations only */
 } elsa_variant;
 
 /* Sizes of the packed form (host-only arithmetic; 0 on invalid arguments). */
@@ -268,7 +270,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_SP24 = 6,
     ELSA_KERNEL_LINEAR_TC_SP24_PAIR = 7,
     ELSA_KERNEL_WEIGHT_IMAGES = 8, /* batched unpack / 2-of-4 re-encoding of a table's weights */
-    ELSA_KERNEL_LINEAR_TC_SP24_WS = 9 /* 2:4 sparse MMA with the weight block resident in tensor memory */
+    ELSA_KERNEL_LINEAR_TC_SP24_WS = 9, /* 2:4 sparse MMA with the weight block resident in tensor memory */
+    ELSA_KERNEL_LINEAR_TC_SP24_ST = 10 /* 2:4 sparse MMA with the weight streaming through tensor memory */
 } elsa_kernel_id;
 
 typedef struct {

@@ -32,6 +32,7 @@ ERR_NAMES = {0: "ELSA_OK", 1: "ELSA_ERR_NULL", 2: "ELSA_ERR_SHAPE", 3: "ELSA_ERR
 F16, BF16 = 0, 1
 VARIANT_AUTO, VARIANT_SIMT, VARIANT_TC_DENSE, VARIANT_TC_PAIR, VARIANT_TC_SPARSE, VARIANT_TC_SPARSE_PAIR = 0, 1, 2, 3, 4, 5
 VARIANT_TC_SPARSE_WS = 6
+VARIANT_TC_SPARSE_ST = 7
 
 _vp, _i, _sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
 
@@ -85,7 +86,7 @@ class ElsaKernelTime(ctypes.Structure):
 
 
 KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images",
-                9: "linear_tc_sp24_ws"}
+                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 

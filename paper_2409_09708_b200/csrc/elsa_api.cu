@@ -136,7 +136,13 @@ elsa_status check_linear(const void* X, int rows, const void* vals, const uint32
     return ELSA_OK;
 }
 
-enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR, KIND_SPARSE_WS };
+enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR, KIND_SPARSE_WS, KIND_SPARSE_ST };
+
+// Form of the 2-of-4 weight image each sparse kernel reads.
+int sp24_layout_of(LinearKind kind)
+{
+    return kind == KIND_SPARSE_WS ? SP24_PERMUTED : kind == KIND_SPARSE_ST ? SP24_TILED : SP24_ROWS;
+}
 
 // Which kernel a layer runs on.  AUTO is the product rule; a forced variant is honoured where it applies.
 elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, LinearKind* kind)
@@ -159,6 +165,11 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
                         "(got %d:%d, in=%d)", N, M, in);
         *kind = KIND_SPARSE_WS;
         return ELSA_OK;
+    case ELSA_VARIANT_TC_SPARSE_ST:
+        if (N == M || !linear_tc_sparse_st_suits(in, N))
+            return fail(ELSA_ERR_NM, "the streaming sparse variant needs N <= 2 < M and in %% 128 == 0 (got %d:%d, in=%d)", N, M, in);
+        *kind = KIND_SPARSE_ST;
+        return ELSA_OK;
     default: break;
     }
     // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K is
@@ -170,7 +181,10 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
         // four blocks of 256 features (qkv, fc1: 10-15 %), equal or slower elsewhere.
         const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in <= 896 && out >= 1024 &&
                         rows >= 256 * (sm_count / 2) / ((out + 255) / 256);
-        *kind = ws ? KIND_SPARSE_WS : KIND_SPARSE_PAIR;
+        // Longer reductions do not fit tensor memory whole: the weight streams through it chunk by chunk, which
+        // still keeps it out of shared memory (measured against staging it there for every row tile).
+        const bool st = !ws && in > 768 && linear_tc_sparse_st_suits(in, N);
+        *kind = ws ? KIND_SPARSE_WS : st ? KIND_SPARSE_ST : KIND_SPARSE_PAIR;
     }
     else
         *kind = linear_tc_pair_suits(rows, out, sm_count) ? KIND_DENSE_PAIR : KIND_DENSE_ONE;
@@ -198,6 +212,9 @@ elsa_status run_linear(const void* X, int rows, const void* vals, const uint32_t
                                             out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
     if (kind == KIND_SPARSE_WS)
         return launch_linear_tc_sparse_ws((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias,
+                                          out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
+    if (kind == KIND_SPARSE_ST)
+        return launch_linear_tc_sparse_st((const uint16_t*)X, rows, (const uint16_t*)vals, idx, (const uint16_t*)bias,
                                           out, in, N, M, dtype, (uint16_t*)Y, workspace, dev_status, stream);
     // Dense-rate path.  The dense level multiplies the stored values as they are; every other level first
     // rebuilds the weight image the MMA reads, in the caller's scratch.
@@ -335,16 +352,17 @@ elsa_status elsa_nm_linear_masked(const void* X, int rows, const void* W_sup, co
     if ((st = pick_kind(rows, out, in, N, M, dev.sm_count, &kind)) != ELSA_OK) return st;
     if (kind == KIND_SIMT || kind == KIND_SPARSE_ONE)
         return fail(ELSA_ERR_NM, "the forced variant has no mask-on-load form");
-    if (kind == KIND_SPARSE_PAIR || kind == KIND_SPARSE_WS) {
+    if (kind == KIND_SPARSE_PAIR || kind == KIND_SPARSE_WS || kind == KIND_SPARSE_ST) {
         uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
-        if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, kind == KIND_SPARSE_WS, (uint16_t*)workspace, meta,
+        if ((st = launch_dense_to_sp24((const uint16_t*)W_sup, out, in, N, M, 128, sp24_layout_of(kind), (uint16_t*)workspace, meta,
                                        stream)) != ELSA_OK)
             return st;
         SparseJob job;
         job.X = (const uint16_t*)X; job.bias = (const uint16_t*)bias; job.Y = (uint16_t*)Y; job.workspace = workspace;
         job.rows = rows; job.in = in; job.out = out;
-        return kind == KIND_SPARSE_WS ? launch_linear_tc_sparse_ws_group(&job, 1, dtype, dev_status, stream)
-                                      : launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
+        return kind == KIND_SPARSE_WS   ? launch_linear_tc_sparse_ws_group(&job, 1, dtype, dev_status, stream)
+               : kind == KIND_SPARSE_ST ? launch_linear_tc_sparse_st_group(&job, 1, dtype, dev_status, stream)
+                                        : launch_linear_tc_sparse_pair_group(&job, 1, dtype, dev_status, stream);
     }
     const uint16_t* Wd = (const uint16_t*)W_sup;     // the dense level multiplies the shared weight as it is
     if (N != M) {
@@ -471,10 +489,10 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
         for (int l = 0; l < n_layers; ++l) {
             const elsa_layer& c = cfg[l];
             if (c.N != c.M) {
-                if (kind[l] == KIND_SPARSE_PAIR || kind[l] == KIND_SPARSE_WS) {
+                if (kind[l] == KIND_SPARSE_PAIR || kind[l] == KIND_SPARSE_WS || kind[l] == KIND_SPARSE_ST) {
                     uint8_t* meta = region[l] + sp24_meta_offset(c.out, c.in);
                     batch_add_to_sp24(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, 128,
-                                      kind[l] == KIND_SPARSE_WS, (uint16_t*)region[l], meta);
+                                      sp24_layout_of(kind[l]), (uint16_t*)region[l], meta);
                 } else {
                     batch_add_unpack(&table, (const uint16_t*)c.vals, c.idx, c.out, c.in, c.N, c.M, (uint16_t*)region[l]);
                 }
@@ -499,6 +517,24 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
             }
             if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_sparse_pair_group_max())) {
                 if ((st = launch_linear_tc_sparse_pair_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
+                    return st;
+                jobs.clear();
+            }
+        }
+    }
+    // sparse-rate layers whose weight block streams through tensor memory, in groups
+    {
+        std::vector<SparseJob> jobs;
+        for (int l = 0; l <= n_layers; ++l) {
+            if (l < n_layers && kind[l] == KIND_SPARSE_ST) {
+                const elsa_layer& c = cfg[l];
+                SparseJob j;
+                j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
+                j.workspace = region[l]; j.rows = c.rows; j.in = c.in; j.out = c.out;
+                jobs.push_back(j);
+            }
+            if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_sparse_st_group_max())) {
+                if ((st = launch_linear_tc_sparse_st_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
                     return st;
                 jobs.clear();
             }
@@ -711,7 +747,8 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
     if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR &&
-        v != ELSA_VARIANT_TC_SPARSE && v != ELSA_VARIANT_TC_SPARSE_PAIR && v != ELSA_VARIANT_TC_SPARSE_WS)
+        v != ELSA_VARIANT_TC_SPARSE && v != ELSA_VARIANT_TC_SPARSE_PAIR && v != ELSA_VARIANT_TC_SPARSE_WS &&
+        v != ELSA_VARIANT_TC_SPARSE_ST)
         return fail(ELSA_ERR_SHAPE, "unknown variant %d", (int)v);
     g_variant.store((int)v, std::memory_order_relaxed);
     return ELSA_OK;

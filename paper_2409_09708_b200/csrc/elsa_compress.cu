@@ -161,10 +161,10 @@ nm_image_batch_kernel(const __grid_constant__ BatchTable t)
         } else {
             uint16_t* a_img = (uint16_t*)it.dst;
             uint16_t* meta16 = (uint16_t*)it.dst2;
-            // aux = K blocks of the metadata layout, aux2 = K steps per block, aux3 = permuted row order
-            if (it.M == 4) to_sp24_segment<4>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3 != 0, local);
-            else if (it.M == 8) to_sp24_segment<8>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3 != 0, local);
-            else to_sp24_segment<16>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3 != 0, local);
+            // aux = K blocks of the metadata layout, aux2 = K steps per block, aux3 = layout of the image
+            if (it.M == 4) to_sp24_segment<4>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3, local);
+            else if (it.M == 8) to_sp24_segment<8>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3, local);
+            else to_sp24_segment<16>(vals, idx, it.out, it.in, it.N, it.wpr, a_img, meta16, it.aux, it.aux2, it.aux3, local);
         }
     }
 }
@@ -262,7 +262,7 @@ void batch_add_unpack(BatchTable* t, const uint16_t* vals, const uint32_t* idx, 
 }
 
 void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                       int block_k, bool permuted, uint16_t* a_img, uint8_t* meta)
+                       int block_k, int layout, uint16_t* a_img, uint8_t* meta)
 {
     BatchItem& it = t->item[t->n++];
     const int tiles_f = (out + 127) / 128;
@@ -271,7 +271,7 @@ void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx,
     it.src = vals; it.src2 = idx; it.dst = a_img; it.dst2 = meta;
     it.out = out; it.in = in; it.N = N; it.M = M;
     it.wpr = (int)index_words_per_row(in, N, M);
-    it.aux = k_blocks; it.aux2 = steps; it.aux3 = permuted ? 1 : 0; it.kind = BATCH_TO_SP24;
+    it.aux = k_blocks; it.aux2 = steps; it.aux3 = layout; it.kind = BATCH_TO_SP24;
     it.first_unit = t->total_units;
     t->total_units += (long long)tiles_f * 128 * k_blocks * steps * 2;
 }

@@ -103,11 +103,17 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                     const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype,
                                     uint16_t* Y, void* workspace, uint32_t* dev_status, cudaStream_t stream);
-// packed weight -> 2-of-4 image [out rounded up to 32][in/2] + metadata blocks of 2 KB per (128 features,
-// block_k of K), block_k = 64 or 128.  `permuted`: row r of every block of 32 image rows holds feature
-// 8 * (r % 4) + r / 4 of the block (the lane order of the weight-stationary kernel), else feature r.
+// Forms of the 2-of-4 image (its rows are rounded up to 32, rows past `out` are zero):
+//   SP24_ROWS      [row][in/2], row r holds feature r                       (TMA-fed kernels)
+//   SP24_PERMUTED  [row][in/2], row r of every block of 32 holds feature 8 * (r % 4) + r / 4 of the block: the
+//                  lane order of the kernels whose epilogue transposes with stmatrix (weight-stationary)
+//   SP24_TILED     permuted rows, and per (block of 32 rows, 256 k) the 16-byte units of all rows interleaved,
+//                  [unit][row][16 bytes], so that a warp reads one unit of 32 rows as one contiguous run
+//                  (streaming kernel); needs in % 128 == 0
+enum Sp24Layout { SP24_ROWS = 0, SP24_PERMUTED = 1, SP24_TILED = 2 };
+// packed weight -> 2-of-4 image + metadata blocks of 2 KB per (128 features, block_k of K), block_k = 64 or 128.
 elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
-                              bool permuted, uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
+                              int layout, uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
 // Where the metadata blocks start in a layer's scratch: after the image, whose rows are rounded up to 32.
 inline size_t sp24_meta_offset(int out, int in) { return round_up((size_t)((out + 31) / 32 * 32) * (size_t)in, 256); }
 // The same on CTA pairs (256 features x 224 rows per pair, K blocks of 128).
@@ -125,7 +131,7 @@ struct SparseJob {
 };
 int linear_tc_sparse_pair_group_max();
 elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                                                 bool permuted, void* workspace, cudaStream_t stream);
+                                                 int layout, void* workspace, cudaStream_t stream);
 elsa_status launch_linear_tc_sparse_pair_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
                                                cudaStream_t stream);
 bool linear_tc_sparse_suits(int in, int N);
@@ -139,6 +145,15 @@ elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16
                                        const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
                                        void* workspace, uint32_t* dev_status, cudaStream_t stream);
 size_t linear_tc_sparse_workspace(int out, int in);
+// The same product with the weight block streaming through tensor memory in K chunks of 256 (in % 128 == 0,
+// any length); jobs as for the pair kernel, weight image in the SP24_TILED form.
+int linear_tc_sparse_st_group_max();
+bool linear_tc_sparse_st_suits(int in, int N);
+elsa_status launch_linear_tc_sparse_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
+                                             cudaStream_t stream);
+elsa_status launch_linear_tc_sparse_st(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
+                                       const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
+                                       void* workspace, uint32_t* dev_status, cudaStream_t stream);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
 constexpr int kMaxLevels = 16;
 struct LevelTable {
@@ -149,7 +164,7 @@ struct LevelTable {
 };
 elsa_status launch_compress_levels(const uint16_t* W, int out, int in, int M, const LevelTable& t, cudaStream_t stream);
 elsa_status launch_mask(const uint16_t* W, int out, int in, int N, int M, uint16_t* Wm, cudaStream_t stream);
-elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, bool permuted,
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, int layout,
                                  uint16_t* a_img, uint8_t* meta, cudaStream_t stream);
 
 // Batched weight-format kernels: one launch over a table of weights (kernel-parameter space).
@@ -172,7 +187,7 @@ void batch_add_compress(BatchTable* t, const uint16_t* W, int out, int in, int N
 void batch_add_unpack(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
                       uint16_t* Wm);
 void batch_add_to_sp24(BatchTable* t, const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                       int block_k, bool permuted, uint16_t* a_img, uint8_t* meta);
+                       int block_k, int layout, uint16_t* a_img, uint8_t* meta);
 elsa_status launch_compress_batch(const BatchTable& t, cudaStream_t stream);
 elsa_status launch_image_batch(const BatchTable& t, cudaStream_t stream);
 

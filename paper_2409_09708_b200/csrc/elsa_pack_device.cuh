@@ -499,15 +499,16 @@ __device__ __forceinline__ void unpack_group(const uint16_t* __restrict__ vals, 
 // Second half of the 2-of-4 re-encoding: given 16 consecutive positions of a weight row with the pruned
 // ones already zero (d) and the kept set (keep), emits two values per aligned chunk of 4 (ascending
 // positions, a zero borrowed where fewer than two are kept) and the chunk nibbles as tensor memory wants them.
-// With `permuted`, weight row o lands in image row (o & ~31) | (4 * (o % 8) + (o % 32) / 8), so that row r of a
-// block of 32 holds feature 8 * (r % 4) + r / 4: the order in which the weight-stationary kernel's transposing
-// stores want the features in tensor-memory lanes.  The image has its rows rounded up to 32; rows past `out`
-// are written as zeros.
+// In the permuted forms (Sp24Layout) weight row o lands in image row (o & ~31) | (4 * (o % 8) + (o % 32) / 8), so
+// that row r of a block of 32 holds feature 8 * (r % 4) + r / 4: the order in which the transposing stores of the
+// tensor-memory-fed kernels want the features in tensor-memory lanes.  The tiled form also interleaves the
+// 16-byte units of the 32 rows of a block inside every 256 k.  The image has its rows rounded up to 32; rows
+// past `out` are written as zeros.
 __device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep, bool real, int o_src, int seg, int k0, int in,
                                           int out, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int k_blocks,
-                                          int steps_per_block, bool permuted)
+                                          int steps_per_block, int layout)
 {
-    const int o = permuted ? ((o_src & ~31) | (4 * (o_src & 7) + ((o_src & 31) >> 3))) : o_src;
+    const int o = layout != SP24_ROWS ? ((o_src & ~31) | (4 * (o_src & 7) + ((o_src & 31) >> 3))) : o_src;
     constexpr int kFeatTile = 128;
     uint32_t nibbles = 0;
     uint16_t sel[8];
@@ -536,7 +537,10 @@ __device__ __forceinline__ void sp24_emit(const uint16_t (&d)[16], uint32_t keep
         r.y = sel[2] | ((uint32_t)sel[3] << 16);
         r.z = sel[4] | ((uint32_t)sel[5] << 16);
         r.w = sel[6] | ((uint32_t)sel[7] << 16);
-        *reinterpret_cast<uint4*>(a_img + (size_t)o * (in / 2) + k0 / 2) = r;
+        size_t at = (size_t)o * (size_t)in + (size_t)k0;        // byte offset of (row o, k0) in the row-major forms
+        if (layout == SP24_TILED)
+            at = (size_t)(o >> 5) * 32 * (size_t)in + (size_t)(k0 >> 8) * 8192 + (size_t)((((k0 & 255) >> 4) * 32 + (o & 31)) * 16);
+        *reinterpret_cast<uint4*>(reinterpret_cast<uint8_t*>(a_img) + at) = r;
     }
     // metadata half-word: block (feature tile, k block) -> lane -> 4 words, one per K step of 32; a
     // block covers steps_per_block (2 or 4) steps and leaves the other words zero
@@ -557,7 +561,7 @@ template <int M>
 __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx,
                                                 int out, int in, int N, int words_per_row,
                                                 uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
-                                                int k_blocks, int steps_per_block, bool permuted, long long tid)
+                                                int k_blocks, int steps_per_block, int layout, long long tid)
 {
     constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
     constexpr int G = 16 / M;                         // groups per 16-k segment
@@ -591,7 +595,7 @@ __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ val
             }
         }
     }
-    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, permuted);
+    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, layout);
 }
 
 // The same from the DENSE shared weight: the 16 positions are projected onto level N:M on the fly
@@ -599,7 +603,7 @@ __device__ __forceinline__ void to_sp24_segment(const uint16_t* __restrict__ val
 template <int M>
 __device__ __forceinline__ void dense_to_sp24_segment(const uint16_t* __restrict__ W, int out, int in, int N,
                                                       uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16,
-                                                      int k_blocks, int steps_per_block, bool permuted, long long tid)
+                                                      int k_blocks, int steps_per_block, int layout, long long tid)
 {
     constexpr int G = 16 / M;
     const int segs = k_blocks * steps_per_block * 2;
@@ -623,7 +627,7 @@ __device__ __forceinline__ void dense_to_sp24_segment(const uint16_t* __restrict
             keep |= kg << (gl * M);
         }
     }
-    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, permuted);
+    sp24_emit(d, keep, real, o, seg, k0, in, out, a_img, meta16, k_blocks, steps_per_block, layout);
 }
 
 }  // namespace

@@ -56,25 +56,25 @@ template <int M>
 __global__ void __launch_bounds__(256)
 nm_to_sp24_kernel(const uint16_t* __restrict__ vals, const uint32_t* __restrict__ idx, int out, int in, int N,
                   int words_per_row, uint16_t* __restrict__ a_img, uint16_t* __restrict__ meta16, int out_tiles,
-                  int k_blocks, int steps_per_block, int permuted)
+                  int k_blocks, int steps_per_block, int layout)
 {
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
     if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
-    to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, permuted != 0, tid);
+    to_sp24_segment<M>(vals, idx, out, in, N, words_per_row, a_img, meta16, k_blocks, steps_per_block, layout, tid);
 }
 
 template <int M>
 __global__ void __launch_bounds__(256)
 dense_to_sp24_kernel(const uint16_t* __restrict__ W, int out, int in, int N, uint16_t* __restrict__ a_img,
-                     uint16_t* __restrict__ meta16, int out_tiles, int k_blocks, int steps_per_block, int permuted)
+                     uint16_t* __restrict__ meta16, int out_tiles, int k_blocks, int steps_per_block, int layout)
 {
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     pdl_wait_for_predecessors();
     pdl_release_successors();
     if (tid >= (long long)out_tiles * kFeatTile * k_blocks * steps_per_block * 2) return;
-    dense_to_sp24_segment<M>(W, out, in, N, a_img, meta16, k_blocks, steps_per_block, permuted != 0, tid);
+    dense_to_sp24_segment<M>(W, out, in, N, a_img, meta16, k_blocks, steps_per_block, layout, tid);
 }
 
 // ------------------------------------------------------------------ GEMM
@@ -270,9 +270,9 @@ linear_tc_sp24_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_co
 }  // namespace
 
 elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M, int block_k,
-                              bool permuted, uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
+                              int layout, uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
 {
-    const int perm = permuted ? 1 : 0;
+    const int perm = layout;
     const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
     const int k_blocks = (in + block_k - 1) / block_k;
     const int steps = block_k / kSpUmmaK;
@@ -292,10 +292,10 @@ elsa_status launch_nm_to_sp24(const uint16_t* vals, const uint32_t* idx, int out
     return launched("nm_to_sp24");
 }
 
-elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, bool permuted,
+elsa_status launch_dense_to_sp24(const uint16_t* W, int out, int in, int N, int M, int block_k, int layout,
                                  uint16_t* a_img, uint8_t* meta, cudaStream_t stream)
 {
-    const int perm = permuted ? 1 : 0;
+    const int perm = layout;
     const int tiles_f = (out + kFeatTile - 1) / kFeatTile;
     const int k_blocks = (in + block_k - 1) / block_k;
     const int steps = block_k / kSpUmmaK;
@@ -343,7 +343,7 @@ elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t*
     uint16_t* a_img = (uint16_t*)workspace;
     uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
 
-    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, false, a_img, meta, stream)) != ELSA_OK) return st;
+    if ((st = launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, SP24_ROWS, a_img, meta, stream)) != ELSA_OK) return st;
 
     SpParams p;
     p.rows = rows; p.in = in; p.out = out;

@@ -426,7 +426,7 @@ elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint
 {
     if (!linear_tc_sparse_suits(in, N) || N == M)
         return fail(ELSA_ERR_NM, "level %d:%d with in=%d does not fit the 2:4 sparse MMA path", N, M, in);
-    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, false, workspace, stream);
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, SP24_ROWS, workspace, stream);
     if (st != ELSA_OK) return st;
     SparseJob job;
     job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;
@@ -436,11 +436,11 @@ elsa_status launch_linear_tc_sparse_pair(const uint16_t* X, int rows, const uint
 
 // Re-encodes one packed weight into `workspace` in the form the pair kernel reads (K blocks of 128).
 elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
-                                                 bool permuted, void* workspace, cudaStream_t stream)
+                                                 int layout, void* workspace, cudaStream_t stream)
 {
     uint16_t* a_img = (uint16_t*)workspace;
     uint8_t* meta = (uint8_t*)workspace + sp24_meta_offset(out, in);
-    return launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, permuted, a_img, meta, stream);
+    return launch_nm_to_sp24(vals, idx, out, in, N, M, kBlockK, layout, a_img, meta, stream);
 }
 
 }  // namespace elsa

@@ -26,7 +26,7 @@
 // are token rows) and Y is row-major, so the epilogue has to turn a lane's column pair into a row's
 // feature run.  stmatrix with .trans does that in one instruction per 8 x 32 outputs if lane t of a
 // quarter holds feature 8 * (t % 4) + t / 4 of its 32; the weight image is therefore built with its
-// rows in that order (`permuted` form of nm_to_sp24), and only the bias index and the store address
+// rows in that order (SP24_PERMUTED form of nm_to_sp24), and only the bias index and the store address
 // here know about it.  Waits are bounded as in the other kernels.
 
 #include <mutex>
@@ -80,101 +80,6 @@ struct WsGroup {
     int stage_bytes;   // one pipeline stage: kStageK / 64 quarters of (largest nt / 2) rows of 128 bytes
     uint32_t* dev_status;
 };
-
-// A from tensor memory: lane = weight row, 8 columns per K step of 32 (16 kept values of 16 bits).
-// Called by the whole (converged) warp; `issue` is non-zero in the one lane that issues.  The predicate
-// lives inside the asm block so that the compiler cannot turn it into a branch around the instruction.
-__device__ __forceinline__ void umma_sp_f16_pair_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t tmem_e,
-                                                    uint32_t idesc, uint32_t accumulate, uint32_t issue)
-{
-    const uint32_t idesc_sel = idesc | (tmem_e & 1u);
-    const uint32_t e_addr = tmem_e & ~1u;
-    asm volatile(
-        "{\n"
-        ".reg .pred p, q;\n"
-        "setp.ne.b32 p, %5, 0;\n"
-        "setp.ne.b32 q, %6, 0;\n"
-        "@q tcgen05.mma.sp.cta_group::2.kind::f16 [%0], [%1], %2, [%3], %4, p;\n"
-        "}\n" ::"r"(d_tmem),
-        "r"(a_tmem), "l"(b_desc), "r"(e_addr), "r"(idesc_sel), "r"(accumulate), "r"(issue)
-        : "memory");
-}
-
-// Lane i of the warp receives 16 consecutive fp32 columns of TMEM lane (lane base + i).
-__device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr)
-        : "memory");
-}
-
-// Four 8 x 8 matrices of 16-bit values, transposed on the way to shared memory: the two halves of
-// register i of lane t go to column t / 4 of rows 2 * (t % 4) and 2 * (t % 4) + 1 of matrix i, whose
-// eight 16-byte rows are at the addresses given by lanes 8 * i .. 8 * i + 7.
-__device__ __forceinline__ void stmatrix_x4_trans(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
-{
-    asm volatile("stmatrix.sync.aligned.m8n8.x4.trans.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r0), "r"(r1),
-                 "r"(r2), "r"(r3)
-                 : "memory");
-}
-
-// Lane i of the warp writes 16 / 4 consecutive columns of TMEM lane (lane base + i).
-__device__ __forceinline__ void tmem_st_32x32b_x16(uint32_t taddr, const uint32_t (&r)[16])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
-        "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
-
-__device__ __forceinline__ void tmem_st_32x32b_x4(uint32_t taddr, const uint32_t (&r)[4])
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%0], {%1, %2, %3, %4};" ::"r"(taddr), "r"(r[0]), "r"(r[1]),
-                 "r"(r[2]), "r"(r[3])
-                 : "memory");
-}
-
-// 3-D TMA load into this CTA's shared memory, completion bytes credited to an mbarrier that may live in
-// the other CTA of the pair.
-__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0,
-                                                 int c1, int c2)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-
-// Row-major 16-bit matrix [rows][in] seen as [in / 64][rows][64]: one box of (64, box_rows, 4) is a K stage
-// of 256 as four 128-byte-swizzled quarters of box_rows rows each.
-elsa_status make_map_x_quarters(CUtensorMap* map, const void* base, uint64_t in, uint64_t rows, uint32_t box_rows)
-{
-    EncodeTiledFn fn = encode_tiled_fn();
-    if (!fn) return fail(ELSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
-    cuuint64_t dims[3] = {64, rows, in / 64};
-    cuuint64_t strides[2] = {in * 2, 128};
-    cuuint32_t box[3] = {64, box_rows, kStageK / 64};
-    cuuint32_t elem[3] = {1, 1, 1};
-    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(base), dims, strides, box, elem,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for X rejected (CUresult %d)", (int)rc);
-    return ELSA_OK;
-}
-
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
-
-// Arrival that publishes this CTA's tensor-memory writes to the MMA issuer of the leader CTA.
-__device__ __forceinline__ void mbar_arrive_cluster_release(uint32_t cluster_addr)
-{
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
-}
 
 template <bool kBf16, int kMaxLayers>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -568,7 +473,7 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         L.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.nt >> 3) << 17) |
                   ((uint32_t)(kPairFeat >> 4) << 24);
         elsa_status st;
-        if ((st = make_map_x_quarters(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, (uint32_t)(L.nt / 2))) != ELSA_OK) return st;
+        if ((st = make_map_x_quarters(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, (uint32_t)(L.nt / 2), kStageK / 64)) != ELSA_OK) return st;
         if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, 32, kStepCols, CU_TENSOR_MAP_SWIZZLE_NONE,
                               "Y")) != ELSA_OK)
             return st;
@@ -615,7 +520,7 @@ elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16
                                        const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
                                        void* workspace, uint32_t* dev_status, cudaStream_t stream)
 {
-    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, true, workspace, stream);
+    elsa_status st = launch_linear_tc_sparse_pair_prepare(vals, idx, out, in, N, M, SP24_PERMUTED, workspace, stream);
     if (st != ELSA_OK) return st;
     SparseJob job;
     job.X = X; job.bias = bias; job.Y = Y; job.workspace = workspace;

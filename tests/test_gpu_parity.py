@@ -122,7 +122,8 @@ VARIANTS = ["simt", "tc_dense", "tc_pair"]
 def variant_code(lib, name):
     return {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
             "tc_sparse": lib.VARIANT_TC_SPARSE, "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR,
-            "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS, "auto": lib.VARIANT_AUTO}[name]
+            "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS, "tc_sparse_st": lib.VARIANT_TC_SPARSE_ST,
+            "auto": lib.VARIANT_AUTO}[name]
 
 
 LINEAR_CASES = [
@@ -271,6 +272,53 @@ def test_weight_stationary_sparse_variant_exact_cases_and_refusals(lib):
         run_linear(lib, torch.eye(192, dtype=dtype), synth.randn((64, 192), 7, synth.W_STD, dtype), None, 2, 4, code)
     with pytest.raises(lib.ElsaError):                         # weight block larger than tensor memory
         run_linear(lib, torch.zeros((8, 2048), dtype=dtype), synth.randn((64, 2048), 8, synth.W_STD, dtype), None, 2, 4, code)
+
+
+ST_CASES = [
+    # rows, in, out, N, M: weight streaming through tensor memory in K chunks of 256 (in % 128 == 0, any length);
+    # ragged row tiles, a half-empty feature block, a last chunk of 128, more chunks than slots, one chunk only
+    (197, 3072, 768, 1, 8), (500, 1152, 384, 2, 4), (449, 2048, 200, 2, 16), (300, 1024, 136, 1, 16),
+    (2300, 768, 2304, 2, 8), (9000, 4096, 1024, 1, 8), (1, 128, 8, 1, 4), (40000, 256, 520, 2, 4),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float16, torch.bfloat16])
+@pytest.mark.parametrize("case", ST_CASES)
+def test_streaming_sparse_variant_matches_oracle(lib, case, dtype):
+    rows, in_, out, N, M = case
+    X = synth.randn((rows, in_), 43 * rows + in_, synth.X_STD, dtype)
+    W = synth.randn((out, in_), 47 * out + in_, synth.W_STD, dtype)
+    bias = synth.randn((out,), 53 * out, synth.B_STD, dtype)
+    Y = run_linear(lib, X, W, bias, N, M, lib.VARIANT_TC_SPARSE_ST)
+    if rows <= 4096:
+        check_close(Y, oracle_linear(X, W, bias, N, M, dtype))
+    else:                                                   # sampled rows: first, last, and a seeded spread
+        pick = torch.from_numpy(synth.sample_rows(rows, 256, 9))
+        check_close(Y.cpu()[pick], oracle_linear(X[pick], W, bias, N, M, dtype))
+
+
+def test_streaming_sparse_variant_exact_cases_and_refusals(lib):
+    code = lib.VARIANT_TC_SPARSE_ST
+    dtype = torch.float16
+    W = synth.randn((320, 1280), 15, synth.W_STD, dtype)
+    bias = synth.randn((320,), 16, synth.B_STD, dtype)
+    X = torch.eye(1280, dtype=dtype)                            # Y = masked W^T + bias, one rounding at most
+    for N, M in [(2, 8), (1, 4), (2, 4), (1, 16)]:
+        Y = run_linear(lib, X, W, bias, N, M, code)
+        expect = torch.from_numpy(oracle_linear(X, W, bias, N, M, dtype)).to(dtype)
+        assert torch.equal(Y.cpu(), expect), (N, M)
+    rng = np.random.default_rng(15)
+    Xi = torch.from_numpy(rng.integers(-4, 5, (300, 896))).to(torch.bfloat16)
+    Wi = torch.from_numpy(rng.integers(-8, 9, (96, 896))).to(torch.bfloat16)
+    for N, M in [(2, 4), (1, 8), (2, 16)]:                      # integer products: fp32 accumulation is exact
+        Y = run_linear(lib, Xi, Wi, None, N, M, code)
+        ref = oracle_linear(Xi, Wi, None, N, M, torch.bfloat16)
+        assert torch.equal(Y.cpu(), torch.from_numpy(ref).to(torch.bfloat16)), (N, M)
+    for N, M in [(4, 8), (3, 4), (8, 8)]:                      # more than 2 per chunk possible: refused
+        with pytest.raises(lib.ElsaError):
+            run_linear(lib, X, W, bias, N, M, code)
+    with pytest.raises(lib.ElsaError):                         # in is not a multiple of 128
+        run_linear(lib, torch.eye(192, dtype=dtype), synth.randn((64, 192), 17, synth.W_STD, dtype), None, 2, 4, code)
 
 
 def test_no_bias_and_zero_rows_of_padding(lib):
