@@ -10,9 +10,11 @@ stack at batch 256 in bf16 with a seeded level per layer from {1:8, 2:8, 4:8, 8:
 
 Prints ONE JSON line.  `value` is dense-equivalent TFLOP/s (2*R*K*O summed over layers / step
 time) with inputs resident in HBM; `e2e` is the same metric through elsa_vit_linears_host with
-pinned host buffers and the copies inside the timed region.  `roofline` is for the dominant
-kernel (the tcgen05 GEMM), timed per launch with CUDA events in a second timed pass; the roofline
-time of a layer is max(kept FLOPs / tensor peak, algorithmic bytes / HBM bandwidth).
+pinned host buffers and the copies inside the timed region.  `roofline` describes the dominant
+kernel family (largest share of kernel time), timed per launch with CUDA events in a second pass;
+`families` gives the same per family and `gemm_frac` over all of them; the roofline time of a
+layer is max(kept FLOPs / tensor peak, algorithmic bytes / HBM bandwidth).  `secondary` carries
+the Swin-B stack measured in the same process.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 With N > 1 (torchrun) every rank runs an independent replica; there is no collective on the path.
 """
@@ -35,14 +37,9 @@ METRIC = "sparse-GEMM dense-equivalent TFLOP/s over the ViT linear stack"
 UNIT = "TFLOP/s"
 GEMM_KERNELS = ("linear_tc_dense", "linear_tc_pair", "linear_tc_sp24", "linear_tc_sp24_pair", "linear_tc_sp24_ws", "linear_tc_sp24_st")   # forms of the tcgen05 GEMM
 
-# dram__bytes_read.sum + dram__bytes_write.sum of each GEMM kernel's launches over ONE step of this
-# benchmark, from a one-pass ncu capture of the same command (the two DRAM counters
-# fit one pass, so the full-size run is captured as it is).  Valid for the kernels as captured; set an
-# entry to None when its kernel changes.
-MEASURED_DRAM_TRAFFIC = {
-    "deit_b_stack_b256": {"linear_tc_pair": 8.773e9, "linear_tc_sp24_ws": 4.70e9, "linear_tc_sp24_pair": 3.571e9},
-    "swin_b_stack_b128": {"linear_tc_pair": 10.458e9, "linear_tc_sp24_pair": 2.485e9},
-}
+# Recorded DRAM traffic (ncu, one-pass captures) lives in profiles/dram_traffic.json: per workload and kernel
+# the bytes of one step, the command that captured them and a hash of the kernel sources at that time.
+DRAM_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "dram_traffic.json")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -198,32 +195,157 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ---------------------------------------------------------------------------------- accounting (no GPU)
+
+def kernel_source_hash():
+    """sha256 over the kernel sources and the public header, in name order: identifies the kernels a
+    recorded counter belongs to."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2409_09708_b200", "csrc")
+    files = sorted(os.path.join(csrc, f) for f in os.listdir(csrc)) + [os.path.join(ROOT, "include", "elsa.h")]
+    for path in files:
+        h.update(os.path.basename(path).encode())
+        with open(path, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic(workload, kernel, source_hash, path=DRAM_TRAFFIC_FILE):
+    """(bytes per step, note) of `kernel` in `workload` from the tracked record, or (None, reason) when there
+    is no capture or the kernel sources have changed since it was taken."""
+    try:
+        with open(path) as f:
+            rec = json.load(f)
+    except (OSError, ValueError):
+        return None, "no record (%s missing or unreadable)" % os.path.basename(path)
+    for c in rec.get("captures", []):
+        if c.get("workload") == workload and c.get("kernel") == kernel:
+            if c.get("csrc_sha256") != source_hash:
+                return None, "kernel sources changed since the capture (recorded %s..., now %s...)" % (
+                    str(c.get("csrc_sha256"))[:12], source_hash[:12])
+            return float(c["dram_bytes_per_step"]), "ncu dram__bytes_read.sum + dram__bytes_write.sum, one pass: " + c.get("command", "")
+    return None, "no capture of %s in %s" % (kernel, workload)
+
+
+def account(layers, peaks, peaks_kind, recs, recs_layer, steps, layer_steps, ms_per_step, workload,
+            source_hash=None, traffic_path=DRAM_TRAFFIC_FILE):
+    """Turns the per-launch records of the profiled passes into the numbers of the JSON line.
+
+    recs: (kernel name, layer, ms) of every launch of `steps` steps as the timed region runs them (layers of a
+    kernel family share launches); recs_layer: the same for `layer_steps` steps with one launch per layer, which
+    tells which family runs which layer.  Roofline time of a layer = max(kept FLOPs / tensor peak, algorithmic
+    bytes / HBM peak).  A family's fraction = summed roofline time of its layers / its measured time per step.
+    `roofline` describes the dominant family (largest share of kernel time) and nothing else."""
+    per_kernel = {}
+    for name, _, ms in recs:
+        k = per_kernel.setdefault(name, [0, 0.0])
+        k[0] += 1
+        k[1] += ms
+    gemm_ms = [0.0] * len(layers)
+    unpack_ms = [0.0] * len(layers)
+    layer_kernel = {}
+    for name, layer, ms in recs_layer:
+        if name in GEMM_KERNELS and layer >= 0:
+            gemm_ms[layer] += ms / layer_steps
+            layer_kernel[layer] = name
+        if name in ("nm_unpack", "nm_to_sp24", "weight_images") and layer >= 0:
+            unpack_ms[layer] += ms / layer_steps
+    kernel_total = sum(v[1] for v in per_kernel.values()) or 1.0
+    roof = [roofline_seconds(l, peaks) for l in layers]
+    roof_sus = [roofline_seconds(l, peaks, "bf16_tflops_sustained") for l in layers]
+    nominal = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}      # data-sheet figures, for context only
+    roof_nom = [roofline_seconds(l, nominal) for l in layers]
+    sum_roof = sum(r[0] for r in roof)
+    sum_gemm = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS) / steps * 1e-3
+
+    families = {}
+    for name in GEMM_KERNELS:
+        idx = [i for i in range(len(layers)) if layer_kernel.get(i) == name]
+        launches, ms = per_kernel.get(name, [0, 0.0])
+        if not idx and not launches:
+            continue
+        t = ms / steps * 1e-3
+        r = sum(roof[i][0] for i in idx)
+        by = {"tensor": sum(roof[i][0] for i in idx if roof[i][1] == "tensor"),
+              "hbm": sum(roof[i][0] for i in idx if roof[i][1] == "hbm")}
+        families[name] = {
+            "layers": len(idx), "launches_per_step": launches / steps, "ms_per_step": t * 1e3, "roofline_ms": r * 1e3,
+            "frac": r / t if t > 0 else None, "bound": "tensor" if by["tensor"] >= by["hbm"] else "hbm",
+            "kept_tflops": sum(layers[i].kept_flops for i in idx) / t / 1e12 if t > 0 else None,
+            "dense_equiv_tflops": sum(layers[i].dense_equiv_flops for i in idx) / t / 1e12 if t > 0 else None,
+            "algorithmic_gbs": sum(algorithmic_bytes(layers[i]) for i in idx) / t / 1e9 if t > 0 else None,
+            "frac_vs_sustained_peak": sum(roof_sus[i][0] for i in idx) / t if t > 0 else None,
+        }
+
+    top = max(families, key=lambda k: families[k]["ms_per_step"]) if families else None
+    roofline = None
+    if top is not None:
+        f = families[top]
+        launches, ms = per_kernel.get(top, [0, 0.0])
+        peak = peaks["bf16_tflops"] if f["bound"] == "tensor" else peaks["hbm_gbs"]
+        idx = [i for i in range(len(layers)) if layer_kernel.get(i) == top]
+        per_launch = steps / launches if launches else None      # steps per launch of this kernel
+        if source_hash is None:
+            source_hash = kernel_source_hash()
+        traffic_step, traffic_note = recorded_traffic(workload, top, source_hash, traffic_path)
+        roofline = {
+            "kernel": top, "layers": f["layers"], "bound": f["bound"],
+            "achieved": f["frac"] * peak if f["frac"] is not None else None, "peak": peak,
+            "unit": "TFLOP/s" if f["bound"] == "tensor" else "GB/s", "frac": f["frac"],
+            "launches": launches, "avg_launch_ms": ms / launches if launches else None,
+            "kept_tflops": f["kept_tflops"], "dense_equiv_tflops": f["dense_equiv_tflops"],
+            "algorithmic_gbs": f["algorithmic_gbs"], "frac_vs_sustained_peak": f["frac_vs_sustained_peak"],
+            "traffic": traffic_step * per_launch if traffic_step is not None and per_launch else None,
+            "traffic_note": traffic_note,
+            "traffic_algorithmic": sum(algorithmic_bytes(layers[i]) for i in idx) * per_launch if per_launch else None,
+            "peaks": peaks_kind,
+            "definition": "all keys describe `kernel`, the family with the largest share of kernel time: frac = summed "
+                          "roofline time of its layers (per layer max(kept FLOPs / tensor peak, algorithmic bytes / HBM "
+                          "peak)) / its CUDA-event time per step (its layers share launches); bound = the resource that "
+                          "bounds most of that roofline time; achieved = frac * peak; traffic and traffic_algorithmic "
+                          "are per launch",
+        }
+    # the step also compresses every weight: its own roofline is the bytes it must move (dense W in, packed
+    # values and index words out) at the HBM peak
+    compress_bytes = sum(l.out * l.in_ * 2 + algorithmic_bytes(l) - 2 * l.rows * (l.in_ + l.out) - l.out * 2 for l in layers)
+    compress_roof = compress_bytes / (peaks["hbm_gbs"] * 1e9)
+    share = {"tensor": sum(r[0] for r in roof if r[1] == "tensor"), "hbm": sum(r[0] for r in roof if r[1] == "hbm")}
+    out = {
+        "stack_roofline_frac": (sum_roof + compress_roof) / (ms_per_step * 1e-3),
+        "stack_roofline_ms": {"linears": sum_roof * 1e3, "compress": compress_roof * 1e3},
+        "gemm_frac": sum_roof / sum_gemm if sum_gemm > 0 else None,
+        "gemm_frac_vs_sustained_peak": sum(r[0] for r in roof_sus) / sum_gemm if sum_gemm > 0 else None,
+        "gemm_frac_vs_nominal_peaks": sum(r[0] for r in roof_nom) / sum_gemm if sum_gemm > 0 else None,
+        "roofline_time_share": {k: v / sum_roof for k, v in share.items()} if sum_roof > 0 else None,
+        "roofline": roofline,
+        "families": families,
+        "kernels": {k: {"launches": v[0], "ms": v[1], "share": v[1] / kernel_total} for k, v in per_kernel.items()},
+        "compress_gbs": (compress_bytes * steps / per_kernel["nm_compress"][1] / 1e6)
+                        if per_kernel.get("nm_compress", [0, 0.0])[1] > 0 else None,
+    }
+    rows = []
+    for i, l in enumerate(layers):
+        rows.append({"layer": l.name, "rows": l.rows, "in": l.in_, "out": l.out, "level": "%d:%d" % (l.N, l.M),
+                     "kernel": layer_kernel.get(i), "gemm_ms": gemm_ms[i], "unpack_ms": unpack_ms[i],
+                     "roofline_ms": roof[i][0] * 1e3, "bound": roof[i][1],
+                     "frac": roof[i][0] * 1e3 / gemm_ms[i] if gemm_ms[i] else None,
+                     "dense_equiv_tflops": l.dense_equiv_flops / gemm_ms[i] / 1e9 if gemm_ms[i] else None,
+                     "algorithmic_gbs": algorithmic_bytes(l) / gemm_ms[i] / 1e6 if gemm_ms[i] else None})
+    return out, rows
+
+
 # ---------------------------------------------------------------------------------- GPU arm
 
-def run_ours(args):
+def measure_stack(lib, synth, workload, steps, warmup, world, barrier, sampler=None):
+    """Builds `workload` resident in HBM, runs it `steps` times three ways (timed; with per-launch events; one
+    launch per layer) and returns what account() and the JSON line need."""
     import torch
-    rank, local_rank, world = dist_env()
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the sparse-linear path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    from paper_2409_09708_b200 import build as _build
-    if rank == 0:
-        _build.build()
-    if world > 1:
-        dist.barrier()
-    from paper_2409_09708_b200 import binding as lib, synth
-
-    layers, dtype_name = synth.workload(args.workload)
+    layers, dtype_name = synth.workload(workload)
     dtype = synth.torch_dtype(dtype_name)
     code = lib.dtype_code(dtype)
-    peaks, peaks_kind = load_peaks()
-
-    # ---- resident inputs (seeded, drawn on the device); every layer owns its X and Y
     dev = []
-    for l in layers:
+    for l in layers:       # seeded, drawn on the device; every layer owns its X and Y
         X, W, b = synth.layer_tensors(l, dtype, device="cuda")
         vals, idx = lib.alloc_packed(l.out, l.in_, l.N, l.M, dtype)
         Y = torch.empty((l.rows, l.out), dtype=dtype, device="cuda")
@@ -231,17 +353,11 @@ def run_ours(args):
     table = lib.make_layer_table(dev)
     ws = lib.alloc_workspace(lib.elsa_vit_workspace_bytes(table, code))
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-
     wtable = lib.make_weight_table(dev)
 
     def step():
         lib.elsa_vit_compress(wtable, code)
         lib.elsa_vit_linears(table, code, ws, dev_status=status)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
 
     def timed(n_steps, profile=False):
         barrier()
@@ -258,88 +374,58 @@ def run_ours(args):
         ms = max_over_ranks(e0.elapsed_time(e1), world)
         return ms, lib.elsa_launch_count() - launches0, recs
 
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         step()
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
+    if sampler is not None:
         sampler.start()
-    total_ms, launches, _ = timed(args.steps)
-    prof_ms, _, recs = timed(args.steps, profile=True)
-    # a third pass with one launch per layer, only for the per-layer report
+    total_ms, launches, _ = timed(steps)
+    prof_ms, _, recs = timed(steps, profile=True)
+    # a third pass with one launch per layer, only for the per-layer report and the layer -> family map
     lib.elsa_set_grouping(False)
-    layer_steps = max(1, args.steps // 2)
+    layer_steps = max(1, steps // 2)
     _, _, recs_layer = timed(layer_steps, profile=True)
     lib.elsa_set_grouping(True)
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop() if sampler is not None else None
     assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    return dict(layers=layers, dtype_name=dtype_name, dtype=dtype, code=code, dev=dev, ms_per_step=total_ms / steps,
+                launches=launches, recs=recs, recs_layer=recs_layer, layer_steps=layer_steps,
+                ms_per_step_profiled=prof_ms / steps, clocks=clocks)
 
-    ms_per_step = total_ms / args.steps
+
+def run_ours(args):
+    import torch
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sparse-linear path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    from paper_2409_09708_b200 import build as _build
+    if rank == 0:
+        _build.build()
+    if world > 1:
+        dist.barrier()
+    from paper_2409_09708_b200 import binding as lib, synth
+    peaks, peaks_kind = load_peaks()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    m = measure_stack(lib, synth, args.workload, args.steps, args.warmup, world, barrier,
+                      ClockSampler(local_rank) if rank == 0 else None)
+    layers, dtype_name = m["layers"], m["dtype_name"]
+    ms_per_step = m["ms_per_step"]
     dense_flops = sum(l.dense_equiv_flops for l in layers)
     kept_flops = sum(l.kept_flops for l in layers)
-    value = whole_job_tflops(dense_flops, world, ms_per_step)
-
-    # ---- per-kernel accounting from the profiled pass
-    per_kernel = {}
-    gemm_ms = [0.0] * len(layers)
-    unpack_ms = [0.0] * len(layers)
-    for name, layer, ms in recs:
-        k = per_kernel.setdefault(name, [0, 0.0])
-        k[0] += 1
-        k[1] += ms
-    layer_kernel = {}                       # which GEMM kernel runs each layer (from the one-launch-per-layer pass)
-    for name, layer, ms in recs_layer:
-        if name in GEMM_KERNELS and layer >= 0:
-            gemm_ms[layer] += ms / layer_steps
-            layer_kernel[layer] = name
-        if name in ("nm_unpack", "nm_to_sp24", "weight_images") and layer >= 0:
-            unpack_ms[layer] += ms / layer_steps
-    kernel_total = sum(v[1] for v in per_kernel.values()) or 1.0
-    roof = [roofline_seconds(l, peaks) for l in layers]
-    roof_sus = [roofline_seconds(l, peaks, "bf16_tflops_sustained") for l in layers]
-    nominal = {"hbm_gbs": 8000.0, "bf16_tflops": 2250.0}      # data-sheet figures, for context only
-    roof_nom = [roofline_seconds(l, nominal) for l in layers]
-    sum_roof = sum(r[0] for r in roof)
-    # GEMM time per step: the shared launches of the profiled pass, as the timed region runs them
-    sum_gemm = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS) / args.steps * 1e-3
-    share = {"tensor": sum(r[0] for r in roof if r[1] == "tensor"), "hbm": sum(r[0] for r in roof if r[1] == "hbm")}
-    bound = "tensor" if share["tensor"] >= share["hbm"] else "hbm"
-    frac = sum_roof / sum_gemm if sum_gemm > 0 else None
-    peak = peaks["bf16_tflops"] if bound == "tensor" else peaks["hbm_gbs"]
-    gemm_launches = sum(per_kernel.get(k, [0, 0.0])[0] for k in GEMM_KERNELS)
-    gemm_total_ms = sum(per_kernel.get(k, [0, 0.0])[1] for k in GEMM_KERNELS)
-    top_kernel = max(GEMM_KERNELS, key=lambda k: per_kernel.get(k, [0, 0.0])[1])
-    top_launches = per_kernel.get(top_kernel, [0, 0.0])[0]
-    roofline = {
-        "kernel": top_kernel, "bound": bound, "achieved": frac * peak if frac else None, "peak": peak,
-        "unit": "TFLOP/s" if bound == "tensor" else "GB/s", "frac": frac,
-        # per launch, like `achieved`: the step's bytes of `kernel` over its launches per step (layers share launches)
-        "traffic": (MEASURED_DRAM_TRAFFIC[args.workload][top_kernel] * args.steps / top_launches
-                    if top_launches and top_kernel in MEASURED_DRAM_TRAFFIC.get(args.workload, {}) else None),
-        "traffic_note": "DRAM bytes (read + written) per launch of `kernel`, whose launches carry all of its layers "
-                        "(ncu, one pass, same command); traffic_algorithmic is the same layers' algorithmic bytes per launch",
-        "traffic_algorithmic": (sum(algorithmic_bytes(l) for i, l in enumerate(layers) if layer_kernel.get(i) == top_kernel)
-                                * args.steps / top_launches if top_launches else None),
-        "peaks": peaks_kind,
-        "definition": "per layer max(kept FLOPs / tensor peak, algorithmic bytes / HBM peak), summed over the "
-                      "layers, divided by the summed CUDA-event durations of the GEMM launches that ran them "
-                      "(layers of a kernel family share launches); achieved = frac * peak of the resource that "
-                      "bounds most of the summed roofline time",
-        "kept_tflops": kept_flops / sum_gemm / 1e12 if sum_gemm else None,
-        "algorithmic_gbs": sum(algorithmic_bytes(l) for l in layers) / sum_gemm / 1e9 if sum_gemm else None,
-        "frac_vs_sustained_peak": sum(r[0] for r in roof_sus) / sum_gemm if sum_gemm else None,
-        "frac_vs_nominal_peaks": sum(r[0] for r in roof_nom) / sum_gemm if sum_gemm else None,
-        "launches": gemm_launches,
-        "avg_launch_ms": gemm_total_ms / max(gemm_launches, 1),
-        "roofline_time_share": {k: v / sum_roof for k, v in share.items()},
-    }
-    # the step also compresses every weight: its own roofline is the bytes it must move (dense W in, packed
-    # values and index words out) at the HBM peak
-    compress_bytes = sum(l.out * l.in_ * 2 + algorithmic_bytes(l) - 2 * l.rows * (l.in_ + l.out) - l.out * 2 for l in layers)
-    compress_roof = compress_bytes / (peaks["hbm_gbs"] * 1e9)
-    stack_frac = (sum_roof + compress_roof) / (ms_per_step * 1e-3)
+    acc, rows = account(layers, peaks, peaks_kind, m["recs"], m["recs_layer"], args.steps, m["layer_steps"], ms_per_step,
+                        args.workload)
 
     line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "metric": METRIC, "value": whole_job_tflops(dense_flops, world, ms_per_step), "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": dtype_name, "data": "synthetic",
         "config": {"workload": args.workload, "layers": len(layers), "rows": layers[0].rows,
@@ -350,26 +436,13 @@ def run_ours(args):
                            "launches)", "multi_gpu": "independent replicas"},
         "actual_tflops": world * kept_flops / (ms_per_step * 1e-3) / 1e12,
         "ms_per_stack": ms_per_step,
-        "stack_roofline_frac": stack_frac,
-        "stack_roofline_ms": {"linears": sum_roof * 1e3, "compress": compress_roof * 1e3},
-        "gpu_launches": launches,
-        "roofline": roofline,
-        "kernels": {k: {"launches": v[0], "ms": v[1], "share": v[1] / kernel_total} for k, v in per_kernel.items()},
-        "ms_per_step_profiled": prof_ms / args.steps,
-        "compress_gbs": (compress_bytes * args.steps / per_kernel["nm_compress"][1] / 1e6)
-                        if per_kernel.get("nm_compress", [0, 0.0])[1] > 0 else None,
-        "clocks": clocks,
+        "gpu_launches": m["launches"],
+        "ms_per_step_profiled": m["ms_per_step_profiled"],
+        "clocks": m["clocks"],
     }
+    line.update(acc)
 
-    # ---- per-layer report (scratch output; the committed summary is made from it)
-    if rank == 0:
-        rows = []
-        for i, l in enumerate(layers):
-            rows.append({"layer": l.name, "rows": l.rows, "in": l.in_, "out": l.out, "level": "%d:%d" % (l.N, l.M),
-                         "gemm_ms": gemm_ms[i], "unpack_ms": unpack_ms[i], "roofline_ms": roof[i][0] * 1e3,
-                         "bound": roof[i][1], "frac": roof[i][0] * 1e3 / gemm_ms[i] if gemm_ms[i] else None,
-                         "dense_equiv_tflops": l.dense_equiv_flops / gemm_ms[i] / 1e9 if gemm_ms[i] else None,
-                         "algorithmic_gbs": algorithmic_bytes(l) / gemm_ms[i] / 1e6 if gemm_ms[i] else None})
+    if rank == 0:       # per-layer report (scratch output; the committed summary is made from it)
         try:
             os.makedirs(os.path.join(ROOT, "bench_out"), exist_ok=True)
             with open(os.path.join(ROOT, "bench_out", "bench_layers_%s.json" % args.workload), "w") as f:
@@ -379,7 +452,7 @@ def run_ours(args):
 
     # ---- end to end from pinned host memory through elsa_vit_linears_host
     if not args.no_e2e:
-        line["e2e"] = run_e2e(args, lib, synth, layers, dtype, code, dev, world, barrier)
+        line["e2e"] = run_e2e(args, lib, synth, layers, m["dtype"], m["code"], m["dev"], world, barrier)
     # ---- the oracle on the host cores, rank 0 at N = 1 only
     if world == 1 and not args.no_cpu_baseline:
         from oracle import elsa_oracle as eo
@@ -387,6 +460,29 @@ def run_ours(args):
         line["cpu_baseline"] = {"value": flops / sec / 1e12, "unit": UNIT, "cores": eo.omp_threads(), "kind": "oracle",
                                 "sample": "%d seeded rows of each of the %d layers, weights compressed in full, "
                                           "%.1f s" % (args.oracle_rows, len(layers), sec)}
+    # ---- the other stack the target is read on, measured in the same process (device timing only)
+    if args.secondary and args.secondary != args.workload and world == 1:
+        del m
+        torch.cuda.empty_cache()
+        sec_steps = max(3, args.steps // 2)
+        m2 = measure_stack(lib, synth, args.secondary, sec_steps, args.warmup, world, barrier)
+        acc2, rows2 = account(m2["layers"], peaks, peaks_kind, m2["recs"], m2["recs_layer"], sec_steps, m2["layer_steps"],
+                              m2["ms_per_step"], args.secondary)
+        l2 = m2["layers"]
+        line["secondary"] = {
+            "workload": args.secondary, "layers": len(l2), "steps": sec_steps, "dtype": m2["dtype_name"],
+            "ms_per_stack": m2["ms_per_step"],
+            "value": whole_job_tflops(sum(l.dense_equiv_flops for l in l2), world, m2["ms_per_step"]), "unit": UNIT,
+            "actual_tflops": sum(l.kept_flops for l in l2) / (m2["ms_per_step"] * 1e-3) / 1e12,
+            "stack_roofline_frac": acc2["stack_roofline_frac"], "stack_roofline_ms": acc2["stack_roofline_ms"],
+            "gemm_frac": acc2["gemm_frac"], "families": acc2["families"], "compress_gbs": acc2["compress_gbs"],
+            "gpu_launches": m2["launches"],
+        }
+        try:
+            with open(os.path.join(ROOT, "bench_out", "bench_layers_%s.json" % args.secondary), "w") as f:
+                json.dump(rows2, f, indent=1)
+        except OSError:
+            pass
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -395,7 +491,8 @@ def run_ours(args):
 
 def run_e2e(args, lib, synth, layers, dtype, code, dev, world, barrier):
     """Same metric through the host-memory entry point: per layer H2D of W, bias and X from pinned
-    memory, compress, linear, D2H of Y.  Layers of equal shape share pinned host buffers."""
+    memory, compress, linear, D2H of Y.  Layers of equal shape share pinned host buffers.  Every step is
+    timed on its own; the value is quoted on the median."""
     import torch
     host_x, host_y = {}, {}
     host = []
@@ -412,20 +509,23 @@ def run_e2e(args, lib, synth, layers, dtype, code, dev, world, barrier):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     h2d = sum(l.rows * l.in_ * 2 + l.out * l.in_ * 2 + l.out * 2 for l in layers)
     d2h = sum(l.rows * l.out * 2 for l in layers)
-    steps = max(1, min(args.steps, args.e2e_steps))
+    steps = max(1, args.e2e_steps)
     lib.elsa_vit_linears_host(table, code, mem, dev_status=status)       # warm-up
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
+    times = []
     for _ in range(steps):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
         lib.elsa_vit_linears_host(table, code, mem, dev_status=status)
-    e1.record()
-    barrier()
-    ms = max_over_ranks(e0.elapsed_time(e1) / steps, world)
+        e1.record()
+        barrier()
+        times.append(max_over_ranks(e0.elapsed_time(e1), world))
     assert int(status.item()) == 0
+    ms = statistics.median(times)
     dense_flops = sum(l.dense_equiv_flops for l in layers)
     return {"value": whole_job_tflops(dense_flops, world, ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "steps": steps,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms, "ms_per_step_min": min(times), "ms_per_step_max": max(times),
+            "steps": steps, "quoted_on": "median of the steps, each timed on its own",
             "api": "elsa_vit_linears_host (pinned host buffers; layers of equal shape share them)"}
 
 
@@ -439,7 +539,9 @@ def main():
                     choices=["single_layer", "deit_b_block_b64", "deit_b_stack_b256", "swin_b_stack_b128"])
     ap.add_argument("--oracle-rows", type=int, default=None,
                     help="rows per layer of the CPU-oracle sample (default 4096 for cpu_baseline, 1024 per step of --impl reference)")
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--secondary", default="swin_b_stack_b128",
+                    help="second workload measured in the same process and reported under `secondary` ('' for none)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -286,6 +286,16 @@ int elsa_profile_stop(elsa_kernel_time* records, int capacity);
 /* Number of kernels the library has launched from this process so far. */
 unsigned long long elsa_launch_count(void);
 
+/*
+ * Test hook for the device-side failure path.  Every wait of the tensor-core kernels is bounded: a wait that
+ * runs out records ELSA_ERR_TIMEOUT | site << 8 in dev_status and the kernel winds down instead of hanging.
+ * This call launches one warp that runs that same wait on a barrier nobody arrives at, with `limit_ns`
+ * (1 ns .. 100 ms) in place of the kernels' two seconds; after synchronising, *dev_status holds
+ * ELSA_ERR_TIMEOUT | 15 << 8 (if it was 0 before) and the device is usable as before.  dev_status: device
+ * pointer, required.  Asynchronous on `stream`.  The paper has no counterpart; it exists for the tests.
+ */
+elsa_status elsa_selftest_wait_timeout(unsigned long long limit_ns, uint32_t* dev_status, void* stream);
+
 /* Message describing the calling thread's last non-OK status ("" if none). */
 const char* elsa_last_error(void);
 

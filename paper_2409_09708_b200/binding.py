@@ -79,6 +79,7 @@ _set_grouping = _sig("elsa_set_grouping", None, [_i])
 _get_variant = _sig("elsa_get_linear_variant", _i, [])
 _launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
 _last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
+_selftest_wait = _sig("elsa_selftest_wait_timeout", _i, [ctypes.c_ulonglong, _vp, _vp])
 
 
 class ElsaKernelTime(ctypes.Structure):
@@ -104,6 +105,11 @@ def _check(status: int):
 
 def elsa_last_error() -> str:
     return (_last_error() or b"").decode()
+
+
+def elsa_selftest_wait_timeout(limit_ns: int, dev_status: torch.Tensor, stream=None):
+    """Launches the bounded wait of the tensor-core kernels on a barrier nobody arrives at (test hook)."""
+    _check(_selftest_wait(int(limit_ns), _ptr(dev_status), _stream(stream)))
 
 
 def elsa_launch_count() -> int:

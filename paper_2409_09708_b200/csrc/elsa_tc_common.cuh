@@ -59,9 +59,10 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
-// Bounded wait.  Returns false if this wait, or any other wait of the CTA, has given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          uint32_t* dev_status, uint32_t site)
+// Bounded wait.  Returns false if this wait, or any other wait of the CTA, has given up: after `limit_ns`
+// the waiter sets the CTA's abort flag and records ELSA_ERR_TIMEOUT | site << 8 in `dev_status`.
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                uint32_t* dev_status, uint32_t site, unsigned long long limit_ns)
 {
     uint32_t spins = 0;
     unsigned long long t0 = 0;
@@ -71,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             const unsigned long long now = global_timer_ns();
             if (t0 == 0) {
                 t0 = now;
-            } else if (now - t0 > kWaitTimeoutNs) {
+            } else if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 if (dev_status) atomicCAS(dev_status, 0u, (uint32_t)ELSA_ERR_TIMEOUT | (site << 8));
                 return false;
@@ -79,6 +80,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         }
     }
     return true;
+}
+
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t* dev_status, uint32_t site)
+{
+    return mbar_wait_limit(bar, parity, abort_flag, dev_status, site, kWaitTimeoutNs);
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,

@@ -64,8 +64,19 @@ def test_compress_and_unpack_match_oracle_bit_for_bit(lib, shape, dtype):
     Wb = synth.bits(W).copy()
     Wb[0, :8] = [0x8000, 0, 0x8000, 0, 0, 0, 0, 0x8000]           # signed zeros
     Wb[1, :16] = Wb[1, 0]                                           # an all-equal stretch
-    W = synth.from_bits(Wb, dtype)
-    Wd = W.cuda()
+    # patterns outside the contract of the linear, inside that of compress / unpack (compare domain: the 15
+    # magnitude bits as an integer, so NaN > Inf > finite and a subnormal is just a small magnitude): infinities of
+    # both signs, quiet and signalling NaNs with different payloads, the largest finite value, subnormals, and
+    # ties among them
+    inf = 0x7C00 if dtype == torch.float16 else 0x7F80
+    sub = [0x0001, 0x8001, 0x03FF, 0x0200] if dtype == torch.float16 else [0x0001, 0x8001, 0x007F, 0x0040]
+    special = [inf, inf | 0x8000, inf + 1, (inf + 1) | 0x8000, 0x7FFF, 0xFFFF, inf - 1, (inf - 1) | 0x8000] + sub + [inf, 0, inf | 0x8000, sub[0]]
+    Wb[2, :16] = special
+    Wb[3, :16] = special[::-1]
+    rng = np.random.default_rng(out * 7 + in_)
+    where = rng.choice(out * in_, size=max(8, out * in_ // 64), replace=False)      # and scattered through the matrix
+    Wb.reshape(-1)[where] = rng.choice(np.asarray(special, dtype=Wb.dtype), size=where.size)
+    Wd = synth.from_bits(Wb, dtype).cuda()                           # exact bit patterns, no conversion
     for N, M in LEVELS:
         if in_ % M:
             continue
@@ -344,7 +355,10 @@ def test_single_layer_config(lib):
         check_close(run_linear(lib, X, W, b, layer.N, layer.M, variant_code(lib, v)), ref)
 
 
-def stack_check(lib, layers, dtype, rows_sampled, seed):
+ROW_TILE_HEIGHTS = (144, 224, 256)    # weight-stationary, streaming / sparse pair, dense pair kernels
+
+
+def stack_check(lib, layers, dtype, rows_sampled, seed, every_tile=False):
     """Run a table through elsa_vit_compress + elsa_vit_linears and check the packed weights in full and
     sampled rows of every layer against the oracle."""
     code = lib.dtype_code(dtype)
@@ -363,6 +377,13 @@ def stack_check(lib, layers, dtype, rows_sampled, seed):
     assert int(status.item()) == 0
     for i, (l, d) in enumerate(zip(layers, dev)):
         pick = synth.sample_rows(l.rows, rows_sampled, seed + i)
+        if every_tile:
+            # one seeded row inside every row tile, for each tile height the kernels use: a persistent launch
+            # walks one tile sequence over many layers, and a wrong tile anywhere in it must show
+            rng = np.random.default_rng(seed + 1000 + i)
+            extra = [np.minimum(np.arange(0, l.rows, t) + rng.integers(0, t, size=-(-l.rows // t)), l.rows - 1)
+                     for t in ROW_TILE_HEIGHTS]
+            pick = np.unique(np.concatenate([pick] + extra))
         sel = torch.from_numpy(pick).cuda()
         Xs = d["X"][sel].cpu()
         ovals, oidx, _ = eo.nm_compress(synth.bits(d["W"]), l.N, l.M)
@@ -385,12 +406,27 @@ def test_deit_b_stack_full_size_sampled_rows(lib):
     layers, dt = synth.workload("deit_b_stack_b256")
     dtype = synth.torch_dtype(dt)
     # run the whole table in one call, a few layers' worth of memory at a time is not needed: 15 GB fits
-    stack_check(lib, layers, dtype, 24, 31)
+    stack_check(lib, layers, dtype, 24, 31, every_tile=True)
 
 
 def test_swin_b_stack_full_size_sampled_rows(lib):
     layers, dt = synth.workload("swin_b_stack_b128")
-    stack_check(lib, layers, synth.torch_dtype(dt), 24, 41)
+    stack_check(lib, layers, synth.torch_dtype(dt), 24, 41, every_tile=True)
+
+
+def test_streaming_layers_share_one_launch(lib):
+    """A table whose layers all take the streaming sparse kernel under the automatic rule (N <= 2, in > 768,
+    in % 128 == 0): reductions of 4, 4.5, 8 and 12 chunks, a last feature block of only 8 features, ragged row
+    tiles; one launch carries them all, its tiles forming one sequence."""
+    dtype = torch.bfloat16
+    layers = [synth.Layer("a", 6000, 1024, 1280, 1, 8, 601, 602, 603),
+              synth.Layer("b", 5001, 1152, 1024, 2, 8, 611, 612, 613),
+              synth.Layer("c", 4100, 2048, 2312, 2, 4, 621, 622, 623),
+              synth.Layer("d", 7777, 3072, 768, 1, 16, 631, 632, 633)]
+    lib.elsa_profile_start()
+    stack_check(lib, layers, dtype, 96, 61, every_tile=True)
+    recs = lib.elsa_profile_stop()
+    assert [k for (k, _, _) in recs if k.startswith("linear")] == ["linear_tc_sp24_st"], recs
 
 
 def test_weight_stationary_layers_share_one_launch(lib):
@@ -545,3 +581,31 @@ def test_mask_on_load_linear_matches_oracle_and_packed_path(lib, case, dtype):
     assert torch.equal(Y, Y_packed)                      # same projection, same kernels
     pick = torch.from_numpy(synth.sample_rows(rows, 48, 5)).cuda()
     check_close(Y[pick], oracle_linear(X[pick].cpu(), W.cpu(), bias.cpu(), N, M, dtype))
+
+
+def test_a_wait_that_runs_out_reports_and_leaves_the_device_usable(lib):
+    """The failure path every tensor-core kernel shares: a bounded wait on a barrier nobody arrives at gives up
+    after its limit (here one millisecond), records ELSA_ERR_TIMEOUT with the site of the wait, and the kernel
+    returns.  Nothing faults and nothing hangs: the next ordinary call runs and is correct."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    lib.elsa_selftest_wait_timeout(1_000_000, status)
+    t1.record()
+    torch.cuda.synchronize()
+    code = int(status.item())
+    assert code & 0xFF == 8 and (code >> 8) == 15, "device status %#x" % code      # ELSA_ERR_TIMEOUT | site << 8
+    assert 0.9 <= t0.elapsed_time(t1) < 100.0                                       # the limit, not the kernels' 2 s
+    # a status that is already set is kept (first failure wins)
+    lib.elsa_selftest_wait_timeout(200_000, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == code
+    with pytest.raises(lib.ElsaError):
+        lib.elsa_selftest_wait_timeout(0, status)
+    # the device is as usable as before
+    dtype = torch.bfloat16
+    X = synth.randn((300, 768), 71, synth.X_STD, dtype)
+    W = synth.randn((256, 768), 72, synth.W_STD, dtype)
+    bias = synth.randn((256,), 73, synth.B_STD, dtype)
+    Y = run_linear(lib, X, W, bias, 2, 8, lib.VARIANT_AUTO)
+    check_close(Y, oracle_linear(X, W, bias, 2, 8, dtype))

@@ -1,12 +1,13 @@
-"""The allocation-free entry point, elsa_nm_linear_static, against elsa_nm_linear.
+"""The allocation-free entry point, elsa_nm_linear_static, against elsa_nm_linear and the CPU oracle.
 
 Some users of the library call it from places where device memory cannot be allocated (a
 runtime plugin's enqueue hook, a process whose framework already owns all of the GPU's memory, a
 loop that must not stall on an allocation).  For them the library keeps the scratch it needs in
 a fixed built-in array.  This file checks, through the C ABI, that the variant returns what the
 ordinary call returns -- on two calls in a row that share the array, the second with a different
-and smaller weight so that leftovers of the first would show -- and that a weight too large for
-the array is refused with a clear message instead of being run.
+and smaller weight so that leftovers of the first would show --, that both agree with the fp64
+oracle within the parity tolerances, and that a weight too large for the array is refused with a
+clear message instead of being run.
 
 It is collected last on purpose: a run that stops at the first failure has then already run
 every other test.
@@ -15,6 +16,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import elsa_oracle as eo
 from paper_2409_09708_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -32,14 +34,28 @@ def lib():
 
 
 def both_ways(lib, layer, dtype):
+    """Y of the allocation-free call, Y of elsa_nm_linear forced onto the kernel the allocation-free call
+    always uses (so that bit-equality does not hang on the dispatch rule), and the oracle on sampled rows."""
     X, W, b = synth.layer_tensors(layer, dtype, device="cuda")
     vals, idx = lib.elsa_nm_compress(W, layer.N, layer.M)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    Y_ref = lib.elsa_nm_linear(X, vals, idx, b, layer.out, layer.in_, layer.N, layer.M, dev_status=status)
+    lib.elsa_set_linear_variant(lib.VARIANT_TC_DENSE)
+    try:
+        Y_ref = lib.elsa_nm_linear(X, vals, idx, b, layer.out, layer.in_, layer.N, layer.M, dev_status=status)
+    finally:
+        lib.elsa_set_linear_variant(lib.VARIANT_AUTO)
     Y = torch.full((layer.rows, layer.out), float("nan"), dtype=dtype, device="cuda")   # caller-owned output
     lib.elsa_nm_linear_static(X, vals, idx, b, layer.out, layer.in_, layer.N, layer.M, Y, dev_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    pick = synth.sample_rows(layer.rows, 64, layer.seed_x)
+    code = eo.F16 if dtype == torch.float16 else eo.BF16
+    ovals, oidx, _ = eo.nm_compress(synth.bits(W), layer.N, layer.M)
+    ref = eo.nm_linear_f64(synth.bits(X.cpu()[torch.from_numpy(pick)]), ovals, oidx, synth.bits(b), layer.out, layer.in_,
+                           layer.N, layer.M, code)
+    got = Y.cpu()[torch.from_numpy(pick)].to(torch.float64).numpy()
+    assert np.linalg.norm(got - ref) <= REL_FRO_TOL * np.linalg.norm(ref), layer.name
+    assert np.max(np.abs(got - ref) / (np.abs(ref) + 1.0)) <= ELEM_TOL, layer.name
     return Y, Y_ref
 
 
