@@ -136,6 +136,33 @@ elsa_status check_linear(const void* X, int rows, const void* vals, const uint32
     return ELSA_OK;
 }
 
+// Side stream of elsa_vit_linears (weight images beside the dense layers), created once per device.
+struct SidePipe {
+    cudaStream_t stream;
+    cudaEvent_t fork, join;
+    bool ready;
+};
+SidePipe g_side[64];
+std::mutex g_side_mutex;
+
+elsa_status side_pipe(int device, SidePipe** pipe)
+{
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    SidePipe& p = g_side[device & 63];
+    if (!p.ready) {
+        const bool ok = cudaStreamCreateWithFlags(&p.stream, cudaStreamNonBlocking) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&p.fork, cudaEventDisableTiming) == cudaSuccess &&
+                        cudaEventCreateWithFlags(&p.join, cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "creating the image stream: %s", cudaGetErrorString(e));
+        }
+        p.ready = true;
+    }
+    *pipe = &p;
+    return ELSA_OK;
+}
+
 enum LinearKind { KIND_SIMT, KIND_DENSE_ONE, KIND_DENSE_PAIR, KIND_SPARSE_ONE, KIND_SPARSE_PAIR, KIND_SPARSE_WS, KIND_SPARSE_ST };
 
 // Form of the 2-of-4 weight image each sparse kernel reads.
@@ -172,14 +199,14 @@ elsa_status pick_kind(int rows, int out, int in, int N, int M, int sm_count, Lin
         return ELSA_OK;
     default: break;
     }
-    // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels once K is
-    // long enough for the mainloop to outweigh its heavier epilogue (K >= 768) and there are enough 256 x 224
-    // tiles to fill the CTA pairs; shorter K ties or loses and stays on the dense-rate path.
-    if (sparse_ok && in >= 768 && (long long)((rows + 223) / 224) * ((out + 255) / 256) >= sm_count / 4) {
+    // Levels with N <= 2 fit the 2:4 sparse MMA.  Measured on B200 it beats the dense-rate kernels from K = 256
+    // up once there are enough tiles to fill the CTA pairs; K = 128 layers are pure streaming problems and
+    // stay on the dense-rate path.
+    if (sparse_ok && in >= 256 && (long long)((rows + 223) / 224) * ((out + 255) / 256) >= sm_count / 4) {
         // With the weight block resident in tensor memory the activations are the only shared-memory
-        // traffic; measured faster than streaming the weight for K around 768 once a layer has at least
-        // four blocks of 256 features (qkv, fc1: 10-15 %), equal or slower elsewhere.
-        const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in <= 896 && out >= 1024 &&
+        // traffic: every layer whose reduction fits (in <= 896) and that has at least two blocks of 256
+        // features goes there.
+        const bool ws = linear_tc_sparse_ws_suits(in, out, N, sm_count) && in <= 896 && out >= 512 &&
                         rows >= 256 * (sm_count / 2) / ((out + 255) / 256);
         // Longer reductions do not fit tensor memory whole: the weight streams through it chunk by chunk, which
         // still keeps it out of shared memory (measured against staging it there for every row tile).
@@ -470,6 +497,11 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
         return ELSA_OK;
     }
 
+    // The weight images are built on a side stream while the dense layers, which need none, already run on
+    // the caller's: the image kernel is a small streaming kernel whose blocks fit beside the persistent GEMM's
+    // one CTA per SM.  Everything else waits for the images.
+    SidePipe* side = nullptr;
+    if ((st = side_pipe(dev.device, &side)) != ELSA_OK) return st;
     std::vector<LinearKind> kind(n_layers);
     std::vector<uint8_t*> region(n_layers);
     size_t off = 0;
@@ -479,6 +511,35 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
         region[l] = (uint8_t*)workspace + off;
         off += round_up(elsa_workspace_bytes(c.rows, c.in, c.out, c.N, c.M, dtype), 256);
     }
+    // dense-rate layers that multiply the stored values as they are (N = M), on CTA pairs, in groups: launched
+    // first, the weight images are built beside them
+    bool forked = false;
+    {
+        std::vector<PairJob> jobs;
+        for (int l = 0; l <= n_layers; ++l) {
+            if (l < n_layers && kind[l] == KIND_DENSE_PAIR && cfg[l].N == cfg[l].M) {
+                const elsa_layer& c = cfg[l];
+                PairJob j;
+                j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
+                j.Wd = (const uint16_t*)c.vals;
+                j.rows = c.rows; j.in = c.in; j.out = c.out;
+                jobs.push_back(j);
+            }
+            if (!jobs.empty() && (l == n_layers || (int)jobs.size() == linear_tc_pair_group_max())) {
+                if (!forked) {
+                    // the side stream starts where the caller's stream stands now (after the compress kernels)
+                    cudaError_t e = cudaEventRecord(side->fork, stream);
+                    if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+                    if (e != cudaSuccess) { cudaGetLastError(); return fail(ELSA_ERR_CUDA, "forking the image stream: %s", cudaGetErrorString(e)); }
+                    forked = true;
+                }
+                if ((st = launch_linear_tc_pair_group(jobs.data(), (int)jobs.size(), dtype, dev_status, stream)) != ELSA_OK)
+                    return st;
+                jobs.clear();
+            }
+        }
+    }
+    cudaStream_t image_stream = forked ? side->stream : stream;
     // weight images of all layers, one launch per 256 layers
     {
         static BatchTable table;          // host staging of the kernel parameters
@@ -498,11 +559,16 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
                 }
             }
             if (table.n == kBatchMax || (l == n_layers - 1 && table.n > 0)) {
-                if ((st = launch_image_batch(table, stream)) != ELSA_OK) return st;
+                if ((st = launch_image_batch(table, image_stream)) != ELSA_OK) return st;
                 table.n = 0;
                 table.total_units = 0;
             }
         }
+    }
+    if (forked) {
+        cudaError_t e = cudaEventRecord(side->join, side->stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join, 0);
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(ELSA_ERR_CUDA, "joining the image stream: %s", cudaGetErrorString(e)); }
     }
     // sparse-rate layers, in groups
     {
@@ -558,11 +624,11 @@ elsa_status elsa_vit_linears(const elsa_layer* cfg, int n_layers, elsa_dtype dty
             }
         }
     }
-    // dense-rate layers on CTA pairs, in groups
+    // dense-rate layers that read a weight image (N < M), on CTA pairs, in groups
     {
         std::vector<PairJob> jobs;
         for (int l = 0; l <= n_layers; ++l) {
-            if (l < n_layers && kind[l] == KIND_DENSE_PAIR) {
+            if (l < n_layers && kind[l] == KIND_DENSE_PAIR && cfg[l].N != cfg[l].M) {
                 const elsa_layer& c = cfg[l];
                 PairJob j;
                 j.X = (const uint16_t*)c.X; j.bias = (const uint16_t*)c.bias; j.Y = (uint16_t*)c.Y;
