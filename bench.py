@@ -337,11 +337,37 @@ def account(layers, peaks, peaks_kind, recs, recs_layer, steps, layer_steps, ms_
 
 # ---------------------------------------------------------------------------------- GPU arm
 
-def measure_stack(lib, synth, workload, steps, warmup, world, barrier, sampler=None):
+def sampled_levels(lib, layers, gmacs_per_image, seed=0):
+    """Levels of an N:4 configuration {1:4, 2:4, 4:4} drawn by the library's two-step sampler (Alg. 3) from the
+    cost interval that holds `gmacs_per_image` (whole-model multiply-accumulates per image, as Table 1 counts
+    them): a level table distributed like the paper's searched models instead of the uniform draw."""
+    import numpy as np
+    tokens = 197
+    shapes = [(tokens, l.in_, l.out) for l in layers]
+    levels = [(1, 4), (2, 4), (4, 4)]
+    fixed = 2 * tokens * tokens * 768 * 12 + 196 * 768 * 768 + 768 * 1000     # attention products, patch embedding, head
+    cost = lib.elsa_cost_table_macs(shapes, levels)
+    dense = lib.elsa_config_cost(cost, [2] * len(layers), fixed)
+    lower = lib.elsa_config_cost(cost, [0] * len(layers), fixed)
+    n_int = 16
+    width = (0.5 * dense - lower) / n_int
+    idx = min(n_int - 1, max(0, int((gmacs_per_image * 1e9 - lower) / width)))
+    u = [(idx + 0.5) / n_int] + [float(v) for v in np.random.default_rng(seed).random(len(layers))]
+    choice, _ = lib.elsa_two_step_sample(cost, [[1.0, 1.0, 1.0]] * len(layers), fixed, 0.5 * dense, n_int,
+                                         tokens * 768 * 768 / 4.0, u)
+    return [levels[c] for c in choice], lib.elsa_config_cost(cost, choice, fixed) / 1e9
+
+
+def measure_stack(lib, synth, workload, steps, warmup, world, barrier, sampler=None, sampled_gmacs=None):
     """Builds `workload` resident in HBM, runs it `steps` times three ways (timed; with per-launch events; one
     launch per layer) and returns what account() and the JSON line need."""
     import torch
     layers, dtype_name = synth.workload(workload)
+    config_gmacs = None
+    if sampled_gmacs:
+        picked, config_gmacs = sampled_levels(lib, layers, sampled_gmacs)
+        import dataclasses
+        layers = [dataclasses.replace(l, N=n, M=m) for l, (n, m) in zip(layers, picked)]
     dtype = synth.torch_dtype(dtype_name)
     code = lib.dtype_code(dtype)
     dev = []
@@ -389,7 +415,7 @@ def measure_stack(lib, synth, workload, steps, warmup, world, barrier, sampler=N
     assert int(status.item()) == 0, "device status %#x" % int(status.item())
     return dict(layers=layers, dtype_name=dtype_name, dtype=dtype, code=code, dev=dev, ms_per_step=total_ms / steps,
                 launches=launches, recs=recs, recs_layer=recs_layer, layer_steps=layer_steps,
-                ms_per_step_profiled=prof_ms / steps, clocks=clocks)
+                ms_per_step_profiled=prof_ms / steps, clocks=clocks, config_gmacs=config_gmacs)
 
 
 def run_ours(args):
@@ -415,7 +441,7 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     m = measure_stack(lib, synth, args.workload, args.steps, args.warmup, world, barrier,
-                      ClockSampler(local_rank) if rank == 0 else None)
+                      ClockSampler(local_rank) if rank == 0 else None, sampled_gmacs=args.sampled_gmacs)
     layers, dtype_name = m["layers"], m["dtype_name"]
     ms_per_step = m["ms_per_step"]
     dense_flops = sum(l.dense_equiv_flops for l in layers)
@@ -441,6 +467,9 @@ def run_ours(args):
         "clocks": m["clocks"],
     }
     line.update(acc)
+    if m["config_gmacs"] is not None:
+        line["config"]["levels_from"] = ("two-step sampler (Alg. 3) over {1:4, 2:4, 4:4} at %.2f GMACs per image "
+                                         "(requested %.2f)" % (m["config_gmacs"], args.sampled_gmacs))
 
     if rank == 0:       # per-layer report (scratch output; the committed summary is made from it)
         try:
@@ -542,6 +571,9 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--secondary", default="swin_b_stack_b128",
                     help="second workload measured in the same process and reported under `secondary` ('' for none)")
+    ap.add_argument("--sampled-gmacs", type=float, default=None,
+                    help="replace the DeiT-B stack's levels by an N:4 configuration drawn by the two-step sampler at this many "
+                         "whole-model GMACs per image (Table 1: 7.0 and 6.0 for ELSA-DeiT-B-N:4)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -286,6 +286,53 @@ int elsa_profile_stop(elsa_kernel_time* records, int capacity);
 /* Number of kernels the library has launched from this process so far. */
 unsigned long long elsa_launch_count(void);
 
+/* ------------------------------------------------------------------------------------------------
+ * Search-side host code (no GPU): cost model, two-step sampling, enumeration of configurations.
+ *
+ * Paper: Sec. 3 defines a configuration alpha = (s^1 .. s^L), one level s^l of the level set S per linear
+ * module (L = 4B: qkv, proj, fc1, fc2 of every block).  Sec. 3.2 and the appendix's settings define the cost
+ * F(alpha) as FLOPs (Table 1's figures are multiply-accumulates: only the linear modules scale with N/M, the
+ * rest of the network stays dense) and the budget C_upper as 50 % of the dense model's.  Alg. 3 (two-step
+ * sampling): cut [C_lower, C_upper] into intervals, draw one uniformly, then draw a configuration whose cost
+ * lies in it from the per-layer level probabilities P_t.  Sec. 2 counts the space: 3 levels over 48 modules
+ * give 3^48 configurations.
+ *
+ * All arrays are HOST memory owned by the caller.  A cost table is cost[l * n_levels + s] = cost of layer l at
+ * level s, in any unit (multiply-accumulates from elsa_cost_table_macs, or measured microseconds); P has the
+ * same shape (non-negative weights, normalised per layer by the callee); a configuration is choice[l] = index
+ * into the level set.  Nothing here is asynchronous.
+ */
+typedef struct { int rows, in, out; } elsa_linear_shape; /* rows = tokens the module processes */
+typedef struct { int N, M; } elsa_level;
+
+/* cost[l][s] = rows * in * out * N_s / M_s multiply-accumulates (Sec. 2: only kept weights are multiplied). */
+elsa_status elsa_cost_table_macs(const elsa_linear_shape* layers, int n_layers, const elsa_level* levels, int n_levels,
+                                 double* cost);
+/* F(alpha) = fixed_cost + sum over layers of cost[l][choice[l]]; fixed_cost carries the part of the network
+ * that is never pruned (attention products, patch embedding, head).  -1 on invalid arguments. */
+double elsa_config_cost(const double* cost, int n_layers, int n_levels, const int* choice, double fixed_cost);
+/*
+ * Alg. 3.  Costs are quantised to multiples of `quantum` (> 0; at most 2^22 quanta over the whole range).
+ * C_lower is the cost of the cheapest configuration; the n_intervals intervals have equal width, are half
+ * open, and the last also contains C_upper (configurations with F <= C_upper take part, Sec. 3.2).
+ * uniforms: 1 + n_layers numbers in [0, 1): the first picks the interval, number 1 + l picks the level of layer
+ * l by inverse CDF over the levels in their given order, under the distribution of Alg. 3's second step: P_t
+ * restricted to the configurations of the interval (computed exactly, without rejection).  Writes choice[l]
+ * and, if not NULL, *interval.  ELSA_ERR_SHAPE when the interval holds no configuration of non-zero
+ * probability, when C_upper is below C_lower, or when an argument is out of range.
+ */
+elsa_status elsa_two_step_sample(const double* cost, int n_layers, int n_levels, const double* P, double fixed_cost,
+                                 double c_upper, int n_intervals, double quantum, const double* uniforms, int* choice,
+                                 int* interval);
+/* mass[i] = probability, under P alone, that a configuration's cost falls into interval i of the same cut. */
+elsa_status elsa_interval_masses(const double* cost, int n_layers, int n_levels, const double* P, double fixed_cost,
+                                 double c_upper, int n_intervals, double quantum, double* mass);
+/* n_levels ^ n_layers as a decimal string (Sec. 2's 3^48); returns its length, -1 if `out` is too small. */
+int elsa_search_space_size(int n_layers, int n_levels, char* out, size_t capacity);
+/* Configuration number `index_decimal` (a decimal string below n_levels ^ n_layers): digit l of the index in base
+ * n_levels is the level of layer l. */
+elsa_status elsa_config_from_index(const char* index_decimal, int n_layers, int n_levels, int* choice);
+
 /*
  * Test hook for the device-side failure path.  Every wait of the tensor-core kernels is bounded: a wait that
  * runs out records ELSA_ERR_TIMEOUT | site << 8 in dev_status and the kernel winds down instead of hanging.

@@ -79,6 +79,22 @@ _set_grouping = _sig("elsa_set_grouping", None, [_i])
 _get_variant = _sig("elsa_get_linear_variant", _i, [])
 _launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
 _last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
+class ElsaLinearShape(ctypes.Structure):
+    _fields_ = [("rows", _i), ("in_", _i), ("out", _i)]
+
+
+class ElsaLevel(ctypes.Structure):
+    _fields_ = [("N", _i), ("M", _i)]
+
+
+_dp = ctypes.POINTER(ctypes.c_double)
+_ip = ctypes.POINTER(_i)
+_cost_table = _sig("elsa_cost_table_macs", _i, [ctypes.POINTER(ElsaLinearShape), _i, ctypes.POINTER(ElsaLevel), _i, _dp])
+_config_cost = _sig("elsa_config_cost", ctypes.c_double, [_dp, _i, _i, _ip, ctypes.c_double])
+_two_step = _sig("elsa_two_step_sample", _i, [_dp, _i, _i, _dp, ctypes.c_double, ctypes.c_double, _i, ctypes.c_double, _dp, _ip, _ip])
+_interval_masses = _sig("elsa_interval_masses", _i, [_dp, _i, _i, _dp, ctypes.c_double, ctypes.c_double, _i, ctypes.c_double, _dp])
+_space_size = _sig("elsa_search_space_size", _i, [_i, _i, ctypes.c_char_p, _sz])
+_config_from_index = _sig("elsa_config_from_index", _i, [ctypes.c_char_p, _i, _i, _ip])
 _selftest_wait = _sig("elsa_selftest_wait_timeout", _i, [ctypes.c_ulonglong, _vp, _vp])
 
 
@@ -105,6 +121,61 @@ def _check(status: int):
 
 def elsa_last_error() -> str:
     return (_last_error() or b"").decode()
+
+
+# ---- search-side host code (lists of numbers in, lists out; argument marshalling only)
+
+def _doubles(values):
+    flat = [float(v) for v in values]
+    return (ctypes.c_double * len(flat))(*flat)
+
+
+def elsa_cost_table_macs(shapes, levels):
+    """shapes: [(rows, in, out)], levels: [(N, M)] -> cost[l][s] as a list of lists."""
+    arr = (ElsaLinearShape * len(shapes))(*[ElsaLinearShape(*s) for s in shapes])
+    lev = (ElsaLevel * len(levels))(*[ElsaLevel(*s) for s in levels])
+    out = (ctypes.c_double * (len(shapes) * len(levels)))()
+    _check(_cost_table(arr, len(shapes), lev, len(levels), out))
+    k = len(levels)
+    return [[out[l * k + s] for s in range(k)] for l in range(len(shapes))]
+
+
+def elsa_config_cost(cost, choice, fixed_cost=0.0):
+    L, k = len(cost), len(cost[0])
+    return float(_config_cost(_doubles(v for row in cost for v in row), L, k, (_i * L)(*choice), float(fixed_cost)))
+
+
+def elsa_two_step_sample(cost, P, fixed_cost, c_upper, n_intervals, quantum, uniforms):
+    """Returns (choice, interval)."""
+    L, k = len(cost), len(cost[0])
+    assert len(uniforms) == L + 1
+    choice = (_i * L)()
+    interval = _i(-1)
+    _check(_two_step(_doubles(v for row in cost for v in row), L, k, _doubles(v for row in P for v in row), float(fixed_cost),
+                     float(c_upper), int(n_intervals), float(quantum), _doubles(uniforms), choice, ctypes.byref(interval)))
+    return list(choice), int(interval.value)
+
+
+def elsa_interval_masses(cost, P, fixed_cost, c_upper, n_intervals, quantum):
+    L, k = len(cost), len(cost[0])
+    mass = (ctypes.c_double * n_intervals)()
+    _check(_interval_masses(_doubles(v for row in cost for v in row), L, k, _doubles(v for row in P for v in row), float(fixed_cost),
+                            float(c_upper), int(n_intervals), float(quantum), mass))
+    return list(mass)
+
+
+def elsa_search_space_size(n_layers, n_levels) -> int:
+    buf = ctypes.create_string_buffer(4096)
+    n = _space_size(n_layers, n_levels, buf, len(buf))
+    if n < 0:
+        raise ElsaError(2)
+    return int(buf.value.decode())
+
+
+def elsa_config_from_index(index: int, n_layers, n_levels):
+    choice = (_i * n_layers)()
+    _check(_config_from_index(str(int(index)).encode(), n_layers, n_levels, choice))
+    return list(choice)
 
 
 def elsa_selftest_wait_timeout(limit_ns: int, dev_status: torch.Tensor, stream=None):

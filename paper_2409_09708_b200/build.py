@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libelsa.so")
 SOURCES = ["elsa_api.cu", "elsa_compress.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu", "elsa_linear_tc2.cu",
-           "elsa_no_alloc.cu", "elsa_selftest.cu", "elsa_sparse24.cu", "elsa_sparse24_pair.cu", "elsa_sparse24_st.cu", "elsa_sparse24_ws.cu"]
+           "elsa_no_alloc.cu", "elsa_search.cu", "elsa_selftest.cu", "elsa_sparse24.cu", "elsa_sparse24_pair.cu", "elsa_sparse24_st.cu", "elsa_sparse24_ws.cu"]
 
 
 def nvcc_path() -> str:

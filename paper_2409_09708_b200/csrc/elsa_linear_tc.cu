@@ -16,6 +16,8 @@
 // Tiles are visited feature-fastest so that the CTAs running together share X row blocks in L2.
 // Every wait is bounded: on expiry the kernel records ELSA_ERR_TIMEOUT and all roles leave.
 
+#include <atomic>
+
 #include "elsa_tc_common.cuh"
 
 namespace elsa {
@@ -315,16 +317,16 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
                           "Y")) != ELSA_OK)
         return st;
 
-    static bool attr_set[64][2] = {};
+    static std::atomic<bool> attr_set[64][2];   // zero-initialised; a double set by racing threads is harmless
     auto kernel = dtype == ELSA_BF16 ? linear_tc_dense_kernel<true> : linear_tc_dense_kernel<false>;
     const int slot = dev.device & 63;
-    if (!attr_set[slot][fmt]) {
+    if (!attr_set[slot][fmt].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         }
-        attr_set[slot][fmt] = true;
+        attr_set[slot][fmt].store(true, std::memory_order_release);
     }
     const int grid = p.num_tiles < dev.sm_count ? p.num_tiles : dev.sm_count;
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_DENSE, stream);

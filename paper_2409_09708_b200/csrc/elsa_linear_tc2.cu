@@ -23,6 +23,7 @@
 // before tensor memory is released keeps either CTA from leaving while its partner may still read
 // its shared memory.
 
+#include <atomic>
 #include <mutex>
 
 #include "elsa_tc_common.cuh"
@@ -426,9 +427,9 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
     const size_t smem = (size_t)stages * kStageBytesMax + fixed;
 
     auto kernel = linear_tc_pair_kernel<kBf16, kMaxLayers>;
-    static int max_pairs[64] = {};
+    static std::atomic<int> max_pairs[64];   // zero-initialised; racing first calls compute the same value
     const int slot = dev.device & 63;
-    if (max_pairs[slot] == 0) {
+    if (max_pairs[slot].load(std::memory_order_acquire) == 0) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
@@ -451,9 +452,9 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
         }
-        max_pairs[slot] = m;
+        max_pairs[slot].store(m, std::memory_order_release);
     }
-    const int pairs = g.num_tiles < max_pairs[slot] ? g.num_tiles : max_pairs[slot];
+    const int pairs = g.num_tiles < max_pairs[slot].load(std::memory_order_acquire) ? g.num_tiles : max_pairs[slot].load(std::memory_order_acquire);
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_PAIR, stream);
     cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, g);
     if (e != cudaSuccess) {

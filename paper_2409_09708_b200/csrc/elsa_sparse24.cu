@@ -22,6 +22,8 @@
 // 0-1, of the second in bits 2-3 (first < second).
 
 #include "elsa_pack_device.cuh"
+#include <atomic>
+
 #include "elsa_tc_common.cuh"
 
 namespace elsa {
@@ -376,16 +378,16 @@ elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t*
         ELSA_OK)
         return st;
 
-    static bool attr_set[64][2] = {};
+    static std::atomic<bool> attr_set[64][2];   // zero-initialised; a double set by racing threads is harmless
     auto kernel = dtype == ELSA_BF16 ? linear_tc_sp24_kernel<true> : linear_tc_sp24_kernel<false>;
     const int slot = dev.device & 63;
-    if (!attr_set[slot][fmt]) {
+    if (!attr_set[slot][fmt].load(std::memory_order_acquire)) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
         }
-        attr_set[slot][fmt] = true;
+        attr_set[slot][fmt].store(true, std::memory_order_release);
     }
     const int grid = p.num_tiles < dev.sm_count ? p.num_tiles : dev.sm_count;
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_SP24, stream);

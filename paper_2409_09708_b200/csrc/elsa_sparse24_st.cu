@@ -27,6 +27,7 @@
 // units of all rows interleaved, so that a warp's load is one contiguous run.  Waits are bounded as
 // in the other kernels.
 
+#include <atomic>
 #include <mutex>
 
 #include "elsa_tc_common.cuh"
@@ -418,9 +419,9 @@ elsa_status launch_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
     const size_t smem = (size_t)kStages * kStageBytes + kStagingTotal + kBarrierBytes + 1024;
     if (smem > dev.smem_optin) return fail(ELSA_ERR_CUDA, "not enough shared memory for the streaming sparse kernel");
 
-    static int max_pairs[64] = {};
+    static std::atomic<int> max_pairs[64];   // zero-initialised; racing first calls compute the same value
     const int slot = dev.device & 63;
-    if (max_pairs[slot] == 0) {
+    if (max_pairs[slot].load(std::memory_order_acquire) == 0) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
@@ -442,7 +443,7 @@ elsa_status launch_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
         }
-        max_pairs[slot] = m;
+        max_pairs[slot].store(m, std::memory_order_release);
     }
 
     static StGroup<kMaxLayers> g;   // host staging of the kernel parameters
@@ -476,7 +477,7 @@ elsa_status launch_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
     g.idesc = (1u << 2) | (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(kRowTile >> 3) << 17) |
               ((uint32_t)(kPairFeat >> 4) << 24);
 
-    const int pairs = g.num_tiles < max_pairs[slot] ? g.num_tiles : max_pairs[slot];
+    const int pairs = g.num_tiles < max_pairs[slot].load(std::memory_order_acquire) ? g.num_tiles : max_pairs[slot].load(std::memory_order_acquire);
     ProfileScope scope(ELSA_KERNEL_LINEAR_TC_SP24_ST, stream);
     cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, g);
     if (e != cudaSuccess) {

@@ -29,6 +29,7 @@
 // rows in that order (SP24_PERMUTED form of nm_to_sp24), and only the bias index and the store address
 // here know about it.  Waits are bounded as in the other kernels.
 
+#include <atomic>
 #include <mutex>
 
 #include "elsa_tc_common.cuh"
@@ -419,9 +420,9 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
     if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
     const size_t smem = (size_t)stages * stage_bytes + fixed;
 
-    static int max_pairs[64] = {};
+    static std::atomic<int> max_pairs[64];   // zero-initialised; racing first calls compute the same value
     const int slot = dev.device & 63;
-    if (max_pairs[slot] == 0) {
+    if (max_pairs[slot].load(std::memory_order_acquire) == 0) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dev.smem_optin) !=
             cudaSuccess) {
             cudaError_t e = cudaGetLastError();
@@ -443,9 +444,9 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
             cudaError_t e = cudaGetLastError();
             return fail(ELSA_ERR_CUDA, "cudaOccupancyMaxActiveClusters: %s", cudaGetErrorString(e));
         }
-        max_pairs[slot] = m;
+        max_pairs[slot].store(m, std::memory_order_release);
     }
-    const int pairs = max_pairs[slot];
+    const int pairs = max_pairs[slot].load(std::memory_order_acquire);
 
     static WsGroup<kMaxLayers> g;   // host staging of the kernel parameters
     static std::mutex g_mutex;
