@@ -91,7 +91,7 @@ __device__ __noinline__ void compress_segment16_call(const uint16_t* W, int in, 
     compress_segment<16>(W, in, N, vals, idx, segs_per_row, words_per_row, seg_id, words);
 }
 
-__global__ void __launch_bounds__(kWarpsPerBlock * 32, 5)
+__global__ void __launch_bounds__(kWarpsPerBlock * 32, 4)
 nm_compress_batch_kernel(const __grid_constant__ BatchTable t)
 {
     __shared__ uint32_t words[kWarpsPerBlock][kMaxIndexWordsPerSegment];
@@ -104,28 +104,77 @@ nm_compress_batch_kernel(const __grid_constant__ BatchTable t)
     pdl_release_successors();
     // A block owns a contiguous range of units and its warps walk it side by side; the table is searched
     // once per block and stepped through afterwards (a search per unit costs several dependent reads of
-    // kernel-parameter memory, more than the unit's own work).
+    // kernel-parameter memory, more than the unit's own work).  The fields of the current weight live in
+    // registers: reading them from the parameter table with a computed index for every unit kept the
+    // pipe that serves such reads busier than any other.
     const long long per_block = (t.total_units + gridDim.x - 1) / gridDim.x;
     const long long begin = (long long)blockIdx.x * per_block;
     const long long end = begin + per_block < t.total_units ? begin + per_block : t.total_units;
     if (begin >= end) return;
     int cur = find_item(t, begin);
-    long long cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
-    for (long long unit = begin + (threadIdx.x >> 5); unit < end; unit += kWarpsPerBlock) {
-        if (unit >= cur_end) {
-            while (unit >= cur_end) {
-                ++cur;
-                cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
-            }
-        }
+    long long cur_end;
+    const uint16_t* W; uint16_t* vals; uint32_t* idx;
+    long long first_unit;
+    int in, N, M, segs_per_row, wpr;
+    auto load_item = [&]() {
         const BatchItem& it = t.item[cur];
-        const long long seg_id = unit - it.first_unit;
-        const uint16_t* W = (const uint16_t*)it.src;
-        uint16_t* vals = (uint16_t*)it.dst;
-        uint32_t* idx = (uint32_t*)it.dst2;
-        if (it.M == 4) compress_segment_fast<4>(W, it.in, it.N, vals, idx, it.aux, seg_id, words, table4);
-        else if (it.M == 8) compress_segment_fast<8>(W, it.in, it.N, vals, idx, it.aux, seg_id, words, table8);
-        else compress_segment16_call(W, it.in, it.N, vals, idx, it.aux, it.wpr, seg_id, words);
+        cur_end = cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units;
+        W = (const uint16_t*)it.src; vals = (uint16_t*)it.dst; idx = (uint32_t*)it.dst2;
+        first_unit = it.first_unit;
+        in = it.in; N = it.N; M = it.M; segs_per_row = it.aux; wpr = it.wpr;
+    };
+    load_item();
+    // Software pipeline: the 16 bytes of the next unit are requested before the current one is worked on.  With
+    // one load per warp in flight the kernel moved exactly (resident warps x 512 bytes) per memory latency.
+    const int lane = threadIdx.x & 31;
+    uint32_t nr[4] = {0u, 0u, 0u, 0u};
+    int n_o = 0, n_seg = 0;
+    auto request = [&](long long unit) {          // `unit` belongs to the weight whose fields are loaded
+        const uint32_t local = (uint32_t)(unit - first_unit);      // a weight has far fewer than 2^32 segments
+        const uint32_t o = local / (uint32_t)segs_per_row;
+        n_o = (int)o;
+        n_seg = (int)(local - o * (uint32_t)segs_per_row);
+        const int g = n_seg * 32 + lane;
+        nr[0] = nr[1] = nr[2] = nr[3] = 0u;
+        if (M == 8) {
+            if (g < in / 8) { const uint4 v = *reinterpret_cast<const uint4*>(W + (size_t)n_o * in + (size_t)g * 8); nr[0] = v.x; nr[1] = v.y; nr[2] = v.z; nr[3] = v.w; }
+        } else if (M == 4) {
+            if (g < in / 4) { const uint2 v = *reinterpret_cast<const uint2*>(W + (size_t)n_o * in + (size_t)g * 4); nr[0] = v.x; nr[1] = v.y; }
+        }
+    };
+    long long unit = begin + (threadIdx.x >> 5);
+    while (unit < end) {
+        if (unit >= cur_end) {
+            while (unit >= (cur + 1 < t.n ? t.item[cur + 1].first_unit : t.total_units)) ++cur;
+            load_item();
+        }
+        // this warp's units inside the current weight: its fields stay put, and the pipeline drains only
+        // where the block's range crosses into the next weight
+        const long long stop = cur_end < end ? cur_end : end;
+        request(unit);
+        for (; unit < stop; unit += kWarpsPerBlock) {
+            const uint32_t r[4] = {nr[0], nr[1], nr[2], nr[3]};
+            const int o = n_o, seg = n_seg;
+            if (unit + kWarpsPerBlock < stop) request(unit + kWarpsPerBlock);
+            // the levels of the ViT tables get the level as a compile-time constant
+            if (M == 8) {
+                switch (N) {
+                case 1: compress_segment_fast_preloaded<8, 1>(r, in, 1, vals, idx, o, seg, words, table8); break;
+                case 2: compress_segment_fast_preloaded<8, 2>(r, in, 2, vals, idx, o, seg, words, table8); break;
+                case 4: compress_segment_fast_preloaded<8, 4>(r, in, 4, vals, idx, o, seg, words, table8); break;
+                case 8: compress_segment_fast_preloaded<8, 8>(r, in, 8, vals, idx, o, seg, words, table8); break;
+                default: compress_segment_fast_preloaded<8>(r, in, N, vals, idx, o, seg, words, table8); break;
+                }
+            } else if (M == 4) {
+                switch (N) {
+                case 1: compress_segment_fast_preloaded<4, 1>(r, in, 1, vals, idx, o, seg, words, table4); break;
+                case 2: compress_segment_fast_preloaded<4, 2>(r, in, 2, vals, idx, o, seg, words, table4); break;
+                case 4: compress_segment_fast_preloaded<4, 4>(r, in, 4, vals, idx, o, seg, words, table4); break;
+                default: compress_segment_fast_preloaded<4>(r, in, N, vals, idx, o, seg, words, table4); break;
+                }
+            }
+            else compress_segment16_call(W, in, N, vals, idx, segs_per_row, wpr, (long long)o * segs_per_row + seg, words);
+        }
     }
 }
 
@@ -283,7 +332,7 @@ elsa_status launch_compress_batch(const BatchTable& t, cudaStream_t stream)
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     long long grid = (t.total_units + kWarpsPerBlock - 1) / kWarpsPerBlock;
-    const long long waves = (long long)dev.sm_count * (2048 / (kWarpsPerBlock * 32)) * 4;   // a few waves of resident blocks
+    const long long waves = (long long)dev.sm_count * 4 * 4;   // a few waves of resident blocks (four per SM)
     if (grid > waves) grid = waves;
     ProfileScope scope(ELSA_KERNEL_COMPRESS, stream);
     launch_pdl(nm_compress_batch_kernel, dim3((unsigned)grid), dim3(kWarpsPerBlock * 32), 0, stream, 1, t);

@@ -250,8 +250,9 @@ __device__ __forceinline__ void compress_fast_load(const uint16_t* __restrict__ 
     }
 }
 
-template <int M>
-__device__ __forceinline__ void compress_fast_emit(const uint32_t (&r)[M / 2], int in, int N,
+// NC: the level's N as a compile-time constant (0 = take `N_runtime`): with N known every branch on it folds.
+template <int M, int NC>
+__device__ __forceinline__ void compress_fast_emit(const uint32_t (&r)[M / 2], int in, int N_runtime,
                                                    uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
                                                    int o, int seg,
                                                    uint32_t (*words)[kMaxIndexWordsPerSegment],
@@ -260,6 +261,7 @@ __device__ __forceinline__ void compress_fast_emit(const uint32_t (&r)[M / 2], i
     static_assert(M == 4 || M == 8, "fast path for groups of 4 and 8");
     constexpr int B = (M == 4) ? 2 : 3;
     constexpr int R = M / 2;
+    const int N = NC ? NC : N_runtime;
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     const int groups_per_row = in / M;
@@ -328,7 +330,7 @@ __device__ __forceinline__ void compress_fast_emit(const uint32_t (&r)[M / 2], i
     __syncwarp();
 }
 
-template <int M>
+template <int M, int NC = 0>
 __device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict__ W, int in, int N,
                                                       uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
                                                       int segs_per_row, long long seg_id,
@@ -340,7 +342,20 @@ __device__ __forceinline__ void compress_segment_fast(const uint16_t* __restrict
     const uint32_t seg = (uint32_t)seg_id - o * (uint32_t)segs_per_row;
     uint32_t r[M / 2];
     compress_fast_load<M>(W, in, (int)o, (int)seg, r);
-    compress_fast_emit<M>(r, in, N, vals, idx, (int)o, (int)seg, words, table);
+    compress_fast_emit<M, NC>(r, in, N, vals, idx, (int)o, (int)seg, words, table);
+}
+
+// The same with the 16 bytes of the group already in registers (requested one unit ahead by the caller).
+template <int M, int NC = 0>
+__device__ __forceinline__ void compress_segment_fast_preloaded(const uint32_t (&r4)[4], int in, int N,
+                                                                uint16_t* __restrict__ vals, uint32_t* __restrict__ idx,
+                                                                int o, int seg, uint32_t (*words)[kMaxIndexWordsPerSegment],
+                                                                const CompactEntry* table)
+{
+    uint32_t r[M / 2];
+#pragma unroll
+    for (int q = 0; q < M / 2; ++q) r[q] = r4[q];
+    compress_fast_emit<M, NC>(r, in, N, vals, idx, o, seg, words, table);
 }
 
 // Single level: the form elsa_nm_compress uses.
