@@ -53,6 +53,37 @@ def compress_table(workload, reps):
     print(json.dumps({"workload": workload, "weights": len(layers), "ms": times, "bytes_read_and_written": nbytes}))
 
 
+def int8_case(args):
+    """One layer in the INT8 form: seeded int8 activations and weights, per-feature scales, 16-bit output."""
+    N, M = (int(v) for v in args.level.split(":"))
+    dtype = synth.torch_dtype(args.dtype)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(5)
+    X = torch.randint(-128, 128, (args.rows, args.in_), dtype=torch.int8, device="cuda", generator=gen)
+    W = torch.randint(-128, 128, (args.out, args.in_), dtype=torch.int8, device="cuda", generator=gen)
+    w_scale = torch.rand(args.out, device="cuda", generator=gen) * 1e-3 + 1e-4
+    bias = synth.randn((args.out,), 3, synth.B_STD, dtype, device="cuda")
+    vals, idx = lib.elsa_nm_compress_i8(W, N, M)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for rep in range(args.reps):
+        flush.fill_(rep)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        lib.elsa_nm_linear_i8(X, 0.02, vals, idx, w_scale, bias, args.out, args.in_, N, M, dtype, dev_status=status)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(status.item()) == 0
+    bits = {4: 2, 8: 3, 16: 4}[M]
+    idx_bytes = 0 if N == M else args.out * (-(-(args.in_ // M * N * bits) // 32)) * 4
+    alg = args.rows * args.in_ + args.rows * args.out * 2 + args.out * (args.in_ // M) * N + idx_bytes + args.out * 6
+    print(json.dumps({"form": "int8", "rows": args.rows, "in": args.in_, "out": args.out, "level": args.level, "out_dtype": args.dtype,
+                      "ms": times, "algorithmic_bytes": alg, "kept_ops": 2.0 * args.rows * args.in_ * args.out * N / M,
+                      "dense_equiv_ops": 2.0 * args.rows * args.in_ * args.out}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--rows", type=int, default=50432)
@@ -64,9 +95,12 @@ def main():
     ap.add_argument("--variant", default="auto", choices=["auto", "simt", "tc_dense", "tc_pair", "tc_sparse", "tc_sparse_pair",
                                                             "tc_sparse_ws", "tc_sparse_st"])
     ap.add_argument("--compress-table", default=None, help="workload whose weights go through elsa_vit_compress")
+    ap.add_argument("--int8", action="store_true", help="the INT8 form: elsa_nm_compress_i8 once, then elsa_nm_linear_i8")
     args = ap.parse_args()
     if args.compress_table:
         return compress_table(args.compress_table, args.reps)
+    if args.int8:
+        return int8_case(args)
     N, M = (int(v) for v in args.level.split(":"))
     dtype = synth.torch_dtype(args.dtype)
     layer = synth.Layer("case", args.rows, args.in_, args.out, N, M, 1, 2, 3)

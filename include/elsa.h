@@ -271,7 +271,9 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_SP24_PAIR = 7,
     ELSA_KERNEL_WEIGHT_IMAGES = 8, /* batched unpack / 2-of-4 re-encoding of a table's weights */
     ELSA_KERNEL_LINEAR_TC_SP24_WS = 9, /* 2:4 sparse MMA with the weight block resident in tensor memory */
-    ELSA_KERNEL_LINEAR_TC_SP24_ST = 10 /* 2:4 sparse MMA with the weight streaming through tensor memory */
+    ELSA_KERNEL_LINEAR_TC_SP24_ST = 10, /* 2:4 sparse MMA with the weight streaming through tensor memory */
+    ELSA_KERNEL_LINEAR_TC_PAIR_I8 = 11, /* INT8 form of the CTA-pair GEMM */
+    ELSA_KERNEL_INT8_FORMAT = 12        /* INT8 compress / unpack */
 } elsa_kernel_id;
 
 typedef struct {
@@ -285,6 +287,29 @@ int elsa_profile_stop(elsa_kernel_time* records, int capacity);
 
 /* Number of kernels the library has launched from this process so far. */
 unsigned long long elsa_launch_count(void);
+
+/* ------------------------------------------------------------------------------------------------
+ * INT8 form of the path (paper: Table 6, the searched N:M models under 8-bit post-training quantisation).
+ * The quantiser is not part of this library: the caller supplies signed 8-bit weights and activations and
+ * their scales (w_scale[o] per output feature, x_scale for the activation tensor).
+ *
+ * elsa_nm_compress_i8: Sec. 3.1 / Eq. 1 with saliency |w| on the integers (|-128| = 128), lowest position first
+ * among equals; vals[out][in / M * N] are the kept bytes in ascending position, idx is the same log2(M)-bit
+ * stream as in the 16-bit form.  elsa_nm_unpack_i8: the dense image, zeros at pruned positions.
+ * elsa_nm_linear_i8: Y[r][o] = round16( float(sum_k X[r][k] * Wm[o][k]) * (x_scale * w_scale[o]) + bias[o] ): the sum
+ * is exact (int32), the int32 -> float conversion, the two products and the sum are each rounded to nearest
+ * in fp32, then one rounding to out_dtype.  bias is out_dtype or NULL.  All pointers are DEVICE pointers
+ * owned by the caller, row-major, 16-byte aligned; in % 16 == 0, out % 8 == 0.  workspace: at least
+ * elsa_workspace_bytes_i8 (0 for N == M), 256-byte aligned.  Asynchronous on `stream`; errors as elsa_nm_linear.
+ */
+size_t elsa_nm_values_bytes_i8(int out, int in, int N, int M);
+size_t elsa_workspace_bytes_i8(int out, int in, int N, int M);
+elsa_status elsa_nm_compress_i8(const int8_t* W, int out, int in, int N, int M, int8_t* vals, uint32_t* idx, void* stream);
+elsa_status elsa_nm_unpack_i8(const int8_t* vals, const uint32_t* idx, int out, int in, int N, int M, int8_t* W_masked,
+                              void* stream);
+elsa_status elsa_nm_linear_i8(const int8_t* X, int rows, float x_scale, const int8_t* vals, const uint32_t* idx,
+                              const float* w_scale, const void* bias, int out, int in, int N, int M, elsa_dtype out_dtype,
+                              void* Y, void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Search-side host code (no GPU): cost model, two-step sampling, enumeration of configurations.

@@ -79,6 +79,13 @@ _set_grouping = _sig("elsa_set_grouping", None, [_i])
 _get_variant = _sig("elsa_get_linear_variant", _i, [])
 _launch_count = _sig("elsa_launch_count", ctypes.c_ulonglong, [])
 _last_error = _sig("elsa_last_error", ctypes.c_char_p, [])
+_values_bytes_i8 = _sig("elsa_nm_values_bytes_i8", _sz, [_i, _i, _i, _i])
+_workspace_bytes_i8 = _sig("elsa_workspace_bytes_i8", _sz, [_i, _i, _i, _i])
+_compress_i8 = _sig("elsa_nm_compress_i8", _i, [_vp, _i, _i, _i, _i, _vp, _vp, _vp])
+_unpack_i8 = _sig("elsa_nm_unpack_i8", _i, [_vp, _vp, _i, _i, _i, _i, _vp, _vp])
+_linear_i8 = _sig("elsa_nm_linear_i8", _i, [_vp, _i, ctypes.c_float, _vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _sz, _vp, _vp])
+
+
 class ElsaLinearShape(ctypes.Structure):
     _fields_ = [("rows", _i), ("in_", _i), ("out", _i)]
 
@@ -103,7 +110,7 @@ class ElsaKernelTime(ctypes.Structure):
 
 
 KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images",
-                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st"}
+                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 
@@ -121,6 +128,37 @@ def _check(status: int):
 
 def elsa_last_error() -> str:
     return (_last_error() or b"").decode()
+
+
+# ---- INT8 form (int8 CUDA tensors; index words as int32 tensors)
+
+def elsa_nm_compress_i8(W: torch.Tensor, N: int, M: int, stream=None):
+    assert W.dtype == torch.int8 and W.is_cuda and W.is_contiguous()
+    out, in_ = W.shape
+    vals = torch.empty((out, in_ // M * N), dtype=torch.int8, device=W.device)
+    words = elsa_nm_index_bytes(out, in_, N, M) // 4
+    idx = torch.empty((out, words // out if out else 0), dtype=torch.int32, device=W.device) if words else None
+    _check(_compress_i8(_ptr(W), out, in_, N, M, _ptr(vals), _ptr(idx), _stream(stream)))
+    return vals, idx
+
+
+def elsa_nm_unpack_i8(vals: torch.Tensor, idx, out: int, in_: int, N: int, M: int, stream=None):
+    Wm = torch.empty((out, in_), dtype=torch.int8, device=vals.device)
+    _check(_unpack_i8(_ptr(vals), _ptr(idx), out, in_, N, M, _ptr(Wm), _stream(stream)))
+    return Wm
+
+
+def elsa_nm_linear_i8(X: torch.Tensor, x_scale: float, vals: torch.Tensor, idx, w_scale: torch.Tensor, bias, out: int,
+                      in_: int, N: int, M: int, out_dtype: torch.dtype, dev_status=None, stream=None):
+    """Y [rows, out] (out_dtype) from int8 activations, the packed int8 weight and the scales."""
+    assert X.dtype == torch.int8 and w_scale.dtype == torch.float32
+    rows = X.shape[0]
+    Y = torch.empty((rows, out), dtype=out_dtype, device=X.device)
+    need = int(_workspace_bytes_i8(out, in_, N, M))
+    ws = alloc_workspace(need) if need else None
+    _check(_linear_i8(_ptr(X), rows, float(x_scale), _ptr(vals), _ptr(idx), _ptr(w_scale), _ptr(bias), out, in_, N, M,
+                      dtype_code(out_dtype), _ptr(Y), _ptr(ws), need, _ptr(dev_status), _stream(stream)))
+    return Y
 
 
 # ---- search-side host code (lists of numbers in, lists out; argument marshalling only)

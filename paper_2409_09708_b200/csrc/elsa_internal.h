@@ -199,10 +199,17 @@ struct PairJob {
     const uint16_t* bias;
     uint16_t* Y;
     int rows, in, out;
+    const float* w_scale = nullptr;   // INT8 form only
+    float x_scale = 0.f;
 };
 int linear_tc_pair_group_max();
 elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,
                                         cudaStream_t stream);
+// INT8 form of the same GEMM: X [rows][in] and the dense weight image Wd [out][in] hold signed 8-bit integers,
+// accumulation is int32, Y[r][o] = round16(float(acc) * (x_scale * w_scale[o]) + bias[o]).
+elsa_status launch_linear_tc_pair_i8(const int8_t* X, int rows, const int8_t* Wd, const float* w_scale, float x_scale,
+                                     const uint16_t* bias, int out, int in, elsa_dtype dtype, uint16_t* Y,
+                                     uint32_t* dev_status, cudaStream_t stream);
 // Whether the problem has enough 256-row tiles to occupy every SM pair.
 bool linear_tc_pair_suits(int rows, int out, int sm_count);
 

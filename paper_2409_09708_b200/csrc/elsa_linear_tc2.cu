@@ -50,6 +50,7 @@ constexpr int kStagingBytes = 32 * kEpiCols * 2;
 constexpr int kStagingBufs = 1;     // one staging buffer per epilogue warp: the shared memory goes to a sixth pipeline stage instead
 constexpr int kStagingTotal = kEpiWarps * kStagingBufs * kStagingBytes;
 constexpr int kBiasBytes = 2 * kMaxBlockN * 2;   // two tiles' bias as stored (16 bit)
+constexpr int kScaleBytes = 2 * kMaxBlockN * 4;  // INT8 form: two tiles' combined scales (fp32)
 constexpr int kBarrierBytes = 256;
 
 // One layer of a launch.  A launch may carry several layers (a group): the persistent CTA pairs walk the
@@ -64,6 +65,8 @@ struct alignas(64) PairLayer {
     int num_k_blocks;
     uint32_t idesc;
     const uint16_t* bias;
+    const float* w_scale;   // INT8 form only: per-feature weight scale, and the activations' scale
+    float x_scale;
 };
 
 template <int kMaxLayers>
@@ -78,7 +81,10 @@ struct PairGroup {
 constexpr int kStageBytesMax = kATileBytes + (kMaxBlockN / 2) * kBlockK * 2;   // stage slots sized for BN = 256
 constexpr int kGroupMax = 72;   // layers per grouped launch (kernel parameters are limited to 32 KB)
 
-template <bool kBf16, int kMaxLayers>
+// kInt8: operands are signed 8-bit integers (rows of 128 elements per 128-byte swizzle row, K = 32 per MMA,
+// int32 accumulators); the epilogue turns an accumulator into float, multiplies by x_scale * w_scale[feature],
+// adds the bias, each in fp32 with one rounding per operation, and rounds once to the 16-bit output type.
+template <bool kBf16, bool kInt8, int kMaxLayers>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 {
@@ -95,14 +101,15 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 
     const uint32_t staging_base = smem_base + (uint32_t)(p.stages * stage_bytes);
     const uint32_t bias_off = (uint32_t)(p.stages * stage_bytes) + kStagingTotal;
-    const uint32_t bar_base = smem_base + bias_off + kBiasBytes;
+    const uint32_t scale_off = bias_off + kBiasBytes;
+    const uint32_t bar_base = smem_base + scale_off + kScaleBytes;
     const uint32_t full_bar = bar_base;                       // used in the leader only
     const uint32_t empty_bar = bar_base + 8 * kMaxStages;     // per CTA
     const uint32_t tmem_full_bar = bar_base + 16 * kMaxStages;                 // per CTA
     const uint32_t tmem_empty_bar = tmem_full_bar + 8 * kNumAccum;             // used in the leader only
     const uint32_t bias_full_bar = tmem_empty_bar + 8 * kNumAccum;             // per CTA
     const uint32_t bias_empty_bar = bias_full_bar + 16;                        // per CTA
-    const uint32_t holder_off = bias_off + kBiasBytes + 16 * kMaxStages + 16 * kNumAccum + 32;
+    const uint32_t holder_off = scale_off + kScaleBytes + 16 * kMaxStages + 16 * kNumAccum + 32;
     volatile uint32_t* tmem_holder = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off);
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_gen + holder_off + 4);
 
@@ -161,8 +168,9 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     if (elected) {
                         // the leader's stage barrier collects the bytes of both CTAs
                         if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
-                        tma_load_2d_pair(a_dst, &L.map_x, bar, kb * kBlockK, m0);
-                        tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * kBlockK, n0);
+                        // a stage is 128 bytes of K per row: 64 16-bit or 128 8-bit elements
+                        tma_load_2d_pair(a_dst, &L.map_x, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), m0);
+                        tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), n0);
                     }
                     __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -205,8 +213,12 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        umma_f16_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
-                                         (uint32_t)((kb | k) != 0), elected);
+                        if constexpr (kInt8)
+                            umma_i8_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                            (uint32_t)((kb | k) != 0), elected);
+                        else
+                            umma_f16_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
+                                             (uint32_t)((kb | k) != 0), elected);
                     }
                     umma_commit_pair_if(empty_bar + 8 * stage, 3, elected);   // frees this stage in both CTAs
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -236,6 +248,12 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 const uint16_t v = (l_bias != nullptr && o < L.out) ? __ldg(l_bias + o) : (uint16_t)0;
                 asm volatile("st.shared.b16 [%0], %1;" ::"r"(smem_base + bias_off + b * (kMaxBlockN * 2) + (uint32_t)(j * 2)), "h"(v)
                              : "memory");
+                if constexpr (kInt8) {
+                    const float sc = o < L.out ? __fmul_rn(L.x_scale, __ldg(L.w_scale + o)) : 0.f;
+                    asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_base + scale_off + b * (kMaxBlockN * 4) + (uint32_t)(j * 4)),
+                                 "r"(__float_as_uint(sc))
+                                 : "memory");
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bias_full_bar + 8 * b);
@@ -265,6 +283,8 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             const int l_rows = L.rows, l_out = L.out;
             const uint32_t bias_b = it & 1u;
             const uint32_t bias_cur = smem_base + bias_off + bias_b * (kMaxBlockN * 2);
+            const uint32_t scale_cur = smem_base + scale_off + bias_b * (kMaxBlockN * 4);
+            (void)scale_cur;
             bool ok = mbar_wait(bias_full_bar + 8 * bias_b, (it >> 1) & 1u, abort_flag, p.dev_status, 6);
             ok = ok && mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
@@ -286,7 +306,16 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                         for (int e = 0; e < 4; ++e) {
                             const float2 bv = raw2_to_float2<kBf16>(bw[e]);
                             const int j = 8 * h + 4 * g + e;
-                            pk[4 * g + e] = pack2<kBf16>(__uint_as_float(r[2 * j]) + bv.x, __uint_as_float(r[2 * j + 1]) + bv.y);
+                            if constexpr (kInt8) {
+                                float sx, sy;
+                                asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];" : "=f"(sx), "=f"(sy)
+                                             : "r"(scale_cur + (uint32_t)((c * kEpiCols + 2 * j) * 4)));
+                                const float vx = __fadd_rn(__fmul_rn((float)(int)r[2 * j], sx), bv.x);
+                                const float vy = __fadd_rn(__fmul_rn((float)(int)r[2 * j + 1], sy), bv.y);
+                                pk[4 * g + e] = pack2<kBf16>(vx, vy);
+                            } else {
+                                pk[4 * g + e] = pack2<kBf16>(__uint_as_float(r[2 * j]) + bv.x, __uint_as_float(r[2 * j + 1]) + bv.y);
+                            }
                         }
                     }
                 };
@@ -384,7 +413,7 @@ bool linear_tc_pair_suits(int rows, int out, int sm_count)
 
 namespace {
 
-template <bool kBf16, int kMaxLayers>
+template <bool kBf16, bool kInt8, int kMaxLayers>
 elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
                          const DeviceInfo& dev)
 {
@@ -401,16 +430,30 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
         L.tiles_n = (j.out + L.bn - 1) / L.bn;
         L.tile_begin = tile_begin;
         tile_begin += ((j.rows + kPairRows - 1) / kPairRows) * L.tiles_n;
-        L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
         L.bias = j.bias;
-        L.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+        L.w_scale = j.w_scale;
+        L.x_scale = j.x_scale;
         elsa_status st;
-        if ((st = make_map_2d(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, kBlockK, kRowsPerCta,
-                              CU_TENSOR_MAP_SWIZZLE_128B, "X")) != ELSA_OK)
-            return st;
-        if ((st = make_map_2d(&L.map_w, j.Wd, (uint64_t)j.in, (uint64_t)j.out, kBlockK, (uint32_t)(L.bn / 2),
-                              CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
-            return st;
+        if constexpr (kInt8) {
+            L.num_k_blocks = (j.in + 2 * kBlockK - 1) / (2 * kBlockK);
+            // int32 accumulate, A and B signed 8-bit, K-major, N = bn, M = 256 over the pair
+            L.idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(L.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+            if ((st = make_map_2d_u8(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, 2 * kBlockK, kRowsPerCta,
+                                     CU_TENSOR_MAP_SWIZZLE_128B, "X")) != ELSA_OK)
+                return st;
+            if ((st = make_map_2d_u8(&L.map_w, j.Wd, (uint64_t)j.in, (uint64_t)j.out, 2 * kBlockK, (uint32_t)(L.bn / 2),
+                                     CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
+                return st;
+        } else {
+            L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
+            L.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(L.bn >> 3) << 17) | ((uint32_t)(kPairRows >> 4) << 24);
+            if ((st = make_map_2d(&L.map_x, j.X, (uint64_t)j.in, (uint64_t)j.rows, kBlockK, kRowsPerCta,
+                                  CU_TENSOR_MAP_SWIZZLE_128B, "X")) != ELSA_OK)
+                return st;
+            if ((st = make_map_2d(&L.map_w, j.Wd, (uint64_t)j.in, (uint64_t)j.out, kBlockK, (uint32_t)(L.bn / 2),
+                                  CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
+                return st;
+        }
         if ((st = make_map_2d(&L.map_y, j.Y, (uint64_t)j.out, (uint64_t)j.rows, kEpiCols, 32, CU_TENSOR_MAP_SWIZZLE_64B,
                               "Y")) != ELSA_OK)
             return st;
@@ -419,14 +462,14 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
     g.num_tiles = tile_begin;
     g.dev_status = dev_status;
 
-    const int fixed = kStagingTotal + kBiasBytes + kBarrierBytes + 1024;
+    const int fixed = kStagingTotal + kBiasBytes + kScaleBytes + kBarrierBytes + 1024;
     int stages = (int)((dev.smem_optin - fixed) / kStageBytesMax);
     if (stages > kMaxStages) stages = kMaxStages;
     if (stages < 2) return fail(ELSA_ERR_CUDA, "not enough shared memory for two pipeline stages");
     g.stages = stages;
     const size_t smem = (size_t)stages * kStageBytesMax + fixed;
 
-    auto kernel = linear_tc_pair_kernel<kBf16, kMaxLayers>;
+    auto kernel = linear_tc_pair_kernel<kBf16, kInt8, kMaxLayers>;
     static std::atomic<int> max_pairs[64];   // zero-initialised; racing first calls compute the same value
     const int slot = dev.device & 63;
     if (max_pairs[slot].load(std::memory_order_acquire) == 0) {
@@ -455,7 +498,7 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
         max_pairs[slot].store(m, std::memory_order_release);
     }
     const int pairs = g.num_tiles < max_pairs[slot].load(std::memory_order_acquire) ? g.num_tiles : max_pairs[slot].load(std::memory_order_acquire);
-    ProfileScope scope(ELSA_KERNEL_LINEAR_TC_PAIR, stream);
+    ProfileScope scope(kInt8 ? ELSA_KERNEL_LINEAR_TC_PAIR_I8 : ELSA_KERNEL_LINEAR_TC_PAIR, stream);
     cudaError_t e = launch_pdl(kernel, dim3((unsigned)(2 * pairs)), dim3(kThreads), smem, stream, 2, g);
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -476,10 +519,26 @@ elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype d
     if (st != ELSA_OK) return st;
     if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
     if (n == 1)
-        return dtype == ELSA_BF16 ? launch_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
-                                  : launch_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
-    return dtype == ELSA_BF16 ? launch_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
-                              : launch_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+        return dtype == ELSA_BF16 ? launch_group<true, false, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_group<false, false, 1>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_group<true, false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_group<false, false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+}
+
+// INT8 form (one layer per launch): X and Wd hold signed 8-bit integers, Y is 16-bit.
+elsa_status launch_linear_tc_pair_i8(const int8_t* X, int rows, const int8_t* Wd, const float* w_scale, float x_scale,
+                                     const uint16_t* bias, int out, int in, elsa_dtype dtype, uint16_t* Y,
+                                     uint32_t* dev_status, cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    PairJob job;
+    job.X = (const uint16_t*)X; job.Wd = (const uint16_t*)Wd; job.bias = bias; job.Y = Y;
+    job.rows = rows; job.in = in; job.out = out;
+    job.w_scale = w_scale; job.x_scale = x_scale;
+    return dtype == ELSA_BF16 ? launch_group<true, true, 1>(&job, 1, dtype, dev_status, stream, dev)
+                              : launch_group<false, true, 1>(&job, 1, dtype, dev_status, stream, dev);
 }
 
 elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias, int out,
@@ -488,6 +547,7 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
     PairJob job;
     job.X = X; job.Wd = Wd; job.bias = bias; job.Y = Y;
     job.rows = rows; job.in = in; job.out = out;
+    job.w_scale = nullptr; job.x_scale = 0.f;
     return launch_linear_tc_pair_group(&job, 1, dtype, dev_status, stream);
 }
 

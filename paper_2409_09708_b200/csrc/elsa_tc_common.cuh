@@ -521,6 +521,21 @@ __device__ __forceinline__ void umma_f16_pair_if(uint32_t d_tmem, uint64_t a_des
         : "memory");
 }
 
+// The same for 8-bit integer operands (K = 32 per instruction, int32 accumulators).
+__device__ __forceinline__ void umma_i8_pair_if(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                                uint32_t accumulate, uint32_t issue)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
+        : "memory");
+}
+
 __device__ __forceinline__ void umma_commit_pair_if(uint32_t bar, uint16_t cta_mask, uint32_t issue)
 {
     asm volatile(
@@ -597,6 +612,23 @@ elsa_status make_map_2d(CUtensorMap* map, const void* base, uint64_t dim0, uint6
     cuuint32_t box[2] = {box0, box1};
     cuuint32_t elem[2] = {1, 1};
     CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for %s rejected (CUresult %d)", what, (int)rc);
+    return ELSA_OK;
+}
+
+// 2-D row-major 8-bit tensor [dim1][dim0], box [box1][box0].
+elsa_status make_map_2d_u8(CUtensorMap* map, const void* base, uint64_t dim0, uint64_t dim1, uint32_t box0,
+                           uint32_t box1, CUtensorMapSwizzle swizzle, const char* what)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(ELSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[2] = {dim0, dim1};
+    cuuint64_t strides[1] = {dim0};
+    cuuint32_t box[2] = {box0, box1};
+    cuuint32_t elem[2] = {1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, elem,
                      CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for %s rejected (CUresult %d)", what, (int)rc);
