@@ -1,0 +1,75 @@
+"""Oracle of the chained transformer block around the four N:M linears (test infrastructure; shares no code
+with the library).  Only tests/, __graft_entry__.smoke() and bench.py's cpu_baseline leg may import it.
+
+What it follows: the ViT encoder block the paper prunes (ELSA, arXiv 2409.09708, Sec. 3: the linear modules
+qkv, proj, fc1, fc2 of every block take one N:M level each; Sec. 4.2 quotes end-to-end speed-ups of whole
+models).  The block is the standard pre-norm one of DeiT:
+    x1 = LayerNorm1(x);  qkv = Linear_qkv(x1);  a = attention(qkv)
+    x2 = x + Linear_proj(a);  x3 = LayerNorm2(x2);  h = GELU(Linear_fc1(x3));  y = x2 + Linear_fc2(h)
+with LayerNorm over the feature dimension (biased variance, eps inside the square root, elementwise gain and
+bias) and GELU(v) = v * Phi(v) = 0.5 * v * (1 + erf(v / sqrt 2)), the exact form (not the tanh approximation).
+The attention products (QK^T, softmax, AV) are NOT part of this oracle: `attention` is the stated stand-in
+a = V, the last third of qkv copied through, so that the linear and elementwise path can be checked and timed.
+
+Every tensor that crosses a stage boundary is a 16-bit tensor (the library writes it to memory in the block's
+dtype), so every stage here computes in fp64 from its 16-bit inputs and rounds its result once, to nearest
+even, to the 16-bit type; the linears are oracle/elsa_oracle.c's (mask, pack, unpack, fp64 product).
+"""
+import math
+
+import numpy as np
+import torch
+
+from oracle import elsa_oracle as eo
+
+
+def _round16(a64, torch_dtype):
+    """fp64 array -> 16-bit type (one rounding to nearest even) -> fp64."""
+    return torch.from_numpy(np.ascontiguousarray(a64)).to(torch_dtype).to(torch.float64).numpy()
+
+
+def _bits(a64, torch_dtype):
+    return torch.from_numpy(np.ascontiguousarray(a64)).to(torch_dtype).contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def layer_norm(x, gain, bias, eps):
+    """fp64: rows normalised to zero mean and unit (biased) variance, then gain and bias per feature."""
+    mean = x.mean(axis=1, keepdims=True)
+    var = ((x - mean) ** 2).mean(axis=1, keepdims=True)
+    return (x - mean) / np.sqrt(var + eps) * gain[None, :] + bias[None, :]
+
+
+_erf = np.vectorize(math.erf, otypes=[np.float64])
+
+
+def gelu(v):
+    return 0.5 * v * (1.0 + _erf(v / math.sqrt(2.0)))
+
+
+def sparse_linear(x16, W_bits, bias_bits, N, M, code):
+    """fp64 product of 16-bit activations (fp64 array of 16-bit values) with the N:M projection of W."""
+    vals, idx, _ = eo.nm_compress(W_bits, N, M)
+    torch_dtype = torch.float16 if code == eo.F16 else torch.bfloat16
+    return eo.nm_linear_f64(_bits(x16, torch_dtype), vals, idx, bias_bits, W_bits.shape[0], W_bits.shape[1], N, M, code)
+
+
+def block_forward(x_bits, p, code, eps=1e-6):
+    """x_bits: uint16 [rows, dim].  p: dict with ln1_g, ln1_b, ln2_g, ln2_b (uint16 [dim]) and, for each of qkv,
+    proj, fc1, fc2: W_<name> (uint16 [out, in]), b_<name> (uint16 [out]), level_<name> = (N, M).
+    Returns a dict of every stage's 16-bit result as fp64 arrays: x1, qkv, a, x2, x3, h, y."""
+    torch_dtype = torch.float16 if code == eo.F16 else torch.bfloat16
+
+    def f64(bits):
+        return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch_dtype).to(torch.float64).numpy()
+
+    x = f64(x_bits)
+    dim = x.shape[1]
+    out = {}
+    out["x1"] = _round16(layer_norm(x, f64(p["ln1_g"]), f64(p["ln1_b"]), eps), torch_dtype)
+    out["qkv"] = _round16(sparse_linear(out["x1"], p["W_qkv"], p["b_qkv"], *p["level_qkv"], code), torch_dtype)
+    out["a"] = out["qkv"][:, 2 * dim:3 * dim].copy()                 # the stated stand-in for attention: a = V
+    out["x2"] = _round16(x + sparse_linear(out["a"], p["W_proj"], p["b_proj"], *p["level_proj"], code), torch_dtype)
+    out["x3"] = _round16(layer_norm(out["x2"], f64(p["ln2_g"]), f64(p["ln2_b"]), eps), torch_dtype)
+    out["h"] = _round16(gelu(sparse_linear(out["x3"], p["W_fc1"], p["b_fc1"], *p["level_fc1"], code)), torch_dtype)
+    out["y"] = _round16(out["x2"] + sparse_linear(out["h"], p["W_fc2"], p["b_fc2"], *p["level_fc2"], code), torch_dtype)
+    return out

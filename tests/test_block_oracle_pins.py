@@ -1,0 +1,77 @@
+"""Pins of the chained-block oracle (no GPU): LayerNorm and GELU against closed forms and hand-worked values, the
+whole chain against the library routines of torch in fp64 on a masked dense weight."""
+import math
+
+import numpy as np
+import torch
+
+from oracle import elsa_block_oracle as bo
+from oracle import elsa_oracle as eo
+from paper_2409_09708_b200 import synth
+
+
+def test_layer_norm_closed_forms():
+    x = np.array([[1.0, 2.0, 3.0, 6.0], [5.0, 5.0, 5.0, 5.0]])
+    g = np.array([1.0, 1.0, 2.0, 1.0])
+    b = np.array([0.0, 0.5, 0.0, 0.0])
+    y = bo.layer_norm(x, g, b, 0.0 + 1e-12)
+    # row 0: mean 3, biased variance (4 + 1 + 0 + 9) / 4 = 3.5
+    s = math.sqrt(3.5)
+    assert np.allclose(y[0], [-2 / s, -1 / s + 0.5, 0.0, 3 / s], atol=1e-9)
+    # a constant row has zero variance: the normalised row is 0 (eps keeps the division finite), leaving the bias
+    assert np.allclose(y[1], b, atol=1e-6)
+    z = bo.layer_norm(np.random.default_rng(0).standard_normal((5, 64)), np.ones(64), np.zeros(64), 0.0)
+    assert np.allclose(z.mean(axis=1), 0, atol=1e-12) and np.allclose(z.var(axis=1), 1, atol=1e-12)
+
+
+def test_gelu_is_the_exact_form():
+    assert bo.gelu(np.array([0.0]))[0] == 0.0
+    # Phi(1) = 0.8413447460685429, Phi(-1) = 1 - Phi(1): standard normal table values
+    assert abs(bo.gelu(np.array([1.0]))[0] - 0.8413447460685429) < 1e-15
+    assert abs(bo.gelu(np.array([-1.0]))[0] + 0.15865525393145707) < 1e-15
+    v = np.linspace(-6, 6, 101)
+    assert np.allclose(bo.gelu(v) - bo.gelu(-v), v, atol=1e-12)              # v Phi(v) + v Phi(-v) = v
+    tanh_form = 0.5 * v * (1 + np.tanh(math.sqrt(2 / math.pi) * (v + 0.044715 * v ** 3)))
+    assert np.abs(bo.gelu(v) - tanh_form).max() > 1e-4                        # not the approximation
+    assert np.allclose(bo.gelu(v), torch.nn.functional.gelu(torch.from_numpy(v)).numpy(), atol=1e-15)
+
+
+def test_block_chain_against_torch_fp64_routines():
+    dtype = torch.bfloat16
+    rows, dim, mlp = 24, 64, 256
+    x = synth.randn((rows, dim), 1, 1.0, dtype)
+    p, tp = {}, {}
+    shapes = {"qkv": (3 * dim, dim), "proj": (dim, dim), "fc1": (mlp, dim), "fc2": (dim, mlp)}
+    levels = {"qkv": (4, 8), "proj": (2, 8), "fc1": (2, 4), "fc2": (1, 4)}
+    for i, (name, (o, k)) in enumerate(shapes.items()):
+        W = synth.randn((o, k), 10 + i, 0.08, dtype)
+        b = synth.randn((o,), 20 + i, 0.02, dtype)
+        p["W_" + name], p["b_" + name], p["level_" + name] = synth.bits(W), synth.bits(b), levels[name]
+        mask = eo.nm_mask(synth.bits(W), *levels[name])
+        tp[name] = (W.double() * torch.from_numpy(mask.astype(np.float64)), b.double())
+    for i, name in enumerate(("ln1_g", "ln1_b", "ln2_g", "ln2_b")):
+        t = synth.randn((dim,), 30 + i, 0.1, dtype) + (1.0 if name.endswith("g") else 0.0)
+        p[name] = synth.bits(t.to(dtype))
+        tp[name] = t.to(dtype).double()
+    got = bo.block_forward(synth.bits(x), p, eo.BF16, eps=1e-6)
+
+    F = torch.nn.functional
+    r = lambda t: t.to(dtype).double()                                  # a stage boundary: one rounding to 16 bits
+    xt = x.double()
+    x1 = r(F.layer_norm(xt, (dim,), tp["ln1_g"], tp["ln1_b"], 1e-6))
+    qkv = r(F.linear(x1, *tp["qkv"]))
+    a = qkv[:, 2 * dim:]
+    x2 = r(xt + F.linear(a, *tp["proj"]))
+    x3 = r(F.layer_norm(x2, (dim,), tp["ln2_g"], tp["ln2_b"], 1e-6))
+    h = r(F.gelu(F.linear(x3, *tp["fc1"])))
+    y = r(x2 + F.linear(h, *tp["fc2"]))
+    for name, ref in (("x1", x1), ("qkv", qkv), ("a", a), ("x2", x2), ("x3", x3), ("h", h), ("y", y)):
+        ref = ref.numpy()
+        # summation order differs between the two fp64 products: a value next to a rounding boundary may land on
+        # the neighbouring 16-bit number, nothing more
+        close = np.abs(got[name] - ref) <= 2.0 ** -7 * np.abs(ref) + 1e-30
+        assert close.all(), name
+        assert (got[name] == ref).mean() > 0.98, name
+    # a mistake anywhere shows: dropping a residual, the wrong GELU, or the wrong third of qkv
+    assert np.abs(got["x2"] - (got["x2"] - x.double().numpy())).max() > 0.1
+    assert not np.array_equal(got["a"], got["qkv"][:, :dim])
