@@ -273,7 +273,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_SP24_WS = 9, /* 2:4 sparse MMA with the weight block resident in tensor memory */
     ELSA_KERNEL_LINEAR_TC_SP24_ST = 10, /* 2:4 sparse MMA with the weight streaming through tensor memory */
     ELSA_KERNEL_LINEAR_TC_PAIR_I8 = 11, /* INT8 form of the CTA-pair GEMM */
-    ELSA_KERNEL_INT8_FORMAT = 12        /* INT8 compress / unpack */
+    ELSA_KERNEL_INT8_FORMAT = 12,       /* INT8 compress / unpack */
+    ELSA_KERNEL_BLOCK_ROWWISE = 13      /* LayerNorm, residual add, GELU, column copy of the chained block */
 } elsa_kernel_id;
 
 typedef struct {
@@ -357,6 +358,72 @@ int elsa_search_space_size(int n_layers, int n_levels, char* out, size_t capacit
 /* Configuration number `index_decimal` (a decimal string below n_levels ^ n_layers): digit l of the index in base
  * n_levels is the level of layer l. */
 elsa_status elsa_config_from_index(const char* index_decimal, int n_layers, int n_levels, int* choice);
+
+/* ------------------------------------------------------------------------------------------------
+ * The chained transformer block around the four pruned linears (Sec. 3: the modules qkv, proj, fc1 and fc2 of
+ * every block each take one N:M level; Sec. 4.2 quotes the speed of whole models).  The block is the pre-norm
+ * ViT block:
+ *     x1 = LayerNorm1(x)        qkv = Linear_qkv(x1)        a = attention(qkv)
+ *     x2 = x + Linear_proj(a)   x3 = LayerNorm2(x2)         h = GELU(Linear_fc1(x3))    y = x2 + Linear_fc2(h)
+ * LayerNorm runs over the `dim` features of a token row (biased variance, eps inside the square root, gain and
+ * bias per feature); GELU is the exact form v * Phi(v).  Statistics, bias, activation and residual are computed
+ * in fp32 and every tensor that crosses a stage boundary is rounded once to `dtype` (where a linear runs on a
+ * kernel whose epilogue cannot take the residual, its output is rounded before the residual is added).
+ * The attention products (QK^T, softmax, AV) are NOT part of this library: elsa_vit_block_qkv runs the block up
+ * to qkv, the caller's attention turns qkv into a [rows][dim], elsa_vit_block_rest runs the block from proj on.
+ * elsa_vit_block runs both with the stand-in a = V (columns 2 dim .. 3 dim of qkv copied through), which is what
+ * the parity tests and the block timing use; it does not compute a transformer block's attention.
+ *
+ * All pointers are DEVICE pointers, 16-byte aligned; dim and mlp_dim multiples of 8 and of every M in use.
+ * Weights are the packed forms elsa_nm_compress writes: qkv [3 dim][dim], proj [dim][dim], fc1 [mlp_dim][dim],
+ * fc2 [dim][mlp_dim].  `scratch`: caller-owned, 256-byte aligned, elsa_vit_block_scratch_bytes(...) bytes; the
+ * intermediates stay there after the call at the byte offsets that call reports, in the order of
+ * elsa_block_region (region T is the unfused linears' output before the residual; WORKSPACE holds the weight
+ * images).  y may not alias x.  Launches are asynchronous on `stream` (weight images are built on a library
+ * stream beside the first LayerNorm); errors as for elsa_nm_linear, nothing is enqueued on a validation error.
+ */
+typedef struct {
+    const void* vals;    /* packed values */
+    const uint32_t* idx; /* packed indices; NULL iff N == M */
+    const void* bias;    /* [out] or NULL */
+    int N, M;
+} elsa_block_linear;
+
+typedef struct {
+    const void* ln1_gain; /* [dim] */
+    const void* ln1_bias;
+    const void* ln2_gain;
+    const void* ln2_bias;
+    elsa_block_linear qkv, proj, fc1, fc2;
+    float eps;            /* LayerNorm epsilon (1e-6 in DeiT) */
+} elsa_block_weights;
+
+typedef enum {
+    ELSA_BLOCK_X1 = 0,  /* [rows][dim]     */
+    ELSA_BLOCK_QKV = 1, /* [rows][3 dim]   */
+    ELSA_BLOCK_A = 2,   /* [rows][dim]     */
+    ELSA_BLOCK_X2 = 3,  /* [rows][dim]     */
+    ELSA_BLOCK_X3 = 4,  /* [rows][dim]     */
+    ELSA_BLOCK_H = 5,   /* [rows][mlp_dim] */
+    ELSA_BLOCK_T = 6,   /* [rows][dim]     */
+    ELSA_BLOCK_WORKSPACE = 7,
+    ELSA_BLOCK_REGIONS = 8
+} elsa_block_region;
+
+/* Bytes of scratch for one block; offsets (may be NULL) receives ELSA_BLOCK_REGIONS byte offsets.  0 on invalid
+ * arguments.  Host-only arithmetic. */
+size_t elsa_vit_block_scratch_bytes(int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                                    size_t* offsets);
+/* x [rows][dim] -> regions X1 and QKV of scratch. */
+elsa_status elsa_vit_block_qkv(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w,
+                               elsa_dtype dtype, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream);
+/* x and region A of scratch (written by the caller's attention) -> y [rows][dim]; fills X2, X3, H. */
+elsa_status elsa_vit_block_rest(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w,
+                                elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status,
+                                void* stream);
+/* Both, with the stand-in a = V between them. */
+elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                           void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream);
 
 /*
  * Test hook for the device-side failure path.  Every wait of the tensor-core kernels is bounded: a wait that

@@ -105,12 +105,30 @@ _config_from_index = _sig("elsa_config_from_index", _i, [ctypes.c_char_p, _i, _i
 _selftest_wait = _sig("elsa_selftest_wait_timeout", _i, [ctypes.c_ulonglong, _vp, _vp])
 
 
+class ElsaBlockLinear(ctypes.Structure):
+    _fields_ = [("vals", _vp), ("idx", _vp), ("bias", _vp), ("N", _i), ("M", _i)]
+
+
+class ElsaBlockWeights(ctypes.Structure):
+    _fields_ = [("ln1_gain", _vp), ("ln1_bias", _vp), ("ln2_gain", _vp), ("ln2_bias", _vp),
+                ("qkv", ElsaBlockLinear), ("proj", ElsaBlockLinear), ("fc1", ElsaBlockLinear), ("fc2", ElsaBlockLinear),
+                ("eps", ctypes.c_float)]
+
+
+BLOCK_REGIONS = ("x1", "qkv", "a", "x2", "x3", "h", "t", "workspace")
+_bw = ctypes.POINTER(ElsaBlockWeights)
+_block_scratch = _sig("elsa_vit_block_scratch_bytes", _sz, [_i, _i, _i, _bw, _i, ctypes.POINTER(_sz)])
+_block_qkv = _sig("elsa_vit_block_qkv", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _sz, _vp, _vp])
+_block_rest = _sig("elsa_vit_block_rest", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
+_block = _sig("elsa_vit_block", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
+
+
 class ElsaKernelTime(ctypes.Structure):
     _fields_ = [("kernel", _i), ("layer", _i), ("ms", ctypes.c_float)]
 
 
 KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images",
-                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format"}
+                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format", 13: "block_rowwise"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 
@@ -351,6 +369,52 @@ def elsa_nm_linear(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_
     _check(_linear(_ptr(X), rows, _ptr(vals), _ptr(idx), _ptr(bias), out, in_, N, M, code, _ptr(Y),
                    _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
     return Y
+
+
+def make_block_weights(ln1_gain, ln1_bias, ln2_gain, ln2_bias, linears, eps=1e-6):
+    """linears: dict name -> (vals, idx or None, bias or None, N, M) for qkv, proj, fc1, fc2 (device tensors).
+    Returns (ElsaBlockWeights, the tensors it points to)."""
+    w = ElsaBlockWeights()
+    keep = [ln1_gain, ln1_bias, ln2_gain, ln2_bias]
+    w.ln1_gain, w.ln1_bias, w.ln2_gain, w.ln2_bias = (_ptr(t) for t in keep)
+    for name in ("qkv", "proj", "fc1", "fc2"):
+        vals, idx, bias, N, M = linears[name]
+        setattr(w, name, ElsaBlockLinear(_ptr(vals), _ptr(idx), _ptr(bias), N, M))
+        keep += [vals, idx, bias]
+    w.eps = eps
+    return w, keep
+
+
+def elsa_vit_block_scratch_bytes(rows, dim, mlp_dim, weights, dtype_c):
+    """(bytes, {region name: byte offset})."""
+    off = (_sz * len(BLOCK_REGIONS))()
+    n = _block_scratch(rows, dim, mlp_dim, ctypes.byref(weights), dtype_c, off)
+    return n, dict(zip(BLOCK_REGIONS, off))
+
+
+def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, stream=None, phase="both"):
+    """One pre-norm ViT block over x [rows, dim] with the four linears in their packed N:M forms.  phase "both"
+    runs the whole block with the stand-in a = V for attention; "qkv" stops after qkv (regions x1, qkv of
+    scratch); "rest" continues from region a of scratch, which the caller's attention has written."""
+    rows, dim = x.shape
+    code = dtype_code(x.dtype)
+    if scratch is None:
+        scratch = alloc_workspace(elsa_vit_block_scratch_bytes(rows, dim, mlp_dim, weights, code)[0], x.device)
+    if y is None and phase != "qkv":
+        y = torch.empty_like(x)
+    if phase == "qkv":
+        _check(_block_qkv(_ptr(x), rows, dim, mlp_dim, ctypes.byref(weights), code, _ptr(scratch), scratch.numel(),
+                          _ptr(dev_status), _stream(stream)))
+    else:
+        fn = _block if phase == "both" else _block_rest
+        _check(fn(_ptr(x), rows, dim, mlp_dim, ctypes.byref(weights), code, _ptr(y), _ptr(scratch), scratch.numel(),
+                  _ptr(dev_status), _stream(stream)))
+    return y, scratch
+
+
+def block_region(scratch, offsets, name, rows, cols, dtype):
+    """View of one region of a block's scratch as a [rows, cols] tensor."""
+    return scratch[offsets[name]:offsets[name] + rows * cols * 2].view(dtype).view(rows, cols)
 
 
 def elsa_nm_linear_static(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_: int, N: int, M: int,

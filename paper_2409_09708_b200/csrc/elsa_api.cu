@@ -810,6 +810,274 @@ elsa_status elsa_vit_linears_host(const elsa_host_layer* cfg, int n_layers, elsa
     return ELSA_OK;
 }
 
+}  // extern "C"
+
+/* ---------------------------------------------------------------------------------------------- */
+/* The chained block                                                                              */
+/* ---------------------------------------------------------------------------------------------- */
+namespace elsa {
+namespace {
+
+struct BlockLinear {
+    const elsa_block_linear* w;
+    int in, out;
+    LinearKind kind;
+    void* ws;          // this linear's part of region WORKSPACE
+    bool image_ready;  // its weight image has been enqueued already
+};
+
+struct BlockPlan {
+    size_t off[ELSA_BLOCK_REGIONS];
+    size_t ws_off[4];   // qkv, proj, fc1, fc2 inside region WORKSPACE
+    size_t total;
+};
+
+bool block_plan(int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype, BlockPlan* p)
+{
+    if (!w || rows <= 0 || dim <= 0 || mlp_dim <= 0 || dim % 8 != 0 || mlp_dim % 8 != 0) return false;
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return false;
+    const size_t row = (size_t)rows * 2;
+    const size_t sizes[7] = {row * dim, row * dim * 3, row * dim, row * dim, row * dim, row * mlp_dim, row * dim};
+    size_t at = 0;
+    for (int r = 0; r < 7; ++r) {
+        p->off[r] = at;
+        at += round_up(sizes[r], 256);
+    }
+    p->off[ELSA_BLOCK_WORKSPACE] = at;
+    const elsa_block_linear* lin[4] = {&w->qkv, &w->proj, &w->fc1, &w->fc2};
+    const int ins[4] = {dim, dim, dim, mlp_dim}, outs[4] = {3 * dim, dim, mlp_dim, dim};
+    for (int l = 0; l < 4; ++l) {
+        if (index_bits(lin[l]->M) < 0 || lin[l]->N < 1 || lin[l]->N > lin[l]->M || ins[l] % lin[l]->M != 0) return false;
+        p->ws_off[l] = at;
+        at += round_up(elsa_workspace_bytes(rows, ins[l], outs[l], lin[l]->N, lin[l]->M, dtype), 256);
+    }
+    p->total = at;
+    return true;
+}
+
+// Validation shared by the three entry points; fills the four linears' descriptions.
+elsa_status block_check(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                        const void* y, bool need_y, void* scratch, size_t scratch_bytes, BlockPlan* plan,
+                        BlockLinear (&lin)[4], const DeviceInfo& dev)
+{
+    if (!x || !w || !scratch || (need_y && !y)) return fail(ELSA_ERR_NULL, "x, w, y and scratch must not be NULL");
+    if (rows <= 0 || dim <= 0 || mlp_dim <= 0) return fail(ELSA_ERR_SHAPE, "non-positive size (rows=%d, dim=%d, mlp_dim=%d)", rows, dim, mlp_dim);
+    if (!w->ln1_gain || !w->ln1_bias || !w->ln2_gain || !w->ln2_bias)
+        return fail(ELSA_ERR_NULL, "the LayerNorm gains and biases must not be NULL");
+    if (!(w->eps >= 0.f)) return fail(ELSA_ERR_SHAPE, "eps must not be negative");
+    const elsa_block_linear* src[4] = {&w->qkv, &w->proj, &w->fc1, &w->fc2};
+    const char* names[4] = {"qkv", "proj", "fc1", "fc2"};
+    const int ins[4] = {dim, dim, dim, mlp_dim}, outs[4] = {3 * dim, dim, mlp_dim, dim};
+    for (int l = 0; l < 4; ++l) {
+        elsa_status st = check_level(outs[l], ins[l], src[l]->N, src[l]->M, dtype);
+        if (st == ELSA_OK && !src[l]->vals) st = fail(ELSA_ERR_NULL, "vals must not be NULL");
+        if (st == ELSA_OK && src[l]->N != src[l]->M && !src[l]->idx) st = fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+        if (st == ELSA_OK && (!aligned16(src[l]->vals) || (src[l]->idx && !aligned16(src[l]->idx)) ||
+                              (src[l]->bias && !aligned16(src[l]->bias))))
+            st = fail(ELSA_ERR_ALIGN, "vals, idx and bias must be 16-byte aligned");
+        if (st != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "%s: %s", names[l], msg);
+        }
+    }
+    if (!aligned16(x) || (y && !aligned16(y)) || !aligned16(w->ln1_gain) || !aligned16(w->ln1_bias) ||
+        !aligned16(w->ln2_gain) || !aligned16(w->ln2_bias))
+        return fail(ELSA_ERR_ALIGN, "x, y and the LayerNorm parameters must be 16-byte aligned");
+    if (y && y == x) return fail(ELSA_ERR_ALIGN, "y may not alias x");
+    if (!block_plan(rows, dim, mlp_dim, w, dtype, plan)) return fail(ELSA_ERR_SHAPE, "dim and mlp_dim must be multiples of 8");
+    if (((uintptr_t)scratch & 255u) != 0) return fail(ELSA_ERR_ALIGN, "scratch must be 256-byte aligned");
+    if (scratch_bytes < plan->total)
+        return fail(ELSA_ERR_WORKSPACE, "scratch of %zu bytes needed, %zu given", plan->total, scratch_bytes);
+    for (int l = 0; l < 4; ++l) {
+        lin[l].w = src[l];
+        lin[l].in = ins[l];
+        lin[l].out = outs[l];
+        lin[l].ws = (uint8_t*)scratch + plan->ws_off[l];
+        lin[l].image_ready = false;
+        elsa_status st = pick_kind(rows, outs[l], ins[l], src[l]->N, src[l]->M, dev.sm_count, &lin[l].kind);
+        if (st != ELSA_OK) return st;
+    }
+    return ELSA_OK;
+}
+
+// The weight image of a linear whose kernel takes it ready-made (the others build theirs when they run).
+elsa_status block_image(BlockLinear& L, cudaStream_t stream)
+{
+    const elsa_block_linear& w = *L.w;
+    elsa_status st = ELSA_OK;
+    if (w.N == w.M) return ELSA_OK;
+    if (L.kind == KIND_DENSE_PAIR)
+        st = launch_unpack((const uint16_t*)w.vals, w.idx, L.out, L.in, w.N, w.M, (uint16_t*)L.ws, stream);
+    else if (L.kind == KIND_SPARSE_WS)
+        st = launch_linear_tc_sparse_pair_prepare((const uint16_t*)w.vals, w.idx, L.out, L.in, w.N, w.M, SP24_PERMUTED,
+                                                  L.ws, stream);
+    else if (L.kind == KIND_SPARSE_ST)
+        st = launch_nm_to_sp24((const uint16_t*)w.vals, w.idx, L.out, L.in, w.N, w.M, 128, SP24_TILED, (uint16_t*)L.ws,
+                               (uint8_t*)L.ws + sp24_meta_offset(L.out, L.in), stream);
+    else
+        return ELSA_OK;
+    L.image_ready = st == ELSA_OK;
+    return st;
+}
+
+// Y = act(X Wm^T + bias) [+ residual].  Returns in *residual_left whether the residual is still to be added:
+// then the linear's output went to `tmp` instead of Y, rounded to 16 bits.
+elsa_status block_linear(BlockLinear& L, const uint16_t* X, int rows, elsa_dtype dtype, uint16_t* Y, int act,
+                         const uint16_t* residual, uint16_t* tmp, bool* residual_left, uint32_t* dev_status,
+                         cudaStream_t stream)
+{
+    const elsa_block_linear& w = *L.w;
+    elsa_status st = ELSA_OK;
+    *residual_left = false;
+    if (L.kind == KIND_DENSE_PAIR) {
+        if (w.N != w.M && !L.image_ready && (st = block_image(L, stream)) != ELSA_OK) return st;
+        PairJob job;
+        job.X = X; job.Wd = w.N == w.M ? (const uint16_t*)w.vals : (const uint16_t*)L.ws;
+        job.bias = (const uint16_t*)w.bias; job.Y = Y;
+        job.rows = rows; job.in = L.in; job.out = L.out;
+        job.act = act; job.residual = residual;
+        return launch_linear_tc_pair_group(&job, 1, dtype, dev_status, stream);
+    }
+    *residual_left = residual != nullptr;
+    uint16_t* dst = residual ? tmp : Y;
+    if (L.kind == KIND_SPARSE_WS || L.kind == KIND_SPARSE_ST) {
+        if (!L.image_ready && (st = block_image(L, stream)) != ELSA_OK) return st;
+        SparseJob job;
+        job.X = X; job.bias = (const uint16_t*)w.bias; job.Y = dst; job.workspace = L.ws;
+        job.rows = rows; job.in = L.in; job.out = L.out; job.act = act;
+        return L.kind == KIND_SPARSE_WS ? launch_linear_tc_sparse_ws_group(&job, 1, dtype, dev_status, stream)
+                                        : launch_linear_tc_sparse_st_group(&job, 1, dtype, dev_status, stream);
+    }
+    st = run_linear(X, rows, w.vals, w.N == w.M ? nullptr : w.idx, w.bias, L.out, L.in, w.N, w.M, dtype, dst, L.ws,
+                    dev_status, stream);
+    if (st != ELSA_OK) return st;
+    return launch_act_inplace(dst, (long long)rows * L.out, act, dtype, stream);
+}
+
+elsa_status block_qkv(const uint16_t* x, int rows, int dim, const elsa_block_weights* w, elsa_dtype dtype,
+                      uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4], uint32_t* dev_status,
+                      cudaStream_t stream)
+{
+    uint16_t* x1 = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_X1]);
+    uint16_t* qkv = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_QKV]);
+    elsa_status st = launch_layer_norm(x, nullptr, nullptr, (const uint16_t*)w->ln1_gain, (const uint16_t*)w->ln1_bias,
+                                       x1, rows, dim, w->eps, dtype, stream);
+    if (st != ELSA_OK) return st;
+    bool left = false;
+    return block_linear(lin[0], x1, rows, dtype, qkv, 0, nullptr, nullptr, &left, dev_status, stream);
+}
+
+elsa_status block_rest(const uint16_t* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                       uint16_t* y, uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4],
+                       uint32_t* dev_status, cudaStream_t stream)
+{
+    (void)mlp_dim;
+    const uint16_t* a = (const uint16_t*)(scratch + plan.off[ELSA_BLOCK_A]);
+    uint16_t* x2 = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_X2]);
+    uint16_t* x3 = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_X3]);
+    uint16_t* h = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_H]);
+    uint16_t* t = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_T]);
+    const uint16_t* g2 = (const uint16_t*)w->ln2_gain;
+    const uint16_t* b2 = (const uint16_t*)w->ln2_bias;
+    bool left = false;
+    elsa_status st = block_linear(lin[1], a, rows, dtype, x2, 0, x, t, &left, dev_status, stream);
+    if (st != ELSA_OK) return st;
+    // x2 = x + proj(a) and x3 = LayerNorm2(x2): one pass where the residual is still to be added
+    st = left ? launch_layer_norm(t, x, x2, g2, b2, x3, rows, dim, w->eps, dtype, stream)
+              : launch_layer_norm(x2, nullptr, nullptr, g2, b2, x3, rows, dim, w->eps, dtype, stream);
+    if (st != ELSA_OK) return st;
+    if ((st = block_linear(lin[2], x3, rows, dtype, h, 1, nullptr, nullptr, &left, dev_status, stream)) != ELSA_OK) return st;
+    if ((st = block_linear(lin[3], h, rows, dtype, y, 0, x2, t, &left, dev_status, stream)) != ELSA_OK) return st;
+    if (left) st = launch_layer_norm(t, x2, y, nullptr, nullptr, nullptr, rows, dim, w->eps, dtype, stream);
+    return st;
+}
+
+}  // namespace
+}  // namespace elsa
+
+extern "C" {
+
+size_t elsa_vit_block_scratch_bytes(int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                                    size_t* offsets)
+{
+    BlockPlan plan;
+    if (!block_plan(rows, dim, mlp_dim, w, dtype, &plan)) return 0;
+    if (offsets)
+        for (int r = 0; r < ELSA_BLOCK_REGIONS; ++r) offsets[r] = plan.off[r];
+    return plan.total;
+}
+
+elsa_status elsa_vit_block_qkv(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w,
+                               elsa_dtype dtype, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    BlockPlan plan;
+    BlockLinear lin[4];
+    if ((st = block_check(x, rows, dim, mlp_dim, w, dtype, nullptr, false, scratch, scratch_bytes, &plan, lin, dev)) != ELSA_OK)
+        return st;
+    return block_qkv((const uint16_t*)x, rows, dim, w, dtype, (uint8_t*)scratch, plan, lin, dev_status, (cudaStream_t)stream);
+}
+
+elsa_status elsa_vit_block_rest(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w,
+                                elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status,
+                                void* stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    BlockPlan plan;
+    BlockLinear lin[4];
+    if ((st = block_check(x, rows, dim, mlp_dim, w, dtype, y, true, scratch, scratch_bytes, &plan, lin, dev)) != ELSA_OK)
+        return st;
+    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, (uint8_t*)scratch, plan, lin,
+                      dev_status, (cudaStream_t)stream);
+}
+
+elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                           void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    BlockPlan plan;
+    BlockLinear lin[4];
+    if ((st = block_check(x, rows, dim, mlp_dim, w, dtype, y, true, scratch, scratch_bytes, &plan, lin, dev)) != ELSA_OK)
+        return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    // The four weight images do not depend on x: they are built on the library's side stream while the first
+    // LayerNorm runs on the caller's, which waits for them before the first linear.
+    bool any_image = false;
+    for (int l = 0; l < 4; ++l)
+        any_image = any_image || (lin[l].w->N != lin[l].w->M && (lin[l].kind == KIND_DENSE_PAIR ||
+                                                                  lin[l].kind == KIND_SPARSE_WS || lin[l].kind == KIND_SPARSE_ST));
+    SidePipe* side = nullptr;
+    if (any_image) {
+        if ((st = side_pipe(dev.device, &side)) != ELSA_OK) return st;
+        cudaError_t e = cudaEventRecord(side->fork, stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(side->stream, side->fork, 0);
+        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "forking the image stream: %s", cudaGetErrorString(e));
+        for (int l = 0; l < 4 && st == ELSA_OK; ++l) st = block_image(lin[l], side->stream);
+        e = cudaEventRecord(side->join, side->stream);   // joined even after a failed launch: the fork must not dangle
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(stream, side->join, 0);
+        if (st != ELSA_OK) return st;
+        if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "joining the image stream: %s", cudaGetErrorString(e));
+    }
+    uint8_t* s8 = (uint8_t*)scratch;
+    if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream)) != ELSA_OK) return st;
+    // the stated stand-in for attention: a = V
+    if ((st = launch_copy_columns((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]),
+                                  rows, 3 * dim, 2 * dim, dim, stream)) != ELSA_OK)
+        return st;
+    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream);
+}
+
+}  // extern "C"
+
+extern "C" {
+
 elsa_status elsa_set_linear_variant(elsa_variant v)
 {
     if (v != ELSA_VARIANT_AUTO && v != ELSA_VARIANT_SIMT && v != ELSA_VARIANT_TC_DENSE && v != ELSA_VARIANT_TC_PAIR &&

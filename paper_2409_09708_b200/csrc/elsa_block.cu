@@ -1,0 +1,243 @@
+// Elementwise and row-wise kernels of the transformer block around the four N:M linears (ELSA, Sec. 3: the
+// pruned modules qkv, proj, fc1, fc2 sit in the standard pre-norm ViT block; Sec. 4.2 measures whole models):
+// LayerNorm, residual add (alone or followed by LayerNorm in the same pass), GELU in place, and the copy of a
+// column range.  All of them are HBM-bound streaming kernels: 16-byte loads and stores, one warp per token row
+// for the row-wise ones, fp32 arithmetic, one rounding to the 16-bit type per stored value.
+#include "elsa_internal.h"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+namespace elsa {
+namespace {
+
+constexpr int kWarpsPerBlock = 8;
+constexpr int kCacheVecs = 4;   // 16-byte vectors of a row each lane keeps in registers (rows up to 1024 values)
+
+template <bool kBf16>
+__device__ __forceinline__ float2 unpack2(uint32_t u)
+{
+    if constexpr (kBf16) {
+        return make_float2(__uint_as_float(u << 16), __uint_as_float(u & 0xffff0000u));
+    } else {
+        __half2 h = *reinterpret_cast<__half2*>(&u);
+        return __half22float2(h);
+    }
+}
+
+template <bool kBf16>
+__device__ __forceinline__ uint32_t pack2_rn(float a, float b)
+{
+    if constexpr (kBf16) {
+        __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+        return *reinterpret_cast<uint32_t*>(&v);
+    } else {
+        __half2 v = __floats2half2_rn(a, b);
+        return *reinterpret_cast<uint32_t*>(&v);
+    }
+}
+
+template <bool kBf16>
+__device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8])
+{
+    const float2 a = unpack2<kBf16>(u.x), b = unpack2<kBf16>(u.y), c = unpack2<kBf16>(u.z), d = unpack2<kBf16>(u.w);
+    f[0] = a.x; f[1] = a.y; f[2] = b.x; f[3] = b.y; f[4] = c.x; f[5] = c.y; f[6] = d.x; f[7] = d.y;
+}
+
+template <bool kBf16>
+__device__ __forceinline__ uint4 pack8(const float (&f)[8])
+{
+    return make_uint4(pack2_rn<kBf16>(f[0], f[1]), pack2_rn<kBf16>(f[2], f[3]), pack2_rn<kBf16>(f[4], f[5]),
+                      pack2_rn<kBf16>(f[6], f[7]));
+}
+
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// One warp per row.  kAdd: the row is S = round16(A + R), written to S (which may be A's or R's own buffer:
+// each lane reads its vectors of a row before it writes them).  The statistics are those of the stored 16-bit
+// row (for kAdd: of S as rounded), mean first, then the biased variance about it; eps sits inside the root.
+// Yn = round16((s - mean) / sqrt(var + eps) * gain + beta), or no normalised output when Yn is NULL.
+template <bool kBf16, bool kAdd>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* __restrict__ gain,
+                  const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, int dim, float eps)
+{
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const int lane = threadIdx.x & 31;
+    const int vecs = dim >> 3;
+    const float inv_dim = 1.0f / (float)dim;
+    for (int row = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); row < rows; row += gridDim.x * kWarpsPerBlock) {
+        const uint4* a4 = reinterpret_cast<const uint4*>(A + (size_t)row * (size_t)dim);
+        const uint4* r4 = kAdd ? reinterpret_cast<const uint4*>(R + (size_t)row * (size_t)dim) : nullptr;
+        uint4* s4 = kAdd ? reinterpret_cast<uint4*>(S + (size_t)row * (size_t)dim) : nullptr;
+        uint4 cache[kCacheVecs];
+        // the row as stored: loaded (and, for kAdd, summed, rounded and written) once
+        auto fetch = [&](int v) -> uint4 {
+            uint4 u = a4[v];
+            if constexpr (kAdd) {
+                const uint4 w = r4[v];
+                float fa[8], fr[8];
+                unpack8<kBf16>(u, fa);
+                unpack8<kBf16>(w, fr);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) fa[e] += fr[e];
+                u = pack8<kBf16>(fa);
+                s4[v] = u;
+            }
+            return u;
+        };
+        // a vector past the register cache is read back from where the row is stored
+        auto again = [&](int v) -> uint4 { return kAdd ? s4[v] : a4[v]; };
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < kCacheVecs; ++c) {
+            const int v = lane + 32 * c;
+            if (v < vecs) {
+                cache[c] = fetch(v);
+                float f[8];
+                unpack8<kBf16>(cache[c], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sum += f[e];
+            }
+        }
+        for (int v = lane + 32 * kCacheVecs; v < vecs; v += 32) {
+            float f[8];
+            unpack8<kBf16>(fetch(v), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sum += f[e];
+        }
+        if (Yn == nullptr) continue;
+        const float mean = warp_sum(sum) * inv_dim;
+        float sq = 0.f;
+#pragma unroll
+        for (int c = 0; c < kCacheVecs; ++c) {
+            if (lane + 32 * c < vecs) {
+                float f[8];
+                unpack8<kBf16>(cache[c], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sq += (f[e] - mean) * (f[e] - mean);
+            }
+        }
+        for (int v = lane + 32 * kCacheVecs; v < vecs; v += 32) {
+            float f[8];
+            unpack8<kBf16>(again(v), f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) sq += (f[e] - mean) * (f[e] - mean);
+        }
+        const float rstd = 1.0f / sqrtf(warp_sum(sq) * inv_dim + eps);
+        uint4* y4 = reinterpret_cast<uint4*>(Yn + (size_t)row * (size_t)dim);
+        auto emit = [&](int v, const uint4& u) {
+            float f[8], g[8], b[8];
+            unpack8<kBf16>(u, f);
+            unpack8<kBf16>(__ldg(reinterpret_cast<const uint4*>(gain) + v), g);
+            unpack8<kBf16>(__ldg(reinterpret_cast<const uint4*>(beta) + v), b);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) f[e] = (f[e] - mean) * rstd * g[e] + b[e];
+            y4[v] = pack8<kBf16>(f);
+        };
+#pragma unroll
+        for (int c = 0; c < kCacheVecs; ++c)
+            if (lane + 32 * c < vecs) emit(lane + 32 * c, cache[c]);
+        for (int v = lane + 32 * kCacheVecs; v < vecs; v += 32) emit(v, again(v));
+    }
+}
+
+// Y = act(Y) in place, eight values per thread and step.
+template <bool kBf16>
+__global__ void __launch_bounds__(256) act_inplace_kernel(uint16_t* Y, long long vecs, int act)
+{
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    uint4* y4 = reinterpret_cast<uint4*>(Y);
+    for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < vecs; v += (long long)gridDim.x * blockDim.x) {
+        float f[8];
+        unpack8<kBf16>(y4[v], f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            f[e] = act == 1 ? 0.5f * f[e] * (1.0f + erff(f[e] * 0.70710678118654752f)) : f[e];
+        y4[v] = pack8<kBf16>(f);
+    }
+}
+
+// dst[r][0 .. cols) = src[r][col0 .. col0 + cols), rows of src_ld values; everything in units of eight values.
+__global__ void __launch_bounds__(256)
+copy_columns_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int rows, int src_ld, int col0, int cols)
+{
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const int vpr = cols >> 3;
+    const long long total = (long long)rows * vpr;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int r = (int)(i / vpr), v = (int)(i % vpr);
+        reinterpret_cast<uint4*>(dst + (size_t)r * (size_t)cols)[v] =
+            __ldg(reinterpret_cast<const uint4*>(src + (size_t)r * (size_t)src_ld + col0) + v);
+    }
+}
+
+unsigned streaming_grid(long long work_items, int per_block, const DeviceInfo& dev)
+{
+    long long blocks = (work_items + per_block - 1) / per_block;
+    const long long cap = (long long)dev.sm_count * 8;   // one wave of resident blocks; the kernels loop
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    return (unsigned)blocks;
+}
+
+}  // namespace
+
+elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* gain,
+                              const uint16_t* beta, uint16_t* Yn, int rows, int dim, float eps, elsa_dtype dtype,
+                              cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (rows <= 0) return ELSA_OK;
+    const unsigned grid = streaming_grid(rows, kWarpsPerBlock, dev);
+    const dim3 block(kWarpsPerBlock * 32);
+    const bool add = R != nullptr;
+    ProfileScope scope(ELSA_KERNEL_BLOCK_ROWWISE, stream);
+    if (dtype == ELSA_BF16) {
+        if (add) launch_pdl(layer_norm_kernel<true, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+        else launch_pdl(layer_norm_kernel<true, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+    } else {
+        if (add) launch_pdl(layer_norm_kernel<false, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+        else launch_pdl(layer_norm_kernel<false, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+    }
+    return launched(add ? "residual_add_layer_norm" : "layer_norm");
+}
+
+elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype dtype, cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (count <= 0 || act == 0) return ELSA_OK;
+    const long long vecs = count / 8;
+    const unsigned grid = streaming_grid(vecs, 256, dev);
+    ProfileScope scope(ELSA_KERNEL_BLOCK_ROWWISE, stream);
+    if (dtype == ELSA_BF16) launch_pdl(act_inplace_kernel<true>, dim3(grid), dim3(256), 0, stream, 1, Y, vecs, act);
+    else launch_pdl(act_inplace_kernel<false>, dim3(grid), dim3(256), 0, stream, 1, Y, vecs, act);
+    return launched("act_inplace");
+}
+
+elsa_status launch_copy_columns(const uint16_t* src, uint16_t* dst, int rows, int src_ld, int col0, int cols,
+                                cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (rows <= 0 || cols <= 0) return ELSA_OK;
+    const unsigned grid = streaming_grid((long long)rows * (cols / 8), 256, dev);
+    ProfileScope scope(ELSA_KERNEL_BLOCK_ROWWISE, stream);
+    launch_pdl(copy_columns_kernel, dim3(grid), dim3(256), 0, stream, 1, src, dst, rows, src_ld, col0, cols);
+    return launched("copy_columns");
+}
+
+}  // namespace elsa

@@ -128,6 +128,7 @@ struct SparseJob {
     uint16_t* Y;
     const void* workspace;
     int rows, in, out;
+    int act = 0;      // epilogue activation: 0 none, 1 GELU (weight-stationary and streaming kernels only)
 };
 int linear_tc_sparse_pair_group_max();
 elsa_status launch_linear_tc_sparse_pair_prepare(const uint16_t* vals, const uint32_t* idx, int out, int in, int N, int M,
@@ -154,6 +155,16 @@ elsa_status launch_linear_tc_sparse_st_group(const SparseJob* jobs, int n, elsa_
 elsa_status launch_linear_tc_sparse_st(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
                                        const uint16_t* bias, int out, int in, int N, int M, elsa_dtype dtype, uint16_t* Y,
                                        void* workspace, uint32_t* dev_status, cudaStream_t stream);
+// Row-wise and elementwise kernels of the chained block (16-bit tensors, fp32 arithmetic, one rounding).
+// R == NULL: Yn = LayerNorm(A).  R != NULL: S = A + R, and Yn = LayerNorm(S) unless Yn is NULL.  dim % 8 == 0.
+elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* gain,
+                              const uint16_t* beta, uint16_t* Yn, int rows, int dim, float eps, elsa_dtype dtype,
+                              cudaStream_t stream);
+// Y = act(Y) over `count` values (count % 8 == 0); act as in the GEMM epilogues.
+elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype dtype, cudaStream_t stream);
+// dst[r][0 .. cols) = src[r][col0 .. col0 + cols); src rows of src_ld values; all multiples of 8.
+elsa_status launch_copy_columns(const uint16_t* src, uint16_t* dst, int rows, int src_ld, int col0, int cols,
+                                cudaStream_t stream);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
 constexpr int kMaxLevels = 16;
 struct LevelTable {
@@ -201,6 +212,8 @@ struct PairJob {
     int rows, in, out;
     const float* w_scale = nullptr;   // INT8 form only
     float x_scale = 0.f;
+    int act = 0;                          // epilogue activation: 0 none, 1 GELU (applied to acc + bias)
+    const uint16_t* residual = nullptr;   // [rows][out], added after the activation, before the one rounding
 };
 int linear_tc_pair_group_max();
 elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,

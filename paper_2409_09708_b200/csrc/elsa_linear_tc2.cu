@@ -67,6 +67,8 @@ struct alignas(64) PairLayer {
     const uint16_t* bias;
     const float* w_scale;   // INT8 form only: per-feature weight scale, and the activations' scale
     float x_scale;
+    int act;                    // epilogue activation (0 none, 1 GELU) on acc + bias
+    const uint16_t* residual;   // [rows][out] added after the activation, or NULL
 };
 
 template <int kMaxLayers>
@@ -79,15 +81,21 @@ struct PairGroup {
 };
 
 constexpr int kStageBytesMax = kATileBytes + (kMaxBlockN / 2) * kBlockK * 2;   // stage slots sized for BN = 256
+// Forms of the kernel: plain (acc + bias), INT8 (integer operands, scaled in the epilogue), fused (activation and
+// residual added in the epilogue). Separate instantiations, so the plain form pays nothing for the other two.
+constexpr int kFormPlain = 0, kFormInt8 = 1, kFormFused = 2;
 constexpr int kGroupMax = 72;   // layers per grouped launch (kernel parameters are limited to 32 KB)
 
 // kInt8: operands are signed 8-bit integers (rows of 128 elements per 128-byte swizzle row, K = 32 per MMA,
 // int32 accumulators); the epilogue turns an accumulator into float, multiplies by x_scale * w_scale[feature],
 // adds the bias, each in fp32 with one rounding per operation, and rounds once to the 16-bit output type.
-template <bool kBf16, bool kInt8, int kMaxLayers>
+template <bool kBf16, int kForm, int kMaxLayers>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 {
+    constexpr bool kInt8 = kForm == kFormInt8;     // 8-bit integer operands, scales in the epilogue
+    constexpr bool kFused = kForm == kFormFused;   // activation and residual in the epilogue
+
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -285,6 +293,10 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             const uint32_t bias_cur = smem_base + bias_off + bias_b * (kMaxBlockN * 2);
             const uint32_t scale_cur = smem_base + scale_off + bias_b * (kMaxBlockN * 4);
             (void)scale_cur;
+            const int l_act = kFused ? L.act : 0;
+            const uint16_t* l_res = kFused ? L.residual : nullptr;
+            (void)l_act;
+            (void)l_res;
             bool ok = mbar_wait(bias_full_bar + 8 * bias_b, (it >> 1) & 1u, abort_flag, p.dev_status, 6);
             ok = ok && mbar_wait(tmem_full_bar + 8 * acc, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
@@ -302,6 +314,18 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                         uint32_t bw[4];
                         asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(bw[0]), "=r"(bw[1]), "=r"(bw[2]), "=r"(bw[3])
                                      : "r"(bias_cur + (uint32_t)(c * kEpiCols * 2 + (2 * h + g) * 16)));
+                        // this lane's row of the residual, eight values (a whole load lies inside or outside the row)
+                        uint32_t res[4] = {0u, 0u, 0u, 0u};
+                        if constexpr (kFused) {
+                            if (l_res != nullptr) {
+                                const int row = row0 + lane;
+                                const int col = n0 + c * kEpiCols + (2 * h + g) * 8;
+                                if (row < l_rows && col < l_out) {
+                                    const uint4 u = __ldg(reinterpret_cast<const uint4*>(l_res + (size_t)row * (size_t)l_out + col));
+                                    res[0] = u.x; res[1] = u.y; res[2] = u.z; res[3] = u.w;
+                                }
+                            }
+                        }
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float2 bv = raw2_to_float2<kBf16>(bw[e]);
@@ -314,7 +338,14 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                                 const float vy = __fadd_rn(__fmul_rn((float)(int)r[2 * j + 1], sy), bv.y);
                                 pk[4 * g + e] = pack2<kBf16>(vx, vy);
                             } else {
-                                pk[4 * g + e] = pack2<kBf16>(__uint_as_float(r[2 * j]) + bv.x, __uint_as_float(r[2 * j + 1]) + bv.y);
+                                float vx = __uint_as_float(r[2 * j]) + bv.x;
+                                float vy = __uint_as_float(r[2 * j + 1]) + bv.y;
+                                if constexpr (kFused) {
+                                    const float2 rv = raw2_to_float2<kBf16>(res[e]);   // zeros without a residual
+                                    vx = apply_act(vx, l_act) + rv.x;
+                                    vy = apply_act(vy, l_act) + rv.y;
+                                }
+                                pk[4 * g + e] = pack2<kBf16>(vx, vy);
                             }
                         }
                     }
@@ -413,10 +444,11 @@ bool linear_tc_pair_suits(int rows, int out, int sm_count)
 
 namespace {
 
-template <bool kBf16, bool kInt8, int kMaxLayers>
+template <bool kBf16, int kForm, int kMaxLayers>
 elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
                          const DeviceInfo& dev)
 {
+    constexpr bool kInt8 = kForm == kFormInt8;
     static PairGroup<kMaxLayers> g;   // host staging of the kernel parameters (single-threaded launch path)
     static std::mutex g_mutex;
     std::lock_guard<std::mutex> lock(g_mutex);
@@ -433,6 +465,8 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
         L.bias = j.bias;
         L.w_scale = j.w_scale;
         L.x_scale = j.x_scale;
+        L.act = j.act;
+        L.residual = j.residual;
         elsa_status st;
         if constexpr (kInt8) {
             L.num_k_blocks = (j.in + 2 * kBlockK - 1) / (2 * kBlockK);
@@ -469,7 +503,7 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
     g.stages = stages;
     const size_t smem = (size_t)stages * kStageBytesMax + fixed;
 
-    auto kernel = linear_tc_pair_kernel<kBf16, kInt8, kMaxLayers>;
+    auto kernel = linear_tc_pair_kernel<kBf16, kForm, kMaxLayers>;
     static std::atomic<int> max_pairs[64];   // zero-initialised; racing first calls compute the same value
     const int slot = dev.device & 63;
     if (max_pairs[slot].load(std::memory_order_acquire) == 0) {
@@ -518,11 +552,20 @@ elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype d
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    bool fused = false;
+    for (int i = 0; i < n; ++i) fused = fused || jobs[i].act != 0 || jobs[i].residual != nullptr;
+    if (fused) {
+        if (n == 1)
+            return dtype == ELSA_BF16 ? launch_group<true, kFormFused, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                      : launch_group<false, kFormFused, 1>(jobs, 1, dtype, dev_status, stream, dev);
+        return dtype == ELSA_BF16 ? launch_group<true, kFormFused, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                                  : launch_group<false, kFormFused, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+    }
     if (n == 1)
-        return dtype == ELSA_BF16 ? launch_group<true, false, 1>(jobs, 1, dtype, dev_status, stream, dev)
-                                  : launch_group<false, false, 1>(jobs, 1, dtype, dev_status, stream, dev);
-    return dtype == ELSA_BF16 ? launch_group<true, false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
-                              : launch_group<false, false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+        return dtype == ELSA_BF16 ? launch_group<true, kFormPlain, 1>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_group<false, kFormPlain, 1>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_group<true, kFormPlain, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_group<false, kFormPlain, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
 }
 
 // INT8 form (one layer per launch): X and Wd hold signed 8-bit integers, Y is 16-bit.
@@ -537,8 +580,8 @@ elsa_status launch_linear_tc_pair_i8(const int8_t* X, int rows, const int8_t* Wd
     job.X = (const uint16_t*)X; job.Wd = (const uint16_t*)Wd; job.bias = bias; job.Y = Y;
     job.rows = rows; job.in = in; job.out = out;
     job.w_scale = w_scale; job.x_scale = x_scale;
-    return dtype == ELSA_BF16 ? launch_group<true, true, 1>(&job, 1, dtype, dev_status, stream, dev)
-                              : launch_group<false, true, 1>(&job, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_group<true, kFormInt8, 1>(&job, 1, dtype, dev_status, stream, dev)
+                              : launch_group<false, kFormInt8, 1>(&job, 1, dtype, dev_status, stream, dev);
 }
 
 elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias, int out,

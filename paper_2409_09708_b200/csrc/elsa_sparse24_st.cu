@@ -76,6 +76,7 @@ struct alignas(64) StLayer {
     int tile_begin;    // index of this layer's first tile in the launch's sequence
     int num_chunks;    // ceil(in / 256)
     int num_k_blocks;  // in / 128
+    int act;           // epilogue activation (0 none, 1 GELU) on acc + bias
 };
 
 constexpr int kGroupMax = 84;   // layers per launch (kernel parameters are limited to 32 KB)
@@ -338,6 +339,7 @@ linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
             const int f = f0 + feat_in_quarter;
             const int l_rows = L.rows, l_out = L.out;
             const float bias_f = (L.bias != nullptr && f < l_out) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
+            const int l_act = L.act;
             bool ok = mbar_wait(tmem_full_bar, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -372,7 +374,8 @@ linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
                 for (int i = 0; i < kRoundSteps; ++i)
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        w[i][j] = pack2<kBf16>(__uint_as_float(rr[i][2 * j]) + bias_f, __uint_as_float(rr[i][2 * j + 1]) + bias_f);
+                        w[i][j] = pack2<kBf16>(apply_act(__uint_as_float(rr[i][2 * j]) + bias_f, l_act),
+                                               apply_act(__uint_as_float(rr[i][2 * j + 1]) + bias_f, l_act));
                 if (rd + 1 < kRounds) {
 #pragma unroll
                     for (int i = 0; i < kRoundSteps; ++i)
@@ -461,6 +464,7 @@ elsa_status launch_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         L.num_chunks = (j.in + kChunkK - 1) / kChunkK;
         L.num_k_blocks = j.in / 128;
         L.bias = j.bias;
+        L.act = j.act;
         L.a_img = (const uint8_t*)j.workspace;
         L.meta = (const uint8_t*)j.workspace + sp24_meta_offset(j.out, j.in);
         elsa_status st;

@@ -67,8 +67,8 @@ struct alignas(64) WsLayer {
     int tiles_f;       // F
     int groups;        // G
     int row_tiles;     // ceil(rows / nt)
-    int num_k_blocks;  // in / 128 (metadata blocks per 128 features)
     uint32_t idesc;
+    int act;           // epilogue activation (0 none, 1 GELU) on acc + bias
 };
 
 constexpr int kGroupMax = 92;   // layers per launch (kernel parameters are limited to 32 KB)
@@ -308,8 +308,8 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                     tmem_st_32x32b_x16(a_col0 + (uint32_t)(16 * c), v);
                 }
                 const uint4* e_blk = reinterpret_cast<const uint4*>(L.meta) +
-                                     (size_t)(blk_ok ? ft128 : 0) * (size_t)L.num_k_blocks * 128 + (size_t)(q * 32 + lane);
-                for (int kb = part; kb < L.num_k_blocks; kb += kEpiParts) {
+                                     (size_t)(blk_ok ? ft128 : 0) * (size_t)(L.in / kBlockK) * 128 + (size_t)(q * 32 + lane);
+                for (int kb = part; kb < L.in / kBlockK; kb += kEpiParts) {
                     uint4 t = make_uint4(0u, 0u, 0u, 0u);
                     if (blk_ok) t = __ldg(e_blk + (size_t)kb * 128);
                     uint32_t v[4] = {t.x, t.y, t.z, t.w};
@@ -321,6 +321,7 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                 if (lane == 0) mbar_arrive_cluster_release(w_ready_remote);
             }
             const float bias_f = (L.bias != nullptr && f_ok) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
+            const int l_act = L.act;
             // this warp's run of token columns: steps of 16, [first_step, first_step + my_steps)
             const int total_steps = nt / kStepCols;
             const int first_step = part * L.steps_per_warp;
@@ -355,7 +356,8 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                     uint32_t w[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        w[j] = pack2<kBf16>(__uint_as_float(rr[s][2 * j]) + bias_f, __uint_as_float(rr[s][2 * j + 1]) + bias_f);
+                        w[j] = pack2<kBf16>(apply_act(__uint_as_float(rr[s][2 * j]) + bias_f, l_act),
+                                            apply_act(__uint_as_float(rr[s][2 * j + 1]) + bias_f, l_act));
                     stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64), w[0], w[1], w[2], w[3]);
                     stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64 + 512), w[4], w[5], w[6], w[7]);
                 }
@@ -466,8 +468,8 @@ elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint
         L.groups = pairs / L.tiles_f;
         if (L.groups > L.row_tiles) L.groups = L.row_tiles;
         if (L.groups * L.tiles_f > used_pairs) used_pairs = L.groups * L.tiles_f;
-        L.num_k_blocks = j.in / kBlockK;
         L.bias = j.bias;
+        L.act = j.act;
         L.a_img = (const uint16_t*)j.workspace;
         L.meta = (const uint8_t*)j.workspace + sp24_meta_offset(j.out, j.in);
         // sparse flag, fp32 accumulate, A and B of type fmt, K-major, N = nt, M = 256 over the pair

@@ -204,6 +204,12 @@ __device__ __forceinline__ float2 raw2_to_float2(uint32_t w)
     else return __half22float2(*reinterpret_cast<const __half2*>(&w));
 }
 
+// GELU in its exact form, v * Phi(v) (the activation of the ViT MLP), in fp32.
+__device__ __forceinline__ float gelu_exact(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752f)); }
+
+// Epilogue activation of a layer: 0 none, 1 GELU.
+__device__ __forceinline__ float apply_act(float v, int act) { return act == 1 ? gelu_exact(v) : v; }
+
 template <bool kBf16>
 __device__ __forceinline__ float bias_to_float(uint16_t u)
 {

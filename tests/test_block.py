@@ -1,0 +1,254 @@
+"""The chained transformer block (elsa_vit_block and its two phases) against oracle/elsa_block_oracle.py.
+
+Two comparisons per case.  Stage by stage: every stage's stored 16-bit result against the oracle's fp64 result of
+that stage computed from the library's own stored inputs, so each kernel is held to one rounding.  Whole chain:
+the library's results against block_forward from x alone, where the stages' roundings compound.
+
+Tolerance of a stage, |got - ref| <= u * (|ref| + |lin|) + 5e-4 with u one unit in the last place of the 16-bit
+type relative to the value (2^-7 bf16, 2^-10 fp16): the library computes in fp32 and rounds once where the
+oracle computes in fp64 and rounds once, so the two can land on neighbouring 16-bit values; |lin| is the
+magnitude of the linear's own output at the stages that add a residual or apply GELU (a kernel whose epilogue
+cannot take the residual or the activation rounds the linear's output first; GELU's slope is at most 1.13); 5e-4 is above the fp32 accumulation bound
+K * 2^-24 * max|x w| ~ 1e-4 of the longest reduction here.  In the chain a stage also inherits the rounding
+of its inputs, which LayerNorm and the linears carry from the large elements of a row to its small ones: each
+element is held to four times the stage tolerance with the largest |ref| of its row added to |ref|, and every
+stage as a whole to a relative Frobenius error of 5e-3 (the bound of the single linears' parity tests).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import elsa_block_oracle as bo
+from oracle import elsa_oracle as eo
+from paper_2409_09708_b200 import synth
+
+STAGES = ("x1", "qkv", "a", "x2", "x3", "h", "y")
+NAMES = ("qkv", "proj", "fc1", "fc2")
+
+
+def shapes_of(dim, mlp):
+    return {"qkv": (3 * dim, dim), "proj": (dim, dim), "fc1": (mlp, dim), "fc2": (dim, mlp)}
+
+
+def make_params(dim, mlp, levels, dtype, seed):
+    """Host tensors of one block: weights N(0, 0.02 .. 0.08), biases, LayerNorm gains near 1."""
+    host = {}
+    for i, (name, (o, k)) in enumerate(shapes_of(dim, mlp).items()):
+        host["W_" + name] = synth.randn((o, k), seed + i, 2.0 / np.sqrt(k), dtype)
+        host["b_" + name] = synth.randn((o,), seed + 10 + i, 0.02, dtype)
+    for i, name in enumerate(("ln1_g", "ln1_b", "ln2_g", "ln2_b")):
+        t = synth.randn((dim,), seed + 20 + i, 0.1, dtype).float() + (1.0 if name.endswith("g") else 0.0)
+        host[name] = t.to(dtype)
+    p = {k: synth.bits(v) for k, v in host.items()}
+    for name in NAMES:
+        p["level_" + name] = levels[name]
+    return host, p
+
+
+def test_scratch_layout_is_host_arithmetic():
+    from paper_2409_09708_b200 import build
+    build.build()
+    from paper_2409_09708_b200 import binding as lib
+    w = lib.ElsaBlockWeights()
+    for name, (N, M) in zip(NAMES, [(8, 8), (2, 8), (4, 8), (1, 8)]):
+        setattr(w, name, lib.ElsaBlockLinear(None, None, None, N, M))
+    rows, dim, mlp = 1000, 768, 3072
+    total, off = lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, lib.BF16)
+    sizes = {"x1": dim, "qkv": 3 * dim, "a": dim, "x2": dim, "x3": dim, "h": mlp, "t": dim}
+    at = 0
+    for name in lib.BLOCK_REGIONS[:-1]:
+        assert off[name] == at and at % 256 == 0
+        at += -(-rows * sizes[name] * 2 // 256) * 256
+    assert off["workspace"] == at
+    ws = sum(-(-lib.elsa_workspace_bytes(rows, k, o, N, M, lib.BF16) // 256) * 256
+             for (o, k), (N, M) in zip(shapes_of(dim, mlp).values(), [(8, 8), (2, 8), (4, 8), (1, 8)]))
+    assert total == at + ws
+    assert lib.elsa_vit_block_scratch_bytes(rows, 772, mlp, w, lib.BF16)[0] == 0       # dim % 8 != 0
+    w.fc2 = lib.ElsaBlockLinear(None, None, None, 9, 8)
+    assert lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, lib.BF16)[0] == 0       # N > M
+
+
+# ------------------------------------------------------------------------------------------------ GPU
+
+def run_block(lib, x, host, levels, mlp, variant=None, phase="both"):
+    """Compresses the four weights, runs the block; returns ({stage: fp64 array}, {stage: bits}, weights)."""
+    dtype = x.dtype
+    rows, dim = x.shape
+    dev = {k: v.cuda() for k, v in host.items()}
+    lin = {}
+    for name in NAMES:
+        N, M = levels[name]
+        vals, idx = lib.elsa_nm_compress(dev["W_" + name], N, M)
+        lin[name] = (vals, idx, dev["b_" + name], N, M)
+    w, keep = lib.make_block_weights(dev["ln1_g"], dev["ln1_b"], dev["ln2_g"], dev["ln2_b"], lin, eps=1e-6)
+    code = lib.dtype_code(dtype)
+    total, off = lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, code)
+    scratch = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    xd = x.cuda()
+    if variant is not None:
+        lib.elsa_set_linear_variant(variant)
+    try:
+        if phase == "both":
+            y, _ = lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status)
+        else:
+            lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status, phase="qkv")
+            qkv = lib.block_region(scratch, off, "qkv", rows, 3 * dim, dtype)
+            lib.block_region(scratch, off, "a", rows, dim, dtype).copy_(qkv[:, 2 * dim:])   # the caller's "attention"
+            y, _ = lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status, phase="rest")
+        torch.cuda.synchronize()
+    finally:
+        lib.elsa_set_linear_variant(lib.VARIANT_AUTO)
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    cols = {"x1": dim, "qkv": 3 * dim, "a": dim, "x2": dim, "x3": dim, "h": mlp}
+    got = {s: lib.block_region(scratch, off, s, rows, cols[s], dtype).cpu() for s in cols}
+    got["y"] = y.cpu()
+    return got
+
+
+def stage_tolerance(ref, lin, dtype):
+    u = 2.0 ** -7 if dtype == torch.bfloat16 else 2.0 ** -10
+    return u * (np.abs(ref) + (0 if lin is None else np.abs(lin))) + 5e-4
+
+
+def check_rows(got, x, p, dtype, rows_idx):
+    """Both comparisons on the given rows (the block treats token rows independently)."""
+    code = eo.F16 if dtype == torch.float16 else eo.BF16
+    f64 = lambda t: t[rows_idx].to(torch.float64).numpy()
+    bits = lambda t: synth.bits(t[rows_idx].contiguous())
+    g = {s: f64(got[s]) for s in STAGES}
+    for s in STAGES:
+        assert np.isfinite(g[s]).all(), s
+    dim = x.shape[1]
+    r16 = lambda a: bo._round16(a, dtype)
+    pf = lambda key: torch.from_numpy(p[key].view(np.int16)).view(dtype).to(torch.float64).numpy()
+    lin = lambda name, inp: bo.sparse_linear(inp, p["W_" + name], p["b_" + name], *p["level_" + name], code)
+    xs = f64(x)
+    # stage by stage, from the library's own stored inputs
+    proj, fc1, fc2 = lin("proj", g["a"]), lin("fc1", g["x3"]), lin("fc2", g["h"])
+    stage_ref = {
+        "x1": (r16(bo.layer_norm(xs, pf("ln1_g"), pf("ln1_b"), 1e-6)), None),
+        "qkv": (r16(lin("qkv", g["x1"])), None),
+        "x2": (r16(xs + proj), proj),
+        "x3": (r16(bo.layer_norm(g["x2"], pf("ln2_g"), pf("ln2_b"), 1e-6)), None),
+        "h": (r16(bo.gelu(fc1)), 1.13 * fc1),
+        "y": (r16(g["x2"] + fc2), fc2),
+    }
+    assert np.array_equal(bits(got["a"]), bits(got["qkv"][:, 2 * dim:3 * dim]))      # the stand-in copies V through
+    for s, (ref, mag) in stage_ref.items():
+        err = np.abs(g[s] - ref)
+        tol = stage_tolerance(ref, mag, dtype)
+        worst = (err - tol).argmax()
+        assert (err <= tol).all(), "stage %s: error %g at tolerance %g" % (s, err.flat[worst], tol.flat[worst])
+    # the whole chain from x alone
+    chain = bo.block_forward(bits(x), p, code, eps=1e-6)
+    for s in STAGES:
+        mag = chain["x2"] - xs if s == "x2" else chain["y"] - chain["x2"] if s == "y" else 1.13 * fc1 if s == "h" else None
+        err = np.abs(g[s] - chain[s])
+        row_max = np.abs(chain[s]).max(axis=1, keepdims=True)
+        tol = 4 * stage_tolerance(chain[s], row_max if mag is None else np.abs(mag) + row_max, dtype)
+        worst = (err - tol).argmax()
+        assert (err <= tol).all(), "chain %s: error %g at tolerance %g" % (s, err.flat[worst], tol.flat[worst])
+        assert np.linalg.norm(g[s] - chain[s]) <= 5e-3 * np.linalg.norm(chain[s]), s
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2409_09708_b200 import build
+    build.build()
+    from paper_2409_09708_b200 import binding
+    return binding
+
+
+SPARSE_LEVELS = {"qkv": (2, 8), "proj": (1, 8), "fc1": (2, 4), "fc2": (1, 4)}
+MIXED_LEVELS = {"qkv": (8, 8), "proj": (4, 8), "fc1": (2, 8), "fc2": (3, 4)}
+SMALL = [("simt", MIXED_LEVELS), ("tc_dense", MIXED_LEVELS), ("tc_pair", MIXED_LEVELS), ("tc_pair", SPARSE_LEVELS),
+         ("tc_sparse_pair", SPARSE_LEVELS), ("tc_sparse_ws", SPARSE_LEVELS), ("tc_sparse_st", SPARSE_LEVELS),
+         ("auto", MIXED_LEVELS)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
+@pytest.mark.parametrize("variant,levels", SMALL, ids=["%s-%s" % (v, "sparse" if l is SPARSE_LEVELS else "mixed") for v, l in SMALL])
+def test_block_matches_oracle_on_every_kernel_family(lib, variant, levels, dtype):
+    rows, dim, mlp = 333, 256, 1024                 # a ragged last tile for every kernel's row tile
+    host, p = make_params(dim, mlp, levels, dtype, 100)
+    x = synth.randn((rows, dim), 7, 1.5, dtype)
+    x[5] = 0.75                                      # a constant row: zero variance, LayerNorm leaves its bias
+    x[6] = 0.0
+    code = {"simt": lib.VARIANT_SIMT, "tc_dense": lib.VARIANT_TC_DENSE, "tc_pair": lib.VARIANT_TC_PAIR,
+            "tc_sparse_pair": lib.VARIANT_TC_SPARSE_PAIR, "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS,
+            "tc_sparse_st": lib.VARIANT_TC_SPARSE_ST, "auto": lib.VARIANT_AUTO}[variant]
+    got = run_block(lib, x, host, levels, mlp, variant=code)
+    check_rows(got, x, p, dtype, np.arange(rows))
+
+
+@pytest.mark.gpu
+def test_rows_longer_than_the_register_cache(lib):
+    # dim > 1024: LayerNorm re-reads the part of the row it does not keep in registers
+    dtype = torch.bfloat16
+    rows, dim, mlp = 70, 1536, 512
+    host, p = make_params(dim, mlp, MIXED_LEVELS, dtype, 300)
+    x = synth.randn((rows, dim), 8, 1.0, dtype)
+    got = run_block(lib, x, host, MIXED_LEVELS, mlp)
+    check_rows(got, x, p, dtype, np.arange(rows))
+
+
+@pytest.mark.gpu
+def test_two_phases_with_the_callers_attention_give_the_same_bits(lib):
+    dtype = torch.bfloat16
+    rows, dim, mlp = 400, 256, 1024
+    host, _ = make_params(dim, mlp, MIXED_LEVELS, dtype, 500)
+    x = synth.randn((rows, dim), 9, 1.0, dtype)
+    whole = run_block(lib, x, host, MIXED_LEVELS, mlp)
+    split = run_block(lib, x, host, MIXED_LEVELS, mlp, phase="split")
+    for s in STAGES:
+        assert torch.equal(whole[s].view(torch.int16), split[s].view(torch.int16)), s
+
+
+DEIT_LEVELS = [{"qkv": (2, 8), "proj": (1, 8), "fc1": (4, 8), "fc2": (2, 8)},     # WS, WS, dense pair + image, ST
+               {"qkv": (8, 8), "proj": (4, 8), "fc1": (1, 8), "fc2": (8, 8)}]     # dense pair (fused residuals), WS
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("levels", DEIT_LEVELS, ids=["sparse_heavy", "dense_heavy"])
+def test_deit_b_block_full_size_sampled_rows(lib, levels):
+    # the block at the size the timing runs (batch 256 x 197 tokens, dim 768, mlp 3072), AUTO kernel choice;
+    # the oracle follows 40 token rows, among them the first and last row of row tiles of every kernel
+    dtype = torch.bfloat16
+    rows, dim, mlp = 256 * 197, 768, 3072
+    host, p = make_params(dim, mlp, levels, dtype, 700)
+    x = synth.randn((rows, dim), 11, 1.0, dtype, "cuda").cpu()
+    got = run_block(lib, x, host, levels, mlp)
+    rng = np.random.default_rng(5)
+    edges = [0, 143, 144, 223, 224, 255, 256, rows - 1, rows - 145, (rows // 224) * 224, (rows // 144) * 144]
+    pick = np.unique(np.concatenate([np.array(edges), rng.integers(0, rows, 29)]))
+    check_rows(got, x, p, dtype, pick)
+
+
+@pytest.mark.gpu
+def test_block_validation(lib):
+    dtype = torch.bfloat16
+    rows, dim, mlp = 64, 256, 512
+    host, _ = make_params(dim, mlp, MIXED_LEVELS, dtype, 900)
+    dev = {k: v.cuda() for k, v in host.items()}
+    lin = {}
+    for name in NAMES:
+        N, M = MIXED_LEVELS[name]
+        vals, idx = lib.elsa_nm_compress(dev["W_" + name], N, M)
+        lin[name] = (vals, idx, dev["b_" + name], N, M)
+    w, keep = lib.make_block_weights(dev["ln1_g"], dev["ln1_b"], dev["ln2_g"], dev["ln2_b"], lin)
+    x = synth.randn((rows, dim), 1, 1.0, dtype).cuda()
+    total, _ = lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, lib.BF16)
+    before = lib.elsa_launch_count()
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_vit_block(x, mlp, w, scratch=torch.empty(total - 256, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == 6                                   # ELSA_ERR_WORKSPACE
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_vit_block(x, mlp, w, y=x)
+    assert e.value.status == 5                                   # y aliases x
+    w.fc1.idx = None
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_vit_block(x, mlp, w)
+    assert e.value.status == 1 and "fc1" in str(e.value)
+    assert lib.elsa_launch_count() == before                     # nothing was enqueued
