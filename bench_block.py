@@ -1,0 +1,105 @@
+"""Timing of the chained transformer block (elsa_vit_block): the twelve blocks of DeiT-B at batch 256, each
+with the levels the stack workload gives its four linears, chained (a block's y is the next block's x).
+
+    python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
+
+Attention is NOT computed: the block runs with the stand-in a = V, so the figure is the speed of the linear and
+elementwise path of the model (LayerNorms, the four N:M linears, GELU, residuals), not of DeiT-B.
+CUDA-event times of `reps` passes over all blocks (activations of one block alone exceed L2), one more pass with
+per-launch events for the split by kernel family, and the roofline of the pass: per linear the larger of kept
+FLOPs / bf16 peak and algorithmic bytes / HBM peak, plus the elementwise stages' bytes (LayerNorm in and out
+twice, the stand-in copy in and out, one residual operand per add) / HBM peak.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import bench
+from paper_2409_09708_b200 import binding as lib
+from paper_2409_09708_b200 import synth
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--blocks", type=int, default=12)
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--out", default="bench_out/block.json")
+    args = ap.parse_args()
+    dtype = torch.bfloat16
+    dim, mlp = 768, 3072
+    layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
+    rows = layers[0].rows
+    peaks, peaks_kind = bench.load_peaks()
+
+    blocks = []
+    for b in range(args.blocks):
+        lin = {}
+        for l in layers[4 * b:4 * b + 4]:
+            _, W, bias = synth.layer_tensors(l, dtype, "cuda", with_x=False)
+            vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+            lin[l.name.split(".")[1]] = (vals, idx, bias, l.N, l.M)
+        ln = [synth.randn((dim,), 9000 + 4 * b + i, 0.1, dtype, "cuda") + (1.0 if i % 2 == 0 else 0.0) for i in range(4)]
+        ln = [t.to(dtype) for t in ln]
+        blocks.append(lib.make_block_weights(ln[0], ln[1], ln[2], ln[3], lin))
+    scratch_bytes = max(lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, lib.BF16)[0] for w, _ in blocks)
+    scratch = lib.alloc_workspace(scratch_bytes)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    x = [synth.randn((rows, dim), 77, 1.0, dtype, "cuda"), torch.empty((rows, dim), dtype=dtype, device="cuda")]
+
+    def one_pass():
+        for b, (w, _) in enumerate(blocks):
+            lib.elsa_vit_block(x[b & 1], mlp, w, y=x[(b + 1) & 1], scratch=scratch, dev_status=status)
+
+    x0 = x[0].clone()
+    for _ in range(3):
+        x[0].copy_(x0)
+        one_pass()
+    times = []
+    for _ in range(args.reps):
+        x[0].copy_(x0)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        one_pass()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    assert torch.isfinite(x[args.blocks & 1].float()).all()
+
+    x[0].copy_(x0)
+    lib.elsa_profile_start()
+    one_pass()
+    families = {}
+    for kernel, _, ms in lib.elsa_profile_stop():
+        f = families.setdefault(kernel, {"launches": 0, "ms": 0.0})
+        f["launches"] += 1
+        f["ms"] += ms
+
+    lin_roof = sum(bench.roofline_seconds(l, peaks)[0] for l in layers)
+    elementwise_bytes = args.blocks * 8 * rows * dim * 2
+    roof_ms = (lin_roof + elementwise_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
+    ms = statistics.median(times)
+    rec = {"workload": "deit_b_blocks_b%d" % args.batch, "blocks": args.blocks, "rows": rows, "dtype": "bf16",
+           "attention": "stand-in a = V (not computed)", "ms_per_pass": ms, "ms_min": min(times), "ms_max": max(times),
+           "images_per_s_linear_and_elementwise_path": args.batch / ms * 1e3,
+           "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "peaks": peaks_kind,
+           "linears_roofline_ms": lin_roof * 1e3, "elementwise_bytes": elementwise_bytes,
+           "families_profiled_pass": families, "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
+    os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
+    json.dump(rec, open(args.out, "w"), indent=1)
+    print(json.dumps(rec))
+
+
+if __name__ == "__main__":
+    main()

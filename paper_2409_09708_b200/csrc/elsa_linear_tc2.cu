@@ -28,6 +28,8 @@
 
 #include "elsa_tc_common.cuh"
 
+#include <type_traits>
+
 namespace elsa {
 namespace {
 
@@ -308,7 +310,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             // converts, stages and stores one 32 x 32 chunk
             auto emit = [&](const uint32_t (&r)[32], int c) {
                 // 16 columns: + bias (read as stored, eight values per load), rounded to 16 bit
-                auto convert16 = [&](int h, uint32_t (&pk)[8]) {
+                auto convert16 = [&](auto with_act, int h, uint32_t (&pk)[8]) {
 #pragma unroll
                     for (int g = 0; g < 2; ++g) {
                         uint32_t bw[4];
@@ -342,8 +344,12 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                                 float vy = __uint_as_float(r[2 * j + 1]) + bv.y;
                                 if constexpr (kFused) {
                                     const float2 rv = raw2_to_float2<kBf16>(res[e]);   // zeros without a residual
-                                    vx = apply_act(vx, l_act) + rv.x;
-                                    vy = apply_act(vy, l_act) + rv.y;
+                                    if constexpr (decltype(with_act)::value) {
+                                        vx = gelu_exact(vx);
+                                        vy = gelu_exact(vy);
+                                    }
+                                    vx += rv.x;
+                                    vy += rv.y;
                                 }
                                 pk[4 * g + e] = pack2<kBf16>(vx, vy);
                             }
@@ -354,12 +360,17 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                 const uint32_t row_addr = buf + (uint32_t)(lane * 64);
                 const uint32_t sw = (uint32_t)((lane >> 1) & 3);   // 64-byte swizzle of the staging rows
                 uint32_t pk[8];
-                convert16(0, pk);
+                // the activation is a warp-uniform property of the layer: one branch per chunk, none per value
+                if (kFused && l_act == 1) convert16(std::true_type{}, 0, pk);
+                else convert16(std::false_type{}, 0, pk);
                 if (lane == 0) bulk_wait_group_read<kStagingBufs - 1>();   // the store that last used this buffer has drained it
                 __syncwarp();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    if (h == 1) convert16(1, pk);
+                    if (h == 1) {
+                        if (kFused && l_act == 1) convert16(std::true_type{}, 1, pk);
+                        else convert16(std::false_type{}, 1, pk);
+                    }
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row_addr + (((uint32_t)(2 * h + j) ^ sw) << 4)),

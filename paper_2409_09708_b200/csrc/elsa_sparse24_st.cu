@@ -92,7 +92,8 @@ struct StGroup {
 
 // (22 warps are allocated as 24: 80 registers per thread is what the register file allows, and a loader warp
 // holds a whole chunk, 72 of them, between its loads and its tensor-memory stores)
-template <bool kBf16, int kMaxLayers>
+// kAct: the instantiation whose epilogue applies the layer's activation (single-layer launches).
+template <bool kBf16, int kMaxLayers, bool kAct>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
 {
@@ -339,7 +340,8 @@ linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
             const int f = f0 + feat_in_quarter;
             const int l_rows = L.rows, l_out = L.out;
             const float bias_f = (L.bias != nullptr && f < l_out) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
-            const int l_act = L.act;
+            const int l_act = kAct ? L.act : 0;
+            (void)l_act;
             bool ok = mbar_wait(tmem_full_bar, acc_phase, abort_flag, p.dev_status, 4);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -374,8 +376,9 @@ linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
                 for (int i = 0; i < kRoundSteps; ++i)
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        w[i][j] = pack2<kBf16>(apply_act(__uint_as_float(rr[i][2 * j]) + bias_f, l_act),
-                                               apply_act(__uint_as_float(rr[i][2 * j + 1]) + bias_f, l_act));
+                        w[i][j] = kAct ? pack2<kBf16>(apply_act(__uint_as_float(rr[i][2 * j]) + bias_f, l_act),
+                                                      apply_act(__uint_as_float(rr[i][2 * j + 1]) + bias_f, l_act))
+                                       : pack2<kBf16>(__uint_as_float(rr[i][2 * j]) + bias_f, __uint_as_float(rr[i][2 * j + 1]) + bias_f);
                 if (rd + 1 < kRounds) {
 #pragma unroll
                     for (int i = 0; i < kRoundSteps; ++i)
@@ -414,11 +417,11 @@ linear_tc_sp24_st_kernel(const __grid_constant__ StGroup<kMaxLayers> p)
     }
 }
 
-template <bool kBf16, int kMaxLayers>
+template <bool kBf16, int kMaxLayers, bool kAct>
 elsa_status launch_st_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
                             const DeviceInfo& dev)
 {
-    auto kernel = linear_tc_sp24_st_kernel<kBf16, kMaxLayers>;
+    auto kernel = linear_tc_sp24_st_kernel<kBf16, kMaxLayers, kAct>;
     const size_t smem = (size_t)kStages * kStageBytes + kStagingTotal + kBarrierBytes + 1024;
     if (smem > dev.smem_optin) return fail(ELSA_ERR_CUDA, "not enough shared memory for the streaming sparse kernel");
 
@@ -504,11 +507,22 @@ elsa_status launch_linear_tc_sparse_st_group(const SparseJob* jobs, int n, elsa_
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    bool act = false;
+    for (int i = 0; i < n; ++i) act = act || jobs[i].act != 0;
+    if (act) {
+        // layers with an activation in the epilogue run one per launch, on the instantiation that has it
+        for (int i = 0; i < n; ++i) {
+            st = dtype == ELSA_BF16 ? launch_st_group<true, 1, true>(jobs + i, 1, dtype, dev_status, stream, dev)
+                                    : launch_st_group<false, 1, true>(jobs + i, 1, dtype, dev_status, stream, dev);
+            if (st != ELSA_OK) return st;
+        }
+        return ELSA_OK;
+    }
     if (n == 1)
-        return dtype == ELSA_BF16 ? launch_st_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
-                                  : launch_st_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
-    return dtype == ELSA_BF16 ? launch_st_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
-                              : launch_st_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+        return dtype == ELSA_BF16 ? launch_st_group<true, 1, false>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_st_group<false, 1, false>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_st_group<true, kGroupMax, false>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_st_group<false, kGroupMax, false>(jobs, n, dtype, dev_status, stream, dev);
 }
 
 elsa_status launch_linear_tc_sparse_st(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,

@@ -82,7 +82,8 @@ struct WsGroup {
     uint32_t* dev_status;
 };
 
-template <bool kBf16, int kMaxLayers>
+// kAct: the instantiation whose epilogue applies the layer's activation (single-layer launches).
+template <bool kBf16, int kMaxLayers, bool kAct>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
 {
@@ -321,7 +322,8 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                 if (lane == 0) mbar_arrive_cluster_release(w_ready_remote);
             }
             const float bias_f = (L.bias != nullptr && f_ok) ? bias_to_float<kBf16>(__ldg(L.bias + f)) : 0.f;
-            const int l_act = L.act;
+            const int l_act = kAct ? L.act : 0;
+            (void)l_act;
             // this warp's run of token columns: steps of 16, [first_step, first_step + my_steps)
             const int total_steps = nt / kStepCols;
             const int first_step = part * L.steps_per_warp;
@@ -356,8 +358,9 @@ linear_tc_sp24_ws_kernel(const __grid_constant__ WsGroup<kMaxLayers> p)
                     uint32_t w[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
-                        w[j] = pack2<kBf16>(apply_act(__uint_as_float(rr[s][2 * j]) + bias_f, l_act),
-                                            apply_act(__uint_as_float(rr[s][2 * j + 1]) + bias_f, l_act));
+                        w[j] = kAct ? pack2<kBf16>(apply_act(__uint_as_float(rr[s][2 * j]) + bias_f, l_act),
+                                                   apply_act(__uint_as_float(rr[s][2 * j + 1]) + bias_f, l_act))
+                                    : pack2<kBf16>(__uint_as_float(rr[s][2 * j]) + bias_f, __uint_as_float(rr[s][2 * j + 1]) + bias_f);
                     stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64), w[0], w[1], w[2], w[3]);
                     stmatrix_x4_trans(st_addr + (uint32_t)(s * kStepCols * 64 + 512), w[4], w[5], w[6], w[7]);
                 }
@@ -402,11 +405,11 @@ int ws_row_tile(int in)
     return nt >= 64 ? nt : 0;
 }
 
-template <bool kBf16, int kMaxLayers>
+template <bool kBf16, int kMaxLayers, bool kAct>
 elsa_status launch_ws_group(const SparseJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status, cudaStream_t stream,
                             const DeviceInfo& dev)
 {
-    auto kernel = linear_tc_sp24_ws_kernel<kBf16, kMaxLayers>;
+    auto kernel = linear_tc_sp24_ws_kernel<kBf16, kMaxLayers, kAct>;
     const int fixed = kStagingTotal + kBarrierBytes + 1024;
     int max_nt = 0;
     for (int i = 0; i < n; ++i) {
@@ -512,11 +515,22 @@ elsa_status launch_linear_tc_sparse_ws_group(const SparseJob* jobs, int n, elsa_
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     if (n < 1 || n > kGroupMax) return fail(ELSA_ERR_SHAPE, "a grouped launch carries 1 to %d layers, got %d", kGroupMax, n);
+    bool act = false;
+    for (int i = 0; i < n; ++i) act = act || jobs[i].act != 0;
+    if (act) {
+        // layers with an activation in the epilogue run one per launch, on the instantiation that has it
+        for (int i = 0; i < n; ++i) {
+            st = dtype == ELSA_BF16 ? launch_ws_group<true, 1, true>(jobs + i, 1, dtype, dev_status, stream, dev)
+                                    : launch_ws_group<false, 1, true>(jobs + i, 1, dtype, dev_status, stream, dev);
+            if (st != ELSA_OK) return st;
+        }
+        return ELSA_OK;
+    }
     if (n == 1)
-        return dtype == ELSA_BF16 ? launch_ws_group<true, 1>(jobs, 1, dtype, dev_status, stream, dev)
-                                  : launch_ws_group<false, 1>(jobs, 1, dtype, dev_status, stream, dev);
-    return dtype == ELSA_BF16 ? launch_ws_group<true, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
-                              : launch_ws_group<false, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+        return dtype == ELSA_BF16 ? launch_ws_group<true, 1, false>(jobs, 1, dtype, dev_status, stream, dev)
+                                  : launch_ws_group<false, 1, false>(jobs, 1, dtype, dev_status, stream, dev);
+    return dtype == ELSA_BF16 ? launch_ws_group<true, kGroupMax, false>(jobs, n, dtype, dev_status, stream, dev)
+                              : launch_ws_group<false, kGroupMax, false>(jobs, n, dtype, dev_status, stream, dev);
 }
 
 elsa_status launch_linear_tc_sparse_ws(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
