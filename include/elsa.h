@@ -274,7 +274,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_SP24_ST = 10, /* 2:4 sparse MMA with the weight streaming through tensor memory */
     ELSA_KERNEL_LINEAR_TC_PAIR_I8 = 11, /* INT8 form of the CTA-pair GEMM */
     ELSA_KERNEL_INT8_FORMAT = 12,       /* INT8 compress / unpack */
-    ELSA_KERNEL_BLOCK_ROWWISE = 13      /* LayerNorm, residual add, GELU, column copy of the chained block */
+    ELSA_KERNEL_BLOCK_ROWWISE = 13,     /* LayerNorm, residual add, GELU, column copy of the chained block */
+    ELSA_KERNEL_BACKWARD_FORMAT = 14    /* transposes, column sums and mask of the backward pass */
 } elsa_kernel_id;
 
 typedef struct {
@@ -424,6 +425,25 @@ elsa_status elsa_vit_block_rest(const void* x, int rows, int dim, int mlp_dim, c
 /* Both, with the stand-in a = V between them. */
 elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                            void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream);
+
+/* ------------------------------------------------------------------------------------------------
+ * Backward pass of the masked linear (Alg. 2, supernet training: the gradient is taken with respect to the
+ * sparse weights W(alpha) derived from the shared weight and applied to the shared weight).  For
+ * Y = X Wm^T + b with Wm = mask .* W and dY the gradient arriving at Y:
+ *     dX [rows][in]  = dY Wm
+ *     dW [out][in]   = mask .* (dY^T X)   dense, exact zeros at pruned positions (a pruned weight takes no part
+ *                                         in the product; the paper states no straight-through estimator)
+ *     db [out]       = sum over rows of dY
+ * fp32 accumulation, one rounding to `dtype` per output.  Any of dX, dW, db may be NULL (not computed); vals is
+ * needed for dX, X for dW; idx names the kept positions (NULL iff N == M).  All DEVICE pointers, 16-byte aligned;
+ * workspace: elsa_backward_workspace_bytes(...) bytes, 256-byte aligned (transposed operands: the tensor-core
+ * GEMM wants the reduction index contiguous in both).  Both contractions run at the dense rate: the 2:4 sparse
+ * MMA needs the zeros along the reduction, which in dX runs over `out`.  Asynchronous on `stream`.
+ */
+size_t elsa_backward_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype dtype);
+elsa_status elsa_nm_linear_backward(const void* dY, const void* X, int rows, const void* vals, const uint32_t* idx,
+                                    int out, int in, int N, int M, elsa_dtype dtype, void* dX, void* dW, void* db,
+                                    void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream);
 
 /*
  * Test hook for the device-side failure path.  Every wait of the tensor-core kernels is bounded: a wait that

@@ -115,6 +115,8 @@ class ElsaBlockWeights(ctypes.Structure):
                 ("eps", ctypes.c_float)]
 
 
+_backward_ws = _sig("elsa_backward_workspace_bytes", _sz, [_i, _i, _i, _i, _i, _i])
+_backward = _sig("elsa_nm_linear_backward", _i, [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp, _sz, _vp, _vp])
 BLOCK_REGIONS = ("x1", "qkv", "a", "x2", "x3", "h", "t", "workspace")
 _bw = ctypes.POINTER(ElsaBlockWeights)
 _block_scratch = _sig("elsa_vit_block_scratch_bytes", _sz, [_i, _i, _i, _bw, _i, ctypes.POINTER(_sz)])
@@ -128,7 +130,7 @@ class ElsaKernelTime(ctypes.Structure):
 
 
 KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images",
-                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format", 13: "block_rowwise"}
+                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format", 13: "block_rowwise", 14: "backward_format"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 
@@ -369,6 +371,26 @@ def elsa_nm_linear(X: torch.Tensor, vals: torch.Tensor, idx, bias, out: int, in_
     _check(_linear(_ptr(X), rows, _ptr(vals), _ptr(idx), _ptr(bias), out, in_, N, M, code, _ptr(Y),
                    _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
     return Y
+
+
+def elsa_backward_workspace_bytes(rows, in_, out, N, M, dtype=F16) -> int:
+    return int(_backward_ws(rows, in_, out, N, M, dtype))
+
+
+def elsa_nm_linear_backward(dY, X, vals, idx, out, in_, N, M, want=("dX", "dW", "db"), workspace=None,
+                            dev_status=None, stream=None):
+    """Backward of Y = X Wm^T + b: returns (dX, dW, db), None for the ones not in `want`.  dW is dense [out, in]
+    with zeros at the pruned positions."""
+    rows = dY.shape[0]
+    code = dtype_code(dY.dtype)
+    dX = torch.empty((rows, in_), dtype=dY.dtype, device=dY.device) if "dX" in want else None
+    dW = torch.empty((out, in_), dtype=dY.dtype, device=dY.device) if "dW" in want else None
+    db = torch.empty((out,), dtype=dY.dtype, device=dY.device) if "db" in want else None
+    if workspace is None:
+        workspace = alloc_workspace(elsa_backward_workspace_bytes(rows, in_, out, N, M, code), dY.device)
+    _check(_backward(_ptr(dY), _ptr(X), rows, _ptr(vals), _ptr(idx), out, in_, N, M, code, _ptr(dX), _ptr(dW), _ptr(db),
+                     _ptr(workspace), workspace.numel(), _ptr(dev_status), _stream(stream)))
+    return dX, dW, db
 
 
 def make_block_weights(ln1_gain, ln1_bias, ln2_gain, ln2_bias, linears, eps=1e-6):

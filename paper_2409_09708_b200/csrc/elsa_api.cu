@@ -1076,6 +1076,106 @@ elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const 
 
 }  // extern "C"
 
+/* ---------------------------------------------------------------------------------------------- */
+/* Backward pass                                                                                  */
+/* ---------------------------------------------------------------------------------------------- */
+namespace elsa {
+namespace {
+
+struct BackwardPlan {
+    size_t wm, wmt, dyt, xt, partial, total;   // byte offsets of the regions
+    int rows_p;                                // rows rounded up to 64: reduction length of the dW product
+};
+
+BackwardPlan backward_plan(int rows, int in, int out)
+{
+    BackwardPlan p;
+    p.rows_p = (rows + 63) / 64 * 64;
+    size_t at = 0;
+    p.wm = at;      at += round_up((size_t)out * in * 2, 256);                 // masked weight [out][in]
+    p.wmt = at;     at += round_up((size_t)out * in * 2, 256);                 // its transpose [in][out]
+    p.dyt = at;     at += round_up((size_t)out * p.rows_p * 2, 256);           // dY^T [out][rows_p]
+    p.xt = at;      at += round_up((size_t)in * p.rows_p * 2, 256);            // X^T  [in][rows_p]
+    p.partial = at; at += round_up((size_t)(p.rows_p / 64) * out * 4, 256);    // column sums of dY per 64 rows
+    p.total = at;
+    return p;
+}
+
+// Y [m][n] = A [m][k] . B [n][k]^T on the dense tensor-core kernels (no bias).
+elsa_status dense_product(const uint16_t* A, int m, const uint16_t* B, int n, int k, elsa_dtype dtype, uint16_t* Y,
+                          uint32_t* dev_status, cudaStream_t stream, int sm_count)
+{
+    const int variant = g_variant.load(std::memory_order_relaxed);
+    const bool pair = variant == ELSA_VARIANT_TC_PAIR || (variant != ELSA_VARIANT_TC_DENSE && linear_tc_pair_suits(m, n, sm_count));
+    return pair ? launch_linear_tc_pair(A, m, B, nullptr, n, k, dtype, Y, dev_status, stream)
+                : launch_linear_tc_dense(A, m, B, nullptr, n, k, dtype, Y, dev_status, stream);
+}
+
+}  // namespace
+}  // namespace elsa
+
+extern "C" {
+
+size_t elsa_backward_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype dtype)
+{
+    if (rows <= 0 || out <= 0 || in <= 0 || index_bits(M) < 0 || N < 1 || N > M || in % M != 0) return 0;
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return 0;
+    return backward_plan(rows, in, out).total;
+}
+
+elsa_status elsa_nm_linear_backward(const void* dY, const void* X, int rows, const void* vals, const uint32_t* idx,
+                                    int out, int in, int N, int M, elsa_dtype dtype, void* dX, void* dW, void* db,
+                                    void* workspace, size_t workspace_bytes, uint32_t* dev_status, void* stream_)
+{
+    if (!dY) return fail(ELSA_ERR_NULL, "dY must not be NULL");
+    elsa_status st = check_level(out, in, N, M, dtype);
+    if (st != ELSA_OK) return st;
+    if (rows <= 0) return fail(ELSA_ERR_SHAPE, "non-positive rows=%d", rows);
+    if (dX && !vals) return fail(ELSA_ERR_NULL, "vals must not be NULL when dX is wanted");
+    if (dW && !X) return fail(ELSA_ERR_NULL, "X must not be NULL when dW is wanted");
+    if ((dX || dW) && N != M && !idx) return fail(ELSA_ERR_NULL, "idx must not be NULL when N < M");
+    if (!aligned16(dY) || (X && !aligned16(X)) || (vals && !aligned16(vals)) || (idx && !aligned16(idx)) ||
+        (dX && !aligned16(dX)) || (dW && !aligned16(dW)) || (db && !aligned16(db)))
+        return fail(ELSA_ERR_ALIGN, "dY, X, vals, idx, dX, dW and db must be 16-byte aligned");
+    const BackwardPlan plan = backward_plan(rows, in, out);
+    if (!workspace || workspace_bytes < plan.total)
+        return fail(ELSA_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", plan.total, workspace ? workspace_bytes : (size_t)0);
+    if (((uintptr_t)workspace & 255u) != 0) return fail(ELSA_ERR_ALIGN, "workspace must be 256-byte aligned");
+    DeviceInfo dev;
+    if ((st = device_info(&dev)) != ELSA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    uint8_t* ws = (uint8_t*)workspace;
+    const uint16_t* dy = (const uint16_t*)dY;
+    if (dX) {
+        // dX = dY Wm: the forward GEMM with the transposed masked weight, reduction over `out`
+        uint16_t* wm = (uint16_t*)(ws + plan.wm);
+        uint16_t* wmt = (uint16_t*)(ws + plan.wmt);
+        const uint16_t* dense = (const uint16_t*)vals;
+        if (N != M) {
+            if ((st = launch_unpack((const uint16_t*)vals, idx, out, in, N, M, wm, stream)) != ELSA_OK) return st;
+            dense = wm;
+        }
+        if ((st = launch_transpose16(dense, wmt, out, in, out, nullptr, dtype, stream)) != ELSA_OK) return st;
+        if ((st = dense_product(dy, rows, wmt, in, out, dtype, (uint16_t*)dX, dev_status, stream, dev.sm_count)) != ELSA_OK) return st;
+    }
+    if (dW || db) {
+        float* partial = (float*)(ws + plan.partial);
+        uint16_t* dyt = (uint16_t*)(ws + plan.dyt);
+        if ((st = launch_transpose16(dy, dyt, rows, out, plan.rows_p, db ? partial : nullptr, dtype, stream)) != ELSA_OK) return st;
+        if (db && (st = launch_colsum_finish(partial, plan.rows_p / 64, out, (uint16_t*)db, dtype, stream)) != ELSA_OK) return st;
+        if (dW) {
+            // dW = dY^T X, reduction over the token rows, then the mask
+            uint16_t* xt = (uint16_t*)(ws + plan.xt);
+            if ((st = launch_transpose16((const uint16_t*)X, xt, rows, in, plan.rows_p, nullptr, dtype, stream)) != ELSA_OK) return st;
+            if ((st = dense_product(dyt, out, xt, in, plan.rows_p, dtype, (uint16_t*)dW, dev_status, stream, dev.sm_count)) != ELSA_OK) return st;
+            if ((st = launch_mask_apply((uint16_t*)dW, idx, out, in, N, M, stream)) != ELSA_OK) return st;
+        }
+    }
+    return ELSA_OK;
+}
+
+}  // extern "C"
+
 extern "C" {
 
 elsa_status elsa_set_linear_variant(elsa_variant v)

@@ -1,0 +1,157 @@
+// Helper kernels of the masked linear's backward pass (ELSA, Alg. 2: the gradient is taken with respect to the
+// sparse weights derived from the shared weight; for Y = X Wm^T + b that is dX = dY Wm, dW = mask .* dY^T X,
+// db = column sums of dY).  The two contractions run on the dense tensor-core GEMM of the forward path, which
+// wants both operands with the reduction index contiguous; these kernels bring the operands into that form:
+//   transpose16   [R][C] -> [C][Rp] (Rp >= R, the tail zero), optionally with the column sums of the source
+//   mask_apply    zeroes the pruned positions of a dense [out][in] gradient in place, from the index stream
+//   colsum_finish sums the per-tile column sums and rounds once
+#include "elsa_internal.h"
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+namespace elsa {
+namespace {
+
+constexpr int kTile = 64;
+
+template <bool kBf16>
+__device__ __forceinline__ float to_float(uint16_t u)
+{
+    if constexpr (kBf16) return __uint_as_float((uint32_t)u << 16);
+    else return __half2float(__ushort_as_half(u));
+}
+
+template <bool kBf16>
+__device__ __forceinline__ uint16_t from_float(float f)
+{
+    if constexpr (kBf16) return __bfloat16_as_ushort(__float2bfloat16_rn(f));
+    else return __half_as_ushort(__float2half_rn(f));
+}
+
+// One block per 64 x 64 tile.  src [R][C] (C % 8 == 0), dst [C][Rp] (Rp % 8 == 0).  Blocks of the last tile row
+// also write the zero tail R..Rp of their dst rows.  partial (or NULL): [tiles over R][C] fp32, the sum of each
+// source column over the tile's rows, summed in row order.
+template <bool kBf16>
+__global__ void __launch_bounds__(256)
+transpose16_kernel(const uint16_t* __restrict__ src, uint16_t* __restrict__ dst, int R, int C, int Rp,
+                   float* __restrict__ partial)
+{
+    __shared__ uint16_t tile[kTile][kTile + 8];
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const int r0 = blockIdx.x * kTile, c0 = blockIdx.y * kTile;   // row tiles on x: their count has no 65535 limit
+    const int t = threadIdx.x;
+    // load: 64 rows x 8 vectors of 8 values
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int slot = t + 256 * i;
+        const int r = slot >> 3, v = slot & 7;
+        uint4 u = make_uint4(0u, 0u, 0u, 0u);
+        if (r0 + r < R && c0 + 8 * v < C)
+            u = __ldg(reinterpret_cast<const uint4*>(src + (size_t)(r0 + r) * (size_t)C + c0 + 8 * v));
+        *reinterpret_cast<uint4*>(&tile[r][8 * v]) = u;
+    }
+    __syncthreads();
+    if (partial != nullptr && t < kTile && c0 + t < C) {
+        float s = 0.f;
+        for (int r = 0; r < kTile; ++r) s += to_float<kBf16>(tile[r][t]);     // rows past R hold zeros
+        partial[(size_t)blockIdx.x * (size_t)C + c0 + t] = s;
+    }
+    // store: 64 dst rows (source columns) x 8 vectors of 8 source rows
+    const bool last = blockIdx.x == gridDim.x - 1;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int slot = t + 256 * i;
+        const int c = slot >> 3, v = slot & 7;
+        if (c0 + c >= C) continue;
+        uint16_t e[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) e[k] = tile[8 * v + k][c];
+        const uint4 u = make_uint4(e[0] | ((uint32_t)e[1] << 16), e[2] | ((uint32_t)e[3] << 16),
+                                   e[4] | ((uint32_t)e[5] << 16), e[6] | ((uint32_t)e[7] << 16));
+        uint16_t* row = dst + (size_t)(c0 + c) * (size_t)Rp;
+        if (r0 + 8 * v < Rp) *reinterpret_cast<uint4*>(row + r0 + 8 * v) = u;
+        if (last)
+            for (int r = r0 + kTile + 8 * v; r < Rp; r += kTile) *reinterpret_cast<uint4*>(row + r) = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// db[c] = round16(sum over tiles of partial[tile][c]), tiles in ascending order.
+template <bool kBf16>
+__global__ void __launch_bounds__(256) colsum_finish_kernel(const float* __restrict__ partial, int tiles, int C, uint16_t* __restrict__ db)
+{
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    float s = 0.f;
+    for (int i = 0; i < tiles; ++i) s += partial[(size_t)i * (size_t)C + c];
+    db[c] = from_float<kBf16>(s);
+}
+
+// One thread per group of M: keeps the N positions the index stream names, zeroes the rest.
+template <int M>
+__global__ void __launch_bounds__(256)
+mask_apply_kernel(uint16_t* __restrict__ dW, const uint32_t* __restrict__ idx, int out, int in, int N, int words_per_row)
+{
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int groups_per_row = in / M;
+    if (gid >= (long long)out * groups_per_row) return;
+    const int o = (int)(gid / groups_per_row), g = (int)(gid % groups_per_row);
+    const uint32_t* row = idx + (size_t)o * (size_t)words_per_row;
+    uint32_t keep = 0;
+    for (int t = 0; t < N; ++t) {
+        const int bit = (g * N + t) * B;
+        const int w = bit >> 5, sh = bit & 31;
+        uint32_t f = row[w] >> sh;
+        if (sh + B > 32) f |= row[w + 1] << (32 - sh);
+        keep |= 1u << (f & (M - 1));
+    }
+    uint32_t* p = reinterpret_cast<uint32_t*>(dW + (size_t)o * (size_t)in + (size_t)g * M);
+#pragma unroll
+    for (int q = 0; q < M / 2; ++q) {
+        const uint32_t m = ((keep >> (2 * q)) & 1u ? 0x0000ffffu : 0u) | ((keep >> (2 * q + 1)) & 1u ? 0xffff0000u : 0u);
+        if (m != 0xffffffffu) p[q] &= m;
+    }
+}
+
+}  // namespace
+
+elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C, int Rp, float* partial,
+                               elsa_dtype dtype, cudaStream_t stream)
+{
+    if (R <= 0 || C <= 0) return ELSA_OK;
+    const dim3 grid((unsigned)((R + kTile - 1) / kTile), (unsigned)((C + kTile - 1) / kTile));
+    ProfileScope scope(ELSA_KERNEL_BACKWARD_FORMAT, stream);
+    if (dtype == ELSA_BF16) launch_pdl(transpose16_kernel<true>, grid, dim3(256), 0, stream, 1, src, dst, R, C, Rp, partial);
+    else launch_pdl(transpose16_kernel<false>, grid, dim3(256), 0, stream, 1, src, dst, R, C, Rp, partial);
+    return launched("transpose16");
+}
+
+elsa_status launch_colsum_finish(const float* partial, int tiles, int C, uint16_t* db, elsa_dtype dtype, cudaStream_t stream)
+{
+    const unsigned grid = (unsigned)((C + 255) / 256);
+    ProfileScope scope(ELSA_KERNEL_BACKWARD_FORMAT, stream);
+    if (dtype == ELSA_BF16) launch_pdl(colsum_finish_kernel<true>, dim3(grid), dim3(256), 0, stream, 1, partial, tiles, C, db);
+    else launch_pdl(colsum_finish_kernel<false>, dim3(grid), dim3(256), 0, stream, 1, partial, tiles, C, db);
+    return launched("colsum_finish");
+}
+
+elsa_status launch_mask_apply(uint16_t* dW, const uint32_t* idx, int out, int in, int N, int M, cudaStream_t stream)
+{
+    if (N == M) return ELSA_OK;
+    const long long groups = (long long)out * (in / M);
+    const unsigned grid = (unsigned)((groups + 255) / 256);
+    const int wpr = (int)index_words_per_row(in, N, M);
+    ProfileScope scope(ELSA_KERNEL_BACKWARD_FORMAT, stream);
+    if (M == 4) launch_pdl(mask_apply_kernel<4>, dim3(grid), dim3(256), 0, stream, 1, dW, idx, out, in, N, wpr);
+    else if (M == 8) launch_pdl(mask_apply_kernel<8>, dim3(grid), dim3(256), 0, stream, 1, dW, idx, out, in, N, wpr);
+    else launch_pdl(mask_apply_kernel<16>, dim3(grid), dim3(256), 0, stream, 1, dW, idx, out, in, N, wpr);
+    return launched("mask_apply");
+}
+
+}  // namespace elsa

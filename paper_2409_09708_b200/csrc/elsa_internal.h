@@ -165,6 +165,13 @@ elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype
 // dst[r][0 .. cols) = src[r][col0 .. col0 + cols); src rows of src_ld values; all multiples of 8.
 elsa_status launch_copy_columns(const uint16_t* src, uint16_t* dst, int rows, int src_ld, int col0, int cols,
                                 cudaStream_t stream);
+// Operand forms of the backward pass.  transpose16: src [R][C] -> dst [C][Rp] with the tail R..Rp zero (C, Rp
+// multiples of 8); partial (or NULL) receives [ceil(R / 64)][C] fp32 column sums per 64-row tile.
+elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C, int Rp, float* partial,
+                               elsa_dtype dtype, cudaStream_t stream);
+elsa_status launch_colsum_finish(const float* partial, int tiles, int C, uint16_t* db, elsa_dtype dtype, cudaStream_t stream);
+// Zeroes the pruned positions of a dense [out][in] tensor in place.
+elsa_status launch_mask_apply(uint16_t* dW, const uint32_t* idx, int out, int in, int N, int M, cudaStream_t stream);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
 constexpr int kMaxLevels = 16;
 struct LevelTable {
