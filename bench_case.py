@@ -9,6 +9,10 @@ calls of elsa_nm_linear), the layer's algorithmic bytes and kept FLOPs.
     python bench_case.py --compress-table deit_b_stack_b256 --reps 3
 
 runs elsa_vit_compress over the weights of a workload table instead (weights only, no activations).
+
+    python bench_case.py --backward --rows 50432 --in 768 --out 3072 --level 2:8 --reps 5
+
+times elsa_nm_linear_backward on that layer: dX alone, dW alone, db alone and all three in one call.
 """
 from __future__ import annotations
 
@@ -84,6 +88,35 @@ def int8_case(args):
                       "dense_equiv_ops": 2.0 * args.rows * args.in_ * args.out}))
 
 
+def backward_case(args):
+    """The backward of one layer; both products run at the dense rate, so their roofline is 2 rows in out flops
+    each against the dense bf16 peak (db: the bytes of dY against the HBM peak)."""
+    N, M = (int(v) for v in args.level.split(":"))
+    dtype = synth.torch_dtype(args.dtype)
+    layer = synth.Layer("case", args.rows, args.in_, args.out, N, M, 1, 2, 3)
+    X, W, _ = synth.layer_tensors(layer, dtype, device="cuda")
+    dY = synth.randn((args.rows, args.out), 4, 0.05, dtype, device="cuda")
+    vals, idx = lib.elsa_nm_compress(W, N, M)
+    ws = lib.alloc_workspace(lib.elsa_backward_workspace_bytes(args.rows, args.in_, args.out, N, M, lib.dtype_code(dtype)))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    out = {"form": "backward", "rows": args.rows, "in": args.in_, "out": args.out, "level": args.level, "dtype": args.dtype,
+           "dense_flops_per_product": layer.dense_equiv_flops, "dY_bytes": args.rows * args.out * 2}
+    for want in (("dX",), ("dW",), ("db",), ("dX", "dW", "db")):
+        times = []
+        for rep in range(args.reps + 1):
+            flush.fill_(rep)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            lib.elsa_nm_linear_backward(dY, X, vals, idx, args.out, args.in_, N, M, want=want, workspace=ws, dev_status=status)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        out["ms_" + "_".join(want)] = times[1:]                    # the first call also allocates its outputs' pages
+    assert int(status.item()) == 0
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--rows", type=int, default=50432)
@@ -96,7 +129,10 @@ def main():
                                                             "tc_sparse_ws", "tc_sparse_st"])
     ap.add_argument("--compress-table", default=None, help="workload whose weights go through elsa_vit_compress")
     ap.add_argument("--int8", action="store_true", help="the INT8 form: elsa_nm_compress_i8 once, then elsa_nm_linear_i8")
+    ap.add_argument("--backward", action="store_true", help="elsa_nm_linear_backward on the layer")
     args = ap.parse_args()
+    if args.backward:
+        return backward_case(args)
     if args.compress_table:
         return compress_table(args.compress_table, args.reps)
     if args.int8:

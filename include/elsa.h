@@ -436,9 +436,9 @@ elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const 
  *     db [out]       = sum over rows of dY
  * fp32 accumulation, one rounding to `dtype` per output.  Any of dX, dW, db may be NULL (not computed); vals is
  * needed for dX, X for dW; idx names the kept positions (NULL iff N == M).  All DEVICE pointers, 16-byte aligned;
- * workspace: elsa_backward_workspace_bytes(...) bytes, 256-byte aligned (transposed operands: the tensor-core
- * GEMM wants the reduction index contiguous in both).  Both contractions run at the dense rate: the 2:4 sparse
- * MMA needs the zeros along the reduction, which in dX runs over `out`.  Asynchronous on `stream`.
+ * workspace: elsa_backward_workspace_bytes(...) bytes, 256-byte aligned (the transposed masked weight for dX,
+ * partial column sums for db).  Both contractions run at the dense rate: the 2:4 sparse MMA needs the zeros along
+ * the reduction, which in dX runs over `out`.  Asynchronous on `stream`.
  */
 size_t elsa_backward_workspace_bytes(int rows, int in, int out, int N, int M, elsa_dtype dtype);
 elsa_status elsa_nm_linear_backward(const void* dY, const void* X, int rows, const void* vals, const uint32_t* idx,

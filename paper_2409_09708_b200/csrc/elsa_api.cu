@@ -1083,20 +1083,16 @@ namespace elsa {
 namespace {
 
 struct BackwardPlan {
-    size_t wm, wmt, dyt, xt, partial, total;   // byte offsets of the regions
-    int rows_p;                                // rows rounded up to 64: reduction length of the dW product
+    size_t wm, wmt, partial, total;   // byte offsets of the regions
 };
 
 BackwardPlan backward_plan(int rows, int in, int out)
 {
     BackwardPlan p;
-    p.rows_p = (rows + 63) / 64 * 64;
     size_t at = 0;
-    p.wm = at;      at += round_up((size_t)out * in * 2, 256);                 // masked weight [out][in]
-    p.wmt = at;     at += round_up((size_t)out * in * 2, 256);                 // its transpose [in][out]
-    p.dyt = at;     at += round_up((size_t)out * p.rows_p * 2, 256);           // dY^T [out][rows_p]
-    p.xt = at;      at += round_up((size_t)in * p.rows_p * 2, 256);            // X^T  [in][rows_p]
-    p.partial = at; at += round_up((size_t)(p.rows_p / 64) * out * 4, 256);    // column sums of dY per 64 rows
+    p.wm = at;      at += round_up((size_t)out * in * 2, 256);                      // masked weight [out][in]
+    p.wmt = at;     at += round_up((size_t)out * in * 2, 256);                      // its transpose [in][out]
+    p.partial = at; at += round_up((size_t)((rows + 511) / 512) * out * 4, 256);    // column sums of dY per 512 rows
     p.total = at;
     return p;
 }
@@ -1155,21 +1151,16 @@ elsa_status elsa_nm_linear_backward(const void* dY, const void* X, int rows, con
             if ((st = launch_unpack((const uint16_t*)vals, idx, out, in, N, M, wm, stream)) != ELSA_OK) return st;
             dense = wm;
         }
-        if ((st = launch_transpose16(dense, wmt, out, in, out, nullptr, dtype, stream)) != ELSA_OK) return st;
+        if ((st = launch_transpose16(dense, wmt, out, in, out, stream)) != ELSA_OK) return st;
         if ((st = dense_product(dy, rows, wmt, in, out, dtype, (uint16_t*)dX, dev_status, stream, dev.sm_count)) != ELSA_OK) return st;
     }
-    if (dW || db) {
-        float* partial = (float*)(ws + plan.partial);
-        uint16_t* dyt = (uint16_t*)(ws + plan.dyt);
-        if ((st = launch_transpose16(dy, dyt, rows, out, plan.rows_p, db ? partial : nullptr, dtype, stream)) != ELSA_OK) return st;
-        if (db && (st = launch_colsum_finish(partial, plan.rows_p / 64, out, (uint16_t*)db, dtype, stream)) != ELSA_OK) return st;
-        if (dW) {
-            // dW = dY^T X, reduction over the token rows, then the mask
-            uint16_t* xt = (uint16_t*)(ws + plan.xt);
-            if ((st = launch_transpose16((const uint16_t*)X, xt, rows, in, plan.rows_p, nullptr, dtype, stream)) != ELSA_OK) return st;
-            if ((st = dense_product(dyt, out, xt, in, plan.rows_p, dtype, (uint16_t*)dW, dev_status, stream, dev.sm_count)) != ELSA_OK) return st;
-            if ((st = launch_mask_apply((uint16_t*)dW, idx, out, in, N, M, stream)) != ELSA_OK) return st;
-        }
+    if (db && (st = launch_colsum(dy, rows, out, (float*)(ws + plan.partial), (uint16_t*)db, dtype, stream)) != ELSA_OK) return st;
+    if (dW) {
+        // dW = dY^T X, reduction over the token rows: both operands are read as they are stored (reduction index
+        // outermost), then the mask
+        if ((st = launch_linear_tc_pair_tn(dy, (const uint16_t*)X, out, in, rows, dtype, (uint16_t*)dW, dev_status, stream)) != ELSA_OK)
+            return st;
+        if ((st = launch_mask_apply((uint16_t*)dW, idx, out, in, N, M, stream)) != ELSA_OK) return st;
     }
     return ELSA_OK;
 }

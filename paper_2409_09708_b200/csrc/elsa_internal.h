@@ -98,6 +98,10 @@ elsa_status launch_linear_tc_dense(const uint16_t* X, int rows, const uint16_t* 
 elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* Wd, const uint16_t* bias,
                                   int out, int in, elsa_dtype dtype, uint16_t* Y, uint32_t* dev_status,
                                   cudaStream_t stream);
+// Y [m][n] = A^T B on the same kernel with both operands stored reduction-outermost, A [k][m] and B [k][n]
+// (m, n multiples of 8): the weight-gradient product dY^T X without transposed copies.
+elsa_status launch_linear_tc_pair_tn(const uint16_t* A, const uint16_t* B, int m, int n, int k, elsa_dtype dtype,
+                                     uint16_t* Y, uint32_t* dev_status, cudaStream_t stream);
 // Levels with N <= 2 on the hardware 2:4 sparse MMA: re-encodes the packed weight into `workspace`
 // (2-of-4 values + metadata), then runs the sparse GEMM.
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
@@ -166,10 +170,9 @@ elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype
 elsa_status launch_copy_columns(const uint16_t* src, uint16_t* dst, int rows, int src_ld, int col0, int cols,
                                 cudaStream_t stream);
 // Operand forms of the backward pass.  transpose16: src [R][C] -> dst [C][Rp] with the tail R..Rp zero (C, Rp
-// multiples of 8); partial (or NULL) receives [ceil(R / 64)][C] fp32 column sums per 64-row tile.
-elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C, int Rp, float* partial,
-                               elsa_dtype dtype, cudaStream_t stream);
-elsa_status launch_colsum_finish(const float* partial, int tiles, int C, uint16_t* db, elsa_dtype dtype, cudaStream_t stream);
+// multiples of 8).  colsum: db [C] = column sums of src [R][C], through ceil(R / 512) * C floats of scratch.
+elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C, int Rp, cudaStream_t stream);
+elsa_status launch_colsum(const uint16_t* src, int R, int C, float* partial, uint16_t* db, elsa_dtype dtype, cudaStream_t stream);
 // Zeroes the pruned positions of a dense [out][in] tensor in place.
 elsa_status launch_mask_apply(uint16_t* dW, const uint32_t* idx, int out, int in, int N, int M, cudaStream_t stream);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.

@@ -84,8 +84,12 @@ struct PairGroup {
 
 constexpr int kStageBytesMax = kATileBytes + (kMaxBlockN / 2) * kBlockK * 2;   // stage slots sized for BN = 256
 // Forms of the kernel: plain (acc + bias), INT8 (integer operands, scaled in the epilogue), fused (activation and
-// residual added in the epilogue). Separate instantiations, so the plain form pays nothing for the other two.
-constexpr int kFormPlain = 0, kFormInt8 = 1, kFormFused = 2;
+// residual added in the epilogue), Tn (both operands stored with the reduction index outermost: A [K][M] and
+// B [K][N], the weight-gradient product dY^T X; tiles arrive as boxes of 64 features x 64 reduction rows and the
+// MMA reads them through MN-major descriptors). Separate instantiations, so the plain form pays nothing for the
+// others.
+constexpr int kFormPlain = 0, kFormInt8 = 1, kFormFused = 2, kFormTn = 3;
+constexpr int kTnBoxBytes = 64 * 64 * 2;   // one box of the Tn form: 64 reduction rows of 128 bytes
 constexpr int kGroupMax = 72;   // layers per grouped launch (kernel parameters are limited to 32 KB)
 
 // kInt8: operands are signed 8-bit integers (rows of 128 elements per 128-byte swizzle row, K = 32 per MMA,
@@ -97,6 +101,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 {
     constexpr bool kInt8 = kForm == kFormInt8;     // 8-bit integer operands, scales in the epilogue
     constexpr bool kFused = kForm == kFormFused;   // activation and residual in the epilogue
+    constexpr bool kTn = kForm == kFormTn;         // operands [K][M] and [K][N]
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -179,8 +184,17 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                         // the leader's stage barrier collects the bytes of both CTAs
                         if (cta_rank == 0) mbar_arrive_expect_tx(full_bar + 8 * stage, tx_bytes);
                         // a stage is 128 bytes of K per row: 64 16-bit or 128 8-bit elements
-                        tma_load_2d_pair(a_dst, &L.map_x, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), m0);
-                        tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), n0);
+                        if constexpr (kTn) {
+                            // boxes of 64 features x 64 reduction rows, 8 KB each: this CTA's 128 rows of A and its
+                            // half of B's columns
+                            for (int i = 0; i < kRowsPerCta / 64; ++i)
+                                tma_load_2d_pair(a_dst + (uint32_t)(i * kTnBoxBytes), &L.map_x, bar, m0 + 64 * i, kb * kBlockK);
+                            for (int i = 0; i < half_bn / 64; ++i)
+                                tma_load_2d_pair(a_dst + kATileBytes + (uint32_t)(i * kTnBoxBytes), &L.map_w, bar, n0 + 64 * i, kb * kBlockK);
+                        } else {
+                            tma_load_2d_pair(a_dst, &L.map_x, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), m0);
+                            tma_load_2d_pair(a_dst + kATileBytes, &L.map_w, bar, kb * (kInt8 ? 2 * kBlockK : kBlockK), n0);
+                        }
                     }
                     __syncwarp();
                     if (++stage == p.stages) { stage = 0; phase ^= 1u; }
@@ -219,11 +233,16 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t a_addr = smem_base + (uint32_t)(stage * stage_bytes);
-                    const uint64_t a_desc = smem_desc_k_major_sw128(a_addr);
-                    const uint64_t b_desc = smem_desc_k_major_sw128(a_addr + kATileBytes);
+                    const uint64_t a_desc = kTn ? smem_desc_mn_major_sw128(a_addr, kTnBoxBytes) : smem_desc_k_major_sw128(a_addr);
+                    const uint64_t b_desc = kTn ? smem_desc_mn_major_sw128(a_addr + kATileBytes, kTnBoxBytes)
+                                                : smem_desc_k_major_sw128(a_addr + kATileBytes);
 #pragma unroll
                     for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-                        if constexpr (kInt8)
+                        if constexpr (kTn)
+                            // 16 reduction rows of 128 bytes per MMA: the start address moves by 2048 bytes
+                            umma_f16_pair_if(d_tmem, a_desc + (uint64_t)(k * (kUmmaK * 128 >> 4)), b_desc + (uint64_t)(k * (kUmmaK * 128 >> 4)),
+                                             idesc, (uint32_t)((kb | k) != 0), elected);
+                        else if constexpr (kInt8)
                             umma_i8_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                             (uint32_t)((kb | k) != 0), elected);
                         else
@@ -431,14 +450,24 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
     }
 }
 
-int pick_pair_block_n(int out)
+// Width of a pair tile in output features.  Cost model: the tiles run in waves over the SM pairs, a tile costs
+// its width plus a fixed share (operand staging, pipeline fill), and features past `out` in the last tile are
+// wasted work; among equals the widest wins (fewest re-reads of X).  For the large layers this picks 256 or
+// the width that divides `out`; below a wave of tiles it narrows the tile until the pairs are occupied.
+int pick_pair_block_n(int out, int rows, int sm_count, bool whole_boxes = false)
 {
-    int best = 64, best_waste = 1 << 30;
+    const int pairs = sm_count / 2 > 0 ? sm_count / 2 : 1;
+    const long long row_tiles = (rows + kPairRows - 1) / kPairRows;
+    int best = 64;
+    long long best_cost = -1;
     const int cand[4] = {256, 192, 128, 64};
     for (int i = 0; i < 4; ++i) {
         const int bn = cand[i];
-        const int waste = (out + bn - 1) / bn * bn - out;
-        if (waste < best_waste) { best = bn; best_waste = waste; }
+        if (whole_boxes && bn % 128 != 0) continue;   // the Tn form loads each CTA's half in boxes of 64 features
+        const long long tiles = row_tiles * ((out + bn - 1) / bn);
+        const long long waves = (tiles + pairs - 1) / pairs;
+        const long long cost = waves * (bn + 32);
+        if (best_cost < 0 || cost < best_cost) { best = bn; best_cost = cost; }
     }
     return best;
 }
@@ -448,7 +477,7 @@ int pick_pair_block_n(int out)
 bool linear_tc_pair_suits(int rows, int out, int sm_count)
 {
     // worth pairing CTAs only when there are enough 256-row tiles to occupy every SM pair
-    const int bn = pick_pair_block_n(out);
+    const int bn = pick_pair_block_n(out, rows, sm_count);
     const long long tiles = (long long)((rows + kPairRows - 1) / kPairRows) * ((out + bn - 1) / bn);
     return tiles >= sm_count / 2;
 }
@@ -469,7 +498,7 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
         const PairJob& j = jobs[i];
         PairLayer& L = g.layer[i];
         L.rows = j.rows; L.out = j.out;
-        L.bn = pick_pair_block_n(j.out);
+        L.bn = pick_pair_block_n(j.out, j.rows, dev.sm_count, kForm == kFormTn);
         L.tiles_n = (j.out + L.bn - 1) / L.bn;
         L.tile_begin = tile_begin;
         tile_begin += ((j.rows + kPairRows - 1) / kPairRows) * L.tiles_n;
@@ -488,6 +517,17 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
                 return st;
             if ((st = make_map_2d_u8(&L.map_w, j.Wd, (uint64_t)j.in, (uint64_t)j.out, 2 * kBlockK, (uint32_t)(L.bn / 2),
                                      CU_TENSOR_MAP_SWIZZLE_128B, "W")) != ELSA_OK)
+                return st;
+        } else if constexpr (kForm == kFormTn) {
+            // A = j.X [in][rows] and B = j.Wd [in][out], `in` the reduction: both MN-major (bits 15 and 16)
+            L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
+            L.idesc = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(L.bn >> 3) << 17) |
+                      ((uint32_t)(kPairRows >> 4) << 24);
+            if ((st = make_map_2d(&L.map_x, j.X, (uint64_t)j.rows, (uint64_t)j.in, 64, kBlockK, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  "A")) != ELSA_OK)
+                return st;
+            if ((st = make_map_2d(&L.map_w, j.Wd, (uint64_t)j.out, (uint64_t)j.in, 64, kBlockK, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  "B")) != ELSA_OK)
                 return st;
         } else {
             L.num_k_blocks = (j.in + kBlockK - 1) / kBlockK;
@@ -577,6 +617,20 @@ elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype d
                                   : launch_group<false, kFormPlain, 1>(jobs, 1, dtype, dev_status, stream, dev);
     return dtype == ELSA_BF16 ? launch_group<true, kFormPlain, kGroupMax>(jobs, n, dtype, dev_status, stream, dev)
                               : launch_group<false, kFormPlain, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
+}
+
+// Y [m][n] = A^T B with A [k][m] and B [k][n] (the reduction index outermost in both), no bias: one launch.
+elsa_status launch_linear_tc_pair_tn(const uint16_t* A, const uint16_t* B, int m, int n, int k, elsa_dtype dtype,
+                                     uint16_t* Y, uint32_t* dev_status, cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    PairJob job;
+    job.X = A; job.Wd = B; job.bias = nullptr; job.Y = Y;
+    job.rows = m; job.in = k; job.out = n;
+    return dtype == ELSA_BF16 ? launch_group<true, kFormTn, 1>(&job, 1, dtype, dev_status, stream, dev)
+                              : launch_group<false, kFormTn, 1>(&job, 1, dtype, dev_status, stream, dev);
 }
 
 // INT8 form (one layer per launch): X and Wd hold signed 8-bit integers, Y is 16-bit.

@@ -184,6 +184,20 @@ __device__ __forceinline__ uint64_t smem_desc_k_major_sw128(uint32_t addr)
     return d;
 }
 
+// Shared-memory matrix descriptor of an MN-major tile: rows of 128 bytes (64 16-bit values along M or N) per
+// reduction index, written by TMA with the 128-byte swizzle.  8 reduction rows form a 1024-byte group (stride
+// offset); blocks of 64 values along M / N are `block_bytes` apart (leading offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_major_sw128(uint32_t addr, uint32_t block_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
 template <bool kBf16>
 __device__ __forceinline__ uint32_t pack2(float lo, float hi)
 {
