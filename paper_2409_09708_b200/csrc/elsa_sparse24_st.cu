@@ -5,27 +5,27 @@
 // re-encoding of the packed weight).  At the sparse MMA rate shared memory cannot carry both operands:
 // the pair kernel stages the compressed weight tile beside the activations for every row tile and
 // runs at about half the sparse rate, and the weight-stationary kernel avoids it only while the whole
-// reduction dimension of a 256-feature block fits tensor memory (in <= 768 beside two accumulators).
+// reduction dimension of a 256-feature block fits tensor memory (in <= 896 beside two accumulators).
 // Here the block's weight is cut into K chunks of 256.  Loader warps read a chunk from
-// global memory (L2-resident image) into registers and write it into one of three tensor-memory
+// global memory (L2-resident image) into registers and write it into one of four tensor-memory
 // slots (tcgen05.st: 64 columns of 2-of-4 values, 8 of metadata, per lane = per feature); every
 // tcgen05.mma.sp takes its A operand and metadata from the slot, and shared memory carries
-// activations only.  The chunk of a row tile that is multiplied, the one being written and the one
-// being fetched occupy the three slots.
+// activations only (three stages of 256 of K).  While one slot is multiplied the next ones are being
+// written and fetched: a load from L2 takes 1.5-2.5 us under this traffic, several chunk times.
 //
-// A CTA pair owns a tile of 256 features x 256 token rows; tiles of all layers of a launch form one
-// sequence walked with the stride of the pairs, feature blocks fastest, so that the pairs that share
-// activation rows read them at the same time (once from HBM, then from L2).  One accumulator of 256
-// columns: with a reduction this long the epilogue's share is small, and the wide tile halves the
-// weight bytes per multiply-accumulate that cross L2.
+// A CTA pair owns a tile of 256 features x 224 token rows (one accumulator of 224 columns beside the
+// four slots of 72); tiles of all layers of a launch form one sequence walked with the stride of the
+// pairs, feature blocks fastest, so that the pairs that share activation rows read them at the same
+// time (once from HBM, then from L2).  With a reduction this long the epilogue's share is small.
 //
-// Per CTA (704 threads): warp 0 TMA producer of this CTA's 128 activation rows, warp 1 tensor-memory
-// allocation and (leader) MMA issue, warps 2-9 epilogue (two per tensor-memory lane quarter, see
-// elsa_sparse24_ws.cu for the transposing stmatrix stores and the lane order of the features),
-// warps 10-21 weight loaders (three per lane quarter, one per slot).  The weight image is read in the `tiled` form of
-// nm_to_sp24: rows in the permuted lane order, and inside a block of 32 rows x 256 k the 16-byte
-// units of all rows interleaved, so that a warp's load is one contiguous run.  Waits are bounded as
-// in the other kernels.
+// Per CTA (640 threads, 96 registers each): warp 0 TMA producer of this CTA's 112 activation rows,
+// warp 1 tensor-memory allocation and (leader) MMA issue, warps 2-9 epilogue (two per tensor-memory
+// lane quarter, see elsa_sparse24_ws.cu for the transposing stmatrix stores and the lane order of the
+// features), warps 10-17 weight loaders (two per lane quarter, taking alternate chunks: the loads of a
+// chunk are issued before the wait for its slot, and the next chunk is requested right after the
+// tcgen05.st of this one).  The weight image is read in the `tiled` form of nm_to_sp24: rows in the
+// permuted lane order, and inside a block of 32 rows x 256 k the 16-byte units of all rows
+// interleaved, so that a warp's load is one contiguous run.  Waits are bounded as in the other kernels.
 
 #include <atomic>
 #include <mutex>
