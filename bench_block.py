@@ -81,7 +81,8 @@ def main():
     lib.elsa_profile_start()
     one_pass()
     families = {}
-    for kernel, _, ms in lib.elsa_profile_stop():
+    launch_list = lib.elsa_profile_stop()
+    for kernel, _, ms in launch_list:
         f = families.setdefault(kernel, {"launches": 0, "ms": 0.0})
         f["launches"] += 1
         f["ms"] += ms
@@ -95,7 +96,8 @@ def main():
            "images_per_s_linear_and_elementwise_path": args.batch / ms * 1e3,
            "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "peaks": peaks_kind,
            "linears_roofline_ms": lin_roof * 1e3, "elementwise_bytes": elementwise_bytes,
-           "families_profiled_pass": families, "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
+           "families_profiled_pass": families,
+           "first_block_launches": [[k, round(ms, 4)] for k, _, ms in launch_list[:len(launch_list) // args.blocks + 2]], "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     json.dump(rec, open(args.out, "w"), indent=1)
     print(json.dumps(rec))
