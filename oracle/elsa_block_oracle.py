@@ -8,8 +8,12 @@ models).  The block is the standard pre-norm one of DeiT:
     x2 = x + Linear_proj(a);  x3 = LayerNorm2(x2);  h = GELU(Linear_fc1(x3));  y = x2 + Linear_fc2(h)
 with LayerNorm over the feature dimension (biased variance, eps inside the square root, elementwise gain and
 bias) and GELU(v) = v * Phi(v) = 0.5 * v * (1 + erf(v / sqrt 2)), the exact form (not the tanh approximation).
-The attention products (QK^T, softmax, AV) are NOT part of this oracle: `attention` is the stated stand-in
-a = V, the last third of qkv copied through, so that the linear and elementwise path can be checked and timed.
+`attention` comes in two forms.  "copy_v": the stated stand-in a = V, the last third of qkv copied through, with
+which the linear and elementwise path can be checked and timed alone.  "softmax": the multi-head self-attention
+of the ViT / DeiT backbones the paper prunes (the paper leaves the attention products unpruned and gives no
+formula of its own: this is the standard one): per image and head, with q, k, v the head's slices of the three
+thirds of qkv and d the head dimension, a = softmax(q k^T / sqrt d) v, the softmax over the keys of the same image;
+heads are laid side by side in a's columns.  All tokens of an image attend to each other (no mask, no dropout).
 
 Every tensor that crosses a stage boundary is a 16-bit tensor (the library writes it to memory in the block's
 dtype), so every stage here computes in fp64 from its 16-bit inputs and rounds its result once, to nearest
@@ -53,9 +57,29 @@ def sparse_linear(x16, W_bits, bias_bits, N, M, code):
     return eo.nm_linear_f64(_bits(x16, torch_dtype), vals, idx, bias_bits, W_bits.shape[0], W_bits.shape[1], N, M, code)
 
 
-def block_forward(x_bits, p, code, eps=1e-6):
+def attention(qkv, tokens, heads):
+    """fp64 multi-head self-attention.  qkv: [images * tokens, 3 * dim] (q | k | v thirds, heads side by side in
+    each); returns [images * tokens, dim].  Plain loops over images and heads; softmax written out."""
+    rows, three_dim = qkv.shape
+    dim = three_dim // 3
+    d = dim // heads
+    out = np.zeros((rows, dim))
+    for b in range(rows // tokens):
+        r = slice(b * tokens, (b + 1) * tokens)
+        for h in range(heads):
+            q = qkv[r, h * d:(h + 1) * d]
+            k = qkv[r, dim + h * d:dim + (h + 1) * d]
+            v = qkv[r, 2 * dim + h * d:2 * dim + (h + 1) * d]
+            s = q @ k.T / math.sqrt(d)
+            e = np.exp(s - s.max(axis=1, keepdims=True))
+            out[r, h * d:(h + 1) * d] = (e / e.sum(axis=1, keepdims=True)) @ v
+    return out
+
+
+def block_forward(x_bits, p, code, eps=1e-6, attn="copy_v", tokens=None, heads=None):
     """x_bits: uint16 [rows, dim].  p: dict with ln1_g, ln1_b, ln2_g, ln2_b (uint16 [dim]) and, for each of qkv,
     proj, fc1, fc2: W_<name> (uint16 [out, in]), b_<name> (uint16 [out]), level_<name> = (N, M).
+    attn: "copy_v" or "softmax" (then tokens per image and heads are required; rows = images * tokens).
     Returns a dict of every stage's 16-bit result as fp64 arrays: x1, qkv, a, x2, x3, h, y."""
     torch_dtype = torch.float16 if code == eo.F16 else torch.bfloat16
 
@@ -67,7 +91,10 @@ def block_forward(x_bits, p, code, eps=1e-6):
     out = {}
     out["x1"] = _round16(layer_norm(x, f64(p["ln1_g"]), f64(p["ln1_b"]), eps), torch_dtype)
     out["qkv"] = _round16(sparse_linear(out["x1"], p["W_qkv"], p["b_qkv"], *p["level_qkv"], code), torch_dtype)
-    out["a"] = out["qkv"][:, 2 * dim:3 * dim].copy()                 # the stated stand-in for attention: a = V
+    if attn == "copy_v":
+        out["a"] = out["qkv"][:, 2 * dim:3 * dim].copy()             # the stated stand-in for attention: a = V
+    else:
+        out["a"] = _round16(attention(out["qkv"], tokens, heads), torch_dtype)
     out["x2"] = _round16(x + sparse_linear(out["a"], p["W_proj"], p["b_proj"], *p["level_proj"], code), torch_dtype)
     out["x3"] = _round16(layer_norm(out["x2"], f64(p["ln2_g"]), f64(p["ln2_b"]), eps), torch_dtype)
     out["h"] = _round16(gelu(sparse_linear(out["x3"], p["W_fc1"], p["b_fc1"], *p["level_fc1"], code)), torch_dtype)

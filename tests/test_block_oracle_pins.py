@@ -75,3 +75,63 @@ def test_block_chain_against_torch_fp64_routines():
     # a mistake anywhere shows: dropping a residual, the wrong GELU, or the wrong third of qkv
     assert np.abs(got["x2"] - (got["x2"] - x.double().numpy())).max() > 0.1
     assert not np.array_equal(got["a"], got["qkv"][:, :dim])
+
+
+def test_attention_against_torch_and_closed_forms():
+    rng = np.random.default_rng(3)
+    images, tokens, heads, d = 3, 7, 2, 4
+    dim = heads * d
+    qkv = rng.standard_normal((images * tokens, 3 * dim))
+    got = bo.attention(qkv, tokens, heads)
+    # torch's fused routine in fp64 on [images, heads, tokens, d] views
+    t = torch.from_numpy(qkv).view(images, tokens, 3, heads, d).permute(2, 0, 3, 1, 4)
+    ref = torch.nn.functional.scaled_dot_product_attention(t[0], t[1], t[2]).permute(0, 2, 1, 3).reshape(images * tokens, dim)
+    assert np.allclose(got, ref.numpy(), rtol=1e-12, atol=1e-12)
+    # hand-worked: one image, one head, two tokens, d = 1: scores q_i k_j, weights by softmax
+    q, k, v = np.array([1.0, 0.0]), np.array([2.0, -1.0]), np.array([10.0, 20.0])
+    w0 = math.exp(2.0) / (math.exp(2.0) + math.exp(-1.0))
+    hand = bo.attention(np.stack([q, k, v], axis=1), 2, 1)
+    assert np.allclose(hand[:, 0], [w0 * 10 + (1 - w0) * 20, 15.0], atol=1e-12)     # q = 0 attends uniformly
+    # zero queries: every token gets the mean of its own image's values, never another image's
+    z = qkv.copy()
+    z[:, :dim] = 0.0
+    mean_v = z[:, 2 * dim:].reshape(images, tokens, dim).mean(axis=1)
+    assert np.allclose(bo.attention(z, tokens, heads).reshape(images, tokens, dim), mean_v[:, None, :], atol=1e-12)
+    # the keys' order inside an image does not matter; the 1 / sqrt d scale does
+    perm = rng.permutation(tokens)
+    shuffled = qkv.reshape(images, tokens, 3 * dim).copy()
+    shuffled[:, :, dim:] = shuffled[:, perm, dim:]
+    assert np.allclose(bo.attention(shuffled.reshape(-1, 3 * dim), tokens, heads), got, atol=1e-12)
+    unscaled = qkv.copy()
+    unscaled[:, :dim] *= math.sqrt(d)
+    assert not np.allclose(bo.attention(unscaled, tokens, heads), got, atol=1e-3)
+    # a shift common to all keys cancels in the softmax
+    shifted = qkv.copy()
+    shifted[:, dim:2 * dim] += 1.0
+    assert np.allclose(bo.attention(shifted, tokens, heads), got, atol=1e-12)
+    # heads are independent: changing head 1's keys leaves head 0's output alone
+    other = qkv.copy()
+    other[:, dim + d:2 * dim] *= 2.0
+    assert np.allclose(bo.attention(other, tokens, heads)[:, :d], got[:, :d], atol=1e-12)
+    assert not np.allclose(bo.attention(other, tokens, heads)[:, d:], got[:, d:], atol=1e-3)
+
+
+def test_block_chain_with_attention_against_torch():
+    dtype = torch.bfloat16
+    images, tokens, heads, dim, mlp = 2, 5, 2, 16, 32
+    rows = images * tokens
+    x = synth.randn((rows, dim), 41, 1.0, dtype)
+    p = {}
+    shapes = {"qkv": (3 * dim, dim), "proj": (dim, dim), "fc1": (mlp, dim), "fc2": (dim, mlp)}
+    for i, (name, (o, k)) in enumerate(shapes.items()):
+        p["W_" + name] = synth.bits(synth.randn((o, k), 50 + i, 0.2, dtype))
+        p["b_" + name] = synth.bits(synth.randn((o,), 60 + i, 0.02, dtype))
+        p["level_" + name] = (2, 4)
+    for i, name in enumerate(("ln1_g", "ln1_b", "ln2_g", "ln2_b")):
+        p[name] = synth.bits((synth.randn((dim,), 70 + i, 0.1, dtype) + (1.0 if name.endswith("g") else 0.0)).to(dtype))
+    got = bo.block_forward(synth.bits(x), p, eo.BF16, attn="softmax", tokens=tokens, heads=heads)
+    qkv = torch.from_numpy(got["qkv"]).view(images, tokens, 3, heads, dim // heads).permute(2, 0, 3, 1, 4)
+    a = torch.nn.functional.scaled_dot_product_attention(qkv[0], qkv[1], qkv[2]).permute(0, 2, 1, 3).reshape(rows, dim)
+    a16 = a.to(dtype).double().numpy()
+    assert (np.abs(got["a"] - a16) <= 2.0 ** -7 * np.abs(a16) + 1e-30).all() and (got["a"] == a16).mean() > 0.95
+    assert not np.allclose(got["a"], got["qkv"][:, 2 * dim:])            # not the stand-in
