@@ -275,7 +275,8 @@ typedef enum {
     ELSA_KERNEL_LINEAR_TC_PAIR_I8 = 11, /* INT8 form of the CTA-pair GEMM */
     ELSA_KERNEL_INT8_FORMAT = 12,       /* INT8 compress / unpack */
     ELSA_KERNEL_BLOCK_ROWWISE = 13,     /* LayerNorm, residual add, GELU, column copy of the chained block */
-    ELSA_KERNEL_BACKWARD_FORMAT = 14    /* transposes, column sums and mask of the backward pass */
+    ELSA_KERNEL_BACKWARD_FORMAT = 14,   /* transposes, column sums and mask of the backward pass */
+    ELSA_KERNEL_ATTENTION = 15          /* multi-head self-attention of the chained block */
 } elsa_kernel_id;
 
 typedef struct {
@@ -370,10 +371,14 @@ elsa_status elsa_config_from_index(const char* index_decimal, int n_layers, int 
  * bias per feature); GELU is the exact form v * Phi(v).  Statistics, bias, activation and residual are computed
  * in fp32 and every tensor that crosses a stage boundary is rounded once to `dtype` (where a linear runs on a
  * kernel whose epilogue cannot take the residual, its output is rounded before the residual is added).
- * The attention products (QK^T, softmax, AV) are NOT part of this library: elsa_vit_block_qkv runs the block up
- * to qkv, the caller's attention turns qkv into a [rows][dim], elsa_vit_block_rest runs the block from proj on.
- * elsa_vit_block runs both with the stand-in a = V (columns 2 dim .. 3 dim of qkv copied through), which is what
- * the parity tests and the block timing use; it does not compute a transformer block's attention.
+ * Attention: the paper prunes the linear modules and leaves the attention products dense.  Three ways to run it:
+ * elsa_vit_block_attn runs the whole block with the library's multi-head self-attention (elsa_attention:
+ * a = softmax(q k^T / sqrt d) v per image and head over the image's own tokens, no mask; at most 256 tokens per
+ * image, head dimension 64, i.e. the ViT / DeiT shapes; windowed attention with a position bias, as in Swin, is not
+ * built); elsa_vit_block_qkv runs the block up to qkv, the caller's own attention turns qkv into a [rows][dim] in
+ * region A, and elsa_vit_block_rest runs the block from proj on; elsa_vit_block runs both halves with the stand-in
+ * a = V (columns 2 dim .. 3 dim of qkv copied through), which times the linear and elementwise path alone and does
+ * not compute a transformer block's attention.
  *
  * All pointers are DEVICE pointers, 16-byte aligned; dim and mlp_dim multiples of 8 and of every M in use.
  * Weights are the packed forms elsa_nm_compress writes: qkv [3 dim][dim], proj [dim][dim], fc1 [mlp_dim][dim],
@@ -425,6 +430,15 @@ elsa_status elsa_vit_block_rest(const void* x, int rows, int dim, int mlp_dim, c
 /* Both, with the stand-in a = V between them. */
 elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                            void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream);
+/* qkv [images * tokens][3 dim] (q | k | v thirds, heads side by side in each) -> a [images * tokens][dim]; the
+ * scores and probabilities stay on chip (fp32 scores, probabilities rounded to `dtype` for the second product, fp32
+ * row sums, one rounding of a).  dim = 64 * heads, tokens <= 256. */
+elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype, void* a,
+                           uint32_t* dev_status, void* stream);
+/* The whole block with elsa_attention between the halves; rows = images * tokens. */
+elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
+                                const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                                uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Backward pass of the masked linear (Alg. 2, supernet training: the gradient is taken with respect to the

@@ -123,6 +123,8 @@ _block_scratch = _sig("elsa_vit_block_scratch_bytes", _sz, [_i, _i, _i, _bw, _i,
 _block_qkv = _sig("elsa_vit_block_qkv", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _sz, _vp, _vp])
 _block_rest = _sig("elsa_vit_block_rest", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _block = _sig("elsa_vit_block", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
+_block_attn = _sig("elsa_vit_block_attn", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
+_attention = _sig("elsa_attention", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 
 
 class ElsaKernelTime(ctypes.Structure):
@@ -130,7 +132,7 @@ class ElsaKernelTime(ctypes.Structure):
 
 
 KERNEL_NAMES = {0: "nm_compress", 1: "nm_unpack", 2: "linear_simt", 3: "linear_tc_dense", 4: "linear_tc_pair", 5: "nm_to_sp24", 6: "linear_tc_sp24", 7: "linear_tc_sp24_pair", 8: "weight_images",
-                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format", 13: "block_rowwise", 14: "backward_format"}
+                9: "linear_tc_sp24_ws", 10: "linear_tc_sp24_st", 11: "linear_tc_pair_i8", 12: "int8_format", 13: "block_rowwise", 14: "backward_format", 15: "attention"}
 _profile_start = _sig("elsa_profile_start", _i, [])
 _profile_stop = _sig("elsa_profile_stop", _i, [ctypes.POINTER(ElsaKernelTime), _i])
 
@@ -414,10 +416,23 @@ def elsa_vit_block_scratch_bytes(rows, dim, mlp_dim, weights, dtype_c):
     return n, dict(zip(BLOCK_REGIONS, off))
 
 
-def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, stream=None, phase="both"):
+def elsa_attention(qkv, tokens, heads, a=None, dev_status=None, stream=None):
+    """a [rows, dim] = multi-head self-attention of qkv [rows, 3 dim], rows = images * tokens."""
+    rows, three_dim = qkv.shape
+    dim = three_dim // 3
+    if a is None:
+        a = torch.empty((rows, dim), dtype=qkv.dtype, device=qkv.device)
+    _check(_attention(_ptr(qkv), rows // tokens, tokens, heads, dim, dtype_code(qkv.dtype), _ptr(a), _ptr(dev_status),
+                      _stream(stream)))
+    return a
+
+
+def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, stream=None, phase="both", tokens=None,
+                   heads=None):
     """One pre-norm ViT block over x [rows, dim] with the four linears in their packed N:M forms.  phase "both"
-    runs the whole block with the stand-in a = V for attention; "qkv" stops after qkv (regions x1, qkv of
-    scratch); "rest" continues from region a of scratch, which the caller's attention has written."""
+    runs the whole block, with the library's attention when tokens (per image) and heads are given and with the
+    stand-in a = V otherwise; "qkv" stops after qkv (regions x1, qkv of scratch); "rest" continues from region a
+    of scratch, which the caller's attention has written."""
     rows, dim = x.shape
     code = dtype_code(x.dtype)
     if scratch is None:
@@ -427,6 +442,9 @@ def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, s
     if phase == "qkv":
         _check(_block_qkv(_ptr(x), rows, dim, mlp_dim, ctypes.byref(weights), code, _ptr(scratch), scratch.numel(),
                           _ptr(dev_status), _stream(stream)))
+    elif phase == "both" and tokens:
+        _check(_block_attn(_ptr(x), rows // tokens, tokens, heads, dim, mlp_dim, ctypes.byref(weights), code, _ptr(y),
+                           _ptr(scratch), scratch.numel(), _ptr(dev_status), _stream(stream)))
     else:
         fn = _block if phase == "both" else _block_rest
         _check(fn(_ptr(x), rows, dim, mlp_dim, ctypes.byref(weights), code, _ptr(y), _ptr(scratch), scratch.numel(),

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libelsa.so")
-SOURCES = ["elsa_api.cu", "elsa_backward.cu", "elsa_block.cu", "elsa_compress.cu", "elsa_int8.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu", "elsa_linear_tc2.cu",
+SOURCES = ["elsa_api.cu", "elsa_attention.cu", "elsa_backward.cu", "elsa_block.cu", "elsa_compress.cu", "elsa_int8.cu", "elsa_linear_simt.cu", "elsa_linear_tc.cu", "elsa_linear_tc2.cu",
            "elsa_no_alloc.cu", "elsa_search.cu", "elsa_selftest.cu", "elsa_sparse24.cu", "elsa_sparse24_pair.cu", "elsa_sparse24_st.cu", "elsa_sparse24_ws.cu"]
 
 

@@ -1036,8 +1036,14 @@ elsa_status elsa_vit_block_rest(const void* x, int rows, int dim, int mlp_dim, c
                       dev_status, (cudaStream_t)stream);
 }
 
-elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
-                           void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_)
+}  // extern "C"
+
+namespace elsa {
+namespace {
+
+// The whole block; tokens == 0 runs the stand-in a = V, otherwise the attention kernel over images of `tokens` rows.
+elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                      void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_, int tokens, int heads)
 {
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
@@ -1067,11 +1073,49 @@ elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const 
     }
     uint8_t* s8 = (uint8_t*)scratch;
     if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream)) != ELSA_OK) return st;
-    // the stated stand-in for attention: a = V
-    if ((st = launch_copy_columns((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]),
-                                  rows, 3 * dim, 2 * dim, dim, stream)) != ELSA_OK)
-        return st;
+    if (tokens == 0) {
+        // the stated stand-in for attention: a = V
+        st = launch_copy_columns((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]),
+                                 rows, 3 * dim, 2 * dim, dim, stream);
+    } else {
+        st = launch_attention((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), rows / tokens, tokens, heads, dim, dtype,
+                              (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]), dev_status, stream);
+    }
+    if (st != ELSA_OK) return st;
     return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream);
+}
+
+}  // namespace
+}  // namespace elsa
+
+extern "C" {
+
+elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
+                           void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream)
+{
+    return run_block(x, rows, dim, mlp_dim, w, dtype, y, scratch, scratch_bytes, dev_status, stream, 0, 0);
+}
+
+elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype, void* a,
+                           uint32_t* dev_status, void* stream)
+{
+    if (!qkv || !a) return fail(ELSA_ERR_NULL, "qkv and a must not be NULL");
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return fail(ELSA_ERR_DTYPE, "dtype %d is neither ELSA_F16 nor ELSA_BF16", (int)dtype);
+    if (images <= 0) return fail(ELSA_ERR_SHAPE, "non-positive images=%d", images);
+    if (!aligned16(qkv) || !aligned16(a)) return fail(ELSA_ERR_ALIGN, "qkv and a must be 16-byte aligned");
+    return launch_attention((const uint16_t*)qkv, images, tokens, heads, dim, dtype, (uint16_t*)a, dev_status, (cudaStream_t)stream);
+}
+
+elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
+                                const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                                uint32_t* dev_status, void* stream)
+{
+    if (images <= 0 || tokens <= 0) return fail(ELSA_ERR_SHAPE, "non-positive images=%d or tokens=%d", images, tokens);
+    if (!attention_suits(tokens, heads, dim))
+        return fail(ELSA_ERR_SHAPE, "attention needs at most 256 tokens per image and dim = 64 * heads (tokens=%d, heads=%d, dim=%d)",
+                    tokens, heads, dim);
+    if ((long long)images * tokens > 0x7fffffffLL) return fail(ELSA_ERR_SHAPE, "images * tokens does not fit an int");
+    return run_block(x, images * tokens, dim, mlp_dim, w, dtype, y, scratch, scratch_bytes, dev_status, stream, tokens, heads);
 }
 
 }  // extern "C"

@@ -1,0 +1,297 @@
+// Multi-head self-attention of the ViT block between the pruned qkv and proj linears (ELSA, Sec. 3: the paper
+// prunes the four linear modules and leaves the attention products dense; Sec. 4.2 measures whole models).
+//     a[img, :, h] = softmax(q k^T / sqrt d) v      per image and head, over the keys of the same image
+// with q, k, v the head's 64 columns in the three thirds of qkv [images * tokens][3 * dim].
+//
+// One CTA per (128 query rows, head, image); tokens <= 256, head dimension 64 (the ViT / DeiT shapes).  Both
+// products run on tcgen05 with everything between them kept on chip:
+//   1. TMA brings the Q tile, all K rows and all V rows of the head into shared memory (128-byte swizzle; a 3-D
+//      tensor map [image][token][column] zero-fills the rows past the image's last token).
+//   2. S = Q K^T: four MMAs (K = 16 each) into Tk = tokens rounded up to 16 fp32 columns of tensor memory.
+//   3. Four warps, one query row per lane: row maximum over the real keys, p = 2^((s - max) * log2(e) / 8), row
+//      sum in fp32, p rounded to the 16-bit type and written back into tensor memory as the A operand of the
+//      second product, two keys per column, over the low half of the columns S occupied.
+//   4. O = P V: Tk / 16 MMAs with A from tensor memory and V as it lies in memory (keys outermost: MN-major
+//      descriptor) into 64 columns of the part of S that is dead by then.
+//   5. The same four warps read O, divide by the row sum, round once and store each row's 128 bytes.
+// 256 columns of tensor memory and 81 KB of shared memory per CTA: two CTAs share an SM, one's products overlap the
+// other's softmax.  Every wait is bounded as in the GEMM kernels.
+#include <atomic>
+#include <mutex>
+
+#include "elsa_tc_common.cuh"
+
+namespace elsa {
+namespace {
+
+constexpr int kHeadDim = 64;
+constexpr int kQRows = 128;          // query rows per CTA = TMEM lanes
+constexpr int kMaxTokens = 256;
+constexpr int kTmemCols = 256;
+constexpr int kSoftmaxWarps = 4;
+constexpr int kThreads = (kSoftmaxWarps + 1) * 32;
+constexpr int kQBytes = kQRows * kHeadDim * 2;
+constexpr int kKvBytesMax = kMaxTokens * kHeadDim * 2;
+constexpr int kSmemBytes = kQBytes + 2 * kKvBytesMax + 1024 /* alignment */ + 256 /* barriers */;
+
+struct AttnParams {
+    CUtensorMap map_q;    // box 64 columns x 128 tokens x 1 image
+    CUtensorMap map_kv;   // box 64 columns x Tk tokens x 1 image
+    uint16_t* out;        // [images * tokens][dim]
+    int tokens, tk, dim;
+    int o_col;            // first tensor-memory column of O
+    uint32_t idesc_s, idesc_o;
+    uint32_t* dev_status;
+};
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+// D[tmem] (+)= A[tmem] * B[smem]: A's 16-bit values two per column, lane = row.  Predicated as the other forms.
+__device__ __forceinline__ void umma_f16_ts_if(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate, uint32_t issue)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "setp.ne.b32 q, %5, 0;\n"
+        "@q tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+        "}\n" ::"r"(d_tmem),
+        "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(issue)
+        : "memory");
+}
+
+__device__ __forceinline__ void tmem_st_32x32b_x8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+
+template <bool kBf16>
+__global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_constant__ AttnParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_smem = smem_base;
+    const uint32_t k_smem = smem_base + kQBytes;
+    const uint32_t v_smem = k_smem + kKvBytesMax;
+    const uint32_t bars = v_smem + kKvBytesMax;
+    const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_o = bars + 32;
+    const uint32_t tmem_holder_addr = bars + 48;
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem_raw + (tmem_holder_addr - smem_u32(smem_raw)));
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 56 - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int mt = blockIdx.x, head = blockIdx.y, img = blockIdx.z;
+
+    if (warp == kSoftmaxWarps) {
+        if (lane == 0) {
+            mbar_init(bar_qk, 1);
+            mbar_init(bar_v, 1);
+            mbar_init(bar_s, 1);
+            mbar_init(bar_p, kSoftmaxWarps);
+            mbar_init(bar_o, 1);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        tmem_alloc(tmem_holder_addr, kTmemCols);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+
+    if (warp == kSoftmaxWarps) {
+        // ------------------------------------------------ loads and both products
+        const uint32_t elected = elect_one() ? 1u : 0u;
+        const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
+        if (elected) {
+            mbar_arrive_expect_tx(bar_qk, (uint32_t)(kQBytes + p.tk * kHeadDim * 2));
+            tma_load_3d(q_smem, &p.map_q, bar_qk, head * kHeadDim, mt * kQRows, img);
+            tma_load_3d(k_smem, &p.map_kv, bar_qk, p.dim + head * kHeadDim, 0, img);
+            mbar_arrive_expect_tx(bar_v, (uint32_t)(p.tk * kHeadDim * 2));
+            tma_load_3d(v_smem, &p.map_kv, bar_v, 2 * p.dim + head * kHeadDim, 0, img);
+        }
+        __syncwarp();
+        bool ok = mbar_wait(bar_qk, 0, abort_flag, p.dev_status, 20);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (ok) {
+            tc_fence_after();
+            const uint64_t a_desc = smem_desc_k_major_sw128(q_smem);
+            const uint64_t b_desc = smem_desc_k_major_sw128(k_smem);
+#pragma unroll
+            for (int k = 0; k < kHeadDim / 16; ++k)
+                umma_f16_if(tmem_u, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc_s, (uint32_t)(k != 0), elected);
+            umma_commit_if(bar_s, elected);
+            ok = mbar_wait(bar_v, 0, abort_flag, p.dev_status, 21);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok) {
+            ok = mbar_wait(bar_p, 0, abort_flag, p.dev_status, 22);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const uint64_t v_desc = smem_desc_mn_major_sw128(v_smem, (uint32_t)(p.tk * kHeadDim * 2));
+            const int steps = p.tk / 16;
+            for (int k = 0; k < steps; ++k)
+                umma_f16_ts_if(tmem_u + (uint32_t)p.o_col, tmem_u + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * 128 >> 4)),
+                               p.idesc_o, (uint32_t)(k != 0), elected);
+            umma_commit_if(bar_o, elected);
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------ softmax and output: lane = query row
+        const int row = mt * kQRows + warp * 32 + lane;           // token index inside the image
+        const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+        const int chunks = p.tk / 16;
+        const float scale = 0.125f * 1.4426950408889634f;         // log2(e) / sqrt(64)
+        bool ok = mbar_wait(bar_s, 0, abort_flag, p.dev_status, 23);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        float sum = 0.f;
+        if (ok) {
+            tc_fence_after();
+            float m = -INFINITY;
+            for (int c = 0; c < chunks; ++c) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(16 * c), r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    if (16 * c + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+            }
+            for (int c = 0; c < chunks; ++c) {
+                uint32_t r[16];
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(16 * c), r);
+                tmem_wait_ld();
+                uint32_t w[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    float e0, e1;
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"((__uint_as_float(r[2 * j]) - m) * scale));
+                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"((__uint_as_float(r[2 * j + 1]) - m) * scale));
+                    if (16 * c + 2 * j >= p.tokens) e0 = 0.f;      // padded keys take no part
+                    if (16 * c + 2 * j + 1 >= p.tokens) e1 = 0.f;
+                    sum += e0 + e1;
+                    w[j] = pack2<kBf16>(e0, e1);
+                }
+                // P's columns 8c .. 8c + 7 lie over S columns that have been read already
+                tmem_st_32x32b_x8(t_lane + (uint32_t)(8 * c), w);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+        }
+        __syncwarp();
+        if (lane == 0 && ok) mbar_arrive(bar_p);
+        if (ok) {
+            ok = mbar_wait(bar_o, 0, abort_flag, p.dev_status, 24);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.0f / sum;
+            uint32_t o[4][16];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 16 * q), o[q]);
+            tmem_wait_ld();
+            if (row < p.tokens) {
+                uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)img * p.tokens + row) * (size_t)p.dim + head * kHeadDim);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t w[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        w[j] = pack2<kBf16>(__uint_as_float(o[q][2 * j]) * inv, __uint_as_float(o[q][2 * j + 1]) * inv);
+                    dst[2 * q] = make_uint4(w[0], w[1], w[2], w[3]);
+                    dst[2 * q + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == kSoftmaxWarps) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+elsa_status make_map_qkv(CUtensorMap* map, const void* qkv, int images, int tokens, int dim, uint32_t box_rows, const char* what)
+{
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return fail(ELSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {(cuuint64_t)(3 * dim), (cuuint64_t)tokens, (cuuint64_t)images};
+    cuuint64_t strides[2] = {(cuuint64_t)(3 * dim) * 2, (cuuint64_t)tokens * (cuuint64_t)(3 * dim) * 2};
+    cuuint32_t box[3] = {(cuuint32_t)kHeadDim, box_rows, 1};
+    cuuint32_t elem[3] = {1, 1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(qkv), dims, strides, box, elem,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for %s rejected (CUresult %d)", what, (int)rc);
+    return ELSA_OK;
+}
+
+template <bool kBf16>
+elsa_status launch(const AttnParams& p, int images, int heads, cudaStream_t stream, const DeviceInfo& dev)
+{
+    auto kernel = attention_kernel<kBf16>;
+    static std::atomic<bool> attr_set[64];
+    const int slot = dev.device & 63;
+    if (!attr_set[slot].load(std::memory_order_acquire)) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess) {
+            cudaError_t e = cudaGetLastError();
+            return fail(ELSA_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+        }
+        attr_set[slot].store(true, std::memory_order_release);
+    }
+    const dim3 grid((unsigned)((p.tokens + kQRows - 1) / kQRows), (unsigned)heads, (unsigned)images);
+    ProfileScope scope(ELSA_KERNEL_ATTENTION, stream);
+    cudaError_t e = launch_pdl(kernel, grid, dim3(kThreads), (size_t)kSmemBytes, stream, 1, p);
+    if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
+    return launched("attention");
+}
+
+}  // namespace
+
+bool attention_suits(int tokens, int heads, int dim)
+{
+    return tokens >= 1 && tokens <= kMaxTokens && heads >= 1 && dim == heads * kHeadDim;
+}
+
+elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype,
+                             uint16_t* out, uint32_t* dev_status, cudaStream_t stream)
+{
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    if (!attention_suits(tokens, heads, dim))
+        return fail(ELSA_ERR_SHAPE, "attention needs 1..%d tokens per image and a head dimension of %d (tokens=%d, heads=%d, dim=%d)",
+                    kMaxTokens, kHeadDim, tokens, heads, dim);
+    if (images > 65535 || heads > 65535) return fail(ELSA_ERR_SHAPE, "at most 65535 images and heads per launch");
+    AttnParams p;
+    p.out = out;
+    p.tokens = tokens;
+    p.tk = (tokens + 15) / 16 * 16;
+    p.dim = dim;
+    // O over the part of S that P does not cover (P: tk / 2 columns from 0); small images: right after S
+    p.o_col = p.tk >= 128 ? (p.tk / 2 + 31) / 32 * 32 : p.tk;
+    const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
+    p.idesc_s = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.tk >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
+    p.idesc_o = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((uint32_t)(kHeadDim >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
+    p.dev_status = dev_status;
+    if ((st = make_map_qkv(&p.map_q, qkv, images, tokens, dim, kQRows, "q")) != ELSA_OK) return st;
+    if ((st = make_map_qkv(&p.map_kv, qkv, images, tokens, dim, (uint32_t)p.tk, "k, v")) != ELSA_OK) return st;
+    return dtype == ELSA_BF16 ? launch<true>(p, images, heads, stream, dev) : launch<false>(p, images, heads, stream, dev);
+}
+
+}  // namespace elsa

@@ -13,6 +13,10 @@ K * 2^-24 * max|x w| ~ 1e-4 of the longest reduction here.  In the chain a stage
 of its inputs, which LayerNorm and the linears carry from the large elements of a row to its small ones: each
 element is held to four times the stage tolerance with the largest |ref| of its row added to |ref|, and every
 stage as a whole to a relative Frobenius error of 5e-3 (the bound of the single linears' parity tests).
+
+Attention (elsa_attention, and the block run with it): the kernel keeps fp32 scores and row sums and rounds the
+probabilities to the 16-bit type for the second product, so |err| <= u |ref| + (u / 2) max|v| + 1e-5 with max|v|
+over the head's values in the image (sum of p |v| <= max|v|; a probability's rounding is u / 4 relative).
 """
 import numpy as np
 import pytest
@@ -70,7 +74,7 @@ def test_scratch_layout_is_host_arithmetic():
 
 # ------------------------------------------------------------------------------------------------ GPU
 
-def run_block(lib, x, host, levels, mlp, variant=None, phase="both"):
+def run_block(lib, x, host, levels, mlp, variant=None, phase="both", attn=None):
     """Compresses the four weights, runs the block; returns ({stage: fp64 array}, {stage: bits}, weights)."""
     dtype = x.dtype
     rows, dim = x.shape
@@ -89,7 +93,9 @@ def run_block(lib, x, host, levels, mlp, variant=None, phase="both"):
     if variant is not None:
         lib.elsa_set_linear_variant(variant)
     try:
-        if phase == "both":
+        if phase == "both" and attn:
+            y, _ = lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status, tokens=attn[0], heads=attn[1])
+        elif phase == "both":
             y, _ = lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status)
         else:
             lib.elsa_vit_block(xd, mlp, w, scratch=scratch, dev_status=status, phase="qkv")
@@ -111,8 +117,18 @@ def stage_tolerance(ref, lin, dtype):
     return u * (np.abs(ref) + (0 if lin is None else np.abs(lin))) + 5e-4
 
 
-def check_rows(got, x, p, dtype, rows_idx):
-    """Both comparisons on the given rows (the block treats token rows independently)."""
+def attention_tolerance(ref, v, tokens, heads, dtype):
+    """ref, v: [rows, dim] fp64 (v = the value third of qkv); per element u |ref| + u / 2 max|v| of its head and image."""
+    u = 2.0 ** -7 if dtype == torch.bfloat16 else 2.0 ** -10
+    rows, dim = v.shape
+    vmax = np.abs(v).reshape(rows // tokens, tokens, heads, dim // heads).max(axis=(1, 3), keepdims=True)
+    vmax = np.broadcast_to(vmax, (rows // tokens, tokens, heads, dim // heads)).reshape(rows, dim)
+    return u * np.abs(ref) + 0.5 * u * vmax + 1e-5
+
+
+def check_rows(got, x, p, dtype, rows_idx, attn=None):
+    """Both comparisons on the given rows (the block treats token rows independently; with attention the rows
+    must be whole images)."""
     code = eo.F16 if dtype == torch.float16 else eo.BF16
     f64 = lambda t: t[rows_idx].to(torch.float64).numpy()
     bits = lambda t: synth.bits(t[rows_idx].contiguous())
@@ -134,14 +150,22 @@ def check_rows(got, x, p, dtype, rows_idx):
         "h": (r16(bo.gelu(fc1)), 1.13 * fc1),
         "y": (r16(g["x2"] + fc2), fc2),
     }
-    assert np.array_equal(bits(got["a"]), bits(got["qkv"][:, 2 * dim:3 * dim]))      # the stand-in copies V through
+    if attn is None:
+        assert np.array_equal(bits(got["a"]), bits(got["qkv"][:, 2 * dim:3 * dim]))  # the stand-in copies V through
+    else:
+        ref = r16(bo.attention(g["qkv"], *attn))
+        tol = attention_tolerance(ref, g["qkv"][:, 2 * dim:], attn[0], attn[1], dtype)
+        err = np.abs(g["a"] - ref)
+        worst = (err - tol).argmax()
+        assert (err <= tol).all(), "stage a: error %g at tolerance %g" % (err.flat[worst], tol.flat[worst])
     for s, (ref, mag) in stage_ref.items():
         err = np.abs(g[s] - ref)
         tol = stage_tolerance(ref, mag, dtype)
         worst = (err - tol).argmax()
         assert (err <= tol).all(), "stage %s: error %g at tolerance %g" % (s, err.flat[worst], tol.flat[worst])
     # the whole chain from x alone
-    chain = bo.block_forward(bits(x), p, code, eps=1e-6)
+    chain = bo.block_forward(bits(x), p, code, eps=1e-6, **({} if attn is None else
+                                                            dict(attn="softmax", tokens=attn[0], heads=attn[1])))
     for s in STAGES:
         mag = chain["x2"] - xs if s == "x2" else chain["y"] - chain["x2"] if s == "y" else 1.13 * fc1 if s == "h" else None
         err = np.abs(g[s] - chain[s])
@@ -252,3 +276,66 @@ def test_block_validation(lib):
         lib.elsa_vit_block(x, mlp, w)
     assert e.value.status == 1 and "fc1" in str(e.value)
     assert lib.elsa_launch_count() == before                     # nothing was enqueued
+
+
+ATTN_CASES = [(3, 197, 2, 1.0), (2, 64, 1, 1.0), (5, 49, 3, 1.0), (2, 256, 2, 1.0), (3, 130, 1, 1.0), (1, 16, 1, 1.0),
+              (2, 7, 2, 1.0), (2, 197, 1, 4.0)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
+@pytest.mark.parametrize("case", ATTN_CASES, ids=["%dx%dx%d_s%g" % c for c in ATTN_CASES])
+def test_attention_matches_oracle(lib, case, dtype):
+    images, tokens, heads, scale = case              # scale 4: scores up to +-60, the row maximum matters
+    dim = 64 * heads
+    qkv = synth.randn((images * tokens, 3 * dim), 17, scale, dtype)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    guard = torch.full((images * tokens + 64, dim), 7.0, dtype=dtype, device="cuda")   # rows after the last image stay
+    a = guard[:images * tokens]
+    lib.elsa_attention(qkv.cuda(), tokens, heads, a=a, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    assert (guard[images * tokens:] == 7.0).all()
+    q64 = qkv.double().numpy()
+    ref = bo._round16(bo.attention(q64, tokens, heads), dtype)
+    got = a.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    tol = attention_tolerance(ref, q64[:, 2 * dim:], tokens, heads, dtype)
+    err = np.abs(got - ref)
+    worst = (err - tol).argmax()
+    assert (err <= tol).all(), "error %g at tolerance %g" % (err.flat[worst], tol.flat[worst])
+
+
+@pytest.mark.gpu
+def test_attention_refuses_shapes_it_does_not_cover(lib):
+    qkv = torch.zeros((300, 3 * 64), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_attention(qkv, 300, 1)                 # more than 256 tokens per image
+    assert e.value.status == 2
+    qkv = torch.zeros((64, 3 * 96), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_attention(qkv, 64, 1)                  # head dimension 96
+    assert e.value.status == 2
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
+def test_block_with_attention_matches_oracle(lib, dtype):
+    images, tokens, heads, mlp = 3, 197, 4, 1024
+    dim = 64 * heads
+    host, p = make_params(dim, mlp, MIXED_LEVELS, dtype, 1100)
+    x = synth.randn((images * tokens, dim), 12, 1.0, dtype)
+    got = run_block(lib, x, host, MIXED_LEVELS, mlp, attn=(tokens, heads))
+    check_rows(got, x, p, dtype, np.arange(images * tokens), attn=(tokens, heads))
+
+
+@pytest.mark.gpu
+def test_deit_b_block_with_attention_full_size_sampled_images(lib):
+    dtype = torch.bfloat16
+    images, tokens, heads, dim, mlp = 256, 197, 12, 768, 3072
+    levels = DEIT_LEVELS[0]
+    host, p = make_params(dim, mlp, levels, dtype, 1300)
+    x = synth.randn((images * tokens, dim), 13, 1.0, dtype, "cuda").cpu()
+    got = run_block(lib, x, host, levels, mlp, attn=(tokens, heads))
+    pick = np.concatenate([np.arange(i * tokens, (i + 1) * tokens) for i in (0, 101, 255)])   # whole images
+    check_rows(got, x, p, dtype, pick, attn=(tokens, heads))
