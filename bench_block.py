@@ -3,12 +3,14 @@ with the levels the stack workload gives its four linears, chained (a block's y 
 
     python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
 
-Attention is NOT computed: the block runs with the stand-in a = V, so the figure is the speed of the linear and
-elementwise path of the model (LayerNorms, the four N:M linears, GELU, residuals), not of DeiT-B.
+Two timings: with the library's multi-head self-attention (elsa_vit_block_attn: the encoder blocks of DeiT-B as
+they run, without patch embedding and classifier head), and with the stand-in a = V in its place (the linear and
+elementwise path alone: LayerNorms, the four N:M linears, GELU, residuals).
 CUDA-event times of `reps` passes over all blocks (activations of one block alone exceed L2), one more pass with
 per-launch events for the split by kernel family, and the roofline of the pass: per linear the larger of kept
 FLOPs / bf16 peak and algorithmic bytes / HBM peak, plus the elementwise stages' bytes (LayerNorm in and out
-twice, the stand-in copy in and out, one residual operand per add) / HBM peak.
+twice, one residual operand per add; the copy in and out for the stand-in) / HBM peak, plus, with attention, the
+larger of its 4 tokens^2 d FLOPs per head and image / bf16 peak and its bytes (qkv in, a out) / HBM peak.
 """
 from __future__ import annotations
 
@@ -57,47 +59,56 @@ def main():
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     x = [synth.randn((rows, dim), 77, 1.0, dtype, "cuda"), torch.empty((rows, dim), dtype=dtype, device="cuda")]
 
-    def one_pass():
-        for b, (w, _) in enumerate(blocks):
-            lib.elsa_vit_block(x[b & 1], mlp, w, y=x[(b + 1) & 1], scratch=scratch, dev_status=status)
-
+    tokens, heads = 197, 12
     x0 = x[0].clone()
-    for _ in range(3):
-        x[0].copy_(x0)
-        one_pass()
-    times = []
-    for _ in range(args.reps):
-        x[0].copy_(x0)
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        one_pass()
-        e1.record()
-        torch.cuda.synchronize()
-        times.append(e0.elapsed_time(e1))
-    assert int(status.item()) == 0, "device status %#x" % int(status.item())
-    assert torch.isfinite(x[args.blocks & 1].float()).all()
-
-    x[0].copy_(x0)
-    lib.elsa_profile_start()
-    one_pass()
-    families = {}
-    launch_list = lib.elsa_profile_stop()
-    for kernel, _, ms in launch_list:
-        f = families.setdefault(kernel, {"launches": 0, "ms": 0.0})
-        f["launches"] += 1
-        f["ms"] += ms
-
     lin_roof = sum(bench.roofline_seconds(l, peaks)[0] for l in layers)
-    elementwise_bytes = args.blocks * 8 * rows * dim * 2
-    roof_ms = (lin_roof + elementwise_bytes / (peaks["hbm_gbs"] * 1e9)) * 1e3
-    ms = statistics.median(times)
+    hbm = peaks["hbm_gbs"] * 1e9
+    attn_roof = max(4.0 * tokens * tokens * 64 * heads * args.batch / (peaks["bf16_tflops"] * 1e12), rows * dim * 4 * 2 / hbm)
+
+    def measure(attention):
+        def one_pass():
+            for b, (w, _) in enumerate(blocks):
+                lib.elsa_vit_block(x[b & 1], mlp, w, y=x[(b + 1) & 1], scratch=scratch, dev_status=status,
+                                   tokens=tokens if attention else None, heads=heads)
+
+        for _ in range(3):
+            x[0].copy_(x0)
+            one_pass()
+        times = []
+        for _ in range(args.reps):
+            x[0].copy_(x0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            one_pass()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        assert int(status.item()) == 0, "device status %#x" % int(status.item())
+        assert torch.isfinite(x[args.blocks & 1].float()).all()
+        x[0].copy_(x0)
+        lib.elsa_profile_start()
+        one_pass()
+        families = {}
+        launch_list = lib.elsa_profile_stop()
+        for kernel, _, ms in launch_list:
+            f = families.setdefault(kernel, {"launches": 0, "ms": 0.0})
+            f["launches"] += 1
+            f["ms"] += ms
+        # elementwise stages per block: LayerNorm twice (in + out), two residual operands; the stand-in adds its copy
+        elementwise_bytes = args.blocks * (6 if attention else 8) * rows * dim * 2
+        roof_ms = (lin_roof + elementwise_bytes / hbm + (args.blocks * attn_roof if attention else 0.0)) * 1e3
+        ms = statistics.median(times)
+        return {"ms_per_pass": ms, "ms_min": min(times), "ms_max": max(times), "images_per_s": args.batch / ms * 1e3,
+                "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "families_profiled_pass": families,
+                "first_block_launches": [[k, round(t, 4)] for k, _, t in launch_list[:len(launch_list) // args.blocks + 2]]}
+
+    with_attention = measure(True)
+    stand_in = measure(False)
     rec = {"workload": "deit_b_blocks_b%d" % args.batch, "blocks": args.blocks, "rows": rows, "dtype": "bf16",
-           "attention": "stand-in a = V (not computed)", "ms_per_pass": ms, "ms_min": min(times), "ms_max": max(times),
-           "images_per_s_linear_and_elementwise_path": args.batch / ms * 1e3,
-           "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "peaks": peaks_kind,
-           "linears_roofline_ms": lin_roof * 1e3, "elementwise_bytes": elementwise_bytes,
-           "families_profiled_pass": families,
-           "first_block_launches": [[k, round(ms, 4)] for k, _, ms in launch_list[:len(launch_list) // args.blocks + 2]], "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
+           "peaks": peaks_kind, "linears_roofline_ms": lin_roof * 1e3, "attention_roofline_ms_per_block": attn_roof * 1e3,
+           "encoder_blocks_with_attention": with_attention,
+           "linear_and_elementwise_path_only_standin_a_eq_v": stand_in,
+           "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     json.dump(rec, open(args.out, "w"), indent=1)
     print(json.dumps(rec))

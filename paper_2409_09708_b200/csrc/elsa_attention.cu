@@ -154,39 +154,79 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
         // ------------------------------------------------ softmax and output: lane = query row
         const int row = mt * kQRows + warp * 32 + lane;           // token index inside the image
         const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const int chunks = p.tk / 16;
         const float scale = 0.125f * 1.4426950408889634f;         // log2(e) / sqrt(64)
         bool ok = mbar_wait(bar_s, 0, abort_flag, p.dev_status, 23);
         ok = __all_sync(0xFFFFFFFFu, ok);
         float sum = 0.f;
         if (ok) {
             tc_fence_after();
+            // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
+            // row maximum from up to 128 columns per round trip, the second pass with the next 32 columns in
+            // flight while the current ones are exponentiated.
+            const int units = p.tk >> 5;            // whole units of 32 columns
+            const bool tail = (p.tk & 31) != 0;     // plus one chunk of 16
             float m = -INFINITY;
-            for (int c = 0; c < chunks; ++c) {
+            for (int u0 = 0; u0 < units; u0 += 4) {
+                uint32_t r[4][32];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (u0 + i < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u0 + i)), r[i]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    if (u0 + i < units) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, __uint_as_float(r[i][j]));
+                    }
+            }
+            if (tail) {
                 uint32_t r[16];
-                tmem_ld_32x32b_x16(t_lane + (uint32_t)(16 * c), r);
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
                 tmem_wait_ld();
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
-                    if (16 * c + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+                    if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
             }
-            for (int c = 0; c < chunks; ++c) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(t_lane + (uint32_t)(16 * c), r);
-                tmem_wait_ld();
-                uint32_t w[8];
+            // p = 2^((s - m) * scale) for 16 columns starting at col0: eight packed pairs
+            auto exp16 = [&](const uint32_t* r, int col0, uint32_t (&w)[8]) {
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     float e0, e1;
                     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"((__uint_as_float(r[2 * j]) - m) * scale));
                     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"((__uint_as_float(r[2 * j + 1]) - m) * scale));
-                    if (16 * c + 2 * j >= p.tokens) e0 = 0.f;      // padded keys take no part
-                    if (16 * c + 2 * j + 1 >= p.tokens) e1 = 0.f;
+                    if (col0 + 2 * j >= p.tokens) e0 = 0.f;        // padded keys take no part
+                    if (col0 + 2 * j + 1 >= p.tokens) e1 = 0.f;
                     sum += e0 + e1;
                     w[j] = pack2<kBf16>(e0, e1);
                 }
-                // P's columns 8c .. 8c + 7 lie over S columns that have been read already
-                tmem_st_32x32b_x8(t_lane + (uint32_t)(8 * c), w);
+            };
+            // P's columns 16u .. 16u + 15 lie over S columns of units that have been read already
+            auto unit = [&](const uint32_t (&r)[32], int u) {
+                uint32_t w[2][8];
+                exp16(&r[0], 32 * u, w[0]);
+                exp16(&r[16], 32 * u + 16, w[1]);
+                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u), w[0]);
+                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u + 8), w[1]);
+            };
+            uint32_t ra[32], rb[32];
+            if (units > 0) tmem_ld_32x32b_x32(t_lane, ra);
+            for (int u = 0; u < units; u += 2) {
+                tmem_wait_ld();
+                if (u + 1 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 1)), rb);
+                unit(ra, u);
+                if (u + 1 < units) {
+                    tmem_wait_ld();
+                    if (u + 2 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 2)), ra);
+                    unit(rb, u + 1);
+                }
+            }
+            if (tail) {
+                uint32_t r[16], w[8];
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                tmem_wait_ld();
+                exp16(r, 32 * units, w);
+                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * units), w);
             }
             tmem_wait_st();
             tc_fence_before();
