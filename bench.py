@@ -14,7 +14,8 @@ pinned host buffers and the copies inside the timed region.  `roofline` describe
 kernel family (largest share of kernel time), timed per launch with CUDA events in a second pass;
 `families` gives the same per family and `gemm_frac` over all of them; the roofline time of a
 layer is max(kept FLOPs / tensor peak, algorithmic bytes / HBM bandwidth).  `secondary` carries
-the Swin-B stack measured in the same process.
+the Swin-B stack measured in the same process; `block_chain` the twelve DeiT-B encoder blocks run as a chain
+(LayerNorms, the four N:M linears, attention, GELU, residuals; bench_block.py), in images per second.
 `--impl reference` times the CPU oracle on a bounded sample of the same workload.
 With N > 1 (torchrun) every rank runs an independent replica; there is no collective on the path.
 """
@@ -512,6 +513,21 @@ def run_ours(args):
                 json.dump(rows2, f, indent=1)
         except OSError:
             pass
+    # ---- the chained encoder blocks (the same 48 linears fed forward, with attention), device timing only
+    if args.block_chain and world == 1 and args.workload == "deit_b_stack_b256":
+        import bench_block
+        torch.cuda.empty_cache()
+        b = bench_block.run(12, 256, 5, peaks, peaks_kind, roofline_seconds)
+        with_attn, stand_in = b["encoder_blocks_with_attention"], b["linear_and_elementwise_path_only_standin_a_eq_v"]
+        line["block_chain"] = {
+            "workload": "deit_b_encoder_blocks_b256 (12 blocks chained, levels of the stack; no patch embedding or head)",
+            "ms_per_pass": with_attn["ms_per_pass"], "images_per_s": with_attn["images_per_s"],
+            "roofline_frac": with_attn["roofline_frac"], "roofline_ms": with_attn["roofline_ms"],
+            "families_ms": {k: v["ms"] for k, v in with_attn["families_profiled_pass"].items()},
+            "without_attention": {"note": "stand-in a = V in place of attention: the linear and elementwise path alone",
+                                  "ms_per_pass": stand_in["ms_per_pass"], "images_per_s": stand_in["images_per_s"],
+                                  "roofline_frac": stand_in["roofline_frac"]},
+        }
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
@@ -574,6 +590,8 @@ def main():
     ap.add_argument("--sampled-gmacs", type=float, default=None,
                     help="replace the DeiT-B stack's levels by an N:4 configuration drawn by the two-step sampler at this many "
                          "whole-model GMACs per image (Table 1: 7.0 and 6.0 for ELSA-DeiT-B-N:4)")
+    ap.add_argument("--no-block-chain", dest="block_chain", action="store_false",
+                    help="skip the chained encoder blocks reported under `block_chain`")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -26,23 +26,22 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-import bench
 from paper_2409_09708_b200 import binding as lib
 from paper_2409_09708_b200 import synth
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--blocks", type=int, default=12)
-    ap.add_argument("--batch", type=int, default=256)
-    ap.add_argument("--reps", type=int, default=5)
-    ap.add_argument("--out", default="bench_out/block.json")
-    args = ap.parse_args()
+def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seconds=None):
+    """Times the chained blocks; returns the record main() prints.  peaks / roofline_seconds: bench.py's (passed in
+    by bench.py itself when it calls this; looked up there otherwise)."""
+    if peaks is None:
+        import bench
+        peaks, peaks_kind = bench.load_peaks()
+        roofline_seconds = bench.roofline_seconds
+    args = argparse.Namespace(blocks=blocks, batch=batch, reps=reps)
     dtype = torch.bfloat16
     dim, mlp = 768, 3072
     layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
     rows = layers[0].rows
-    peaks, peaks_kind = bench.load_peaks()
 
     blocks = []
     for b in range(args.blocks):
@@ -61,7 +60,7 @@ def main():
 
     tokens, heads = 197, 12
     x0 = x[0].clone()
-    lin_roof = sum(bench.roofline_seconds(l, peaks)[0] for l in layers)
+    lin_roof = sum(roofline_seconds(l, peaks)[0] for l in layers)
     hbm = peaks["hbm_gbs"] * 1e9
     attn_roof = max(4.0 * tokens * tokens * 64 * heads * args.batch / (peaks["bf16_tflops"] * 1e12), rows * dim * 4 * 2 / hbm)
 
@@ -109,6 +108,17 @@ def main():
            "encoder_blocks_with_attention": with_attention,
            "linear_and_elementwise_path_only_standin_a_eq_v": stand_in,
            "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
+    return rec
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--blocks", type=int, default=12)
+    ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--out", default="bench_out/block.json")
+    args = ap.parse_args()
+    rec = run(args.blocks, args.batch, args.reps)
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     json.dump(rec, open(args.out, "w"), indent=1)
     print(json.dumps(rec))

@@ -13,6 +13,10 @@ runs elsa_vit_compress over the weights of a workload table instead (weights onl
     python bench_case.py --backward --rows 50432 --in 768 --out 3072 --level 2:8 --reps 5
 
 times elsa_nm_linear_backward on that layer: dX alone, dW alone, db alone and all three in one call.
+
+    python bench_case.py --attention --images 256 --tokens 197 --heads 12 --reps 5
+
+times elsa_attention alone (qkv of that many images in, a out).
 """
 from __future__ import annotations
 
@@ -117,6 +121,31 @@ def backward_case(args):
     print(json.dumps(out))
 
 
+def attention_case(args):
+    """elsa_attention alone.  Its roofline is the larger of 4 tokens^2 64 FLOPs per head and image at the bf16 peak
+    and the bytes of qkv in and a out at the HBM peak."""
+    dtype = synth.torch_dtype(args.dtype)
+    dim = 64 * args.heads
+    rows = args.images * args.tokens
+    qkv = synth.randn((rows, 3 * dim), 5, 1.0, dtype, device="cuda")
+    a = torch.empty((rows, dim), dtype=dtype, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    for rep in range(args.reps + 1):
+        flush.fill_(rep)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        lib.elsa_attention(qkv, args.tokens, args.heads, a=a, dev_status=status)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(status.item()) == 0
+    print(json.dumps({"form": "attention", "images": args.images, "tokens": args.tokens, "heads": args.heads, "dtype": args.dtype,
+                      "ms": times[1:], "flops": 4.0 * args.tokens * args.tokens * 64 * args.heads * args.images,
+                      "algorithmic_bytes": rows * dim * 4 * 2}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--rows", type=int, default=50432)
@@ -130,7 +159,13 @@ def main():
     ap.add_argument("--compress-table", default=None, help="workload whose weights go through elsa_vit_compress")
     ap.add_argument("--int8", action="store_true", help="the INT8 form: elsa_nm_compress_i8 once, then elsa_nm_linear_i8")
     ap.add_argument("--backward", action="store_true", help="elsa_nm_linear_backward on the layer")
+    ap.add_argument("--attention", action="store_true", help="elsa_attention on --images x --tokens x --heads")
+    ap.add_argument("--images", type=int, default=256)
+    ap.add_argument("--tokens", type=int, default=197)
+    ap.add_argument("--heads", type=int, default=12)
     args = ap.parse_args()
+    if args.attention:
+        return attention_case(args)
     if args.backward:
         return backward_case(args)
     if args.compress_table:

@@ -3,7 +3,7 @@
 //     a[img, :, h] = softmax(q k^T / sqrt d) v      per image and head, over the keys of the same image
 // with q, k, v the head's 64 columns in the three thirds of qkv [images * tokens][3 * dim].
 //
-// One CTA per (128 query rows, head, image); tokens <= 256, head dimension 64 (the ViT / DeiT shapes).  Both
+// Work item = (128 query rows, head, image); tokens <= 256, head dimension 64 (the ViT / DeiT shapes).  Both
 // products run on tcgen05 with everything between them kept on chip:
 //   1. TMA brings the Q tile, all K rows and all V rows of the head into shared memory (128-byte swizzle; a 3-D
 //      tensor map [image][token][column] zero-fills the rows past the image's last token).
@@ -14,8 +14,11 @@
 //   4. O = P V: Tk / 16 MMAs with A from tensor memory and V as it lies in memory (keys outermost: MN-major
 //      descriptor) into 64 columns of the part of S that is dead by then.
 //   5. The same four warps read O, divide by the row sum, round once and store each row's 128 bytes.
-// 256 columns of tensor memory and 81 KB of shared memory per CTA: two CTAs share an SM, one's products overlap the
-// other's softmax.  Every wait is bounded as in the GEMM kernels.
+// Persistent: one CTA per SM walks the items with the stride of the grid, two items in flight.  Shared memory holds
+// two stages of (Q, K, V), tensor memory two halves of 256 columns, and there are two groups of four softmax warps:
+// item n uses stage, half and group n % 2.  The producer warp loads item n + 1 (and n + 2 once its stage is free)
+// while item n is computed; the MMA warp issues S of item n, then P V of item n - 1, so one group's softmax runs
+// under the other group's products and epilogue.  Every wait is bounded as in the GEMM kernels.
 #include <atomic>
 #include <mutex>
 
@@ -25,21 +28,24 @@ namespace elsa {
 namespace {
 
 constexpr int kHeadDim = 64;
-constexpr int kQRows = 128;          // query rows per CTA = TMEM lanes
+constexpr int kQRows = 128;          // query rows per item = TMEM lanes
 constexpr int kMaxTokens = 256;
-constexpr int kTmemCols = 256;
-constexpr int kSoftmaxWarps = 4;
-constexpr int kThreads = (kSoftmaxWarps + 1) * 32;
+constexpr int kBufCols = 256;        // tensor-memory columns per item in flight
+constexpr int kTmemCols = 2 * kBufCols;
+constexpr int kGroupWarps = 4;       // softmax warps per group, one per TMEM lane quarter
+constexpr int kThreads = (2 + 2 * kGroupWarps) * 32;
 constexpr int kQBytes = kQRows * kHeadDim * 2;
 constexpr int kKvBytesMax = kMaxTokens * kHeadDim * 2;
-constexpr int kSmemBytes = kQBytes + 2 * kKvBytesMax + 1024 /* alignment */ + 256 /* barriers */;
+constexpr int kStageBytes = kQBytes + 2 * kKvBytesMax;
+constexpr int kSmemBytes = 2 * kStageBytes + 1024 /* alignment */ + 256 /* barriers */;
 
 struct AttnParams {
     CUtensorMap map_q;    // box 64 columns x 128 tokens x 1 image
     CUtensorMap map_kv;   // box 64 columns x Tk tokens x 1 image
     uint16_t* out;        // [images * tokens][dim]
     int tokens, tk, dim;
-    int o_col;            // first tensor-memory column of O
+    int m_tiles, heads, items;   // items = images * heads * m_tiles, query tile fastest
+    int o_col;            // first column of O inside an item's half of tensor memory
     uint32_t idesc_s, idesc_o;
     uint32_t* dev_status;
 };
@@ -75,29 +81,33 @@ __device__ __forceinline__ void tmem_st_32x32b_x8(uint32_t taddr, const uint32_t
 }
 
 template <bool kBf16>
-__global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_constant__ AttnParams p)
+__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_smem = smem_base;
-    const uint32_t k_smem = smem_base + kQBytes;
-    const uint32_t v_smem = k_smem + kKvBytesMax;
-    const uint32_t bars = v_smem + kKvBytesMax;
-    const uint32_t bar_qk = bars, bar_v = bars + 8, bar_s = bars + 16, bar_p = bars + 24, bar_o = bars + 32;
-    const uint32_t tmem_holder_addr = bars + 48;
+    const uint32_t bars = smem_base + 2 * kStageBytes;
+    // per buffer b: +0 qk_full, +8 v_full, +16 smem_empty, +24 s_full, +32 p_full, +40 o_full, +48 tmem_empty
+    auto bar = [&](int which, int b) { return bars + (uint32_t)(64 * b + 8 * which); };
+    enum { kQkFull = 0, kVFull, kSmemEmpty, kSFull, kPFull, kOFull, kTmemEmpty };
+    const uint32_t tmem_holder_addr = bars + 128;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem_raw + (tmem_holder_addr - smem_u32(smem_raw)));
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 56 - smem_u32(smem_raw)));
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 136 - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int mt = blockIdx.x, head = blockIdx.y, img = blockIdx.z;
+    const int first = blockIdx.x, stride = gridDim.x;
+    const int n_items = first < p.items ? (p.items - first + stride - 1) / stride : 0;   // items of this CTA
 
-    if (warp == kSoftmaxWarps) {
+    if (warp == 1) {
         if (lane == 0) {
-            mbar_init(bar_qk, 1);
-            mbar_init(bar_v, 1);
-            mbar_init(bar_s, 1);
-            mbar_init(bar_p, kSoftmaxWarps);
-            mbar_init(bar_o, 1);
+            for (int b = 0; b < 2; ++b) {
+                mbar_init(bar(kQkFull, b), 1);
+                mbar_init(bar(kVFull, b), 1);
+                mbar_init(bar(kSmemEmpty, b), 1);
+                mbar_init(bar(kSFull, b), 1);
+                mbar_init(bar(kPFull, b), kGroupWarps);
+                mbar_init(bar(kOFull, b), 1);
+                mbar_init(bar(kTmemEmpty, b), kGroupWarps);
+            }
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -111,156 +121,217 @@ __global__ void __launch_bounds__(kThreads, 2) attention_kernel(const __grid_con
     pdl_wait_for_predecessors();
     pdl_release_successors();
 
-    if (warp == kSoftmaxWarps) {
-        // ------------------------------------------------ loads and both products
+    if (warp == 0) {
+        // ------------------------------------------------ TMA producer
+        const bool elected = elect_one();
+        bool ok = true;
+        for (int n = 0; ok && n < n_items; ++n) {
+            const int b = n & 1;
+            const uint32_t ph = (uint32_t)((n >> 1) & 1);
+            ok = mbar_wait(bar(kSmemEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 20);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const int item = first + n * stride;
+            const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
+            const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
+            if (elected) {
+                mbar_arrive_expect_tx(bar(kQkFull, b), (uint32_t)(kQBytes + p.tk * kHeadDim * 2));
+                tma_load_3d(q_smem, &p.map_q, bar(kQkFull, b), head * kHeadDim, mt * kQRows, img);
+                tma_load_3d(q_smem + kQBytes, &p.map_kv, bar(kQkFull, b), p.dim + head * kHeadDim, 0, img);
+                mbar_arrive_expect_tx(bar(kVFull, b), (uint32_t)(p.tk * kHeadDim * 2));
+                tma_load_3d(q_smem + kQBytes + kKvBytesMax, &p.map_kv, bar(kVFull, b), 2 * p.dim + head * kHeadDim, 0, img);
+            }
+            __syncwarp();
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------ MMA issuer: S of item n, then P V of item n - 1
         const uint32_t elected = elect_one() ? 1u : 0u;
         const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
-        if (elected) {
-            mbar_arrive_expect_tx(bar_qk, (uint32_t)(kQBytes + p.tk * kHeadDim * 2));
-            tma_load_3d(q_smem, &p.map_q, bar_qk, head * kHeadDim, mt * kQRows, img);
-            tma_load_3d(k_smem, &p.map_kv, bar_qk, p.dim + head * kHeadDim, 0, img);
-            mbar_arrive_expect_tx(bar_v, (uint32_t)(p.tk * kHeadDim * 2));
-            tma_load_3d(v_smem, &p.map_kv, bar_v, 2 * p.dim + head * kHeadDim, 0, img);
-        }
-        __syncwarp();
-        bool ok = mbar_wait(bar_qk, 0, abort_flag, p.dev_status, 20);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        if (ok) {
-            tc_fence_after();
-            const uint64_t a_desc = smem_desc_k_major_sw128(q_smem);
-            const uint64_t b_desc = smem_desc_k_major_sw128(k_smem);
+        const int steps = p.tk / 16;
+        bool ok = true;
+        for (int n = 0; ok && n <= n_items; ++n) {
+            if (n < n_items) {
+                const int b = n & 1;
+                const uint32_t ph = (uint32_t)((n >> 1) & 1);
+                ok = mbar_wait(bar(kTmemEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 21);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                ok = mbar_wait(bar(kQkFull, b), ph, abort_flag, p.dev_status, 22);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
+                const uint64_t a_desc = smem_desc_k_major_sw128(q_smem);
+                const uint64_t b_desc = smem_desc_k_major_sw128(q_smem + kQBytes);
 #pragma unroll
-            for (int k = 0; k < kHeadDim / 16; ++k)
-                umma_f16_if(tmem_u, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc_s, (uint32_t)(k != 0), elected);
-            umma_commit_if(bar_s, elected);
-            ok = mbar_wait(bar_v, 0, abort_flag, p.dev_status, 21);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-        }
-        if (ok) {
-            ok = mbar_wait(bar_p, 0, abort_flag, p.dev_status, 22);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-        }
-        if (ok) {
-            tc_fence_after();
-            const uint64_t v_desc = smem_desc_mn_major_sw128(v_smem, (uint32_t)(p.tk * kHeadDim * 2));
-            const int steps = p.tk / 16;
-            for (int k = 0; k < steps; ++k)
-                umma_f16_ts_if(tmem_u + (uint32_t)p.o_col, tmem_u + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * 128 >> 4)),
-                               p.idesc_o, (uint32_t)(k != 0), elected);
-            umma_commit_if(bar_o, elected);
+                for (int k = 0; k < kHeadDim / 16; ++k)
+                    umma_f16_if(tmem_u + (uint32_t)(b * kBufCols), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc_s,
+                                (uint32_t)(k != 0), elected);
+                umma_commit_if(bar(kSFull, b), elected);
+            }
+            if (n >= 1) {
+                const int m = n - 1, b = m & 1;
+                const uint32_t ph = (uint32_t)((m >> 1) & 1);
+                ok = mbar_wait(bar(kVFull, b), ph, abort_flag, p.dev_status, 23);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                ok = mbar_wait(bar(kPFull, b), ph, abort_flag, p.dev_status, 24);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_buf = tmem_u + (uint32_t)(b * kBufCols);
+                const uint64_t v_desc = smem_desc_mn_major_sw128(smem_base + (uint32_t)(b * kStageBytes + kQBytes + kKvBytesMax),
+                                                                 (uint32_t)(p.tk * kHeadDim * 2));
+                for (int k = 0; k < steps; ++k)
+                    umma_f16_ts_if(t_buf + (uint32_t)p.o_col, t_buf + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * 128 >> 4)),
+                                   p.idesc_o, (uint32_t)(k != 0), elected);
+                umma_commit_if(bar(kOFull, b), elected);
+                umma_commit_if(bar(kSmemEmpty, b), elected);   // both products of the item have read its stage
+            }
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------ softmax and output: lane = query row
-        const int row = mt * kQRows + warp * 32 + lane;           // token index inside the image
-        const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
-        const float scale = 0.125f * 1.4426950408889634f;         // log2(e) / sqrt(64)
-        bool ok = mbar_wait(bar_s, 0, abort_flag, p.dev_status, 23);
-        ok = __all_sync(0xFFFFFFFFu, ok);
-        float sum = 0.f;
-        if (ok) {
+        // ------------------------------------------------ softmax and output: group g takes the items n = g, g + 2, ...
+        const int g = (warp - 2) / kGroupWarps;
+        const int quarter = warp & 3;                                  // the TMEM lanes this warp may touch
+        const float scale = 0.125f * 1.4426950408889634f;              // log2(e) / sqrt(64)
+        bool ok = true;
+        for (int n = g; ok && n < n_items; n += 2) {
+            const uint32_t ph = (uint32_t)((n >> 1) & 1);
+            const int item = first + n * stride;
+            const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
+            const int row = mt * kQRows + quarter * 32 + lane;         // token index inside the image
+            const uint32_t t_lane = tmem_base + (uint32_t)(g * kBufCols) + ((uint32_t)(quarter * 32) << 16);
+            ok = mbar_wait(bar(kSFull, g), ph, abort_flag, p.dev_status, 25);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
             tc_fence_after();
-            // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
-            // row maximum from up to 128 columns per round trip, the second pass with the next 32 columns in
-            // flight while the current ones are exponentiated.
-            const int units = p.tk >> 5;            // whole units of 32 columns
-            const bool tail = (p.tk & 31) != 0;     // plus one chunk of 16
-            float m = -INFINITY;
-            for (int u0 = 0; u0 < units; u0 += 4) {
-                uint32_t r[4][32];
+            float sum = 0.f;
+            {
+                // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
+                // row maximum from up to 64 columns per round trip, the second pass with the next 32 columns in
+                // flight while the current ones are exponentiated.
+                const int units = p.tk >> 5;            // whole units of 32 columns
+                const bool tail = (p.tk & 31) != 0;     // plus one chunk of 16
+                float m = -INFINITY;
+                for (int u0 = 0; u0 < units; u0 += 2) {
+                    uint32_t r[2][32];
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (u0 + i < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u0 + i)), r[i]);
-                tmem_wait_ld();
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (u0 + i < units) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, __uint_as_float(r[i][j]));
-                    }
-            }
-            if (tail) {
-                uint32_t r[16];
-                tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
-                tmem_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j)
-                    if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
-            }
-            // p = 2^((s - m) * scale) for 16 columns starting at col0: eight packed pairs
-            auto exp16 = [&](const uint32_t* r, int col0, uint32_t (&w)[8]) {
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float e0, e1;
-                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"((__uint_as_float(r[2 * j]) - m) * scale));
-                    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"((__uint_as_float(r[2 * j + 1]) - m) * scale));
-                    if (col0 + 2 * j >= p.tokens) e0 = 0.f;        // padded keys take no part
-                    if (col0 + 2 * j + 1 >= p.tokens) e1 = 0.f;
-                    sum += e0 + e1;
-                    w[j] = pack2<kBf16>(e0, e1);
-                }
-            };
-            // P's columns 16u .. 16u + 15 lie over S columns of units that have been read already
-            auto unit = [&](const uint32_t (&r)[32], int u) {
-                uint32_t w[2][8];
-                exp16(&r[0], 32 * u, w[0]);
-                exp16(&r[16], 32 * u + 16, w[1]);
-                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u), w[0]);
-                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u + 8), w[1]);
-            };
-            uint32_t ra[32], rb[32];
-            if (units > 0) tmem_ld_32x32b_x32(t_lane, ra);
-            for (int u = 0; u < units; u += 2) {
-                tmem_wait_ld();
-                if (u + 1 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 1)), rb);
-                unit(ra, u);
-                if (u + 1 < units) {
+                    for (int i = 0; i < 2; ++i)
+                        if (u0 + i < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u0 + i)), r[i]);
                     tmem_wait_ld();
-                    if (u + 2 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 2)), ra);
-                    unit(rb, u + 1);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+                        if (u0 + i < units) {
+                            if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
+                                float m0 = m, m1 = -INFINITY;
+#pragma unroll
+                                for (int j = 0; j < 32; j += 2) {
+                                    m0 = fmaxf(m0, __uint_as_float(r[i][j]));
+                                    m1 = fmaxf(m1, __uint_as_float(r[i][j + 1]));
+                                }
+                                m = fmaxf(m0, m1);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, __uint_as_float(r[i][j]));
+                            }
+                        }
                 }
-            }
-            if (tail) {
-                uint32_t r[16], w[8];
-                tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
-                tmem_wait_ld();
-                exp16(r, 32 * units, w);
-                tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * units), w);
+                if (tail) {
+                    uint32_t r[16];
+                    tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int j = 0; j < 16; ++j)
+                        if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+                }
+                // p = 2^(s * scale - m * scale) for 16 columns starting at col0: eight packed pairs
+                const float m_scaled = m * scale;
+                float sum1 = 0.f;
+                auto exp16 = [&](const uint32_t* r, int col0, uint32_t (&w)[8]) {
+                    const bool all_real = col0 + 16 <= p.tokens;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float e0, e1;
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(fmaf(__uint_as_float(r[2 * j]), scale, -m_scaled)));
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(fmaf(__uint_as_float(r[2 * j + 1]), scale, -m_scaled)));
+                        if (!all_real) {                                  // padded keys take no part
+                            if (col0 + 2 * j >= p.tokens) e0 = 0.f;
+                            if (col0 + 2 * j + 1 >= p.tokens) e1 = 0.f;
+                        }
+                        sum += e0;
+                        sum1 += e1;
+                        w[j] = pack2<kBf16>(e0, e1);
+                    }
+                };
+                // P's columns 16u .. 16u + 15 lie over S columns of units that have been read already
+                auto unit = [&](const uint32_t (&r)[32], int u) {
+                    uint32_t w[2][8];
+                    exp16(&r[0], 32 * u, w[0]);
+                    exp16(&r[16], 32 * u + 16, w[1]);
+                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u), w[0]);
+                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u + 8), w[1]);
+                };
+                uint32_t ra[32], rb[32];
+                if (units > 0) tmem_ld_32x32b_x32(t_lane, ra);
+                for (int u = 0; u < units; u += 2) {
+                    tmem_wait_ld();
+                    if (u + 1 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 1)), rb);
+                    unit(ra, u);
+                    if (u + 1 < units) {
+                        tmem_wait_ld();
+                        if (u + 2 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 2)), ra);
+                        unit(rb, u + 1);
+                    }
+                }
+                if (tail) {
+                    uint32_t r[16], w[8];
+                    tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                    tmem_wait_ld();
+                    exp16(r, 32 * units, w);
+                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * units), w);
+                }
+                sum += sum1;
             }
             tmem_wait_st();
             tc_fence_before();
-        }
-        __syncwarp();
-        if (lane == 0 && ok) mbar_arrive(bar_p);
-        if (ok) {
-            ok = mbar_wait(bar_o, 0, abort_flag, p.dev_status, 24);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kPFull, g));
+            ok = mbar_wait(bar(kOFull, g), ph, abort_flag, p.dev_status, 26);
             ok = __all_sync(0xFFFFFFFFu, ok);
-        }
-        if (ok) {
+            if (!ok) break;
             tc_fence_after();
             const float inv = 1.0f / sum;
-            uint32_t o[4][16];
+            uint32_t w[4][8];                                          // the row's 64 outputs, packed
 #pragma unroll
-            for (int q = 0; q < 4; ++q) tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 16 * q), o[q]);
-            tmem_wait_ld();
+            for (int half = 0; half < 2; ++half) {
+                uint32_t o[2][16];
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 32 * half), o[0]);
+                tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 32 * half + 16), o[1]);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 2; ++q)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        w[2 * half + q][j] = pack2<kBf16>(__uint_as_float(o[q][2 * j]) * inv, __uint_as_float(o[q][2 * j + 1]) * inv);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(kTmemEmpty, g));            // the half may take the S of item n + 2
             if (row < p.tokens) {
                 uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)img * p.tokens + row) * (size_t)p.dim + head * kHeadDim);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    uint32_t w[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j)
-                        w[j] = pack2<kBf16>(__uint_as_float(o[q][2 * j]) * inv, __uint_as_float(o[q][2 * j + 1]) * inv);
-                    dst[2 * q] = make_uint4(w[0], w[1], w[2], w[3]);
-                    dst[2 * q + 1] = make_uint4(w[4], w[5], w[6], w[7]);
+                    dst[2 * q] = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
+                    dst[2 * q + 1] = make_uint4(w[q][4], w[q][5], w[q][6], w[q][7]);
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == kSoftmaxWarps) {
+    if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -294,7 +365,9 @@ elsa_status launch(const AttnParams& p, int images, int heads, cudaStream_t stre
         }
         attr_set[slot].store(true, std::memory_order_release);
     }
-    const dim3 grid((unsigned)((p.tokens + kQRows - 1) / kQRows), (unsigned)heads, (unsigned)images);
+    (void)images;
+    (void)heads;
+    const dim3 grid((unsigned)(p.items < dev.sm_count ? p.items : dev.sm_count));   // one persistent CTA per SM
     ProfileScope scope(ELSA_KERNEL_ATTENTION, stream);
     cudaError_t e = launch_pdl(kernel, grid, dim3(kThreads), (size_t)kSmemBytes, stream, 1, p);
     if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "attention launch: %s", cudaGetErrorString(e));
@@ -317,12 +390,16 @@ elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int he
     if (!attention_suits(tokens, heads, dim))
         return fail(ELSA_ERR_SHAPE, "attention needs 1..%d tokens per image and a head dimension of %d (tokens=%d, heads=%d, dim=%d)",
                     kMaxTokens, kHeadDim, tokens, heads, dim);
-    if (images > 65535 || heads > 65535) return fail(ELSA_ERR_SHAPE, "at most 65535 images and heads per launch");
+    if ((long long)images * heads * ((tokens + kQRows - 1) / kQRows) > 0x7fffffffLL)
+        return fail(ELSA_ERR_SHAPE, "images * heads does not fit an int");
     AttnParams p;
     p.out = out;
     p.tokens = tokens;
     p.tk = (tokens + 15) / 16 * 16;
     p.dim = dim;
+    p.m_tiles = (tokens + kQRows - 1) / kQRows;
+    p.heads = heads;
+    p.items = images * heads * p.m_tiles;
     // O over the part of S that P does not cover (P: tk / 2 columns from 0); small images: right after S
     p.o_col = p.tk >= 128 ? (p.tk / 2 + 31) / 32 * 32 : p.tk;
     const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;

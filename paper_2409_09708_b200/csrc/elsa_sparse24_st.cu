@@ -18,7 +18,7 @@
 // pairs, feature blocks fastest, so that the pairs that share activation rows read them at the same
 // time (once from HBM, then from L2).  With a reduction this long the epilogue's share is small.
 //
-// Per CTA (640 threads, 96 registers each): warp 0 TMA producer of this CTA's 112 activation rows,
+// Per CTA (576 threads, 96 registers each): warp 0 TMA producer of this CTA's 112 activation rows,
 // warp 1 tensor-memory allocation and (leader) MMA issue, warps 2-9 epilogue (two per tensor-memory
 // lane quarter, see elsa_sparse24_ws.cu for the transposing stmatrix stores and the lane order of the
 // features), warps 10-17 weight loaders (two per lane quarter, taking alternate chunks: the loads of a
