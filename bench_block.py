@@ -3,8 +3,8 @@ with the levels the stack workload gives its four linears, chained (a block's y 
 
     python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
 
-Two timings: with the library's multi-head self-attention (elsa_vit_block_attn: the encoder blocks of DeiT-B as
-they run, without patch embedding and classifier head), and with the stand-in a = V in its place (the linear and
+Two timings: with the library's multi-head self-attention (elsa_vit_encoder: the encoder blocks of DeiT-B as
+they run, without patch embedding, final norm and classifier head), and with the stand-in a = V in its place (the linear and
 elementwise path alone: LayerNorms, the four N:M linears, GELU, residuals).
 CUDA-event times of `reps` passes over all blocks (activations of one block alone exceed L2), one more pass with
 per-launch events for the split by kernel family, and the roofline of the pass: per linear the larger of kept
@@ -64,11 +64,16 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     hbm = peaks["hbm_gbs"] * 1e9
     attn_roof = max(4.0 * tokens * tokens * 64 * heads * args.batch / (peaks["bf16_tflops"] * 1e12), rows * dim * 4 * 2 / hbm)
 
+    table = lib.make_encoder_table([w for w, _ in blocks])
+    enc_scratch = lib.alloc_workspace(int(lib._encoder_scratch(args.batch, tokens, dim, mlp, table, len(blocks), lib.BF16)))
+
     def measure(attention):
         def one_pass():
+            if attention:      # one call for the whole encoder
+                lib.elsa_vit_encoder(x[0], tokens, heads, mlp, table, y=x[args.blocks & 1], scratch=enc_scratch, dev_status=status)
+                return
             for b, (w, _) in enumerate(blocks):
-                lib.elsa_vit_block(x[b & 1], mlp, w, y=x[(b + 1) & 1], scratch=scratch, dev_status=status,
-                                   tokens=tokens if attention else None, heads=heads)
+                lib.elsa_vit_block(x[b & 1], mlp, w, y=x[(b + 1) & 1], scratch=scratch, dev_status=status)
 
         for _ in range(3):
             x[0].copy_(x0)

@@ -439,6 +439,21 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
 elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
                                 const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
                                 uint32_t* dev_status, void* stream);
+/*
+ * n_blocks such blocks in a row (`blocks`: HOST array, one level table per block: the paper's configuration alpha
+ * over the whole encoder), optionally followed by the model's final LayerNorm (final_gain / final_bias: [dim] device,
+ * or both NULL).  Same results, bit for bit, as n_blocks calls of elsa_vit_block_attn; where a block's last linear runs
+ * on a kernel that cannot add the residual, the next block's first LayerNorm (or the final one) adds it in the same
+ * pass instead of a kernel of its own.  scratch: elsa_vit_encoder_scratch_bytes(...) bytes, 256-byte aligned (the
+ * largest block's scratch plus two activation buffers); y [images * tokens][dim] may not alias x.  All blocks are
+ * validated before the first launch.
+ */
+size_t elsa_vit_encoder_scratch_bytes(int images, int tokens, int dim, int mlp_dim, const elsa_block_weights* blocks,
+                                      int n_blocks, elsa_dtype dtype);
+elsa_status elsa_vit_encoder(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
+                             const elsa_block_weights* blocks, int n_blocks, const void* final_gain, const void* final_bias,
+                             float final_eps, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                             uint32_t* dev_status, void* stream);
 
 /* ------------------------------------------------------------------------------------------------
  * Backward pass of the masked linear (Alg. 2, supernet training: the gradient is taken with respect to the

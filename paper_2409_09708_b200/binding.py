@@ -125,6 +125,8 @@ _block_rest = _sig("elsa_vit_block_rest", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _v
 _block = _sig("elsa_vit_block", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _block_attn = _sig("elsa_vit_block_attn", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _attention = _sig("elsa_attention", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
+_encoder_scratch = _sig("elsa_vit_encoder_scratch_bytes", _sz, [_i, _i, _i, _i, _bw, _i, _i])
+_encoder = _sig("elsa_vit_encoder", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, ctypes.c_float, _i, _vp, _vp, _sz, _vp, _vp])
 
 
 class ElsaKernelTime(ctypes.Structure):
@@ -449,6 +451,26 @@ def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, s
         fn = _block if phase == "both" else _block_rest
         _check(fn(_ptr(x), rows, dim, mlp_dim, ctypes.byref(weights), code, _ptr(y), _ptr(scratch), scratch.numel(),
                   _ptr(dev_status), _stream(stream)))
+    return y, scratch
+
+
+def make_encoder_table(block_weights):
+    """ctypes array of ElsaBlockWeights from a list of them (as make_block_weights returns)."""
+    return (ElsaBlockWeights * len(block_weights))(*block_weights)
+
+
+def elsa_vit_encoder(x, tokens, heads, mlp_dim, table, final_gain=None, final_bias=None, final_eps=1e-6, y=None, scratch=None,
+                     dev_status=None, stream=None):
+    """The encoder: len(table) blocks with attention, each under its own levels, then the optional final LayerNorm."""
+    rows, dim = x.shape
+    code = dtype_code(x.dtype)
+    n = len(table)
+    if scratch is None:
+        scratch = alloc_workspace(int(_encoder_scratch(rows // tokens, tokens, dim, mlp_dim, table, n, code)), x.device)
+    if y is None:
+        y = torch.empty_like(x)
+    _check(_encoder(_ptr(x), rows // tokens, tokens, heads, dim, mlp_dim, table, n, _ptr(final_gain), _ptr(final_bias),
+                    final_eps, code, _ptr(y), _ptr(scratch), scratch.numel(), _ptr(dev_status), _stream(stream)))
     return y, scratch
 
 

@@ -955,13 +955,23 @@ elsa_status block_linear(BlockLinear& L, const uint16_t* X, int rows, elsa_dtype
     return launch_act_inplace(dst, (long long)rows * L.out, act, dtype, stream);
 }
 
+// What a block leaves to its successor when the residual of its last linear has not been added yet: the block's
+// output is t + r, and the successor's first LayerNorm adds, stores and normalises it in one pass.
+struct BlockCarry {
+    const uint16_t* t = nullptr;   // fc2's output, rounded to 16 bits
+    const uint16_t* r = nullptr;   // x2
+};
+
+// carry (or NULL) + x_sum: the block's input is carry->t + carry->r, written to x_sum; otherwise it is x.
 elsa_status block_qkv(const uint16_t* x, int rows, int dim, const elsa_block_weights* w, elsa_dtype dtype,
                       uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4], uint32_t* dev_status,
-                      cudaStream_t stream)
+                      cudaStream_t stream, const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr)
 {
     uint16_t* x1 = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_X1]);
     uint16_t* qkv = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_QKV]);
-    elsa_status st = launch_layer_norm(x, nullptr, nullptr, (const uint16_t*)w->ln1_gain, (const uint16_t*)w->ln1_bias,
+    const bool add = carry != nullptr && carry->t != nullptr;
+    elsa_status st = launch_layer_norm(add ? carry->t : x, add ? carry->r : nullptr, add ? x_sum : nullptr,
+                                       (const uint16_t*)w->ln1_gain, (const uint16_t*)w->ln1_bias,
                                        x1, rows, dim, w->eps, dtype, stream);
     if (st != ELSA_OK) return st;
     bool left = false;
@@ -970,7 +980,7 @@ elsa_status block_qkv(const uint16_t* x, int rows, int dim, const elsa_block_wei
 
 elsa_status block_rest(const uint16_t* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                        uint16_t* y, uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4],
-                       uint32_t* dev_status, cudaStream_t stream)
+                       uint32_t* dev_status, cudaStream_t stream, BlockCarry* defer = nullptr)
 {
     (void)mlp_dim;
     const uint16_t* a = (const uint16_t*)(scratch + plan.off[ELSA_BLOCK_A]);
@@ -989,6 +999,11 @@ elsa_status block_rest(const uint16_t* x, int rows, int dim, int mlp_dim, const 
     if (st != ELSA_OK) return st;
     if ((st = block_linear(lin[2], x3, rows, dtype, h, 1, nullptr, nullptr, &left, dev_status, stream)) != ELSA_OK) return st;
     if ((st = block_linear(lin[3], h, rows, dtype, y, 0, x2, t, &left, dev_status, stream)) != ELSA_OK) return st;
+    if (left && defer != nullptr) {          // the successor's first LayerNorm adds the residual
+        defer->t = t;
+        defer->r = x2;
+        return ELSA_OK;
+    }
     if (left) st = launch_layer_norm(t, x2, y, nullptr, nullptr, nullptr, rows, dim, w->eps, dtype, stream);
     return st;
 }
@@ -1043,7 +1058,8 @@ namespace {
 
 // The whole block; tokens == 0 runs the stand-in a = V, otherwise the attention kernel over images of `tokens` rows.
 elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
-                      void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_, int tokens, int heads)
+                      void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_, int tokens, int heads,
+                      const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr, BlockCarry* defer = nullptr)
 {
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
@@ -1072,7 +1088,9 @@ elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_
         if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "joining the image stream: %s", cudaGetErrorString(e));
     }
     uint8_t* s8 = (uint8_t*)scratch;
-    if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream)) != ELSA_OK) return st;
+    if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream, carry, x_sum)) != ELSA_OK)
+        return st;
+    if (carry != nullptr && carry->t != nullptr) x = x_sum;      // the block's input, as just stored
     if (tokens == 0) {
         // the stated stand-in for attention: a = V
         st = launch_copy_columns((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]),
@@ -1082,13 +1100,105 @@ elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_
                               (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]), dev_status, stream);
     }
     if (st != ELSA_OK) return st;
-    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream);
+    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream, defer);
+}
+
+struct EncoderPlan {
+    size_t block_bytes;   // scratch of the largest block
+    size_t buf[2];        // byte offsets of the two activation buffers the blocks alternate between
+    size_t total;
+};
+
+bool encoder_plan(int rows, int dim, int mlp_dim, const elsa_block_weights* blocks, int n_blocks, elsa_dtype dtype, EncoderPlan* p)
+{
+    if (!blocks || n_blocks <= 0) return false;
+    p->block_bytes = 0;
+    for (int b = 0; b < n_blocks; ++b) {
+        BlockPlan plan;
+        if (!block_plan(rows, dim, mlp_dim, blocks + b, dtype, &plan)) return false;
+        if (plan.total > p->block_bytes) p->block_bytes = plan.total;
+    }
+    size_t at = round_up(p->block_bytes, 256);
+    for (int i = 0; i < 2; ++i) {
+        p->buf[i] = at;
+        at += round_up((size_t)rows * dim * 2, 256);
+    }
+    p->total = at;
+    return true;
 }
 
 }  // namespace
 }  // namespace elsa
 
 extern "C" {
+
+size_t elsa_vit_encoder_scratch_bytes(int images, int tokens, int dim, int mlp_dim, const elsa_block_weights* blocks,
+                                      int n_blocks, elsa_dtype dtype)
+{
+    EncoderPlan p;
+    if (images <= 0 || tokens <= 0 || (long long)images * tokens > 0x7fffffffLL) return 0;
+    return encoder_plan(images * tokens, dim, mlp_dim, blocks, n_blocks, dtype, &p) ? p.total : 0;
+}
+
+elsa_status elsa_vit_encoder(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
+                             const elsa_block_weights* blocks, int n_blocks, const void* final_gain, const void* final_bias,
+                             float final_eps, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                             uint32_t* dev_status, void* stream)
+{
+    if (!x || !y || !blocks || !scratch) return fail(ELSA_ERR_NULL, "x, y, blocks and scratch must not be NULL");
+    if (images <= 0 || tokens <= 0 || n_blocks <= 0)
+        return fail(ELSA_ERR_SHAPE, "non-positive images=%d, tokens=%d or n_blocks=%d", images, tokens, n_blocks);
+    if (!attention_suits(tokens, heads, dim))
+        return fail(ELSA_ERR_SHAPE, "attention needs at most 256 tokens per image and dim = 64 * heads (tokens=%d, heads=%d, dim=%d)",
+                    tokens, heads, dim);
+    if ((long long)images * tokens > 0x7fffffffLL) return fail(ELSA_ERR_SHAPE, "images * tokens does not fit an int");
+    if ((final_gain == nullptr) != (final_bias == nullptr)) return fail(ELSA_ERR_NULL, "final_gain and final_bias go together");
+    if (final_gain && (!aligned16(final_gain) || !aligned16(final_bias)))
+        return fail(ELSA_ERR_ALIGN, "final_gain and final_bias must be 16-byte aligned");
+    if (final_gain && !(final_eps >= 0.f)) return fail(ELSA_ERR_SHAPE, "final_eps must not be negative");
+    const int rows = images * tokens;
+    EncoderPlan plan;
+    if (!encoder_plan(rows, dim, mlp_dim, blocks, n_blocks, dtype, &plan))
+        return fail(ELSA_ERR_SHAPE, "dim and mlp_dim must be multiples of 8 and every level valid");
+    if (((uintptr_t)scratch & 255u) != 0) return fail(ELSA_ERR_ALIGN, "scratch must be 256-byte aligned");
+    if (scratch_bytes < plan.total) return fail(ELSA_ERR_WORKSPACE, "scratch of %zu bytes needed, %zu given", plan.total, scratch_bytes);
+    DeviceInfo dev;
+    elsa_status st = device_info(&dev);
+    if (st != ELSA_OK) return st;
+    uint8_t* s8 = (uint8_t*)scratch;
+    uint16_t* buf[2] = {(uint16_t*)(s8 + plan.buf[0]), (uint16_t*)(s8 + plan.buf[1])};
+    // every block is validated before the first launch
+    for (int b = 0; b < n_blocks; ++b) {
+        BlockPlan bp;
+        BlockLinear lin[4];
+        if ((st = block_check(x, rows, dim, mlp_dim, blocks + b, dtype, buf[0], true, scratch, plan.block_bytes, &bp, lin, dev)) != ELSA_OK) {
+            char msg[400];
+            snprintf(msg, sizeof msg, "%s", elsa_last_error());
+            return fail(st, "block %d: %s", b, msg);
+        }
+    }
+    // Block b reads its input from buf[b % 2] (block 0: from x) and writes its output to buf[(b + 1) % 2]; where a
+    // block's last residual is still to be added, the next block's first LayerNorm does it while it normalises.
+    BlockCarry carry;
+    const void* in = x;
+    for (int b = 0; b < n_blocks; ++b) {
+        const bool last = b + 1 == n_blocks;
+        void* out = (last && final_gain == nullptr) ? y : (void*)buf[(b + 1) & 1];
+        BlockCarry next;
+        st = run_block(in, rows, dim, mlp_dim, blocks + b, dtype, out, scratch, plan.block_bytes, dev_status, stream, tokens, heads,
+                       &carry, buf[b & 1], last && final_gain == nullptr ? nullptr : &next);
+        if (st != ELSA_OK) return st;
+        carry = next;
+        in = buf[(b + 1) & 1];
+    }
+    if (final_gain != nullptr) {
+        const bool add = carry.t != nullptr;
+        st = launch_layer_norm(add ? carry.t : buf[n_blocks & 1], add ? carry.r : nullptr, add ? buf[n_blocks & 1] : nullptr,
+                               (const uint16_t*)final_gain, (const uint16_t*)final_bias, (uint16_t*)y, rows, dim, final_eps, dtype,
+                               (cudaStream_t)stream);
+    }
+    return st;
+}
 
 elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                            void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream)

@@ -339,3 +339,74 @@ def test_deit_b_block_with_attention_full_size_sampled_images(lib):
     got = run_block(lib, x, host, levels, mlp, attn=(tokens, heads))
     pick = np.concatenate([np.arange(i * tokens, (i + 1) * tokens) for i in (0, 101, 255)])   # whole images
     check_rows(got, x, p, dtype, pick, attn=(tokens, heads))
+
+
+def _encoder_case(lib, dtype, images, tokens, heads, mlp, level_sets, seed):
+    dim = 64 * heads
+    x = synth.randn((images * tokens, dim), seed, 1.0, dtype)
+    blocks, params, keep = [], [], []
+    for b, levels in enumerate(level_sets):
+        host, p = make_params(dim, mlp, levels, dtype, seed + 100 * (b + 1))
+        dev = {k: v.cuda() for k, v in host.items()}
+        lin = {}
+        for name in NAMES:
+            N, M = levels[name]
+            vals, idx = lib.elsa_nm_compress(dev["W_" + name], N, M)
+            lin[name] = (vals, idx, dev["b_" + name], N, M)
+        w, k = lib.make_block_weights(dev["ln1_g"], dev["ln1_b"], dev["ln2_g"], dev["ln2_b"], lin, eps=1e-6)
+        blocks.append(w)
+        params.append(p)
+        keep.append((dev, lin, k))
+    return x, blocks, params, keep
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("variant", ["auto", "tc_pair", "tc_sparse_ws"])
+def test_encoder_equals_block_by_block_and_follows_the_oracle(lib, variant):
+    # auto at this size: kernels without a residual epilogue, so every block hands its last add to the next LayerNorm;
+    # tc_pair: every residual fused; tc_sparse_ws: proj and fc2 unfused, fc1's GELU fused
+    dtype = torch.bfloat16
+    images, tokens, heads, mlp = 3, 50, 2, 256
+    sets = [SPARSE_LEVELS, {"qkv": (1, 8), "proj": (2, 8), "fc1": (1, 4), "fc2": (2, 4)}, SPARSE_LEVELS] if variant == "tc_sparse_ws" \
+        else [MIXED_LEVELS, SPARSE_LEVELS, {"qkv": (2, 4), "proj": (8, 8), "fc1": (4, 8), "fc2": (1, 16)}]
+    x, blocks, params, keep = _encoder_case(lib, dtype, images, tokens, heads, mlp, sets, 2000)
+    code = {"auto": lib.VARIANT_AUTO, "tc_pair": lib.VARIANT_TC_PAIR, "tc_sparse_ws": lib.VARIANT_TC_SPARSE_WS}[variant]
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fg = (synth.randn((64 * heads,), 31, 0.1, dtype).float() + 1.0).to(dtype).cuda()
+    fb = synth.randn((64 * heads,), 32, 0.1, dtype).cuda()
+    lib.elsa_set_linear_variant(code)
+    try:
+        cur = x.cuda()
+        for w in blocks:
+            cur, _ = lib.elsa_vit_block(cur, mlp, w, dev_status=status, tokens=tokens, heads=heads)
+        table = lib.make_encoder_table(blocks)
+        y_plain, _ = lib.elsa_vit_encoder(x.cuda(), tokens, heads, mlp, table, dev_status=status)
+        y_norm, _ = lib.elsa_vit_encoder(x.cuda(), tokens, heads, mlp, table, final_gain=fg, final_bias=fb, dev_status=status)
+        torch.cuda.synchronize()
+    finally:
+        lib.elsa_set_linear_variant(lib.VARIANT_AUTO)
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    assert torch.equal(y_plain.view(torch.int16), cur.view(torch.int16))         # bit for bit the block-by-block result
+    # the final LayerNorm, from the library's own block output
+    ref_norm = bo._round16(bo.layer_norm(cur.double().cpu().numpy(), fg.double().cpu().numpy(), fb.double().cpu().numpy(), 1e-6), dtype)
+    err = np.abs(y_norm.double().cpu().numpy() - ref_norm)
+    assert (err <= stage_tolerance(ref_norm, None, dtype)).all()
+    # the oracle's chain of the same blocks
+    bits = synth.bits(x)
+    for p in params:
+        out = bo.block_forward(bits, p, eo.BF16, eps=1e-6, attn="softmax", tokens=tokens, heads=heads)
+        bits = bo._bits(out["y"], dtype)
+    got = cur.double().cpu().numpy()
+    assert np.linalg.norm(got - out["y"]) <= 1e-2 * np.linalg.norm(out["y"])     # three blocks of seven 16-bit stages each
+
+
+@pytest.mark.gpu
+def test_encoder_validates_every_block_before_launching(lib):
+    dtype = torch.bfloat16
+    x, blocks, params, keep = _encoder_case(lib, dtype, 2, 20, 1, 128, [MIXED_LEVELS, MIXED_LEVELS], 2500)
+    blocks[1].fc2.idx = None
+    before = lib.elsa_launch_count()
+    with pytest.raises(lib.ElsaError) as e:
+        lib.elsa_vit_encoder(x.cuda(), 20, 1, 128, lib.make_encoder_table(blocks))
+    assert e.value.status == 1 and "block 1" in str(e.value)
+    assert lib.elsa_launch_count() == before
