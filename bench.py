@@ -515,19 +515,22 @@ def run_ours(args):
             pass
     # ---- the chained encoder blocks (the same 48 linears fed forward, with attention), device timing only
     if args.block_chain and world == 1 and args.workload == "deit_b_stack_b256":
-        import bench_block
-        torch.cuda.empty_cache()
-        b = bench_block.run(12, 256, 5, peaks, peaks_kind, roofline_seconds)
-        with_attn, stand_in = b["encoder_blocks_with_attention"], b["linear_and_elementwise_path_only_standin_a_eq_v"]
-        line["block_chain"] = {
-            "workload": "deit_b_encoder_blocks_b256 (12 blocks chained, levels of the stack; no patch embedding or head)",
-            "ms_per_pass": with_attn["ms_per_pass"], "images_per_s": with_attn["images_per_s"],
-            "roofline_frac": with_attn["roofline_frac"], "roofline_ms": with_attn["roofline_ms"],
-            "families_ms": {k: v["ms"] for k, v in with_attn["families_profiled_pass"].items()},
-            "without_attention": {"note": "stand-in a = V in place of attention: the linear and elementwise path alone",
-                                  "ms_per_pass": stand_in["ms_per_pass"], "images_per_s": stand_in["images_per_s"],
-                                  "roofline_frac": stand_in["roofline_frac"]},
-        }
+        try:
+            import bench_block
+            torch.cuda.empty_cache()
+            b = bench_block.run(12, 256, 5, peaks, peaks_kind, roofline_seconds)
+            with_attn, stand_in = b["encoder_blocks_with_attention"], b["linear_and_elementwise_path_only_standin_a_eq_v"]
+            line["block_chain"] = {
+                "workload": "deit_b_encoder_blocks_b256 (12 blocks chained, levels of the stack; no patch embedding or head)",
+                "ms_per_pass": with_attn["ms_per_pass"], "images_per_s": with_attn["images_per_s"],
+                "roofline_frac": with_attn["roofline_frac"], "roofline_ms": with_attn["roofline_ms"],
+                "families_ms": {k: v["ms"] for k, v in with_attn["families_profiled_pass"].items()},
+                "without_attention": {"note": "stand-in a = V in place of attention: the linear and elementwise path alone",
+                                      "ms_per_pass": stand_in["ms_per_pass"], "images_per_s": stand_in["images_per_s"],
+                                      "roofline_frac": stand_in["roofline_frac"]},
+            }
+        except Exception as exc:          # the headline line must not depend on this extra measurement
+            line["block_chain"] = {"error": "%s: %s" % (type(exc).__name__, exc)}
     if rank == 0:
         print(json.dumps(line))
     if world > 1:
