@@ -1237,8 +1237,18 @@ namespace elsa {
 namespace {
 
 struct BackwardPlan {
-    size_t wm, wmt, partial, total;   // byte offsets of the regions
+    size_t wm, wmt, partial, sums, total;   // byte offsets of the regions
 };
+
+// Upper bound, from host arithmetic alone, of the ranges the dW product may be cut into: what a device of 256 SMs
+// would use.  The call clamps its choice to it.
+int wgrad_splits_bound(int in, int out)
+{
+    const long long tiles = (long long)((out + 255) / 256) * ((in + 255) / 256);
+    long long s = 128 / tiles;
+    if (s > 8) s = 8;
+    return s < 1 ? 1 : (int)s;
+}
 
 BackwardPlan backward_plan(int rows, int in, int out)
 {
@@ -1247,6 +1257,8 @@ BackwardPlan backward_plan(int rows, int in, int out)
     p.wm = at;      at += round_up((size_t)out * in * 2, 256);                      // masked weight [out][in]
     p.wmt = at;     at += round_up((size_t)out * in * 2, 256);                      // its transpose [in][out]
     p.partial = at; at += round_up((size_t)((rows + 511) / 512) * out * 4, 256);    // column sums of dY per 512 rows
+    const int bound = wgrad_splits_bound(in, out);                                  // fp32 sums of dW per range of rows
+    p.sums = at;    at += bound > 1 ? round_up((size_t)bound * out * in * 4, 256) : 0;
     p.total = at;
     return p;
 }
@@ -1312,9 +1324,16 @@ elsa_status elsa_nm_linear_backward(const void* dY, const void* X, int rows, con
     if (dW) {
         // dW = dY^T X, reduction over the token rows: both operands are read as they are stored (reduction index
         // outermost), then the mask
-        if ((st = launch_linear_tc_pair_tn(dy, (const uint16_t*)X, out, in, rows, dtype, (uint16_t*)dW, dev_status, stream)) != ELSA_OK)
+        // when 256 x 256 tiles alone leave SM pairs idle, the rows are cut into ranges summed afterwards
+        int splits = linear_tc_pair_tn_splits(out, in, rows, dev.sm_count);
+        if (splits > wgrad_splits_bound(in, out)) splits = wgrad_splits_bound(in, out);
+        float* sums = (float*)(ws + plan.sums);
+        if ((st = launch_linear_tc_pair_tn(dy, (const uint16_t*)X, out, in, rows, dtype, (uint16_t*)dW, splits, sums, dev_status,
+                                           stream)) != ELSA_OK)
             return st;
-        if ((st = launch_mask_apply((uint16_t*)dW, idx, out, in, N, M, stream)) != ELSA_OK) return st;
+        st = splits > 1 ? launch_wgrad_finish(sums, splits, idx, out, in, N, M, dtype, (uint16_t*)dW, stream)
+                        : launch_mask_apply((uint16_t*)dW, idx, out, in, N, M, stream);
+        if (st != ELSA_OK) return st;
     }
     return ELSA_OK;
 }

@@ -175,6 +175,56 @@ mask_apply_kernel(uint16_t* __restrict__ dW, const uint32_t* __restrict__ idx, i
     }
 }
 
+// One thread per group of M weights: adds the ranges' fp32 sums in ascending order, rounds once, zeroes what the
+// index stream does not keep (everything is kept when idx is NULL).
+template <int M, bool kBf16>
+__global__ void __launch_bounds__(256)
+wgrad_finish_kernel(const float* __restrict__ partial, int splits, const uint32_t* __restrict__ idx, int out, int in, int N,
+                    int words_per_row, uint16_t* __restrict__ dW)
+{
+    constexpr int B = (M == 4) ? 2 : (M == 8) ? 3 : 4;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int groups_per_row = in / M;
+    if (gid >= (long long)out * groups_per_row) return;
+    const int o = (int)(gid / groups_per_row), g = (int)(gid % groups_per_row);
+    uint32_t keep = 0xffffffffu;
+    if (idx != nullptr) {
+        keep = 0;
+        const uint32_t* row = idx + (size_t)o * (size_t)words_per_row;
+        for (int t = 0; t < N; ++t) {
+            const int bit = (g * N + t) * B;
+            const int w = bit >> 5, sh = bit & 31;
+            uint32_t f = row[w] >> sh;
+            if (sh + B > 32) f |= row[w + 1] << (32 - sh);
+            keep |= 1u << (f & (M - 1));
+        }
+    }
+    const size_t at = (size_t)o * (size_t)in + (size_t)g * M;
+    const size_t plane = (size_t)out * (size_t)in;
+    float acc[M];
+#pragma unroll
+    for (int q = 0; q < M / 4; ++q) {
+        const float4 v = *reinterpret_cast<const float4*>(partial + at + 4 * q);
+        acc[4 * q] = v.x; acc[4 * q + 1] = v.y; acc[4 * q + 2] = v.z; acc[4 * q + 3] = v.w;
+    }
+    for (int s = 1; s < splits; ++s) {
+#pragma unroll
+        for (int q = 0; q < M / 4; ++q) {
+            const float4 v = *reinterpret_cast<const float4*>(partial + (size_t)s * plane + at + 4 * q);
+            acc[4 * q] += v.x; acc[4 * q + 1] += v.y; acc[4 * q + 2] += v.z; acc[4 * q + 3] += v.w;
+        }
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(dW + at);
+#pragma unroll
+    for (int q = 0; q < M / 2; ++q) {
+        const uint32_t lo = (keep >> (2 * q)) & 1u ? from_float<kBf16>(acc[2 * q]) : 0u;
+        const uint32_t hi = (keep >> (2 * q + 1)) & 1u ? from_float<kBf16>(acc[2 * q + 1]) : 0u;
+        dst[q] = lo | (hi << 16);
+    }
+}
+
 }  // namespace
 
 elsa_status launch_colsum_finish(const float* partial, int tiles, int C, uint16_t* db, elsa_dtype dtype, cudaStream_t stream);
@@ -210,6 +260,27 @@ elsa_status launch_colsum_finish(const float* partial, int tiles, int C, uint16_
     if (dtype == ELSA_BF16) launch_pdl(colsum_finish_kernel<true>, dim3(grid), dim3(256), 0, stream, 1, partial, tiles, C, db);
     else launch_pdl(colsum_finish_kernel<false>, dim3(grid), dim3(256), 0, stream, 1, partial, tiles, C, db);
     return launched("colsum_finish");
+}
+
+elsa_status launch_wgrad_finish(const float* partial, int splits, const uint32_t* idx, int out, int in, int N, int M,
+                                elsa_dtype dtype, uint16_t* dW, cudaStream_t stream)
+{
+    const long long groups = (long long)out * (in / M);
+    const unsigned grid = (unsigned)((groups + 255) / 256);
+    const int wpr = (int)index_words_per_row(in, N, M);
+    const uint32_t* ix = N == M ? nullptr : idx;
+    const bool bf = dtype == ELSA_BF16;
+    ProfileScope scope(ELSA_KERNEL_BACKWARD_FORMAT, stream);
+#define ELSA_FINISH(MM)                                                                                                     \
+    do {                                                                                                                  \
+        if (bf) launch_pdl(wgrad_finish_kernel<MM, true>, dim3(grid), dim3(256), 0, stream, 1, partial, splits, ix, out, in, N, wpr, dW); \
+        else launch_pdl(wgrad_finish_kernel<MM, false>, dim3(grid), dim3(256), 0, stream, 1, partial, splits, ix, out, in, N, wpr, dW);   \
+    } while (0)
+    if (M == 4) ELSA_FINISH(4);
+    else if (M == 8) ELSA_FINISH(8);
+    else ELSA_FINISH(16);
+#undef ELSA_FINISH
+    return launched("wgrad_finish");
 }
 
 elsa_status launch_mask_apply(uint16_t* dW, const uint32_t* idx, int out, int in, int N, int M, cudaStream_t stream)

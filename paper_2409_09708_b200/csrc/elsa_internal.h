@@ -100,8 +100,11 @@ elsa_status launch_linear_tc_pair(const uint16_t* X, int rows, const uint16_t* W
                                   cudaStream_t stream);
 // Y [m][n] = A^T B on the same kernel with both operands stored reduction-outermost, A [k][m] and B [k][n]
 // (m, n multiples of 8): the weight-gradient product dY^T X without transposed copies.
+// With splits > 1 the reduction is cut into that many ranges whose fp32 sums go to partial [splits][m][n] (Y is then
+// not written); linear_tc_pair_tn_splits says how many ranges keep the SM pairs occupied.
+int linear_tc_pair_tn_splits(int m, int n, int k, int sm_count);
 elsa_status launch_linear_tc_pair_tn(const uint16_t* A, const uint16_t* B, int m, int n, int k, elsa_dtype dtype,
-                                     uint16_t* Y, uint32_t* dev_status, cudaStream_t stream);
+                                     uint16_t* Y, int splits, float* partial, uint32_t* dev_status, cudaStream_t stream);
 // Levels with N <= 2 on the hardware 2:4 sparse MMA: re-encodes the packed weight into `workspace`
 // (2-of-4 values + metadata), then runs the sparse GEMM.
 elsa_status launch_linear_tc_sparse(const uint16_t* X, int rows, const uint16_t* vals, const uint32_t* idx,
@@ -180,6 +183,9 @@ elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C,
 elsa_status launch_colsum(const uint16_t* src, int R, int C, float* partial, uint16_t* db, elsa_dtype dtype, cudaStream_t stream);
 // Zeroes the pruned positions of a dense [out][in] tensor in place.
 elsa_status launch_mask_apply(uint16_t* dW, const uint32_t* idx, int out, int in, int N, int M, cudaStream_t stream);
+// dW [out][in] = mask .* round16(sum over ranges of partial [splits][out][in]); idx NULL (N == M) keeps everything.
+elsa_status launch_wgrad_finish(const float* partial, int splits, const uint32_t* idx, int out, int in, int N, int M,
+                                elsa_dtype dtype, uint16_t* dW, cudaStream_t stream);
 // Several levels of one weight in one pass, and the dense projections used by the mask-on-load linear.
 constexpr int kMaxLevels = 16;
 struct LevelTable {
@@ -229,6 +235,8 @@ struct PairJob {
     float x_scale = 0.f;
     int act = 0;                          // epilogue activation: 0 none, 1 GELU (applied to acc + bias)
     const uint16_t* residual = nullptr;   // [rows][out], added after the activation, before the one rounding
+    int splits = 1;                       // Tn form: ranges the reduction is cut into; > 1 writes fp32 sums to `partial`
+    float* partial = nullptr;             // [splits][rows][out]
 };
 int linear_tc_pair_group_max();
 elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t* dev_status,

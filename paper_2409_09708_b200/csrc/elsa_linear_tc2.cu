@@ -80,6 +80,10 @@ struct PairGroup {
     int num_tiles;     // over all layers
     int stages;
     uint32_t* dev_status;
+    // Tn form only (one layer per launch): the reduction is cut into `splits` ranges of K blocks, a tile index t is
+    // tile t / splits over range t % splits, and each range's fp32 sums go to partial[range][rows][out].
+    int splits;
+    float* partial;
 };
 
 constexpr int kStageBytesMax = kATileBytes + (kMaxBlockN / 2) * kBlockK * 2;   // stage slots sized for BN = 256
@@ -169,12 +173,19 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
                 while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
                 const PairLayer& L = p.layer[cur];
-                const int t = tile - L.tile_begin;
+                int t = tile - L.tile_begin;
+                int kb0 = 0, kb1 = L.num_k_blocks;
+                if constexpr (kTn) {
+                    const int range = t % p.splits;
+                    t /= p.splits;
+                    kb0 = (int)((long long)L.num_k_blocks * range / p.splits);
+                    kb1 = (int)((long long)L.num_k_blocks * (range + 1) / p.splits);
+                }
                 const int half_bn = L.bn >> 1;
                 const int m0 = (t / L.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
                 const int n0 = (t % L.tiles_n) * L.bn + (int)cta_rank * half_bn;
                 const uint32_t tx_bytes = (uint32_t)(2 * (kATileBytes + half_bn * kBlockK * 2));
-                for (int kb = 0; kb < L.num_k_blocks; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(empty_bar + 8 * stage, phase ^ 1u, abort_flag, p.dev_status, 1);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
@@ -220,14 +231,19 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
             int cur = 0;
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
                 while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
-                const int num_k_blocks = p.layer[cur].num_k_blocks;
+                int kb0 = 0, kb1 = p.layer[cur].num_k_blocks;
+                if constexpr (kTn) {
+                    const int range = (tile - p.layer[cur].tile_begin) % p.splits;
+                    kb0 = (int)((long long)p.layer[cur].num_k_blocks * range / p.splits);
+                    kb1 = (int)((long long)p.layer[cur].num_k_blocks * (range + 1) / p.splits);
+                }
                 const uint32_t idesc = p.layer[cur].idesc;
                 ok = mbar_wait(tmem_empty_bar + 8 * acc, acc_phase ^ 1u, abort_flag, p.dev_status, 2);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_u + (uint32_t)(acc * kMaxBlockN);
-                for (int kb = 0; kb < num_k_blocks; ++kb) {
+                for (int kb = kb0; kb < kb1; ++kb) {
                     ok = mbar_wait(full_bar + 8 * stage, phase, abort_flag, p.dev_status, 3);
                     ok = __all_sync(0xFFFFFFFFu, ok);
                     if (!ok) break;
@@ -241,7 +257,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
                         if constexpr (kTn)
                             // 16 reduction rows of 128 bytes per MMA: the start address moves by 2048 bytes
                             umma_f16_pair_if(d_tmem, a_desc + (uint64_t)(k * (kUmmaK * 128 >> 4)), b_desc + (uint64_t)(k * (kUmmaK * 128 >> 4)),
-                                             idesc, (uint32_t)((kb | k) != 0), elected);
+                                             idesc, (uint32_t)(kb != kb0 || k != 0), elected);
                         else if constexpr (kInt8)
                             umma_i8_pair_if(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), idesc,
                                             (uint32_t)((kb | k) != 0), elected);
@@ -266,7 +282,7 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++it) {
             while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
             const PairLayer& L = p.layer[cur];
-            const int n0 = ((tile - L.tile_begin) % L.tiles_n) * L.bn;
+            const int n0 = (((tile - L.tile_begin) / (kTn ? p.splits : 1)) % L.tiles_n) * L.bn;
             const uint32_t b = it & 1u;
             bool ok = mbar_wait(bias_empty_bar + 8 * b, ((it >> 1) & 1u) ^ 1u, abort_flag, p.dev_status, 5);
             ok = __all_sync(0xFFFFFFFFu, ok);
@@ -304,7 +320,13 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
         for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++it) {
             while (cur + 1 < p.n_layers && tile >= p.layer[cur + 1].tile_begin) ++cur;
             const PairLayer& L = p.layer[cur];
-            const int t = tile - L.tile_begin;
+            int t = tile - L.tile_begin;
+            int range = 0;
+            if constexpr (kTn) {
+                range = t % p.splits;
+                t /= p.splits;
+            }
+            (void)range;
             const int chunks = L.bn / kEpiCols;
             const int my_chunks = (chunks - part + kEpiParts - 1) / kEpiParts;
             const int m0 = (t / L.tiles_n) * kPairRows + (int)cta_rank * kRowsPerCta;
@@ -328,6 +350,21 @@ linear_tc_pair_kernel(const __grid_constant__ PairGroup<kMaxLayers> p)
 
             // converts, stages and stores one 32 x 32 chunk
             auto emit = [&](const uint32_t (&r)[32], int c) {
+                if constexpr (kTn) {
+                    if (p.partial != nullptr) {
+                        // a range's fp32 sums as they are: this lane's row, 32 consecutive columns
+                        const int row = row0 + lane, col0 = n0 + c * kEpiCols;
+                        if (row < l_rows) {
+                            float4* dst = reinterpret_cast<float4*>(p.partial + ((size_t)range * (size_t)l_rows + row) * (size_t)l_out + col0);
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                if (col0 + 4 * v < l_out)
+                                    dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                         __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                        }
+                        return;
+                    }
+                }
                 // 16 columns: + bias (read as stored, eight values per load), rounded to 16 bit
                 auto convert16 = [&](auto with_act, int h, uint32_t (&pk)[8]) {
 #pragma unroll
@@ -498,10 +535,10 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
         const PairJob& j = jobs[i];
         PairLayer& L = g.layer[i];
         L.rows = j.rows; L.out = j.out;
-        L.bn = pick_pair_block_n(j.out, j.rows, dev.sm_count, kForm == kFormTn);
+        L.bn = (kForm == kFormTn && j.splits > 1) ? 256 : pick_pair_block_n(j.out, j.rows, dev.sm_count, kForm == kFormTn);
         L.tiles_n = (j.out + L.bn - 1) / L.bn;
         L.tile_begin = tile_begin;
-        tile_begin += ((j.rows + kPairRows - 1) / kPairRows) * L.tiles_n;
+        tile_begin += ((j.rows + kPairRows - 1) / kPairRows) * L.tiles_n * (kForm == kFormTn ? j.splits : 1);
         L.bias = j.bias;
         L.w_scale = j.w_scale;
         L.x_scale = j.x_scale;
@@ -544,6 +581,8 @@ elsa_status launch_group(const PairJob* jobs, int n, elsa_dtype dtype, uint32_t*
             return st;
     }
     g.n_layers = n;
+    g.splits = kForm == kFormTn ? jobs[0].splits : 1;
+    g.partial = kForm == kFormTn && jobs[0].splits > 1 ? jobs[0].partial : nullptr;
     g.num_tiles = tile_begin;
     g.dev_status = dev_status;
 
@@ -619,9 +658,23 @@ elsa_status launch_linear_tc_pair_group(const PairJob* jobs, int n, elsa_dtype d
                               : launch_group<false, kFormPlain, kGroupMax>(jobs, n, dtype, dev_status, stream, dev);
 }
 
+// How many ranges the reduction of an m x n product is cut into: with 256 x 256 tiles, as many as keep one wave of
+// work units on the SM pairs (1 when the tiles alone fill them).
+int linear_tc_pair_tn_splits(int m, int n, int k, int sm_count)
+{
+    const int pairs = sm_count / 2 > 0 ? sm_count / 2 : 1;
+    const long long tiles = (long long)((m + kPairRows - 1) / kPairRows) * ((n + 255) / 256);
+    long long s = pairs / tiles;
+    const int k_blocks = (k + kBlockK - 1) / kBlockK;
+    if (s > 8) s = 8;
+    if (s > k_blocks) s = k_blocks;
+    return s < 1 ? 1 : (int)s;
+}
+
 // Y [m][n] = A^T B with A [k][m] and B [k][n] (the reduction index outermost in both), no bias: one launch.
+// splits > 1: nothing is written to Y; partial [splits][m][n] receives the fp32 sums of each range of the reduction.
 elsa_status launch_linear_tc_pair_tn(const uint16_t* A, const uint16_t* B, int m, int n, int k, elsa_dtype dtype,
-                                     uint16_t* Y, uint32_t* dev_status, cudaStream_t stream)
+                                     uint16_t* Y, int splits, float* partial, uint32_t* dev_status, cudaStream_t stream)
 {
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
@@ -629,6 +682,8 @@ elsa_status launch_linear_tc_pair_tn(const uint16_t* A, const uint16_t* B, int m
     PairJob job;
     job.X = A; job.Wd = B; job.bias = nullptr; job.Y = Y;
     job.rows = m; job.in = k; job.out = n;
+    job.splits = splits < 1 ? 1 : splits;
+    job.partial = partial;
     return dtype == ELSA_BF16 ? launch_group<true, kFormTn, 1>(&job, 1, dtype, dev_status, stream, dev)
                               : launch_group<false, kFormTn, 1>(&job, 1, dtype, dev_status, stream, dev);
 }

@@ -46,7 +46,7 @@ def run(lib, dY, X, W, N, M, want=("dX", "dW", "db"), variant=None):
 
 
 CASES = [(333, 256, 192, 2, 8), (70, 64, 40, 1, 4), (1000, 768, 768, 4, 8), (129, 128, 264, 8, 8), (200, 96, 64, 3, 16),
-         (65, 24, 8, 3, 8)]
+         (65, 24, 8, 3, 8), (5000, 768, 768, 1, 8)]     # the last: nine 256 x 256 tiles, so the rows are cut into eight uneven ranges
 
 
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
