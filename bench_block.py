@@ -2,6 +2,7 @@
 with the levels the stack workload gives its four linears, chained (a block's y is the next block's x).
 
     python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
+    python bench_block.py --compare          # dense 4:4 against N:4 configurations at the paper's operating points
 
 Two timings: with the library's multi-head self-attention (elsa_vit_encoder: the encoder blocks of DeiT-B as
 they run, without patch embedding, final norm and classifier head), and with the stand-in a = V in its place (the linear and
@@ -11,6 +12,12 @@ per-launch events for the split by kernel family, and the roofline of the pass: 
 FLOPs / bf16 peak and algorithmic bytes / HBM peak, plus the elementwise stages' bytes (LayerNorm in and out
 twice, one residual operand per add; the copy in and out for the stand-in) / HBM peak, plus, with attention, the
 larger of its 4 tokens^2 d FLOPs per head and image / bf16 peak and its bytes (qkv in, a out) / HBM peak.
+
+--compare runs the encoder three times: every linear dense (4:4), and under two N:4 configurations {1:4, 2:4, 4:4}
+drawn by the library's two-step sampler (Alg. 3) at 7.0 and 6.0 whole-model GMACs per image, the two operating
+points Table 1 lists for ELSA-DeiT-B-N:4 (the paper expects up to 2.9x at 6.0 G from a cited accelerator's
+MAC-proportional model; it measures no speed itself).  The searched configurations themselves need the trained
+supernet; these are draws from the same search space at the same cost.
 """
 from __future__ import annotations
 
@@ -30,9 +37,10 @@ from paper_2409_09708_b200 import binding as lib
 from paper_2409_09708_b200 import synth
 
 
-def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seconds=None):
+def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seconds=None, levels=None, stand_in=True):
     """Times the chained blocks; returns the record main() prints.  peaks / roofline_seconds: bench.py's (passed in
-    by bench.py itself when it calls this; looked up there otherwise)."""
+    by bench.py itself when it calls this; looked up there otherwise).  levels: one (N, M) per linear in the order
+    of the stack workload, or None for that workload's own seeded draw."""
     if peaks is None:
         import bench
         peaks, peaks_kind = bench.load_peaks()
@@ -41,6 +49,9 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     dtype = torch.bfloat16
     dim, mlp = 768, 3072
     layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
+    if levels is not None:
+        import dataclasses
+        layers = [dataclasses.replace(l, N=n, M=m) for l, (n, m) in zip(layers, levels)]
     rows = layers[0].rows
 
     blocks = []
@@ -107,7 +118,7 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
                 "first_block_launches": [[k, round(t, 4)] for k, _, t in launch_list[:len(launch_list) // args.blocks + 2]]}
 
     with_attention = measure(True)
-    stand_in = measure(False)
+    stand_in = measure(False) if stand_in else None
     rec = {"workload": "deit_b_blocks_b%d" % args.batch, "blocks": args.blocks, "rows": rows, "dtype": "bf16",
            "peaks": peaks_kind, "linears_roofline_ms": lin_roof * 1e3, "attention_roofline_ms_per_block": attn_roof * 1e3,
            "encoder_blocks_with_attention": with_attention,
@@ -116,14 +127,41 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     return rec
 
 
+def compare(args):
+    import bench
+    layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
+    runs = [("dense 4:4", [(4, 4)] * len(layers), None)]
+    for gmacs in (7.0, 6.0):
+        picked, cost = bench.sampled_levels(lib, layers, gmacs)
+        runs.append(("N:4 sampled at %.1f GMACs" % gmacs, picked, cost))
+    out = []
+    for name, levels, cost in runs:
+        r = run(args.blocks, args.batch, args.reps, levels=levels, stand_in=False)["encoder_blocks_with_attention"]
+        kept = sum(n / m for n, m in levels) / len(levels)
+        out.append({"configuration": name, "whole_model_gmacs_per_image": cost, "mean_linear_density": kept,
+                    "levels": ["%d:%d" % lv for lv in levels], "ms_per_pass": r["ms_per_pass"], "ms_min": r["ms_min"],
+                    "images_per_s": r["images_per_s"], "roofline_frac": r["roofline_frac"],
+                    "families_ms": {k: round(v["ms"], 3) for k, v in r["families_profiled_pass"].items()}})
+    for o in out:
+        o["speedup_over_dense"] = out[0]["ms_per_pass"] / o["ms_per_pass"]
+    return {"workload": "deit_b_encoder_blocks_b%d" % args.batch, "blocks": args.blocks, "dtype": "bf16",
+            "note": "encoder blocks only (no patch embedding, final norm or head); configurations are draws of the "
+                    "two-step sampler from the N:4 space at the paper's operating points, not the paper's searched ones",
+            "runs": out}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--blocks", type=int, default=12)
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--out", default="bench_out/block.json")
+    ap.add_argument("--compare", action="store_true", help="dense 4:4 against sampled N:4 configurations at 7.0 and 6.0 GMACs")
     args = ap.parse_args()
-    rec = run(args.blocks, args.batch, args.reps)
+    if args.compare:
+        rec = compare(args)
+    else:
+        rec = run(args.blocks, args.batch, args.reps)
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     json.dump(rec, open(args.out, "w"), indent=1)
     print(json.dumps(rec))
