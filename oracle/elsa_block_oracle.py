@@ -14,6 +14,13 @@ of the ViT / DeiT backbones the paper prunes (the paper leaves the attention pro
 formula of its own: this is the standard one): per image and head, with q, k, v the head's slices of the three
 thirds of qkv and d the head dimension, a = softmax(q k^T / sqrt d) v, the softmax over the keys of the same image;
 heads are laid side by side in a's columns.  All tokens of an image attend to each other (no mask, no dropout).
+"window": the shifted-window attention of the Swin backbones the paper also prunes (Table 1, Swin-S / Swin-B; again
+the paper gives no formula, this is the backbone's): the H x W token grid of an image is rolled by -shift along both
+axes, cut into windows of ws x ws tokens, every window attends within itself as above with a per-head additive
+bias [ws^2, ws^2] on the scores (the relative-position bias, given as a dense table) and, when shift > 0, with
+-100 added where two tokens of a window come from different sides of the roll's seam (the three bands
+[0, H - ws), [H - ws, H - shift), [H - shift, H) of each axis number the regions); the result is put back and rolled
+by +shift.
 
 Every tensor that crosses a stage boundary is a 16-bit tensor (the library writes it to memory in the block's
 dtype), so every stage here computes in fp64 from its 16-bit inputs and rounds its result once, to nearest
@@ -76,10 +83,55 @@ def attention(qkv, tokens, heads):
     return out
 
 
-def block_forward(x_bits, p, code, eps=1e-6, attn="copy_v", tokens=None, heads=None):
+def window_order(H, W, ws, shift):
+    """Row index, inside one image's H * W tokens, of every window token: [windows, ws * ws] in the order
+    (window row, window column; token row, token column) of the grid rolled by -shift."""
+    i, j = np.meshgrid(np.arange(H), np.arange(W), indexing="ij")
+    src = ((i + shift) % H) * W + (j + shift) % W          # rolled[i, j] = x[(i + shift) % H, (j + shift) % W]
+    return src.reshape(H // ws, ws, W // ws, ws).transpose(0, 2, 1, 3).reshape(-1, ws * ws)
+
+
+def shift_mask(H, W, ws, shift):
+    """[windows, ws * ws, ws * ws]: 0 where two tokens of a window may attend to each other, -100 where the roll
+    brought them together from different regions."""
+    region = np.zeros((H, W))
+    bands = lambda n: (slice(0, n - ws), slice(n - ws, n - shift), slice(n - shift, n))
+    k = 0
+    for hs in bands(H):
+        for wsl in bands(W):
+            region[hs, wsl] = k
+            k += 1
+    r = region.reshape(H // ws, ws, W // ws, ws).transpose(0, 2, 1, 3).reshape(-1, ws * ws)
+    return np.where(r[:, :, None] != r[:, None, :], -100.0, 0.0)
+
+
+def window_attention(qkv, H, W, ws, shift, heads, rel_bias):
+    """fp64 shifted-window attention.  qkv: [images * H * W, 3 * dim] in the images' own token order; rel_bias:
+    [heads, ws * ws, ws * ws]; returns [images * H * W, dim] in the same token order."""
+    rows, three_dim = qkv.shape
+    dim = three_dim // 3
+    d = dim // heads
+    order = window_order(H, W, ws, shift)
+    mask = shift_mask(H, W, ws, shift) if shift > 0 else np.zeros((order.shape[0], ws * ws, ws * ws))
+    out = np.zeros((rows, dim))
+    for b in range(rows // (H * W)):
+        for w in range(order.shape[0]):
+            r = b * H * W + order[w]
+            for h in range(heads):
+                q = qkv[r, h * d:(h + 1) * d]
+                k = qkv[r, dim + h * d:dim + (h + 1) * d]
+                v = qkv[r, 2 * dim + h * d:2 * dim + (h + 1) * d]
+                s = q @ k.T / math.sqrt(d) + rel_bias[h] + mask[w]
+                e = np.exp(s - s.max(axis=1, keepdims=True))
+                out[r, h * d:(h + 1) * d] = (e / e.sum(axis=1, keepdims=True)) @ v
+    return out
+
+
+def block_forward(x_bits, p, code, eps=1e-6, attn="copy_v", tokens=None, heads=None, window=None):
     """x_bits: uint16 [rows, dim].  p: dict with ln1_g, ln1_b, ln2_g, ln2_b (uint16 [dim]) and, for each of qkv,
     proj, fc1, fc2: W_<name> (uint16 [out, in]), b_<name> (uint16 [out]), level_<name> = (N, M).
-    attn: "copy_v" or "softmax" (then tokens per image and heads are required; rows = images * tokens).
+    attn: "copy_v", "softmax" (then tokens per image and heads are required; rows = images * tokens) or "window"
+    (then heads and window = dict(H, W, ws, shift, rel_bias [heads, ws^2, ws^2] fp64); rows = images * H * W).
     Returns a dict of every stage's 16-bit result as fp64 arrays: x1, qkv, a, x2, x3, h, y."""
     torch_dtype = torch.float16 if code == eo.F16 else torch.bfloat16
 
@@ -93,6 +145,9 @@ def block_forward(x_bits, p, code, eps=1e-6, attn="copy_v", tokens=None, heads=N
     out["qkv"] = _round16(sparse_linear(out["x1"], p["W_qkv"], p["b_qkv"], *p["level_qkv"], code), torch_dtype)
     if attn == "copy_v":
         out["a"] = out["qkv"][:, 2 * dim:3 * dim].copy()             # the stated stand-in for attention: a = V
+    elif attn == "window":
+        out["a"] = _round16(window_attention(out["qkv"], window["H"], window["W"], window["ws"], window["shift"], heads,
+                                             window["rel_bias"]), torch_dtype)
     else:
         out["a"] = _round16(attention(out["qkv"], tokens, heads), torch_dtype)
     out["x2"] = _round16(x + sparse_linear(out["a"], p["W_proj"], p["b_proj"], *p["level_proj"], code), torch_dtype)

@@ -135,3 +135,64 @@ def test_block_chain_with_attention_against_torch():
     a16 = a.to(dtype).double().numpy()
     assert (np.abs(got["a"] - a16) <= 2.0 ** -7 * np.abs(a16) + 1e-30).all() and (got["a"] == a16).mean() > 0.95
     assert not np.allclose(got["a"], got["qkv"][:, 2 * dim:])            # not the stand-in
+
+
+def _swin_reference(qkv, B, H, W, ws, shift, heads, rel_bias):
+    """The backbone's formulation with torch's own roll / view / permute and its fused attention, in fp64."""
+    dim = qkv.shape[1] // 3
+    d = dim // heads
+    t = torch.from_numpy(qkv).view(B, H, W, 3 * dim)
+    if shift:
+        t = torch.roll(t, shifts=(-shift, -shift), dims=(1, 2))
+    t = t.view(B, H // ws, ws, W // ws, ws, 3 * dim).permute(0, 1, 3, 2, 4, 5).reshape(-1, ws * ws, 3, heads, d)
+    q, k, v = (t[:, :, i].permute(0, 2, 1, 3) for i in range(3))                    # [windows, heads, tokens, d]
+    bias = torch.from_numpy(rel_bias)[None]                                          # [1, heads, T, T]
+    if shift:
+        img = torch.zeros(1, H, W, 1, dtype=torch.float64)
+        cnt = 0
+        for hs in (slice(0, -ws), slice(-ws, -shift), slice(-shift, None)):
+            for wsl in (slice(0, -ws), slice(-ws, -shift), slice(-shift, None)):
+                img[:, hs, wsl, :] = cnt
+                cnt += 1
+        mw = img.view(1, H // ws, ws, W // ws, ws, 1).permute(0, 1, 3, 2, 4, 5).reshape(-1, ws * ws)
+        m = (mw[:, None, :] - mw[:, :, None] != 0).double() * -100.0                 # [nW, T, T]
+        bias = bias + m.repeat(B, 1, 1)[:, None]
+    o = torch.nn.functional.scaled_dot_product_attention(q, k, v, attn_mask=bias)
+    o = o.permute(0, 2, 1, 3).reshape(B, H // ws, W // ws, ws, ws, dim).permute(0, 1, 3, 2, 4, 5).reshape(B, H, W, dim)
+    if shift:
+        o = torch.roll(o, shifts=(shift, shift), dims=(1, 2))
+    return o.reshape(B * H * W, dim).numpy()
+
+
+def test_window_attention_against_the_backbones_formulation():
+    rng = np.random.default_rng(5)
+    for (B, H, W, ws, shift, heads, d) in [(2, 6, 6, 3, 0, 2, 4), (2, 6, 6, 3, 1, 2, 4), (1, 8, 4, 4, 2, 1, 8), (3, 14, 14, 7, 3, 2, 4)]:
+        dim = heads * d
+        qkv = rng.standard_normal((B * H * W, 3 * dim))
+        rel_bias = rng.standard_normal((heads, ws * ws, ws * ws))
+        got = bo.window_attention(qkv, H, W, ws, shift, heads, rel_bias)
+        assert np.allclose(got, _swin_reference(qkv, B, H, W, ws, shift, heads, rel_bias), rtol=1e-10, atol=1e-10)
+    # one window covering the whole image, no shift, no bias: plain attention over the image
+    qkv = rng.standard_normal((2 * 16, 3 * 8))
+    assert np.allclose(bo.window_attention(qkv, 4, 4, 4, 0, 2, np.zeros((2, 16, 16))), bo.attention(qkv, 16, 2), atol=1e-12)
+    # the order of windows: every token exactly once, windows are ws x ws patches of the rolled grid
+    order = bo.window_order(6, 9, 3, 1)
+    assert sorted(order.ravel().tolist()) == list(range(54))
+    assert order[0].tolist() == [10, 11, 12, 19, 20, 21, 28, 29, 30]               # rows 1..3, columns 1..3
+    assert order[-1].tolist() == [43, 44, 36, 52, 53, 45, 7, 8, 0]                 # the wrapped corner
+    # the mask: nothing is masked inside the windows away from the seam; the last window mixes four regions
+    m = bo.shift_mask(6, 9, 3, 1)
+    assert (m[0] == 0).all() and (m[-1] != 0).any()
+    r_last = np.array([0, 0, 1, 0, 0, 1, 2, 2, 3])                                # regions of the last window's tokens
+    assert np.array_equal(m[-1] != 0, r_last[:, None] != r_last[None, :])
+    # tokens from different regions of a window do not influence each other
+    B, H, W, ws, shift, heads, d = 1, 6, 6, 3, 1, 1, 4
+    qkv = rng.standard_normal((36, 12))
+    bias = np.zeros((1, 9, 9))
+    base = bo.window_attention(qkv, H, W, ws, shift, heads, bias)
+    changed = qkv.copy()
+    changed[0, 4:] += 5.0                        # token (0, 0) ends up alone in its region of the last window
+    after = bo.window_attention(changed, H, W, ws, shift, heads, bias)
+    others = np.ones(36, bool)
+    others[0] = False
+    assert np.allclose(after[others], base[others], atol=1e-12) and not np.allclose(after[0], base[0], atol=1e-3)
