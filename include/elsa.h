@@ -432,9 +432,17 @@ elsa_status elsa_vit_block(const void* x, int rows, int dim, int mlp_dim, const 
                            void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream);
 /* qkv [images * tokens][3 dim] (q | k | v thirds, heads side by side in each) -> a [images * tokens][dim]; the
  * scores and probabilities stay on chip (fp32 scores, probabilities rounded to `dtype` for the second product, fp32
- * row sums, one rounding of a).  dim = 64 * heads, tokens <= 256. */
+ * row sums, one rounding of a).  dim = 64 * heads or 32 * heads, tokens <= 256. */
 elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype, void* a,
                            uint32_t* dev_status, void* stream);
+/* The same over windows of `tokens` consecutive rows with additive tables on the scores (Swin's window attention once
+ * the rows are in window order): a = softmax(q k^T / sqrt d + bias[head] + mask[window % n_masks]) v.  bias: fp32
+ * [heads][tokens][bias_pitch] (the relative-position bias as a dense table), mask: fp32 [n_masks][tokens][bias_pitch] or
+ * NULL (the seam mask of shifted windows, one table per window position of an image); bias_pitch >= tokens floats per
+ * row.  Head dimension 32 or 64 (dim = heads * 32 or heads * 64), tokens <= 256. */
+elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int heads, int dim, const float* bias,
+                                  int bias_pitch, const float* mask, int n_masks, elsa_dtype dtype, void* a,
+                                  uint32_t* dev_status, void* stream);
 /* The whole block with elsa_attention between the halves; rows = images * tokens. */
 elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
                                 const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,

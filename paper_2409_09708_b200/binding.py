@@ -125,6 +125,7 @@ _block_rest = _sig("elsa_vit_block_rest", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _v
 _block = _sig("elsa_vit_block", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _block_attn = _sig("elsa_vit_block_attn", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _attention = _sig("elsa_attention", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
+_window_attention = _sig("elsa_window_attention", _i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _i, _i, _vp, _vp, _vp])
 _encoder_scratch = _sig("elsa_vit_encoder_scratch_bytes", _sz, [_i, _i, _i, _i, _bw, _i, _i])
 _encoder = _sig("elsa_vit_encoder", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, ctypes.c_float, _i, _vp, _vp, _sz, _vp, _vp])
 
@@ -426,6 +427,18 @@ def elsa_attention(qkv, tokens, heads, a=None, dev_status=None, stream=None):
         a = torch.empty((rows, dim), dtype=qkv.dtype, device=qkv.device)
     _check(_attention(_ptr(qkv), rows // tokens, tokens, heads, dim, dtype_code(qkv.dtype), _ptr(a), _ptr(dev_status),
                       _stream(stream)))
+    return a
+
+
+def elsa_window_attention(qkv, tokens, heads, bias, mask=None, a=None, dev_status=None, stream=None):
+    """Attention over windows of `tokens` consecutive rows of qkv [rows, 3 dim] with fp32 tables on the scores:
+    bias [heads, tokens, pitch], mask [n_masks, tokens, pitch] or None (window w takes table w % n_masks)."""
+    rows, three_dim = qkv.shape
+    dim = three_dim // 3
+    if a is None:
+        a = torch.empty((rows, dim), dtype=qkv.dtype, device=qkv.device)
+    _check(_window_attention(_ptr(qkv), rows // tokens, tokens, heads, dim, _ptr(bias), bias.shape[-1], _ptr(mask),
+                             0 if mask is None else mask.shape[0], dtype_code(qkv.dtype), _ptr(a), _ptr(dev_status), _stream(stream)))
     return a
 
 

@@ -1216,6 +1216,19 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
     return launch_attention((const uint16_t*)qkv, images, tokens, heads, dim, dtype, (uint16_t*)a, dev_status, (cudaStream_t)stream);
 }
 
+elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int heads, int dim, const float* bias,
+                                  int bias_pitch, const float* mask, int n_masks, elsa_dtype dtype, void* a,
+                                  uint32_t* dev_status, void* stream)
+{
+    if (!qkv || !a || !bias) return fail(ELSA_ERR_NULL, "qkv, a and bias must not be NULL");
+    if (dtype != ELSA_F16 && dtype != ELSA_BF16) return fail(ELSA_ERR_DTYPE, "dtype %d is neither ELSA_F16 nor ELSA_BF16", (int)dtype);
+    if (windows <= 0) return fail(ELSA_ERR_SHAPE, "non-positive windows=%d", windows);
+    if (!aligned16(qkv) || !aligned16(a) || ((uintptr_t)bias & 3u) || ((uintptr_t)mask & 3u))
+        return fail(ELSA_ERR_ALIGN, "qkv and a must be 16-byte aligned, the tables 4-byte aligned");
+    return launch_attention((const uint16_t*)qkv, windows, tokens, heads, dim, dtype, (uint16_t*)a, dev_status, (cudaStream_t)stream,
+                            bias, mask, n_masks, bias_pitch);
+}
+
 elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
                                 const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
                                 uint32_t* dev_status, void* stream)

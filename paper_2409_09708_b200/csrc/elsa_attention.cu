@@ -3,7 +3,10 @@
 //     a[img, :, h] = softmax(q k^T / sqrt d) v      per image and head, over the keys of the same image
 // with q, k, v the head's 64 columns in the three thirds of qkv [images * tokens][3 * dim].
 //
-// Work item = (128 query rows, head, image); tokens <= 256, head dimension 64 (the ViT / DeiT shapes).  Both
+// Work item = (128 query rows, head, image); tokens <= 256, head dimension 64 (the ViT / DeiT shapes) or 32 (Swin).
+// An "image" is whatever set of consecutive rows attends within itself: for Swin, one window of the rolled grid, with
+// an additive fp32 table per head on the scores (relative-position bias) and a second one per window position
+// (the seam mask of shifted windows); the biased form is an instantiation of its own.  Both
 // products run on tcgen05 with everything between them kept on chip:
 //   1. TMA brings the Q tile, all K rows and all V rows of the head into shared memory (128-byte swizzle; a 3-D
 //      tensor map [image][token][column] zero-fills the rows past the image's last token).
@@ -27,15 +30,15 @@
 namespace elsa {
 namespace {
 
-constexpr int kHeadDim = 64;
+constexpr int kMaxHeadDim = 64;
 constexpr int kQRows = 128;          // query rows per item = TMEM lanes
 constexpr int kMaxTokens = 256;
 constexpr int kBufCols = 256;        // tensor-memory columns per item in flight
 constexpr int kTmemCols = 2 * kBufCols;
 constexpr int kGroupWarps = 4;       // softmax warps per group, one per TMEM lane quarter
 constexpr int kThreads = (2 + 2 * kGroupWarps) * 32;
-constexpr int kQBytes = kQRows * kHeadDim * 2;
-constexpr int kKvBytesMax = kMaxTokens * kHeadDim * 2;
+constexpr int kQBytes = kQRows * kMaxHeadDim * 2;          // the shared-memory slots are laid out for head dimension 64
+constexpr int kKvBytesMax = kMaxTokens * kMaxHeadDim * 2;
 constexpr int kStageBytes = kQBytes + 2 * kKvBytesMax;
 constexpr int kSmemBytes = 2 * kStageBytes + 1024 /* alignment */ + 256 /* barriers */;
 
@@ -48,7 +51,24 @@ struct AttnParams {
     int o_col;            // first column of O inside an item's half of tensor memory
     uint32_t idesc_s, idesc_o;
     uint32_t* dev_status;
+    // biased form: scores get bias[head][row][key] + mask[image % n_masks][row][key] (fp32, rows of bias_pitch floats)
+    const float* bias;
+    const float* mask;    // or NULL
+    int n_masks, bias_pitch;
 };
+
+// MN-major tile of rows of 64 bytes (32 16-bit values along N per reduction index) with the 64-byte swizzle: 8
+// reduction rows form a 512-byte group.
+__device__ __forceinline__ uint64_t smem_desc_mn_major_sw64(uint32_t addr, uint32_t block_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(512 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)4 << 61;
+    return d;
+}
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2)
 {
@@ -80,9 +100,12 @@ __device__ __forceinline__ void tmem_st_32x32b_x8(uint32_t taddr, const uint32_t
                  : "memory");
 }
 
-template <bool kBf16>
+template <bool kBf16, int kD, bool kBias>
 __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnParams p)
 {
+    static_assert(kD == 64 || kD == 32, "head dimension");
+    constexpr int kHeadDim = kD;
+    constexpr int kItemQBytes = kQRows * kD * 2;      // bytes TMA delivers for the Q tile; K and V: tk * kD * 2
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = smem_base + 2 * kStageBytes;
@@ -135,7 +158,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
             const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
             if (elected) {
-                mbar_arrive_expect_tx(bar(kQkFull, b), (uint32_t)(kQBytes + p.tk * kHeadDim * 2));
+                mbar_arrive_expect_tx(bar(kQkFull, b), (uint32_t)(kItemQBytes + p.tk * kHeadDim * 2));
                 tma_load_3d(q_smem, &p.map_q, bar(kQkFull, b), head * kHeadDim, mt * kQRows, img);
                 tma_load_3d(q_smem + kQBytes, &p.map_kv, bar(kQkFull, b), p.dim + head * kHeadDim, 0, img);
                 mbar_arrive_expect_tx(bar(kVFull, b), (uint32_t)(p.tk * kHeadDim * 2));
@@ -161,8 +184,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
-                const uint64_t a_desc = smem_desc_k_major_sw128(q_smem);
-                const uint64_t b_desc = smem_desc_k_major_sw128(q_smem + kQBytes);
+                const uint64_t a_desc = kD == 64 ? smem_desc_k_major_sw128(q_smem) : smem_desc_k_major_sw64(q_smem);
+                const uint64_t b_desc = kD == 64 ? smem_desc_k_major_sw128(q_smem + kQBytes) : smem_desc_k_major_sw64(q_smem + kQBytes);
 #pragma unroll
                 for (int k = 0; k < kHeadDim / 16; ++k)
                     umma_f16_if(tmem_u + (uint32_t)(b * kBufCols), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc_s,
@@ -180,10 +203,12 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t t_buf = tmem_u + (uint32_t)(b * kBufCols);
-                const uint64_t v_desc = smem_desc_mn_major_sw128(smem_base + (uint32_t)(b * kStageBytes + kQBytes + kKvBytesMax),
-                                                                 (uint32_t)(p.tk * kHeadDim * 2));
+                const uint32_t v_smem = smem_base + (uint32_t)(b * kStageBytes + kQBytes + kKvBytesMax);
+                const uint64_t v_desc = kD == 64 ? smem_desc_mn_major_sw128(v_smem, (uint32_t)(p.tk * kHeadDim * 2))
+                                                 : smem_desc_mn_major_sw64(v_smem, (uint32_t)(p.tk * kHeadDim * 2));
+                // 16 keys of kD * 2 bytes per MMA
                 for (int k = 0; k < steps; ++k)
-                    umma_f16_ts_if(t_buf + (uint32_t)p.o_col, t_buf + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * 128 >> 4)),
+                    umma_f16_ts_if(t_buf + (uint32_t)p.o_col, t_buf + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * kD * 2 >> 4)),
                                    p.idesc_o, (uint32_t)(k != 0), elected);
                 umma_commit_if(bar(kOFull, b), elected);
                 umma_commit_if(bar(kSmemEmpty, b), elected);   // both products of the item have read its stage
@@ -194,7 +219,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         // ------------------------------------------------ softmax and output: group g takes the items n = g, g + 2, ...
         const int g = (warp - 2) / kGroupWarps;
         const int quarter = warp & 3;                                  // the TMEM lanes this warp may touch
-        const float scale = 0.125f * 1.4426950408889634f;              // log2(e) / sqrt(64)
+        const float scale = (kD == 64 ? 0.125f : 0.17677669529663687f) * 1.4426950408889634f;   // log2(e) / sqrt(kD)
         bool ok = true;
         for (int n = g; ok && n < n_items; n += 2) {
             const uint32_t ph = (uint32_t)((n >> 1) & 1);
@@ -207,6 +232,23 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             if (!ok) break;
             tc_fence_after();
             float sum = 0.f;
+            // biased form: what is exponentiated is s * scale + (bias + mask) * log2(e); the tables' rows of this lane
+            const float* brow = nullptr;
+            const float* mrow = nullptr;
+            if constexpr (kBias) {
+                if (row < p.tokens) {
+                    brow = p.bias + ((size_t)head * p.tokens + row) * (size_t)p.bias_pitch;
+                    if (p.mask != nullptr) mrow = p.mask + ((size_t)(img % p.n_masks) * p.tokens + row) * (size_t)p.bias_pitch;
+                }
+            }
+            auto biased = [&](uint32_t raw, int col) -> float {     // kBias only: the score in the exponent's domain
+                float b = 0.f;
+                if (brow != nullptr && col < p.tokens) {
+                    b = __ldg(brow + col);
+                    if (mrow != nullptr) b += __ldg(mrow + col);
+                }
+                return fmaf(__uint_as_float(raw), scale, b * 1.4426950408889634f);
+            };
             {
                 // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
                 // row maximum from up to 64 columns per round trip, the second pass with the next 32 columns in
@@ -223,7 +265,11 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 #pragma unroll
                     for (int i = 0; i < 2; ++i)
                         if (u0 + i < units) {
-                            if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
+                            if constexpr (kBias) {
+#pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, biased(r[i][j], 32 * (u0 + i) + j));
+                            } else if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
                                 float m0 = m, m1 = -INFINITY;
 #pragma unroll
                                 for (int j = 0; j < 32; j += 2) {
@@ -244,18 +290,22 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+                        if (32 * units + j < p.tokens)
+                            m = fmaxf(m, kBias ? biased(r[j], 32 * units + j) : __uint_as_float(r[j]));
                 }
                 // p = 2^(s * scale - m * scale) for 16 columns starting at col0: eight packed pairs
-                const float m_scaled = m * scale;
+                const float m_scaled = kBias ? m : m * scale;      // the biased maximum is in the exponent's domain already
                 float sum1 = 0.f;
                 auto exp16 = [&](const uint32_t* r, int col0, uint32_t (&w)[8]) {
                     const bool all_real = col0 + 16 <= p.tokens;
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         float e0, e1;
-                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(fmaf(__uint_as_float(r[2 * j]), scale, -m_scaled)));
-                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(fmaf(__uint_as_float(r[2 * j + 1]), scale, -m_scaled)));
+                        const float a0 = kBias ? biased(r[2 * j], col0 + 2 * j) - m_scaled : fmaf(__uint_as_float(r[2 * j]), scale, -m_scaled);
+                        const float a1 = kBias ? biased(r[2 * j + 1], col0 + 2 * j + 1) - m_scaled
+                                               : fmaf(__uint_as_float(r[2 * j + 1]), scale, -m_scaled);
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(a0));
+                        asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(a1));
                         if (!all_real) {                                  // padded keys take no part
                             if (col0 + 2 * j >= p.tokens) e0 = 0.f;
                             if (col0 + 2 * j + 1 >= p.tokens) e1 = 0.f;
@@ -303,9 +353,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             if (!ok) break;
             tc_fence_after();
             const float inv = 1.0f / sum;
-            uint32_t w[4][8];                                          // the row's 64 outputs, packed
+            uint32_t w[kD / 16][8];                                    // the row's kD outputs, packed
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int half = 0; half < kD / 32; ++half) {
                 uint32_t o[2][16];
                 tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 32 * half), o[0]);
                 tmem_ld_32x32b_x16(t_lane + (uint32_t)(p.o_col + 32 * half + 16), o[1]);
@@ -322,7 +372,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             if (row < p.tokens) {
                 uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)img * p.tokens + row) * (size_t)p.dim + head * kHeadDim);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
+                for (int q = 0; q < kD / 16; ++q) {
                     dst[2 * q] = make_uint4(w[q][0], w[q][1], w[q][2], w[q][3]);
                     dst[2 * q + 1] = make_uint4(w[q][4], w[q][5], w[q][6], w[q][7]);
                 }
@@ -337,25 +387,26 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
     }
 }
 
-elsa_status make_map_qkv(CUtensorMap* map, const void* qkv, int images, int tokens, int dim, uint32_t box_rows, const char* what)
+elsa_status make_map_qkv(CUtensorMap* map, const void* qkv, int images, int tokens, int dim, int head_dim, uint32_t box_rows,
+                         const char* what)
 {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return fail(ELSA_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[3] = {(cuuint64_t)(3 * dim), (cuuint64_t)tokens, (cuuint64_t)images};
     cuuint64_t strides[2] = {(cuuint64_t)(3 * dim) * 2, (cuuint64_t)tokens * (cuuint64_t)(3 * dim) * 2};
-    cuuint32_t box[3] = {(cuuint32_t)kHeadDim, box_rows, 1};
+    cuuint32_t box[3] = {(cuuint32_t)head_dim, box_rows, 1};
     cuuint32_t elem[3] = {1, 1, 1};
     CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT16, 3, const_cast<void*>(qkv), dims, strides, box, elem,
-                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, head_dim == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc != CUDA_SUCCESS) return fail(ELSA_ERR_CUDA, "tensor map for %s rejected (CUresult %d)", what, (int)rc);
     return ELSA_OK;
 }
 
-template <bool kBf16>
+template <bool kBf16, int kD, bool kBias>
 elsa_status launch(const AttnParams& p, int images, int heads, cudaStream_t stream, const DeviceInfo& dev)
 {
-    auto kernel = attention_kernel<kBf16>;
+    auto kernel = attention_kernel<kBf16, kD, kBias>;
     static std::atomic<bool> attr_set[64];
     const int slot = dev.device & 63;
     if (!attr_set[slot].load(std::memory_order_acquire)) {
@@ -378,18 +429,23 @@ elsa_status launch(const AttnParams& p, int images, int heads, cudaStream_t stre
 
 bool attention_suits(int tokens, int heads, int dim)
 {
-    return tokens >= 1 && tokens <= kMaxTokens && heads >= 1 && dim == heads * kHeadDim;
+    return tokens >= 1 && tokens <= kMaxTokens && heads >= 1 && (dim == heads * 64 || dim == heads * 32);
 }
 
 elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype,
-                             uint16_t* out, uint32_t* dev_status, cudaStream_t stream)
+                             uint16_t* out, uint32_t* dev_status, cudaStream_t stream, const float* bias, const float* mask,
+                             int n_masks, int bias_pitch)
 {
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     if (!attention_suits(tokens, heads, dim))
-        return fail(ELSA_ERR_SHAPE, "attention needs 1..%d tokens per image and a head dimension of %d (tokens=%d, heads=%d, dim=%d)",
-                    kMaxTokens, kHeadDim, tokens, heads, dim);
+        return fail(ELSA_ERR_SHAPE, "attention needs 1..%d tokens per image and a head dimension of 32 or 64 (tokens=%d, heads=%d, dim=%d)",
+                    kMaxTokens, tokens, heads, dim);
+    const int head_dim = dim / heads;
+    if (bias == nullptr && mask != nullptr) return fail(ELSA_ERR_NULL, "a mask table needs a bias table");
+    if (bias != nullptr && (bias_pitch < tokens || (mask != nullptr && n_masks < 1)))
+        return fail(ELSA_ERR_SHAPE, "bias_pitch=%d must be at least tokens=%d, n_masks=%d at least 1", bias_pitch, tokens, n_masks);
     if ((long long)images * heads * ((tokens + kQRows - 1) / kQRows) > 0x7fffffffLL)
         return fail(ELSA_ERR_SHAPE, "images * heads does not fit an int");
     AttnParams p;
@@ -400,15 +456,22 @@ elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int he
     p.m_tiles = (tokens + kQRows - 1) / kQRows;
     p.heads = heads;
     p.items = images * heads * p.m_tiles;
-    // O over the part of S that P does not cover (P: tk / 2 columns from 0); small images: right after S
+    // O (head_dim columns) over the part of S that P does not cover (P: tk / 2 columns from 0); small images: right after S
     p.o_col = p.tk >= 128 ? (p.tk / 2 + 31) / 32 * 32 : p.tk;
     const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
     p.idesc_s = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.tk >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
-    p.idesc_o = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((uint32_t)(kHeadDim >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
+    p.idesc_o = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((uint32_t)(head_dim >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
     p.dev_status = dev_status;
-    if ((st = make_map_qkv(&p.map_q, qkv, images, tokens, dim, kQRows, "q")) != ELSA_OK) return st;
-    if ((st = make_map_qkv(&p.map_kv, qkv, images, tokens, dim, (uint32_t)p.tk, "k, v")) != ELSA_OK) return st;
-    return dtype == ELSA_BF16 ? launch<true>(p, images, heads, stream, dev) : launch<false>(p, images, heads, stream, dev);
+    p.bias = bias; p.mask = mask; p.n_masks = n_masks > 0 ? n_masks : 1; p.bias_pitch = bias_pitch;
+    if ((st = make_map_qkv(&p.map_q, qkv, images, tokens, dim, head_dim, kQRows, "q")) != ELSA_OK) return st;
+    if ((st = make_map_qkv(&p.map_kv, qkv, images, tokens, dim, head_dim, (uint32_t)p.tk, "k, v")) != ELSA_OK) return st;
+    const bool bf = dtype == ELSA_BF16, biased = bias != nullptr;
+    if (head_dim == 64) {
+        if (biased) return bf ? launch<true, 64, true>(p, images, heads, stream, dev) : launch<false, 64, true>(p, images, heads, stream, dev);
+        return bf ? launch<true, 64, false>(p, images, heads, stream, dev) : launch<false, 64, false>(p, images, heads, stream, dev);
+    }
+    if (biased) return bf ? launch<true, 32, true>(p, images, heads, stream, dev) : launch<false, 32, true>(p, images, heads, stream, dev);
+    return bf ? launch<true, 32, false>(p, images, heads, stream, dev) : launch<false, 32, false>(p, images, heads, stream, dev);
 }
 
 }  // namespace elsa

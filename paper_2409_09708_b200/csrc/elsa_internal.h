@@ -172,11 +172,13 @@ elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype
 // dst[r][0 .. cols) = src[r][col0 .. col0 + cols); src rows of src_ld values; all multiples of 8.
 elsa_status launch_copy_columns(const uint16_t* src, uint16_t* dst, int rows, int src_ld, int col0, int cols,
                                 cudaStream_t stream);
-// Multi-head self-attention a = softmax(q k^T / sqrt d) v per image and head on tcgen05 (tokens <= 256, head
-// dimension 64): qkv [images * tokens][3 * dim] -> out [images * tokens][dim].
+// Multi-head self-attention a = softmax(q k^T / sqrt d + bias + mask) v per image and head on tcgen05 (tokens <= 256,
+// head dimension 64 or 32): qkv [images * tokens][3 * dim] -> out [images * tokens][dim].  bias (or NULL):
+// fp32 [heads][tokens][bias_pitch]; mask (or NULL): fp32 [n_masks][tokens][bias_pitch], image i takes table i % n_masks.
 bool attention_suits(int tokens, int heads, int dim);
 elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int heads, int dim, elsa_dtype dtype,
-                             uint16_t* out, uint32_t* dev_status, cudaStream_t stream);
+                             uint16_t* out, uint32_t* dev_status, cudaStream_t stream, const float* bias = nullptr,
+                             const float* mask = nullptr, int n_masks = 0, int bias_pitch = 0);
 // Operand forms of the backward pass.  transpose16: src [R][C] -> dst [C][Rp] with the tail R..Rp zero (C, Rp
 // multiples of 8).  colsum: db [C] = column sums of src [R][C], through ceil(R / 512) * C floats of scratch.
 elsa_status launch_transpose16(const uint16_t* src, uint16_t* dst, int R, int C, int Rp, cudaStream_t stream);

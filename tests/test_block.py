@@ -410,3 +410,35 @@ def test_encoder_validates_every_block_before_launching(lib):
         lib.elsa_vit_encoder(x.cuda(), 20, 1, 128, lib.make_encoder_table(blocks))
     assert e.value.status == 1 and "block 1" in str(e.value)
     assert lib.elsa_launch_count() == before
+
+
+WINDOW_CASES = [(2, 14, 14, 7, 0, 2, 32), (2, 14, 14, 7, 3, 2, 32), (1, 28, 14, 7, 3, 4, 32), (2, 14, 14, 7, 3, 1, 64),
+                (3, 8, 8, 4, 2, 3, 32), (1, 16, 16, 16, 5, 2, 32)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
+@pytest.mark.parametrize("case", WINDOW_CASES, ids=["%dx%dx%d_w%d_s%d_h%d_d%d" % c for c in WINDOW_CASES])
+def test_window_attention_matches_oracle(lib, case, dtype):
+    B, H, W, ws, shift, heads, d = case
+    dim, T = heads * d, ws * ws
+    qkv = synth.randn((B * H * W, 3 * dim), 23, 1.0, dtype)
+    rel_bias = np.random.default_rng(7).standard_normal((heads, T, T)) * 0.5
+    # the rows in window order: what the block's first LayerNorm writes
+    order = bo.window_order(H, W, ws, shift)
+    perm = np.concatenate([b * H * W + order.ravel() for b in range(B)])
+    mask = bo.shift_mask(H, W, ws, shift) if shift else None
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    a_win = lib.elsa_window_attention(qkv[perm].contiguous().cuda(), T, heads,
+                                      torch.from_numpy(rel_bias).float().cuda(),
+                                      None if mask is None else torch.from_numpy(mask).float().cuda(), dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    q64 = qkv.double().numpy()
+    ref = bo._round16(bo.window_attention(q64, H, W, ws, shift, heads, rel_bias), dtype)[perm]
+    got = a_win.double().cpu().numpy()
+    assert np.isfinite(got).all()
+    tol = attention_tolerance(ref, q64[perm][:, 2 * dim:], T, heads, dtype)
+    err = np.abs(got - ref)
+    worst = (err - tol).argmax()
+    assert (err <= tol).all(), "error %g at tolerance %g" % (err.flat[worst], tol.flat[worst])
