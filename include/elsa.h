@@ -443,6 +443,28 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
 elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int heads, int dim, const float* bias,
                                   int bias_pitch, const float* mask, int n_masks, elsa_dtype dtype, void* a,
                                   uint32_t* dev_status, void* stream);
+/*
+ * The Swin form of the block (Table 1 and Fig. 10 of the paper evaluate Swin-S / Swin-B): tokens are an H x W grid per
+ * image, attention runs inside windows of window x window tokens of the grid rolled by -shift (shift = 0 or, in every
+ * second block, window / 2), with the relative-position bias and, for shift > 0, the seam mask on the scores.  The
+ * first LayerNorm writes its rows in window order, qkv, attention and proj work on windows as runs of rows, and the
+ * residual add brings proj's rows back to the grid's order.  Regions X1, QKV, A and T of scratch are therefore in
+ * window order.  rel_bias: fp32 [heads][window^2][bias_pitch], device; mask: fp32 [(H / window) (W / window)]
+ * [window^2][bias_pitch], device, as elsa_swin_mask writes it (required iff shift > 0).  dim = 32 or 64 times heads.
+ * Patch merging between stages is a separate linear and not part of this call.
+ */
+typedef struct {
+    int H, W, window, shift;
+    const float* rel_bias;
+    const float* mask;
+    int bias_pitch;
+} elsa_swin_attn;
+/* HOST arithmetic: fills mask [windows of an image][window^2][pitch] (host memory) with 0 / -100 and returns the number
+ * of windows, -1 on invalid arguments (needs 0 < shift < window). */
+int elsa_swin_mask(int H, int W, int window, int shift, int pitch, float* mask);
+elsa_status elsa_swin_block(const void* x, int images, int heads, int dim, int mlp_dim, const elsa_block_weights* w,
+                            const elsa_swin_attn* attn, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                            uint32_t* dev_status, void* stream);
 /* The whole block with elsa_attention between the halves; rows = images * tokens. */
 elsa_status elsa_vit_block_attn(const void* x, int images, int tokens, int heads, int dim, int mlp_dim,
                                 const elsa_block_weights* w, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,

@@ -126,6 +126,12 @@ _block = _sig("elsa_vit_block", _i, [_vp, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _v
 _block_attn = _sig("elsa_vit_block_attn", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, _sz, _vp, _vp])
 _attention = _sig("elsa_attention", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 _window_attention = _sig("elsa_window_attention", _i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _i, _i, _vp, _vp, _vp])
+class ElsaSwinAttn(ctypes.Structure):
+    _fields_ = [("H", _i), ("W", _i), ("window", _i), ("shift", _i), ("rel_bias", _vp), ("mask", _vp), ("bias_pitch", _i)]
+
+
+_swin_mask = _sig("elsa_swin_mask", _i, [_i, _i, _i, _i, _i, ctypes.POINTER(ctypes.c_float)])
+_swin_block = _sig("elsa_swin_block", _i, [_vp, _i, _i, _i, _i, _bw, ctypes.POINTER(ElsaSwinAttn), _i, _vp, _vp, _sz, _vp, _vp])
 _encoder_scratch = _sig("elsa_vit_encoder_scratch_bytes", _sz, [_i, _i, _i, _i, _bw, _i, _i])
 _encoder = _sig("elsa_vit_encoder", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, ctypes.c_float, _i, _vp, _vp, _sz, _vp, _vp])
 
@@ -440,6 +446,33 @@ def elsa_window_attention(qkv, tokens, heads, bias, mask=None, a=None, dev_statu
     _check(_window_attention(_ptr(qkv), rows // tokens, tokens, heads, dim, _ptr(bias), bias.shape[-1], _ptr(mask),
                              0 if mask is None else mask.shape[0], dtype_code(qkv.dtype), _ptr(a), _ptr(dev_status), _stream(stream)))
     return a
+
+
+def elsa_swin_mask(H, W, window, shift, pitch=None):
+    """The seam mask of shifted windows as a host fp32 tensor [windows, window^2, pitch]."""
+    T = window * window
+    pitch = pitch or T
+    n = (H // window) * (W // window)
+    out = torch.empty((n, T, pitch), dtype=torch.float32)
+    got = _swin_mask(H, W, window, shift, pitch, ctypes.cast(out.data_ptr(), ctypes.POINTER(ctypes.c_float)))
+    if got != n:
+        raise ValueError("elsa_swin_mask rejected its arguments")
+    return out
+
+
+def elsa_swin_block(x, H, W, window, shift, heads, mlp_dim, weights, rel_bias, mask=None, y=None, scratch=None,
+                    dev_status=None, stream=None):
+    """One Swin block over x [images * H * W, dim]; rel_bias [heads, T, pitch] and mask [windows, T, pitch] fp32 on the device."""
+    rows, dim = x.shape
+    code = dtype_code(x.dtype)
+    if scratch is None:
+        scratch = alloc_workspace(elsa_vit_block_scratch_bytes(rows, dim, mlp_dim, weights, code)[0], x.device)
+    if y is None:
+        y = torch.empty_like(x)
+    attn = ElsaSwinAttn(H, W, window, shift, _ptr(rel_bias), _ptr(mask), rel_bias.shape[-1])
+    _check(_swin_block(_ptr(x), rows // (H * W), heads, dim, mlp_dim, ctypes.byref(weights), ctypes.byref(attn), code, _ptr(y),
+                       _ptr(scratch), scratch.numel(), _ptr(dev_status), _stream(stream)))
+    return y, scratch
 
 
 def elsa_vit_block(x, mlp_dim, weights, y=None, scratch=None, dev_status=None, stream=None, phase="both", tokens=None,

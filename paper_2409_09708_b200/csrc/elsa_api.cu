@@ -965,14 +965,17 @@ struct BlockCarry {
 // carry (or NULL) + x_sum: the block's input is carry->t + carry->r, written to x_sum; otherwise it is x.
 elsa_status block_qkv(const uint16_t* x, int rows, int dim, const elsa_block_weights* w, elsa_dtype dtype,
                       uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4], uint32_t* dev_status,
-                      cudaStream_t stream, const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr)
+                      cudaStream_t stream, const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr,
+                      const elsa_swin_attn* swin = nullptr)
 {
     uint16_t* x1 = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_X1]);
     uint16_t* qkv = (uint16_t*)(scratch + plan.off[ELSA_BLOCK_QKV]);
     const bool add = carry != nullptr && carry->t != nullptr;
+    RowMap out_map = {0, 0, 0, 0, 0, 1};      // Swin: x1 is written in window order, so that windows are runs of rows
+    if (swin) { out_map.H = swin->H; out_map.W = swin->W; out_map.ws = swin->window; out_map.shift = swin->shift; }
     elsa_status st = launch_layer_norm(add ? carry->t : x, add ? carry->r : nullptr, add ? x_sum : nullptr,
                                        (const uint16_t*)w->ln1_gain, (const uint16_t*)w->ln1_bias,
-                                       x1, rows, dim, w->eps, dtype, stream);
+                                       x1, rows, dim, w->eps, dtype, stream, swin ? &out_map : nullptr);
     if (st != ELSA_OK) return st;
     bool left = false;
     return block_linear(lin[0], x1, rows, dtype, qkv, 0, nullptr, nullptr, &left, dev_status, stream);
@@ -980,7 +983,8 @@ elsa_status block_qkv(const uint16_t* x, int rows, int dim, const elsa_block_wei
 
 elsa_status block_rest(const uint16_t* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                        uint16_t* y, uint8_t* scratch, const BlockPlan& plan, BlockLinear (&lin)[4],
-                       uint32_t* dev_status, cudaStream_t stream, BlockCarry* defer = nullptr)
+                       uint32_t* dev_status, cudaStream_t stream, BlockCarry* defer = nullptr,
+                       const elsa_swin_attn* swin = nullptr)
 {
     (void)mlp_dim;
     const uint16_t* a = (const uint16_t*)(scratch + plan.off[ELSA_BLOCK_A]);
@@ -991,11 +995,18 @@ elsa_status block_rest(const uint16_t* x, int rows, int dim, int mlp_dim, const 
     const uint16_t* g2 = (const uint16_t*)w->ln2_gain;
     const uint16_t* b2 = (const uint16_t*)w->ln2_bias;
     bool left = false;
-    elsa_status st = block_linear(lin[1], a, rows, dtype, x2, 0, x, t, &left, dev_status, stream);
-    if (st != ELSA_OK) return st;
-    // x2 = x + proj(a) and x3 = LayerNorm2(x2): one pass where the residual is still to be added
-    st = left ? launch_layer_norm(t, x, x2, g2, b2, x3, rows, dim, w->eps, dtype, stream)
-              : launch_layer_norm(x2, nullptr, nullptr, g2, b2, x3, rows, dim, w->eps, dtype, stream);
+    elsa_status st;
+    if (swin) {
+        // proj runs on rows in window order; the add that follows reads them back in the grid's order
+        RowMap in_map = {swin->H, swin->W, swin->window, swin->shift, 1, 0};
+        if ((st = block_linear(lin[1], a, rows, dtype, t, 0, nullptr, nullptr, &left, dev_status, stream)) != ELSA_OK) return st;
+        st = launch_layer_norm(t, x, x2, g2, b2, x3, rows, dim, w->eps, dtype, stream, &in_map);
+    } else {
+        if ((st = block_linear(lin[1], a, rows, dtype, x2, 0, x, t, &left, dev_status, stream)) != ELSA_OK) return st;
+        // x2 = x + proj(a) and x3 = LayerNorm2(x2): one pass where the residual is still to be added
+        st = left ? launch_layer_norm(t, x, x2, g2, b2, x3, rows, dim, w->eps, dtype, stream)
+                  : launch_layer_norm(x2, nullptr, nullptr, g2, b2, x3, rows, dim, w->eps, dtype, stream);
+    }
     if (st != ELSA_OK) return st;
     if ((st = block_linear(lin[2], x3, rows, dtype, h, 1, nullptr, nullptr, &left, dev_status, stream)) != ELSA_OK) return st;
     if ((st = block_linear(lin[3], h, rows, dtype, y, 0, x2, t, &left, dev_status, stream)) != ELSA_OK) return st;
@@ -1059,7 +1070,8 @@ namespace {
 // The whole block; tokens == 0 runs the stand-in a = V, otherwise the attention kernel over images of `tokens` rows.
 elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_block_weights* w, elsa_dtype dtype,
                       void* y, void* scratch, size_t scratch_bytes, uint32_t* dev_status, void* stream_, int tokens, int heads,
-                      const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr, BlockCarry* defer = nullptr)
+                      const BlockCarry* carry = nullptr, uint16_t* x_sum = nullptr, BlockCarry* defer = nullptr,
+                      const elsa_swin_attn* swin = nullptr)
 {
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
@@ -1088,10 +1100,16 @@ elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_
         if (e != cudaSuccess) return fail(ELSA_ERR_CUDA, "joining the image stream: %s", cudaGetErrorString(e));
     }
     uint8_t* s8 = (uint8_t*)scratch;
-    if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream, carry, x_sum)) != ELSA_OK)
+    if ((st = block_qkv((const uint16_t*)x, rows, dim, w, dtype, s8, plan, lin, dev_status, stream, carry, x_sum, swin)) != ELSA_OK)
         return st;
     if (carry != nullptr && carry->t != nullptr) x = x_sum;      // the block's input, as just stored
-    if (tokens == 0) {
+    if (swin) {
+        const int T = swin->window * swin->window;
+        st = launch_attention((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), rows / T, T, heads, dim, dtype,
+                              (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]), dev_status, stream, swin->rel_bias,
+                              swin->shift > 0 ? swin->mask : nullptr, (swin->H / swin->window) * (swin->W / swin->window),
+                              swin->bias_pitch);
+    } else if (tokens == 0) {
         // the stated stand-in for attention: a = V
         st = launch_copy_columns((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]),
                                  rows, 3 * dim, 2 * dim, dim, stream);
@@ -1100,7 +1118,7 @@ elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_
                               (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]), dev_status, stream);
     }
     if (st != ELSA_OK) return st;
-    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream, defer);
+    return block_rest((const uint16_t*)x, rows, dim, mlp_dim, w, dtype, (uint16_t*)y, s8, plan, lin, dev_status, stream, defer, swin);
 }
 
 struct EncoderPlan {
@@ -1214,6 +1232,52 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
     if (images <= 0) return fail(ELSA_ERR_SHAPE, "non-positive images=%d", images);
     if (!aligned16(qkv) || !aligned16(a)) return fail(ELSA_ERR_ALIGN, "qkv and a must be 16-byte aligned");
     return launch_attention((const uint16_t*)qkv, images, tokens, heads, dim, dtype, (uint16_t*)a, dev_status, (cudaStream_t)stream);
+}
+
+int elsa_swin_mask(int H, int W, int window, int shift, int pitch, float* mask)
+{
+    if (H <= 0 || W <= 0 || window <= 0 || H % window != 0 || W % window != 0 || shift <= 0 || shift >= window ||
+        pitch < window * window || !mask)
+        return -1;
+    const int T = window * window, nww = W / window;
+    // region of a position of the rolled grid: the bands [0, n - window), [n - window, n - shift), [n - shift, n) of each axis
+    auto band = [&](int v, int n) { return v < n - window ? 0 : v < n - shift ? 1 : 2; };
+    for (int wi = 0; wi < H / window; ++wi)
+        for (int wj = 0; wj < nww; ++wj) {
+            float* m = mask + (size_t)(wi * nww + wj) * T * pitch;
+            for (int p = 0; p < T; ++p) {
+                const int rp = 3 * band(wi * window + p / window, H) + band(wj * window + p % window, W);
+                for (int q = 0; q < pitch; ++q) {
+                    float v = 0.f;
+                    if (q < T) {
+                        const int rq = 3 * band(wi * window + q / window, H) + band(wj * window + q % window, W);
+                        v = rp != rq ? -100.f : 0.f;
+                    }
+                    m[(size_t)p * pitch + q] = v;
+                }
+            }
+        }
+    return (H / window) * nww;
+}
+
+elsa_status elsa_swin_block(const void* x, int images, int heads, int dim, int mlp_dim, const elsa_block_weights* w,
+                            const elsa_swin_attn* attn, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
+                            uint32_t* dev_status, void* stream)
+{
+    if (!attn) return fail(ELSA_ERR_NULL, "attn must not be NULL");
+    if (images <= 0 || attn->H <= 0 || attn->W <= 0 || attn->window <= 0 || attn->H % attn->window != 0 ||
+        attn->W % attn->window != 0 || attn->shift < 0 || attn->shift >= attn->window)
+        return fail(ELSA_ERR_SHAPE, "windows of %d do not tile a %d x %d grid, or shift=%d is outside [0, window)", attn->window,
+                    attn->H, attn->W, attn->shift);
+    const int T = attn->window * attn->window;
+    if (!attention_suits(T, heads, dim))
+        return fail(ELSA_ERR_SHAPE, "window attention needs at most 256 tokens per window and dim = 32 or 64 times heads "
+                    "(window=%d, heads=%d, dim=%d)", attn->window, heads, dim);
+    if (!attn->rel_bias || (attn->shift > 0 && !attn->mask)) return fail(ELSA_ERR_NULL, "rel_bias (and mask when shift > 0) must not be NULL");
+    if (attn->bias_pitch < T) return fail(ELSA_ERR_SHAPE, "bias_pitch=%d is below the %d tokens of a window", attn->bias_pitch, T);
+    if ((long long)images * attn->H * attn->W > 0x7fffffffLL) return fail(ELSA_ERR_SHAPE, "images * H * W does not fit an int");
+    return run_block(x, images * attn->H * attn->W, dim, mlp_dim, w, dtype, y, scratch, scratch_bytes, dev_status, stream, T, heads,
+                     nullptr, nullptr, nullptr, attn);
 }
 
 elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int heads, int dim, const float* bias,

@@ -74,14 +74,28 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
-// One warp per row.  kAdd: the row is S = round16(A + R), written to S (which may be A's or R's own buffer:
+// Where a row of the token grid goes in window order (Swin): the H x W grid of an image rolled by -shift along both
+// axes and cut into ws x ws windows, windows row-major, tokens row-major inside a window.  H == 0: identity.
+__device__ __forceinline__ int window_row(const RowMap& m, int row)
+{
+    if (m.H == 0) return row;
+    const int hw = m.H * m.W;
+    const int b = row / hw, t = row - b * hw;
+    const int i = t / m.W, j = t - i * m.W;
+    const int ir = (i - m.shift + m.H) % m.H, jr = (j - m.shift + m.W) % m.W;      // position in the rolled grid
+    const int win = (ir / m.ws) * (m.W / m.ws) + jr / m.ws;
+    return b * hw + win * m.ws * m.ws + (ir % m.ws) * m.ws + jr % m.ws;
+}
+
+// One warp per row.  map.on_input: A's row r is read at window_row(r) (a tensor in window order brought back to the
+// grid's order); map.on_output: Yn's row r is written at window_row(r).  kAdd: the row is S = round16(A + R), written to S (which may be A's or R's own buffer:
 // each lane reads its vectors of a row before it writes them).  The statistics are those of the stored 16-bit
 // row (for kAdd: of S as rounded), mean first, then the biased variance about it; eps sits inside the root.
 // Yn = round16((s - mean) / sqrt(var + eps) * gain + beta), or no normalised output when Yn is NULL.
 template <bool kBf16, bool kAdd>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* __restrict__ gain,
-                  const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, int dim, float eps)
+                  const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, int dim, float eps, const RowMap map)
 {
     pdl_wait_for_predecessors();
     pdl_release_successors();
@@ -89,7 +103,8 @@ layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint1
     const int vecs = dim >> 3;
     const float inv_dim = 1.0f / (float)dim;
     for (int row = blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); row < rows; row += gridDim.x * kWarpsPerBlock) {
-        const uint4* a4 = reinterpret_cast<const uint4*>(A + (size_t)row * (size_t)dim);
+        const int mapped = window_row(map, row);
+        const uint4* a4 = reinterpret_cast<const uint4*>(A + (size_t)(map.on_input ? mapped : row) * (size_t)dim);
         const uint4* r4 = kAdd ? reinterpret_cast<const uint4*>(R + (size_t)row * (size_t)dim) : nullptr;
         uint4* s4 = kAdd ? reinterpret_cast<uint4*>(S + (size_t)row * (size_t)dim) : nullptr;
         uint4 cache[kCacheVecs];
@@ -147,7 +162,7 @@ layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint1
             for (int e = 0; e < 8; ++e) sq += (f[e] - mean) * (f[e] - mean);
         }
         const float rstd = 1.0f / sqrtf(warp_sum(sq) * inv_dim + eps);
-        uint4* y4 = reinterpret_cast<uint4*>(Yn + (size_t)row * (size_t)dim);
+        uint4* y4 = reinterpret_cast<uint4*>(Yn + (size_t)(map.on_output ? mapped : row) * (size_t)dim);
         auto emit = [&](int v, const uint4& u) {
             float f[8], g[8], b[8];
             unpack8<kBf16>(u, f);
@@ -209,8 +224,10 @@ unsigned streaming_grid(long long work_items, int per_block, const DeviceInfo& d
 
 elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* gain,
                               const uint16_t* beta, uint16_t* Yn, int rows, int dim, float eps, elsa_dtype dtype,
-                              cudaStream_t stream)
+                              cudaStream_t stream, const RowMap* row_map)
 {
+    RowMap map = {0, 0, 0, 0, 0, 0};
+    if (row_map != nullptr) map = *row_map;
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
@@ -220,11 +237,11 @@ elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S,
     const bool add = R != nullptr;
     ProfileScope scope(ELSA_KERNEL_BLOCK_ROWWISE, stream);
     if (dtype == ELSA_BF16) {
-        if (add) launch_pdl(layer_norm_kernel<true, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
-        else launch_pdl(layer_norm_kernel<true, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+        if (add) launch_pdl(layer_norm_kernel<true, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);
+        else launch_pdl(layer_norm_kernel<true, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);
     } else {
-        if (add) launch_pdl(layer_norm_kernel<false, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
-        else launch_pdl(layer_norm_kernel<false, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps);
+        if (add) launch_pdl(layer_norm_kernel<false, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);
+        else launch_pdl(layer_norm_kernel<false, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);
     }
     return launched(add ? "residual_add_layer_norm" : "layer_norm");
 }

@@ -164,9 +164,15 @@ elsa_status launch_linear_tc_sparse_st(const uint16_t* X, int rows, const uint16
                                        void* workspace, uint32_t* dev_status, cudaStream_t stream);
 // Row-wise and elementwise kernels of the chained block (16-bit tensors, fp32 arithmetic, one rounding).
 // R == NULL: Yn = LayerNorm(A).  R != NULL: S = A + R, and Yn = LayerNorm(S) unless Yn is NULL.  dim % 8 == 0.
+// row_map (or NULL): Swin's window order of the token rows (grid H x W, windows of ws x ws, roll by shift), applied
+// to where A is read (on_input) or where Yn is written (on_output).
+struct RowMap {
+    int H, W, ws, shift;
+    int on_input, on_output;
+};
 elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* gain,
                               const uint16_t* beta, uint16_t* Yn, int rows, int dim, float eps, elsa_dtype dtype,
-                              cudaStream_t stream);
+                              cudaStream_t stream, const RowMap* row_map = nullptr);
 // Y = act(Y) over `count` values (count % 8 == 0); act as in the GEMM epilogues.
 elsa_status launch_act_inplace(uint16_t* Y, long long count, int act, elsa_dtype dtype, cudaStream_t stream);
 // dst[r][0 .. cols) = src[r][col0 .. col0 + cols); src rows of src_ld values; all multiples of 8.

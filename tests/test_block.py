@@ -152,6 +152,13 @@ def check_rows(got, x, p, dtype, rows_idx, attn=None):
     }
     if attn is None:
         assert np.array_equal(bits(got["a"]), bits(got["qkv"][:, 2 * dim:3 * dim]))  # the stand-in copies V through
+    elif isinstance(attn, dict):                                                      # Swin's windows
+        ref = r16(bo.window_attention(g["qkv"], attn["H"], attn["W"], attn["ws"], attn["shift"], attn["heads"], attn["rel_bias"]))
+        u = 2.0 ** -7 if dtype == torch.bfloat16 else 2.0 ** -10
+        tol = u * np.abs(ref) + 0.5 * u * np.abs(g["qkv"][:, 2 * dim:]).max() + 1e-5
+        err = np.abs(g["a"] - ref)
+        worst = (err - tol).argmax()
+        assert (err <= tol).all(), "stage a: error %g at tolerance %g" % (err.flat[worst], tol.flat[worst])
     else:
         ref = r16(bo.attention(g["qkv"], *attn))
         tol = attention_tolerance(ref, g["qkv"][:, 2 * dim:], attn[0], attn[1], dtype)
@@ -164,8 +171,13 @@ def check_rows(got, x, p, dtype, rows_idx, attn=None):
         worst = (err - tol).argmax()
         assert (err <= tol).all(), "stage %s: error %g at tolerance %g" % (s, err.flat[worst], tol.flat[worst])
     # the whole chain from x alone
-    chain = bo.block_forward(bits(x), p, code, eps=1e-6, **({} if attn is None else
-                                                            dict(attn="softmax", tokens=attn[0], heads=attn[1])))
+    if attn is None:
+        how = {}
+    elif isinstance(attn, dict):
+        how = dict(attn="window", heads=attn["heads"], window=attn)
+    else:
+        how = dict(attn="softmax", tokens=attn[0], heads=attn[1])
+    chain = bo.block_forward(bits(x), p, code, eps=1e-6, **how)
     for s in STAGES:
         mag = chain["x2"] - xs if s == "x2" else chain["y"] - chain["x2"] if s == "y" else 1.13 * fc1 if s == "h" else None
         err = np.abs(g[s] - chain[s])
@@ -442,3 +454,56 @@ def test_window_attention_matches_oracle(lib, case, dtype):
     err = np.abs(got - ref)
     worst = (err - tol).argmax()
     assert (err <= tol).all(), "error %g at tolerance %g" % (err.flat[worst], tol.flat[worst])
+
+
+def test_swin_mask_is_the_oracles():
+    from paper_2409_09708_b200 import build
+    build.build()
+    from paper_2409_09708_b200 import binding as lib
+    for H, W, ws, shift in [(14, 14, 7, 3), (6, 9, 3, 1), (28, 14, 7, 3), (8, 8, 4, 2)]:
+        got = lib.elsa_swin_mask(H, W, ws, shift).numpy()
+        assert np.array_equal(got, bo.shift_mask(H, W, ws, shift).astype(np.float32))
+        padded = lib.elsa_swin_mask(H, W, ws, shift, pitch=ws * ws + 7).numpy()
+        assert np.array_equal(padded[:, :, :ws * ws], got) and (padded[:, :, ws * ws:] == 0).all()
+
+
+SWIN_CASES = [(2, 14, 14, 7, 0, 2, 32), (2, 14, 14, 7, 3, 2, 32), (1, 28, 28, 7, 3, 4, 32), (2, 14, 14, 7, 3, 1, 64)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
+@pytest.mark.parametrize("case", SWIN_CASES, ids=["%dx%dx%d_w%d_s%d_h%d_d%d" % c for c in SWIN_CASES])
+def test_swin_block_matches_oracle(lib, case, dtype):
+    B, H, W, ws, shift, heads, d = case
+    dim, T, mlp = heads * d, ws * ws, 4 * heads * d
+    rows = B * H * W
+    host, p = make_params(dim, mlp, MIXED_LEVELS, dtype, 3100)
+    x = synth.randn((rows, dim), 14, 1.0, dtype)
+    rel_bias = np.random.default_rng(9).standard_normal((heads, T, T)) * 0.5
+    dev = {k: v.cuda() for k, v in host.items()}
+    lin = {}
+    for name in NAMES:
+        N, M = MIXED_LEVELS[name]
+        vals, idx = lib.elsa_nm_compress(dev["W_" + name], N, M)
+        lin[name] = (vals, idx, dev["b_" + name], N, M)
+    w, keep = lib.make_block_weights(dev["ln1_g"], dev["ln1_b"], dev["ln2_g"], dev["ln2_b"], lin, eps=1e-6)
+    code = lib.dtype_code(dtype)
+    total, off = lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, code)
+    scratch = torch.zeros(total, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mask = lib.elsa_swin_mask(H, W, ws, shift).cuda() if shift else None
+    y, _ = lib.elsa_swin_block(x.cuda(), H, W, ws, shift, heads, mlp, w, torch.from_numpy(rel_bias).float().cuda(), mask,
+                               scratch=scratch, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    cols = {"x1": dim, "qkv": 3 * dim, "a": dim, "x2": dim, "x3": dim, "h": mlp}
+    got = {s: lib.block_region(scratch, off, s, rows, cols[s], dtype).cpu() for s in cols}
+    got["y"] = y.cpu()
+    # x1, qkv and a are stored in window order: bring them back to the grid's order for the comparison
+    order = bo.window_order(H, W, ws, shift)
+    perm = torch.from_numpy(np.concatenate([b * H * W + order.ravel() for b in range(B)]))
+    for s in ("x1", "qkv", "a"):
+        back = torch.empty_like(got[s])
+        back[perm] = got[s]
+        got[s] = back
+    check_rows(got, x, p, dtype, np.arange(rows), attn=dict(H=H, W=W, ws=ws, shift=shift, heads=heads, rel_bias=rel_bias))
