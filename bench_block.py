@@ -3,6 +3,7 @@ with the levels the stack workload gives its four linears, chained (a block's y 
 
     python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
     python bench_block.py --compare          # dense 4:4 against N:4 configurations at the paper's operating points
+    python bench_block.py --swin             # the 24 blocks of Swin-B at batch 128, stage by stage
 
 Two timings: with the library's multi-head self-attention (elsa_vit_encoder: the encoder blocks of DeiT-B as
 they run, without patch embedding, final norm and classifier head), and with the stand-in a = V in its place (the linear and
@@ -127,6 +128,85 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     return rec
 
 
+def run_swin(batch=128, reps=5):
+    """The 24 blocks of Swin-B (elsa_swin_block), chained inside each stage, with the levels of the Swin-B stack
+    workload; window 7, every second block shifted by 3 (none in the last stage, whose grid is one window).  Patch
+    embedding, the patch-merging linears between the stages, final norm and head are not part of it: each stage
+    starts from a seeded input of its own shape."""
+    import bench
+    peaks, peaks_kind = bench.load_peaks()
+    hbm = peaks["hbm_gbs"] * 1e9
+    dtype = torch.bfloat16
+    layers = synth.swin_b_stack(batch)
+    grids = (56, 28, 14, 7)
+    heads_of = (4, 8, 16, 32)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stages, li = [], 0
+    for st, (dim, depth, g) in enumerate(zip(synth.SWIN_B_DIMS, synth.SWIN_B_DEPTHS, grids)):
+        rows, heads, mlp, T = batch * g * g, heads_of[st], 4 * dim, 49
+        blocks = []
+        for b in range(depth):
+            lin = {}
+            for l in layers[li:li + 4]:
+                _, W, bias = synth.layer_tensors(l, dtype, "cuda", with_x=False)
+                vals, idx = lib.elsa_nm_compress(W, l.N, l.M)
+                lin[l.name.split(".")[2]] = (vals, idx, bias, l.N, l.M)
+            li += 4
+            ln = [(synth.randn((dim,), 9500 + 4 * li + i, 0.1, dtype, "cuda") + (1.0 if i % 2 == 0 else 0.0)).to(dtype) for i in range(4)]
+            shift = 3 if (b % 2 == 1 and g > 7) else 0
+            rel = lib.pad_score_table(torch.randn((heads, T, T), generator=torch.Generator(device="cuda").manual_seed(9700 + li),
+                                                  device="cuda") * 0.5)
+            mask = lib.elsa_swin_mask(g, g, 7, shift).cuda() if shift else None
+            blocks.append((lib.make_block_weights(ln[0], ln[1], ln[2], ln[3], lin), shift, rel, mask))
+        scratch = lib.alloc_workspace(max(lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w[0], lib.BF16)[0] for w, _, _, _ in blocks))
+        x = [synth.randn((rows, dim), 78 + st, 1.0, dtype, "cuda"), torch.empty((rows, dim), dtype=dtype, device="cuda")]
+        stages.append(dict(dim=dim, g=g, heads=heads, mlp=mlp, rows=rows, blocks=blocks, scratch=scratch, x=x, x0=x[0].clone()))
+
+    def one_pass():
+        for s in stages:
+            for b, (w, shift, rel, mask) in enumerate(s["blocks"]):
+                lib.elsa_swin_block(s["x"][b & 1], s["g"], s["g"], 7, shift, s["heads"], s["mlp"], w[0], rel, mask,
+                                    y=s["x"][(b + 1) & 1], scratch=s["scratch"], dev_status=status)
+
+    def reset():
+        for s in stages:
+            s["x"][0].copy_(s["x0"])
+
+    for _ in range(3):
+        reset()
+        one_pass()
+    times = []
+    for _ in range(reps):
+        reset()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        one_pass()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert int(status.item()) == 0, "device status %#x" % int(status.item())
+    for s in stages:
+        assert torch.isfinite(s["x"][len(s["blocks"]) & 1].float()).all()
+    reset()
+    lib.elsa_profile_start()
+    one_pass()
+    families = {}
+    for kernel, _, ms in lib.elsa_profile_stop():
+        f = families.setdefault(kernel, {"launches": 0, "ms": 0.0})
+        f["launches"] += 1
+        f["ms"] += ms
+    lin_roof = sum(bench.roofline_seconds(l, peaks)[0] for l in layers)
+    # per block: LayerNorm in and out twice, two residual operands, attention's qkv in and a out
+    other_bytes = sum(len(s["blocks"]) * (6 + 4) * s["rows"] * s["dim"] * 2 for s in stages)
+    roof_ms = (lin_roof + other_bytes / hbm) * 1e3
+    ms = statistics.median(times)
+    return {"workload": "swin_b_blocks_b%d" % batch, "blocks": 24, "dtype": "bf16", "peaks": peaks_kind,
+            "note": "blocks chained inside each stage; no patch embedding, patch merging, final norm or head",
+            "ms_per_pass": ms, "ms_min": min(times), "ms_max": max(times), "images_per_s": batch / ms * 1e3,
+            "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "linears_roofline_ms": lin_roof * 1e3,
+            "families_profiled_pass": families, "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
+
+
 def compare(args):
     import bench
     layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
@@ -157,8 +237,11 @@ def main():
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--out", default="bench_out/block.json")
     ap.add_argument("--compare", action="store_true", help="dense 4:4 against sampled N:4 configurations at 7.0 and 6.0 GMACs")
+    ap.add_argument("--swin", action="store_true", help="the 24 blocks of Swin-B at batch 128")
     args = ap.parse_args()
-    if args.compare:
+    if args.swin:
+        rec = run_swin(128, args.reps)
+    elif args.compare:
         rec = compare(args)
     else:
         rec = run(args.blocks, args.batch, args.reps)

@@ -438,8 +438,8 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
 /* The same over windows of `tokens` consecutive rows with additive tables on the scores (Swin's window attention once
  * the rows are in window order): a = softmax(q k^T / sqrt d + bias[head] + mask[window % n_masks]) v.  bias: fp32
  * [heads][tokens][bias_pitch] (the relative-position bias as a dense table), mask: fp32 [n_masks][tokens][bias_pitch] or
- * NULL (the seam mask of shifted windows, one table per window position of an image); bias_pitch >= tokens floats per
- * row.  Head dimension 32 or 64 (dim = heads * 32 or heads * 64), tokens <= 256. */
+ * NULL (the seam mask of shifted windows, one table per window position of an image); rows of bias_pitch >= tokens floats,
+ * bias_pitch a multiple of 4, tables 16-byte aligned.  Head dimension 32 or 64 (dim = heads * 32 or heads * 64), tokens <= 256. */
 elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int heads, int dim, const float* bias,
                                   int bias_pitch, const float* mask, int n_masks, elsa_dtype dtype, void* a,
                                   uint32_t* dev_status, void* stream);
@@ -450,7 +450,7 @@ elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int 
  * first LayerNorm writes its rows in window order, qkv, attention and proj work on windows as runs of rows, and the
  * residual add brings proj's rows back to the grid's order.  Regions X1, QKV, A and T of scratch are therefore in
  * window order.  rel_bias: fp32 [heads][window^2][bias_pitch], device; mask: fp32 [(H / window) (W / window)]
- * [window^2][bias_pitch], device, as elsa_swin_mask writes it (required iff shift > 0).  dim = 32 or 64 times heads.
+ * [window^2][bias_pitch], device, as elsa_swin_mask writes it (required iff shift > 0); bias_pitch a multiple of 4.  dim = 32 or 64 times heads.
  * Patch merging between stages is a separate linear and not part of this call.
  */
 typedef struct {

@@ -448,10 +448,19 @@ def elsa_window_attention(qkv, tokens, heads, bias, mask=None, a=None, dev_statu
     return a
 
 
+def pad_score_table(t):
+    """fp32 table [..., T, T] with its rows padded to whole float4s, as the attention kernel reads them."""
+    T = t.shape[-1]
+    pitch = (T + 3) // 4 * 4
+    out = torch.zeros(t.shape[:-1] + (pitch,), dtype=torch.float32, device=t.device)
+    out[..., :T] = t
+    return out
+
+
 def elsa_swin_mask(H, W, window, shift, pitch=None):
     """The seam mask of shifted windows as a host fp32 tensor [windows, window^2, pitch]."""
     T = window * window
-    pitch = pitch or T
+    pitch = pitch or (T + 3) // 4 * 4          # rows padded to whole float4s
     n = (H // window) * (W // window)
     out = torch.empty((n, T, pitch), dtype=torch.float32)
     got = _swin_mask(H, W, window, shift, pitch, ctypes.cast(out.data_ptr(), ctypes.POINTER(ctypes.c_float)))

@@ -241,13 +241,23 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                     if (p.mask != nullptr) mrow = p.mask + ((size_t)(img % p.n_masks) * p.tokens + row) * (size_t)p.bias_pitch;
                 }
             }
-            auto biased = [&](uint32_t raw, int col) -> float {     // kBias only: the score in the exponent's domain
-                float b = 0.f;
-                if (brow != nullptr && col < p.tokens) {
-                    b = __ldg(brow + col);
-                    if (mrow != nullptr) b += __ldg(mrow + col);
+            // (bias + mask) * log2(e) for `count` columns from col0 (multiples of 4; rows of the tables are 16-byte
+            // aligned and padded to bias_pitch, so whole float4 loads stay inside a row); zeros without tables
+            auto load_bias = [&](float* bb, int col0, int count) {
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    if (4 * v >= count) break;
+                    float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (brow != nullptr && col0 + 4 * v < p.bias_pitch) {
+                        b4 = __ldg(reinterpret_cast<const float4*>(brow + col0) + v);
+                        if (mrow != nullptr) {
+                            const float4 m4 = __ldg(reinterpret_cast<const float4*>(mrow + col0) + v);
+                            b4.x += m4.x; b4.y += m4.y; b4.z += m4.z; b4.w += m4.w;
+                        }
+                    }
+                    bb[4 * v] = b4.x * 1.4426950408889634f; bb[4 * v + 1] = b4.y * 1.4426950408889634f;
+                    bb[4 * v + 2] = b4.z * 1.4426950408889634f; bb[4 * v + 3] = b4.w * 1.4426950408889634f;
                 }
-                return fmaf(__uint_as_float(raw), scale, b * 1.4426950408889634f);
             };
             {
                 // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
@@ -256,7 +266,44 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                 const int units = p.tk >> 5;            // whole units of 32 columns
                 const bool tail = (p.tk & 31) != 0;     // plus one chunk of 16
                 float m = -INFINITY;
-                for (int u0 = 0; u0 < units; u0 += 2) {
+                if constexpr (kBias) {
+                    // first pass of the biased form: t = s * scale + (bias + mask) * log2(e) replaces s in tensor memory,
+                    // so the tables are read once
+                    for (int u = 0; u < units; ++u) {
+                        uint32_t r[32];
+                        float bb[32];
+                        tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * u), r);
+                        load_bias(bb, 32 * u, 32);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const float t = fmaf(__uint_as_float(r[j]), scale, bb[j]);
+                            r[j] = __float_as_uint(t);
+                            if (32 * u + j < p.tokens) m = fmaxf(m, t);
+                        }
+                        uint32_t lo[16], hi[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) { lo[j] = r[j]; hi[j] = r[16 + j]; }
+                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * u), lo);
+                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * u + 16), hi);
+                    }
+                    if (tail) {
+                        uint32_t r[16];
+                        float bb[16];
+                        tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                        load_bias(bb, 32 * units, 16);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const float t = fmaf(__uint_as_float(r[j]), scale, bb[j]);
+                            r[j] = __float_as_uint(t);
+                            if (32 * units + j < p.tokens) m = fmaxf(m, t);
+                        }
+                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                    }
+                    tmem_wait_st();
+                }
+                for (int u0 = 0; !kBias && u0 < units; u0 += 2) {
                     uint32_t r[2][32];
 #pragma unroll
                     for (int i = 0; i < 2; ++i)
@@ -265,11 +312,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 #pragma unroll
                     for (int i = 0; i < 2; ++i)
                         if (u0 + i < units) {
-                            if constexpr (kBias) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, biased(r[i][j], 32 * (u0 + i) + j));
-                            } else if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
+                            if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
                                 float m0 = m, m1 = -INFINITY;
 #pragma unroll
                                 for (int j = 0; j < 32; j += 2) {
@@ -284,14 +327,13 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                             }
                         }
                 }
-                if (tail) {
+                if (!kBias && tail) {
                     uint32_t r[16];
                     tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
                     tmem_wait_ld();
 #pragma unroll
                     for (int j = 0; j < 16; ++j)
-                        if (32 * units + j < p.tokens)
-                            m = fmaxf(m, kBias ? biased(r[j], 32 * units + j) : __uint_as_float(r[j]));
+                        if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
                 }
                 // p = 2^(s * scale - m * scale) for 16 columns starting at col0: eight packed pairs
                 const float m_scaled = kBias ? m : m * scale;      // the biased maximum is in the exponent's domain already
@@ -301,8 +343,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         float e0, e1;
-                        const float a0 = kBias ? biased(r[2 * j], col0 + 2 * j) - m_scaled : fmaf(__uint_as_float(r[2 * j]), scale, -m_scaled);
-                        const float a1 = kBias ? biased(r[2 * j + 1], col0 + 2 * j + 1) - m_scaled
+                        const float a0 = kBias ? __uint_as_float(r[2 * j]) - m_scaled : fmaf(__uint_as_float(r[2 * j]), scale, -m_scaled);
+                        const float a1 = kBias ? __uint_as_float(r[2 * j + 1]) - m_scaled
                                                : fmaf(__uint_as_float(r[2 * j + 1]), scale, -m_scaled);
                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(a0));
                         asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(a1));
@@ -444,8 +486,11 @@ elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int he
                     kMaxTokens, tokens, heads, dim);
     const int head_dim = dim / heads;
     if (bias == nullptr && mask != nullptr) return fail(ELSA_ERR_NULL, "a mask table needs a bias table");
-    if (bias != nullptr && (bias_pitch < tokens || (mask != nullptr && n_masks < 1)))
-        return fail(ELSA_ERR_SHAPE, "bias_pitch=%d must be at least tokens=%d, n_masks=%d at least 1", bias_pitch, tokens, n_masks);
+    if (bias != nullptr && (bias_pitch < tokens || bias_pitch % 4 != 0 || (mask != nullptr && n_masks < 1)))
+        return fail(ELSA_ERR_SHAPE, "bias_pitch=%d must be a multiple of 4 and at least tokens=%d, n_masks=%d at least 1", bias_pitch,
+                    tokens, n_masks);
+    if (bias != nullptr && ((((uintptr_t)bias) & 15u) != 0 || (((uintptr_t)mask) & 15u) != 0))
+        return fail(ELSA_ERR_ALIGN, "the bias and mask tables must be 16-byte aligned");
     if ((long long)images * heads * ((tokens + kQRows - 1) / kQRows) > 0x7fffffffLL)
         return fail(ELSA_ERR_SHAPE, "images * heads does not fit an int");
     AttnParams p;

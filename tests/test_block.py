@@ -442,8 +442,9 @@ def test_window_attention_matches_oracle(lib, case, dtype):
     mask = bo.shift_mask(H, W, ws, shift) if shift else None
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     a_win = lib.elsa_window_attention(qkv[perm].contiguous().cuda(), T, heads,
-                                      torch.from_numpy(rel_bias).float().cuda(),
-                                      None if mask is None else torch.from_numpy(mask).float().cuda(), dev_status=status)
+                                      lib.pad_score_table(torch.from_numpy(rel_bias).float().cuda()),
+                                      None if mask is None else lib.pad_score_table(torch.from_numpy(mask).float().cuda()),
+                                      dev_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status %#x" % int(status.item())
     q64 = qkv.double().numpy()
@@ -461,7 +462,7 @@ def test_swin_mask_is_the_oracles():
     build.build()
     from paper_2409_09708_b200 import binding as lib
     for H, W, ws, shift in [(14, 14, 7, 3), (6, 9, 3, 1), (28, 14, 7, 3), (8, 8, 4, 2)]:
-        got = lib.elsa_swin_mask(H, W, ws, shift).numpy()
+        got = lib.elsa_swin_mask(H, W, ws, shift, pitch=ws * ws).numpy()
         assert np.array_equal(got, bo.shift_mask(H, W, ws, shift).astype(np.float32))
         padded = lib.elsa_swin_mask(H, W, ws, shift, pitch=ws * ws + 7).numpy()
         assert np.array_equal(padded[:, :, :ws * ws], got) and (padded[:, :, ws * ws:] == 0).all()
@@ -492,7 +493,7 @@ def test_swin_block_matches_oracle(lib, case, dtype):
     scratch = torch.zeros(total, dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     mask = lib.elsa_swin_mask(H, W, ws, shift).cuda() if shift else None
-    y, _ = lib.elsa_swin_block(x.cuda(), H, W, ws, shift, heads, mlp, w, torch.from_numpy(rel_bias).float().cuda(), mask,
+    y, _ = lib.elsa_swin_block(x.cuda(), H, W, ws, shift, heads, mlp, w, lib.pad_score_table(torch.from_numpy(rel_bias).float().cuda()), mask,
                                scratch=scratch, dev_status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status %#x" % int(status.item())
