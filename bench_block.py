@@ -128,11 +128,11 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     return rec
 
 
-def run_swin(batch=128, reps=5):
+def run_swin(batch=128, reps=5, pack=2):
     """The 24 blocks of Swin-B (elsa_swin_block), chained inside each stage, with the levels of the Swin-B stack
     workload; window 7, every second block shifted by 3 (none in the last stage, whose grid is one window).  Patch
     embedding, the patch-merging linears between the stages, final norm and head are not part of it: each stage
-    starts from a seeded input of its own shape."""
+    starts from a seeded input of its own shape.  pack: windows per attention item."""
     import bench
     peaks, peaks_kind = bench.load_peaks()
     hbm = peaks["hbm_gbs"] * 1e9
@@ -154,9 +154,9 @@ def run_swin(batch=128, reps=5):
             li += 4
             ln = [(synth.randn((dim,), 9500 + 4 * li + i, 0.1, dtype, "cuda") + (1.0 if i % 2 == 0 else 0.0)).to(dtype) for i in range(4)]
             shift = 3 if (b % 2 == 1 and g > 7) else 0
-            rel = lib.pad_score_table(torch.randn((heads, T, T), generator=torch.Generator(device="cuda").manual_seed(9700 + li),
-                                                  device="cuda") * 0.5)
-            mask = lib.elsa_swin_mask(g, g, 7, shift).cuda() if shift else None
+            rel = lib.elsa_swin_pack_bias(torch.randn((heads, T, T), generator=torch.Generator().manual_seed(9700 + li)) * 0.5,
+                                          7, pack=pack).cuda()
+            mask = lib.elsa_swin_mask(g, g, 7, shift, pack=pack).cuda() if shift else None
             blocks.append((lib.make_block_weights(ln[0], ln[1], ln[2], ln[3], lin), shift, rel, mask))
         scratch = lib.alloc_workspace(max(lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w[0], lib.BF16)[0] for w, _, _, _ in blocks))
         x = [synth.randn((rows, dim), 78 + st, 1.0, dtype, "cuda"), torch.empty((rows, dim), dtype=dtype, device="cuda")]
@@ -166,7 +166,7 @@ def run_swin(batch=128, reps=5):
         for s in stages:
             for b, (w, shift, rel, mask) in enumerate(s["blocks"]):
                 lib.elsa_swin_block(s["x"][b & 1], s["g"], s["g"], 7, shift, s["heads"], s["mlp"], w[0], rel, mask,
-                                    y=s["x"][(b + 1) & 1], scratch=s["scratch"], dev_status=status)
+                                    y=s["x"][(b + 1) & 1], scratch=s["scratch"], dev_status=status, pack=pack)
 
     def reset():
         for s in stages:
@@ -200,7 +200,7 @@ def run_swin(batch=128, reps=5):
     other_bytes = sum(len(s["blocks"]) * (6 + 4) * s["rows"] * s["dim"] * 2 for s in stages)
     roof_ms = (lin_roof + other_bytes / hbm) * 1e3
     ms = statistics.median(times)
-    return {"workload": "swin_b_blocks_b%d" % batch, "blocks": 24, "dtype": "bf16", "peaks": peaks_kind,
+    return {"workload": "swin_b_blocks_b%d" % batch, "blocks": 24, "dtype": "bf16", "peaks": peaks_kind, "windows_per_attention_item": pack,
             "note": "blocks chained inside each stage; no patch embedding, patch merging, final norm or head",
             "ms_per_pass": ms, "ms_min": min(times), "ms_max": max(times), "images_per_s": batch / ms * 1e3,
             "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms, "linears_roofline_ms": lin_roof * 1e3,
@@ -238,9 +238,10 @@ def main():
     ap.add_argument("--out", default="bench_out/block.json")
     ap.add_argument("--compare", action="store_true", help="dense 4:4 against sampled N:4 configurations at 7.0 and 6.0 GMACs")
     ap.add_argument("--swin", action="store_true", help="the 24 blocks of Swin-B at batch 128")
+    ap.add_argument("--pack", type=int, default=2, help="--swin: windows per attention item (1 or 2)")
     args = ap.parse_args()
     if args.swin:
-        rec = run_swin(128, args.reps)
+        rec = run_swin(128, args.reps, args.pack)
     elif args.compare:
         rec = compare(args)
     else:

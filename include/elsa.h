@@ -452,16 +452,24 @@ elsa_status elsa_window_attention(const void* qkv, int windows, int tokens, int 
  * window order.  rel_bias: fp32 [heads][window^2][bias_pitch], device; mask: fp32 [(H / window) (W / window)]
  * [window^2][bias_pitch], device, as elsa_swin_mask writes it (required iff shift > 0); bias_pitch a multiple of 4.  dim = 32 or 64 times heads.
  * Patch merging between stages is a separate linear and not part of this call.
+ * pack: windows per attention item (1, or more while pack * window^2 <= 256; consecutive windows are consecutive rows,
+ * so an item of `pack` windows is a run of rows too, and the 128-row tiles of the tensor cores are better filled: 2 for
+ * 7 x 7 windows).  The tables are then per group of windows, [heads][pack window^2][bias_pitch] with -30000 between
+ * tokens of different windows (elsa_swin_pack_bias builds it) and [windows of an image / pack][pack window^2][bias_pitch].
  */
 typedef struct {
     int H, W, window, shift;
     const float* rel_bias;
     const float* mask;
     int bias_pitch;
+    int pack;
 } elsa_swin_attn;
-/* HOST arithmetic: fills mask [windows of an image][window^2][pitch] (host memory) with 0 / -100 and returns the number
- * of windows, -1 on invalid arguments (needs 0 < shift < window). */
-int elsa_swin_mask(int H, int W, int window, int shift, int pitch, float* mask);
+/* HOST arithmetic: fills mask [windows of an image / pack][pack window^2][pitch] (host memory) with 0 / -100 and
+ * returns the number of tables, -1 on invalid arguments (needs 0 < shift < window). */
+int elsa_swin_mask(int H, int W, int window, int shift, int pack, int pitch, float* mask);
+/* HOST arithmetic: rel_bias [heads][window^2][window^2] -> packed [heads][pack window^2][pitch], the bias on the
+ * diagonal blocks and -30000 elsewhere.  0, or -1 on invalid arguments. */
+int elsa_swin_pack_bias(const float* rel_bias, int heads, int window, int pack, int pitch, float* packed);
 elsa_status elsa_swin_block(const void* x, int images, int heads, int dim, int mlp_dim, const elsa_block_weights* w,
                             const elsa_swin_attn* attn, elsa_dtype dtype, void* y, void* scratch, size_t scratch_bytes,
                             uint32_t* dev_status, void* stream);

@@ -127,10 +127,13 @@ _block_attn = _sig("elsa_vit_block_attn", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i,
 _attention = _sig("elsa_attention", _i, [_vp, _i, _i, _i, _i, _i, _vp, _vp, _vp])
 _window_attention = _sig("elsa_window_attention", _i, [_vp, _i, _i, _i, _i, _vp, _i, _vp, _i, _i, _vp, _vp, _vp])
 class ElsaSwinAttn(ctypes.Structure):
-    _fields_ = [("H", _i), ("W", _i), ("window", _i), ("shift", _i), ("rel_bias", _vp), ("mask", _vp), ("bias_pitch", _i)]
+    _fields_ = [("H", _i), ("W", _i), ("window", _i), ("shift", _i), ("rel_bias", _vp), ("mask", _vp), ("bias_pitch", _i),
+                ("pack", _i)]
 
 
-_swin_mask = _sig("elsa_swin_mask", _i, [_i, _i, _i, _i, _i, ctypes.POINTER(ctypes.c_float)])
+_fp = ctypes.POINTER(ctypes.c_float)
+_swin_mask = _sig("elsa_swin_mask", _i, [_i, _i, _i, _i, _i, _i, _fp])
+_swin_pack_bias = _sig("elsa_swin_pack_bias", _i, [_fp, _i, _i, _i, _i, _fp])
 _swin_block = _sig("elsa_swin_block", _i, [_vp, _i, _i, _i, _i, _bw, ctypes.POINTER(ElsaSwinAttn), _i, _vp, _vp, _sz, _vp, _vp])
 _encoder_scratch = _sig("elsa_vit_encoder_scratch_bytes", _sz, [_i, _i, _i, _i, _bw, _i, _i])
 _encoder = _sig("elsa_vit_encoder", _i, [_vp, _i, _i, _i, _i, _i, _bw, _i, _vp, _vp, ctypes.c_float, _i, _vp, _vp, _sz, _vp, _vp])
@@ -457,28 +460,41 @@ def pad_score_table(t):
     return out
 
 
-def elsa_swin_mask(H, W, window, shift, pitch=None):
-    """The seam mask of shifted windows as a host fp32 tensor [windows, window^2, pitch]."""
-    T = window * window
+def elsa_swin_mask(H, W, window, shift, pitch=None, pack=1):
+    """The seam mask of shifted windows as a host fp32 tensor [windows / pack, pack window^2, pitch]."""
+    T = window * window * pack
     pitch = pitch or (T + 3) // 4 * 4          # rows padded to whole float4s
-    n = (H // window) * (W // window)
+    n = (H // window) * (W // window) // pack
     out = torch.empty((n, T, pitch), dtype=torch.float32)
-    got = _swin_mask(H, W, window, shift, pitch, ctypes.cast(out.data_ptr(), ctypes.POINTER(ctypes.c_float)))
+    got = _swin_mask(H, W, window, shift, pack, pitch, ctypes.cast(out.data_ptr(), _fp))
     if got != n:
         raise ValueError("elsa_swin_mask rejected its arguments")
     return out
 
 
+def elsa_swin_pack_bias(rel_bias, window, pack=1, pitch=None):
+    """rel_bias: host fp32 [heads, T, T] -> host fp32 [heads, pack T, pitch] (bias on the diagonal blocks, -30000 between
+    tokens of different windows)."""
+    rel_bias = rel_bias.detach().to(torch.float32).cpu().contiguous()
+    heads, T = rel_bias.shape[0], window * window
+    pitch = pitch or (pack * T + 3) // 4 * 4
+    out = torch.empty((heads, pack * T, pitch), dtype=torch.float32)
+    if _swin_pack_bias(ctypes.cast(rel_bias.data_ptr(), _fp), heads, window, pack, pitch, ctypes.cast(out.data_ptr(), _fp)) != 0:
+        raise ValueError("elsa_swin_pack_bias rejected its arguments")
+    return out
+
+
 def elsa_swin_block(x, H, W, window, shift, heads, mlp_dim, weights, rel_bias, mask=None, y=None, scratch=None,
-                    dev_status=None, stream=None):
-    """One Swin block over x [images * H * W, dim]; rel_bias [heads, T, pitch] and mask [windows, T, pitch] fp32 on the device."""
+                    dev_status=None, stream=None, pack=1):
+    """One Swin block over x [images * H * W, dim]; rel_bias [heads, pack T, pitch] and mask [windows / pack, pack T, pitch]
+    fp32 on the device, as elsa_swin_pack_bias and elsa_swin_mask build them for `pack` windows per attention item."""
     rows, dim = x.shape
     code = dtype_code(x.dtype)
     if scratch is None:
         scratch = alloc_workspace(elsa_vit_block_scratch_bytes(rows, dim, mlp_dim, weights, code)[0], x.device)
     if y is None:
         y = torch.empty_like(x)
-    attn = ElsaSwinAttn(H, W, window, shift, _ptr(rel_bias), _ptr(mask), rel_bias.shape[-1])
+    attn = ElsaSwinAttn(H, W, window, shift, _ptr(rel_bias), _ptr(mask), rel_bias.shape[-1], pack)
     _check(_swin_block(_ptr(x), rows // (H * W), heads, dim, mlp_dim, ctypes.byref(weights), ctypes.byref(attn), code, _ptr(y),
                        _ptr(scratch), scratch.numel(), _ptr(dev_status), _stream(stream)))
     return y, scratch

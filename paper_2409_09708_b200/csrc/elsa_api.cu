@@ -1104,10 +1104,11 @@ elsa_status run_block(const void* x, int rows, int dim, int mlp_dim, const elsa_
         return st;
     if (carry != nullptr && carry->t != nullptr) x = x_sum;      // the block's input, as just stored
     if (swin) {
-        const int T = swin->window * swin->window;
+        const int pack = swin->pack < 1 ? 1 : swin->pack;
+        const int T = swin->window * swin->window * pack;
         st = launch_attention((const uint16_t*)(s8 + plan.off[ELSA_BLOCK_QKV]), rows / T, T, heads, dim, dtype,
                               (uint16_t*)(s8 + plan.off[ELSA_BLOCK_A]), dev_status, stream, swin->rel_bias,
-                              swin->shift > 0 ? swin->mask : nullptr, (swin->H / swin->window) * (swin->W / swin->window),
+                              swin->shift > 0 ? swin->mask : nullptr, (swin->H / swin->window) * (swin->W / swin->window) / pack,
                               swin->bias_pitch);
     } else if (tokens == 0) {
         // the stated stand-in for attention: a = V
@@ -1234,30 +1235,44 @@ elsa_status elsa_attention(const void* qkv, int images, int tokens, int heads, i
     return launch_attention((const uint16_t*)qkv, images, tokens, heads, dim, dtype, (uint16_t*)a, dev_status, (cudaStream_t)stream);
 }
 
-int elsa_swin_mask(int H, int W, int window, int shift, int pitch, float* mask)
+int elsa_swin_mask(int H, int W, int window, int shift, int pack, int pitch, float* mask)
 {
-    if (H <= 0 || W <= 0 || window <= 0 || H % window != 0 || W % window != 0 || shift <= 0 || shift >= window ||
-        pitch < window * window || !mask)
+    if (H <= 0 || W <= 0 || window <= 0 || H % window != 0 || W % window != 0 || shift <= 0 || shift >= window || pack < 1 ||
+        pitch < pack * window * window || !mask)
         return -1;
-    const int T = window * window, nww = W / window;
+    const int T = window * window, nww = W / window, n_windows = (H / window) * nww;
+    if (n_windows % pack != 0) return -1;
     // region of a position of the rolled grid: the bands [0, n - window), [n - window, n - shift), [n - shift, n) of each axis
     auto band = [&](int v, int n) { return v < n - window ? 0 : v < n - shift ? 1 : 2; };
-    for (int wi = 0; wi < H / window; ++wi)
-        for (int wj = 0; wj < nww; ++wj) {
-            float* m = mask + (size_t)(wi * nww + wj) * T * pitch;
-            for (int p = 0; p < T; ++p) {
-                const int rp = 3 * band(wi * window + p / window, H) + band(wj * window + p % window, W);
-                for (int q = 0; q < pitch; ++q) {
-                    float v = 0.f;
-                    if (q < T) {
-                        const int rq = 3 * band(wi * window + q / window, H) + band(wj * window + q % window, W);
-                        v = rp != rq ? -100.f : 0.f;
-                    }
-                    m[(size_t)p * pitch + q] = v;
-                }
+    auto region = [&](int win, int t) {
+        const int wi = win / nww, wj = win % nww;
+        return 3 * band(wi * window + t / window, H) + band(wj * window + t % window, W);
+    };
+    for (int g = 0; g < n_windows / pack; ++g) {
+        float* m = mask + (size_t)g * pack * T * pitch;
+        for (int p = 0; p < pack * T; ++p)
+            for (int q = 0; q < pitch; ++q) {
+                float v = 0.f;
+                // tokens of different windows of a group are kept apart by the bias table; here: the seam inside a window
+                if (q < pack * T && p / T == q / T) v = region(g * pack + p / T, p % T) != region(g * pack + q / T, q % T) ? -100.f : 0.f;
+                m[(size_t)p * pitch + q] = v;
             }
-        }
-    return (H / window) * nww;
+    }
+    return n_windows / pack;
+}
+
+int elsa_swin_pack_bias(const float* rel_bias, int heads, int window, int pack, int pitch, float* packed)
+{
+    if (!rel_bias || !packed || heads <= 0 || window <= 0 || pack < 1 || pitch < pack * window * window) return -1;
+    const int T = window * window;
+    for (int h = 0; h < heads; ++h)
+        for (int p = 0; p < pack * T; ++p)
+            for (int q = 0; q < pitch; ++q) {
+                float v = 0.f;
+                if (q < pack * T) v = p / T == q / T ? rel_bias[((size_t)h * T + p % T) * T + q % T] : -30000.f;
+                packed[((size_t)h * pack * T + p) * pitch + q] = v;
+            }
+    return 0;
 }
 
 elsa_status elsa_swin_block(const void* x, int images, int heads, int dim, int mlp_dim, const elsa_block_weights* w,
@@ -1269,10 +1284,15 @@ elsa_status elsa_swin_block(const void* x, int images, int heads, int dim, int m
         attn->W % attn->window != 0 || attn->shift < 0 || attn->shift >= attn->window)
         return fail(ELSA_ERR_SHAPE, "windows of %d do not tile a %d x %d grid, or shift=%d is outside [0, window)", attn->window,
                     attn->H, attn->W, attn->shift);
-    const int T = attn->window * attn->window;
+    const int pack = attn->pack < 1 ? 1 : attn->pack;
+    const int T = attn->window * attn->window * pack;         // tokens of one attention item: `pack` windows
     if (!attention_suits(T, heads, dim))
-        return fail(ELSA_ERR_SHAPE, "window attention needs at most 256 tokens per window and dim = 32 or 64 times heads "
-                    "(window=%d, heads=%d, dim=%d)", attn->window, heads, dim);
+        return fail(ELSA_ERR_SHAPE, "window attention needs at most 256 tokens per group of windows and dim = 32 or 64 times heads "
+                    "(window=%d, pack=%d, heads=%d, dim=%d)", attn->window, pack, heads, dim);
+    if (((long long)images * (attn->H / attn->window) * (attn->W / attn->window)) % pack != 0)
+        return fail(ELSA_ERR_SHAPE, "the windows do not divide into groups of %d", pack);
+    if (attn->shift > 0 && ((attn->H / attn->window) * (attn->W / attn->window)) % pack != 0)
+        return fail(ELSA_ERR_SHAPE, "with a shift the windows of one image must divide into groups of %d", pack);
     if (!attn->rel_bias || (attn->shift > 0 && !attn->mask)) return fail(ELSA_ERR_NULL, "rel_bias (and mask when shift > 0) must not be NULL");
     if (attn->bias_pitch < T) return fail(ELSA_ERR_SHAPE, "bias_pitch=%d is below the %d tokens of a window", attn->bias_pitch, T);
     if ((long long)images * attn->H * attn->W > 0x7fffffffLL) return fail(ELSA_ERR_SHAPE, "images * H * W does not fit an int");

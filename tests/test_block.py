@@ -463,18 +463,30 @@ def test_swin_mask_is_the_oracles():
     from paper_2409_09708_b200 import binding as lib
     for H, W, ws, shift in [(14, 14, 7, 3), (6, 9, 3, 1), (28, 14, 7, 3), (8, 8, 4, 2)]:
         got = lib.elsa_swin_mask(H, W, ws, shift, pitch=ws * ws).numpy()
-        assert np.array_equal(got, bo.shift_mask(H, W, ws, shift).astype(np.float32))
+        ref = bo.shift_mask(H, W, ws, shift).astype(np.float32)
+        assert np.array_equal(got, ref)
         padded = lib.elsa_swin_mask(H, W, ws, shift, pitch=ws * ws + 7).numpy()
         assert np.array_equal(padded[:, :, :ws * ws], got) and (padded[:, :, ws * ws:] == 0).all()
+        # two windows per item: the seam masks on the diagonal blocks, nothing (the bias table separates the windows) elsewhere
+        T = ws * ws
+        two = lib.elsa_swin_mask(H, W, ws, shift, pitch=2 * T, pack=2).numpy()
+        assert two.shape == (ref.shape[0] // 2, 2 * T, 2 * T)
+        assert np.array_equal(two[:, :T, :T], ref[0::2]) and np.array_equal(two[:, T:, T:], ref[1::2])
+        assert (two[:, :T, T:] == 0).all() and (two[:, T:, :T] == 0).all()
+    bias = torch.from_numpy(np.random.default_rng(1).standard_normal((3, 9, 9)).astype(np.float32))
+    packed = lib.elsa_swin_pack_bias(bias, 3, pack=2, pitch=20).numpy()
+    assert np.array_equal(packed[:, :9, :9], bias.numpy()) and np.array_equal(packed[:, 9:, 9:18], bias.numpy())
+    assert (packed[:, :9, 9:18] == -30000).all() and (packed[:, 9:, :9] == -30000).all() and (packed[:, :, 18:] == 0).all()
 
 
 SWIN_CASES = [(2, 14, 14, 7, 0, 2, 32), (2, 14, 14, 7, 3, 2, 32), (1, 28, 28, 7, 3, 4, 32), (2, 14, 14, 7, 3, 1, 64)]
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("pack", [1, 2])
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
 @pytest.mark.parametrize("case", SWIN_CASES, ids=["%dx%dx%d_w%d_s%d_h%d_d%d" % c for c in SWIN_CASES])
-def test_swin_block_matches_oracle(lib, case, dtype):
+def test_swin_block_matches_oracle(lib, case, dtype, pack):
     B, H, W, ws, shift, heads, d = case
     dim, T, mlp = heads * d, ws * ws, 4 * heads * d
     rows = B * H * W
@@ -492,9 +504,10 @@ def test_swin_block_matches_oracle(lib, case, dtype):
     total, off = lib.elsa_vit_block_scratch_bytes(rows, dim, mlp, w, code)
     scratch = torch.zeros(total, dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
-    mask = lib.elsa_swin_mask(H, W, ws, shift).cuda() if shift else None
-    y, _ = lib.elsa_swin_block(x.cuda(), H, W, ws, shift, heads, mlp, w, lib.pad_score_table(torch.from_numpy(rel_bias).float().cuda()), mask,
-                               scratch=scratch, dev_status=status)
+    mask = lib.elsa_swin_mask(H, W, ws, shift, pack=pack).cuda() if shift else None
+    bias_table = lib.elsa_swin_pack_bias(torch.from_numpy(rel_bias), ws, pack=pack).cuda()
+    y, _ = lib.elsa_swin_block(x.cuda(), H, W, ws, shift, heads, mlp, w, bias_table, mask, scratch=scratch, dev_status=status,
+                               pack=pack)
     torch.cuda.synchronize()
     assert int(status.item()) == 0, "device status %#x" % int(status.item())
     cols = {"x1": dim, "qkv": 3 * dim, "a": dim, "x2": dim, "x3": dim, "h": mlp}
