@@ -128,7 +128,7 @@ def run(blocks=12, batch=256, reps=5, peaks=None, peaks_kind=None, roofline_seco
     return rec
 
 
-def run_swin(batch=128, reps=5, pack=2):
+def run_swin(batch=128, reps=5, pack=1):
     """The 24 blocks of Swin-B (elsa_swin_block), chained inside each stage, with the levels of the Swin-B stack
     workload; window 7, every second block shifted by 3 (none in the last stage, whose grid is one window).  Patch
     embedding, the patch-merging linears between the stages, final norm and head are not part of it: each stage
@@ -238,7 +238,7 @@ def main():
     ap.add_argument("--out", default="bench_out/block.json")
     ap.add_argument("--compare", action="store_true", help="dense 4:4 against sampled N:4 configurations at 7.0 and 6.0 GMACs")
     ap.add_argument("--swin", action="store_true", help="the 24 blocks of Swin-B at batch 128")
-    ap.add_argument("--pack", type=int, default=2, help="--swin: windows per attention item (1 or 2)")
+    ap.add_argument("--pack", type=int, default=1, help="--swin: windows per attention item (1 or 2)")
     args = ap.parse_args()
     if args.swin:
         rec = run_swin(128, args.reps, args.pack)

@@ -17,11 +17,12 @@
 //   4. O = P V: Tk / 16 MMAs with A from tensor memory and V as it lies in memory (keys outermost: MN-major
 //      descriptor) into 64 columns of the part of S that is dead by then.
 //   5. The same four warps read O, divide by the row sum, round once and store each row's 128 bytes.
-// Persistent: one CTA per SM walks the items with the stride of the grid, two items in flight.  Shared memory holds
-// two stages of (Q, K, V), tensor memory two halves of 256 columns, and there are two groups of four softmax warps:
-// item n uses stage, half and group n % 2.  The producer warp loads item n + 1 (and n + 2 once its stage is free)
-// while item n is computed; the MMA warp issues S of item n, then P V of item n - 1, so one group's softmax runs
-// under the other group's products and epilogue.  Every wait is bounded as in the GEMM kernels.
+// Persistent: one CTA per SM walks the items with the stride of the grid, with several items in flight: two for up
+// to 256 keys, four for up to 128 (Swin's windows), each with its own shared-memory stage (Q, K, V), its own share
+// of tensor memory (256 or 128 columns) and its own group of four softmax warps: item n uses stage, share and group
+// n % 2 (n % 4).  The producer warp loads ahead as stages come free; the MMA warp issues S of item n, then P V of the
+// oldest item whose probabilities are due, so one group's softmax runs under the others' products and epilogues.
+// Every wait is bounded as in the GEMM kernels.
 #include <atomic>
 #include <mutex>
 
@@ -33,14 +34,21 @@ namespace {
 constexpr int kMaxHeadDim = 64;
 constexpr int kQRows = 128;          // query rows per item = TMEM lanes
 constexpr int kMaxTokens = 256;
-constexpr int kBufCols = 256;        // tensor-memory columns per item in flight
-constexpr int kTmemCols = 2 * kBufCols;
+constexpr int kTmemCols = 512;
 constexpr int kGroupWarps = 4;       // softmax warps per group, one per TMEM lane quarter
-constexpr int kThreads = (2 + 2 * kGroupWarps) * 32;
 constexpr int kQBytes = kQRows * kMaxHeadDim * 2;          // the shared-memory slots are laid out for head dimension 64
-constexpr int kKvBytesMax = kMaxTokens * kMaxHeadDim * 2;
-constexpr int kStageBytes = kQBytes + 2 * kKvBytesMax;
-constexpr int kSmemBytes = 2 * kStageBytes + 1024 /* alignment */ + 256 /* barriers */;
+
+// kBufs items in flight per CTA: 2 for up to 256 keys (256 tensor-memory columns each), 4 for up to 128 keys (the
+// windows of Swin), where an item's on-chip chain is short and only more of them in flight fill the SM.
+template <int kBufs>
+struct Shape {
+    static constexpr int kBufCols = kTmemCols / kBufs;
+    static constexpr int kThreads = (2 + kBufs * kGroupWarps) * 32;
+    static constexpr int kKvBytes = (kBufs == 2 ? 256 : 128) * kMaxHeadDim * 2;
+    static constexpr int kStageBytes = kQBytes + 2 * kKvBytes;
+    static constexpr int kSmemBytes = kBufs * kStageBytes + 1024 /* alignment */ + 512 /* barriers */;
+    static constexpr int kUnit = kBufs == 2 ? 32 : 16;      // score columns a softmax warp handles at a time (registers)
+};
 
 struct AttnParams {
     CUtensorMap map_q;    // box 64 columns x 128 tokens x 1 image
@@ -100,21 +108,25 @@ __device__ __forceinline__ void tmem_st_32x32b_x8(uint32_t taddr, const uint32_t
                  : "memory");
 }
 
-template <bool kBf16, int kD, bool kBias>
-__global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_constant__ AttnParams p)
+template <bool kBf16, int kD, bool kBias, int kBufs>
+__global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(const __grid_constant__ AttnParams p)
 {
     static_assert(kD == 64 || kD == 32, "head dimension");
+    static_assert(kBufs == 2 || kBufs == 4, "items in flight");
+    constexpr int kBufCols = Shape<kBufs>::kBufCols, kStageBytes = Shape<kBufs>::kStageBytes, kKvBytesMax = Shape<kBufs>::kKvBytes;
+    constexpr int U = Shape<kBufs>::kUnit;
+    constexpr int kLag = kBufs - 1;                   // P V of item n - kLag is issued after S of item n
     constexpr int kHeadDim = kD;
     constexpr int kItemQBytes = kQRows * kD * 2;      // bytes TMA delivers for the Q tile; K and V: tk * kD * 2
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = smem_base + 2 * kStageBytes;
+    const uint32_t bars = smem_base + kBufs * kStageBytes;
     // per buffer b: +0 qk_full, +8 v_full, +16 smem_empty, +24 s_full, +32 p_full, +40 o_full, +48 tmem_empty
     auto bar = [&](int which, int b) { return bars + (uint32_t)(64 * b + 8 * which); };
     enum { kQkFull = 0, kVFull, kSmemEmpty, kSFull, kPFull, kOFull, kTmemEmpty };
-    const uint32_t tmem_holder_addr = bars + 128;
+    const uint32_t tmem_holder_addr = bars + 64 * kBufs;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem_raw + (tmem_holder_addr - smem_u32(smem_raw)));
-    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 136 - smem_u32(smem_raw)));
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 64 * kBufs + 8 - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int first = blockIdx.x, stride = gridDim.x;
@@ -122,7 +134,7 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
 
     if (warp == 1) {
         if (lane == 0) {
-            for (int b = 0; b < 2; ++b) {
+            for (int b = 0; b < kBufs; ++b) {
                 mbar_init(bar(kQkFull, b), 1);
                 mbar_init(bar(kVFull, b), 1);
                 mbar_init(bar(kSmemEmpty, b), 1);
@@ -149,8 +161,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         const bool elected = elect_one();
         bool ok = true;
         for (int n = 0; ok && n < n_items; ++n) {
-            const int b = n & 1;
-            const uint32_t ph = (uint32_t)((n >> 1) & 1);
+            const int b = n % kBufs;
+            const uint32_t ph = (uint32_t)((n / kBufs) & 1);
             ok = mbar_wait(bar(kSmemEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 20);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -172,10 +184,10 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         const uint32_t tmem_u = __reduce_or_sync(0xFFFFFFFFu, tmem_base);
         const int steps = p.tk / 16;
         bool ok = true;
-        for (int n = 0; ok && n <= n_items; ++n) {
+        for (int n = 0; ok && n < n_items + kLag; ++n) {
             if (n < n_items) {
-                const int b = n & 1;
-                const uint32_t ph = (uint32_t)((n >> 1) & 1);
+                const int b = n % kBufs;
+                const uint32_t ph = (uint32_t)((n / kBufs) & 1);
                 ok = mbar_wait(bar(kTmemEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 21);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
@@ -192,9 +204,9 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                                 (uint32_t)(k != 0), elected);
                 umma_commit_if(bar(kSFull, b), elected);
             }
-            if (n >= 1) {
-                const int m = n - 1, b = m & 1;
-                const uint32_t ph = (uint32_t)((m >> 1) & 1);
+            if (n >= kLag) {
+                const int m = n - kLag, b = m % kBufs;
+                const uint32_t ph = (uint32_t)((m / kBufs) & 1);
                 ok = mbar_wait(bar(kVFull, b), ph, abort_flag, p.dev_status, 23);
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
@@ -221,8 +233,8 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
         const int quarter = warp & 3;                                  // the TMEM lanes this warp may touch
         const float scale = (kD == 64 ? 0.125f : 0.17677669529663687f) * 1.4426950408889634f;   // log2(e) / sqrt(kD)
         bool ok = true;
-        for (int n = g; ok && n < n_items; n += 2) {
-            const uint32_t ph = (uint32_t)((n >> 1) & 1);
+        for (int n = g; ok && n < n_items; n += kBufs) {
+            const uint32_t ph = (uint32_t)((n / kBufs) & 1);
             const int item = first + n * stride;
             const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
             const int row = mt * kQRows + quarter * 32 + lane;         // token index inside the image
@@ -261,79 +273,86 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
             };
             {
                 // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
-                // row maximum from up to 64 columns per round trip, the second pass with the next 32 columns in
-                // flight while the current ones are exponentiated.
-                const int units = p.tk >> 5;            // whole units of 32 columns
-                const bool tail = (p.tk & 31) != 0;     // plus one chunk of 16
+                // row maximum from two units per round trip, the second pass with the next unit in flight while
+                // the current one is exponentiated.  A unit is U = 32 score columns (16 with four items in flight).
+                auto ld_unit = [&](uint32_t taddr, uint32_t (&r)[U]) {
+                    if constexpr (U == 32) tmem_ld_32x32b_x32(taddr, r);
+                    else tmem_ld_32x32b_x16(taddr, r);
+                };
+                const int units = p.tk / U;                      // whole units
+                const bool tail = U == 32 && (p.tk & 31) != 0;   // plus one chunk of 16
                 float m = -INFINITY;
                 if constexpr (kBias) {
                     // first pass of the biased form: t = s * scale + (bias + mask) * log2(e) replaces s in tensor memory,
                     // so the tables are read once
                     for (int u = 0; u < units; ++u) {
-                        uint32_t r[32];
-                        float bb[32];
-                        tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * u), r);
-                        load_bias(bb, 32 * u, 32);
+                        uint32_t r[U];
+                        float bb[U];
+                        ld_unit(t_lane + (uint32_t)(U * u), r);
+                        load_bias(bb, U * u, U);
                         tmem_wait_ld();
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
+                        for (int j = 0; j < U; ++j) {
                             const float t = fmaf(__uint_as_float(r[j]), scale, bb[j]);
                             r[j] = __float_as_uint(t);
-                            if (32 * u + j < p.tokens) m = fmaxf(m, t);
+                            if (U * u + j < p.tokens) m = fmaxf(m, t);
                         }
-                        uint32_t lo[16], hi[16];
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) { lo[j] = r[j]; hi[j] = r[16 + j]; }
-                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * u), lo);
-                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * u + 16), hi);
+                        for (int h = 0; h < U / 16; ++h) {
+                            uint32_t part[16];
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) part[j] = r[16 * h + j];
+                            tmem_st_32x32b_x16(t_lane + (uint32_t)(U * u + 16 * h), part);
+                        }
                     }
                     if (tail) {
                         uint32_t r[16];
                         float bb[16];
-                        tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
-                        load_bias(bb, 32 * units, 16);
+                        tmem_ld_32x32b_x16(t_lane + (uint32_t)(U * units), r);
+                        load_bias(bb, U * units, 16);
                         tmem_wait_ld();
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const float t = fmaf(__uint_as_float(r[j]), scale, bb[j]);
                             r[j] = __float_as_uint(t);
-                            if (32 * units + j < p.tokens) m = fmaxf(m, t);
+                            if (U * units + j < p.tokens) m = fmaxf(m, t);
                         }
-                        tmem_st_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                        tmem_st_32x32b_x16(t_lane + (uint32_t)(U * units), r);
                     }
                     tmem_wait_st();
-                }
-                for (int u0 = 0; !kBias && u0 < units; u0 += 2) {
-                    uint32_t r[2][32];
+                } else {
+                    for (int u0 = 0; u0 < units; u0 += 2) {
+                        uint32_t r[2][U];
 #pragma unroll
-                    for (int i = 0; i < 2; ++i)
-                        if (u0 + i < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u0 + i)), r[i]);
-                    tmem_wait_ld();
+                        for (int i = 0; i < 2; ++i)
+                            if (u0 + i < units) ld_unit(t_lane + (uint32_t)(U * (u0 + i)), r[i]);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int i = 0; i < 2; ++i)
-                        if (u0 + i < units) {
-                            if (32 * (u0 + i) + 32 <= p.tokens) {       // a unit of real keys only: no per-column test
-                                float m0 = m, m1 = -INFINITY;
+                        for (int i = 0; i < 2; ++i)
+                            if (u0 + i < units) {
+                                if (U * (u0 + i) + U <= p.tokens) {       // a unit of real keys only: no per-column test
+                                    float m0 = m, m1 = -INFINITY;
 #pragma unroll
-                                for (int j = 0; j < 32; j += 2) {
-                                    m0 = fmaxf(m0, __uint_as_float(r[i][j]));
-                                    m1 = fmaxf(m1, __uint_as_float(r[i][j + 1]));
+                                    for (int j = 0; j < U; j += 2) {
+                                        m0 = fmaxf(m0, __uint_as_float(r[i][j]));
+                                        m1 = fmaxf(m1, __uint_as_float(r[i][j + 1]));
+                                    }
+                                    m = fmaxf(m0, m1);
+                                } else {
+#pragma unroll
+                                    for (int j = 0; j < U; ++j)
+                                        if (U * (u0 + i) + j < p.tokens) m = fmaxf(m, __uint_as_float(r[i][j]));
                                 }
-                                m = fmaxf(m0, m1);
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j)
-                                    if (32 * (u0 + i) + j < p.tokens) m = fmaxf(m, __uint_as_float(r[i][j]));
                             }
-                        }
-                }
-                if (!kBias && tail) {
-                    uint32_t r[16];
-                    tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
-                    tmem_wait_ld();
+                    }
+                    if (tail) {
+                        uint32_t r[16];
+                        tmem_ld_32x32b_x16(t_lane + (uint32_t)(U * units), r);
+                        tmem_wait_ld();
 #pragma unroll
-                    for (int j = 0; j < 16; ++j)
-                        if (32 * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+                        for (int j = 0; j < 16; ++j)
+                            if (U * units + j < p.tokens) m = fmaxf(m, __uint_as_float(r[j]));
+                    }
                 }
                 // p = 2^(s * scale - m * scale) for 16 columns starting at col0: eight packed pairs
                 const float m_scaled = kBias ? m : m * scale;      // the biased maximum is in the exponent's domain already
@@ -357,32 +376,33 @@ __global__ void __launch_bounds__(kThreads, 1) attention_kernel(const __grid_con
                         w[j] = pack2<kBf16>(e0, e1);
                     }
                 };
-                // P's columns 16u .. 16u + 15 lie over S columns of units that have been read already
-                auto unit = [&](const uint32_t (&r)[32], int u) {
-                    uint32_t w[2][8];
-                    exp16(&r[0], 32 * u, w[0]);
-                    exp16(&r[16], 32 * u + 16, w[1]);
-                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u), w[0]);
-                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * u + 8), w[1]);
+                // P's columns of a unit lie over S columns of units that have been read already
+                auto unit = [&](const uint32_t (&r)[U], int u) {
+#pragma unroll
+                    for (int h = 0; h < U / 16; ++h) {
+                        uint32_t w[8];
+                        exp16(&r[16 * h], U * u + 16 * h, w);
+                        tmem_st_32x32b_x8(t_lane + (uint32_t)(U / 2 * u + 8 * h), w);
+                    }
                 };
-                uint32_t ra[32], rb[32];
-                if (units > 0) tmem_ld_32x32b_x32(t_lane, ra);
+                uint32_t ra[U], rb[U];
+                if (units > 0) ld_unit(t_lane, ra);
                 for (int u = 0; u < units; u += 2) {
                     tmem_wait_ld();
-                    if (u + 1 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 1)), rb);
+                    if (u + 1 < units) ld_unit(t_lane + (uint32_t)(U * (u + 1)), rb);
                     unit(ra, u);
                     if (u + 1 < units) {
                         tmem_wait_ld();
-                        if (u + 2 < units) tmem_ld_32x32b_x32(t_lane + (uint32_t)(32 * (u + 2)), ra);
+                        if (u + 2 < units) ld_unit(t_lane + (uint32_t)(U * (u + 2)), ra);
                         unit(rb, u + 1);
                     }
                 }
                 if (tail) {
                     uint32_t r[16], w[8];
-                    tmem_ld_32x32b_x16(t_lane + (uint32_t)(32 * units), r);
+                    tmem_ld_32x32b_x16(t_lane + (uint32_t)(U * units), r);
                     tmem_wait_ld();
-                    exp16(r, 32 * units, w);
-                    tmem_st_32x32b_x8(t_lane + (uint32_t)(16 * units), w);
+                    exp16(r, U * units, w);
+                    tmem_st_32x32b_x8(t_lane + (uint32_t)(U / 2 * units), w);
                 }
                 sum += sum1;
             }
@@ -445,10 +465,11 @@ elsa_status make_map_qkv(CUtensorMap* map, const void* qkv, int images, int toke
     return ELSA_OK;
 }
 
-template <bool kBf16, int kD, bool kBias>
+template <bool kBf16, int kD, bool kBias, int kBufs>
 elsa_status launch(const AttnParams& p, int images, int heads, cudaStream_t stream, const DeviceInfo& dev)
 {
-    auto kernel = attention_kernel<kBf16, kD, kBias>;
+    constexpr int kSmemBytes = Shape<kBufs>::kSmemBytes, kThreads = Shape<kBufs>::kThreads;
+    auto kernel = attention_kernel<kBf16, kD, kBias, kBufs>;
     static std::atomic<bool> attr_set[64];
     const int slot = dev.device & 63;
     if (!attr_set[slot].load(std::memory_order_acquire)) {
@@ -501,8 +522,8 @@ elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int he
     p.m_tiles = (tokens + kQRows - 1) / kQRows;
     p.heads = heads;
     p.items = images * heads * p.m_tiles;
-    // O (head_dim columns) over the part of S that P does not cover (P: tk / 2 columns from 0); small images: right after S
-    p.o_col = p.tk >= 128 ? (p.tk / 2 + 31) / 32 * 32 : p.tk;
+    // O (head_dim columns) over the part of S that P does not cover (P: tk / 2 columns from 0; S is dead by then)
+    p.o_col = (p.tk / 2 + 31) / 32 * 32;
     const uint32_t fmt = dtype == ELSA_BF16 ? 1u : 0u;
     p.idesc_s = (1u << 4) | (fmt << 7) | (fmt << 10) | ((uint32_t)(p.tk >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
     p.idesc_o = (1u << 4) | (fmt << 7) | (fmt << 10) | (1u << 16) | ((uint32_t)(head_dim >> 3) << 17) | ((uint32_t)(kQRows >> 4) << 24);
@@ -511,12 +532,15 @@ elsa_status launch_attention(const uint16_t* qkv, int images, int tokens, int he
     if ((st = make_map_qkv(&p.map_q, qkv, images, tokens, dim, head_dim, kQRows, "q")) != ELSA_OK) return st;
     if ((st = make_map_qkv(&p.map_kv, qkv, images, tokens, dim, head_dim, (uint32_t)p.tk, "k, v")) != ELSA_OK) return st;
     const bool bf = dtype == ELSA_BF16, biased = bias != nullptr;
+    const bool four = p.tk <= 128;       // short chains: four items in flight per CTA
+#define ELSA_ATTN(D, B, N) (bf ? launch<true, D, B, N>(p, images, heads, stream, dev) : launch<false, D, B, N>(p, images, heads, stream, dev))
     if (head_dim == 64) {
-        if (biased) return bf ? launch<true, 64, true>(p, images, heads, stream, dev) : launch<false, 64, true>(p, images, heads, stream, dev);
-        return bf ? launch<true, 64, false>(p, images, heads, stream, dev) : launch<false, 64, false>(p, images, heads, stream, dev);
+        if (biased) return four ? ELSA_ATTN(64, true, 4) : ELSA_ATTN(64, true, 2);
+        return four ? ELSA_ATTN(64, false, 4) : ELSA_ATTN(64, false, 2);
     }
-    if (biased) return bf ? launch<true, 32, true>(p, images, heads, stream, dev) : launch<false, 32, true>(p, images, heads, stream, dev);
-    return bf ? launch<true, 32, false>(p, images, heads, stream, dev) : launch<false, 32, false>(p, images, heads, stream, dev);
+    if (biased) return four ? ELSA_ATTN(32, true, 4) : ELSA_ATTN(32, true, 2);
+    return four ? ELSA_ATTN(32, false, 4) : ELSA_ATTN(32, false, 2);
+#undef ELSA_ATTN
 }
 
 }  // namespace elsa
