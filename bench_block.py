@@ -4,6 +4,7 @@ with the levels the stack workload gives its four linears, chained (a block's y 
     python bench_block.py [--blocks 12] [--batch 256] [--reps 5] [--out bench_out/block.json]
     python bench_block.py --compare          # dense 4:4 against N:4 configurations at the paper's operating points
     python bench_block.py --swin             # the 24 blocks of Swin-B at batch 128, stage by stage
+    python bench_block.py --latency-cost     # F(alpha) with measured latencies as the cost table (Sec. 3.2)
 
 Two timings: with the library's multi-head self-attention (elsa_vit_encoder: the encoder blocks of DeiT-B as
 they run, without patch embedding, final norm and classifier head), and with the stand-in a = V in its place (the linear and
@@ -207,6 +208,71 @@ def run_swin(batch=128, reps=5, pack=1):
             "families_profiled_pass": families, "levels": ["%d:%d" % (l.N, l.M) for l in layers]}
 
 
+def latency_cost(args):
+    """F(alpha) of Sec. 3.2 with measured latency in place of MACs: time each DeiT-B linear shape at each level of the
+    N:4 space through elsa_nm_linear, hand the table (in microseconds) to the library's cost model and two-step
+    sampler, and compare the cost it predicts for the drawn configurations with the encoder's measured time."""
+    import numpy as np
+    dtype = torch.bfloat16
+    rows = args.batch * 197
+    shapes = {"qkv": (768, 2304), "proj": (768, 768), "fc1": (768, 3072), "fc2": (3072, 768)}
+    levels = [(1, 4), (2, 4), (4, 4)]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    table = {}
+    for name, (k, o) in shapes.items():
+        X = synth.randn((rows, k), 5, 1.0, dtype, "cuda")
+        W = synth.randn((o, k), 6, synth.W_STD, dtype, "cuda")
+        b = synth.randn((o,), 7, synth.B_STD, dtype, "cuda")
+        Y = torch.empty((rows, o), dtype=dtype, device="cuda")
+        row = []
+        for N, M in levels:
+            vals, idx = lib.elsa_nm_compress(W, N, M)
+            ws = lib.alloc_workspace(lib.elsa_workspace_bytes(rows, k, o, N, M, lib.BF16))
+            # sustained latency: many calls back to back between one pair of events, as the layer runs inside a model
+            # (a single cold call runs at a clock the power cap does not allow for long)
+            calls = 40
+            for _ in range(10):
+                lib.elsa_nm_linear(X, vals, idx, b, o, k, N, M, Y=Y, workspace=ws, dev_status=status)
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(calls):
+                lib.elsa_nm_linear(X, vals, idx, b, o, k, N, M, Y=Y, workspace=ws, dev_status=status)
+            e1.record()
+            torch.cuda.synchronize()
+            row.append(e0.elapsed_time(e1) * 1e3 / calls)
+        table[name] = row
+        del X, Y
+    order = ["qkv", "proj", "fc1", "fc2"] * args.blocks
+    cost = [table[n] for n in order]
+    dense = run(args.blocks, args.batch, args.reps, levels=[(4, 4)] * len(order), stand_in=False)["encoder_blocks_with_attention"]
+    # what is not a pruned linear, calibrated at the dense end: the dense encoder's time minus its linears' table cost
+    # (attention, the row-wise kernels, and the gaps between dependent launches that a per-kernel sum does not see)
+    fixed = dense["ms_per_pass"] * 1e3 - sum(c[2] for c in cost)
+    other_kernels = sum(v["ms"] for k, v in dense["families_profiled_pass"].items() if k in ("attention", "block_rowwise")) * 1e3
+    lower = lib.elsa_config_cost(cost, [0] * len(cost), fixed)
+    upper = lib.elsa_config_cost(cost, [2] * len(cost), fixed)
+    n_int = 8
+    out = []
+    rng = np.random.default_rng(0)
+    for interval in (1, 4, 6):
+        u = [(interval + 0.5) / n_int] + [float(v) for v in rng.random(len(cost))]
+        choice, got_interval = lib.elsa_two_step_sample(cost, [[1.0, 1.0, 1.0]] * len(cost), fixed, upper, n_int, 1.0, u)
+        picked = [levels[c] for c in choice]
+        predicted = lib.elsa_config_cost(cost, choice, fixed)
+        m = run(args.blocks, args.batch, args.reps, levels=picked, stand_in=False)["encoder_blocks_with_attention"]
+        out.append({"interval": got_interval, "interval_bounds_us": [lower + (upper - lower) * got_interval / n_int,
+                                                                     lower + (upper - lower) * (got_interval + 1) / n_int],
+                    "levels": ["%d:%d" % lv for lv in picked], "predicted_us": predicted, "measured_us": m["ms_per_pass"] * 1e3,
+                    "measured_over_predicted": m["ms_per_pass"] * 1e3 / predicted})
+    return {"workload": "deit_b_encoder_blocks_b%d" % args.batch,
+            "cost_unit": "microseconds per call of elsa_nm_linear, 40 calls back to back",
+            "levels": ["%d:%d" % lv for lv in levels], "latency_table_us": table, "fixed_cost_us": fixed,
+            "attention_and_rowwise_kernels_us": other_kernels,
+            "dense_encoder_us": dense["ms_per_pass"] * 1e3, "cost_range_us": [lower, upper], "draws": out}
+
+
 def compare(args):
     import bench
     layers = synth.deit_b_stack(args.batch)[:4 * args.blocks]
@@ -238,9 +304,12 @@ def main():
     ap.add_argument("--out", default="bench_out/block.json")
     ap.add_argument("--compare", action="store_true", help="dense 4:4 against sampled N:4 configurations at 7.0 and 6.0 GMACs")
     ap.add_argument("--swin", action="store_true", help="the 24 blocks of Swin-B at batch 128")
+    ap.add_argument("--latency-cost", action="store_true", help="measured latencies as the cost table of F(alpha)")
     ap.add_argument("--pack", type=int, default=1, help="--swin: windows per attention item (1 or 2)")
     args = ap.parse_args()
-    if args.swin:
+    if args.latency_cost:
+        rec = latency_cost(args)
+    elif args.swin:
         rec = run_swin(128, args.reps, args.pack)
     elif args.compare:
         rec = compare(args)
