@@ -7,7 +7,9 @@ x level in {1:4, 2:4, 1:8, 2:8, 4:8, 1:16, 2:16, 4:16, 8:16} x {fp16, bf16}: per
 CUDA-event time of elsa_nm_linear (weight-image rebuild + GEMM) with L2 flushed between repetitions
 (small points are otherwise L2-resident), dense-equivalent and kept TFLOP/s, algorithmic GB/s and
 the fraction of the layer's roofline; per weight shape, level and dtype the time and GB/s (bytes
-read + written) of elsa_nm_compress.  Writes a JSON list and prints a short table.
+read + written) of elsa_nm_compress.  For scale, under the same timing: an empty kernel (what the method itself
+costs) and the library's dense product of every (rows, K, O) in bf16 (torch.matmul, i.e. cuBLAS; context, not a
+path of this library).  Writes a JSON list and prints a short table.
 """
 from __future__ import annotations
 
@@ -93,6 +95,21 @@ def main():
                             "algorithmic_gbs": alg / ms / 1e6, "roofline_ms": roof, "roofline_frac": roof / ms,
                             "bound": "tensor" if l.kept_flops / (tf * 1e12) >= alg / (hbm * 1e9) else "hbm"})
             del X, Y
+    # scale: what the timing method costs for an empty kernel, and the library's dense GEMM on the same shapes
+    tiny = torch.zeros(32, device="cuda")
+    tiny.add_(1)
+    ms, best = timed(lambda: tiny.add_(1), max(args.reps, 9), flush)
+    results.append({"op": "empty_kernel", "ms": ms, "ms_min": best})
+    for rows in ([synth.SWEEP_ROWS[0]] if args.quick else synth.SWEEP_ROWS):
+        for K, O in synth.SWEEP_SHAPES:
+            X = synth.randn((rows, K), 1, synth.X_STD, torch.bfloat16, "cuda")
+            W = synth.randn((O, K), 2, synth.W_STD, torch.bfloat16, "cuda")
+            Y = torch.empty((rows, O), dtype=torch.bfloat16, device="cuda")
+            run = lambda: torch.matmul(X, W.t(), out=Y)
+            run(); run()
+            ms, best = timed(run, args.reps, flush)
+            results.append({"op": "library_dense", "dtype": "bf16", "rows": rows, "in": K, "out": O, "ms": ms, "ms_min": best})
+            del X, Y
     assert int(status.item()) == 0
     os.makedirs(os.path.dirname(args.out) or ".", exist_ok=True)
     json.dump({"peaks": {"hbm_gbs": hbm, "bf16_tflops": tf, "kind": kind}, "results": results}, open(args.out, "w"), indent=0)
@@ -106,10 +123,10 @@ def main():
 
 
     if args.summary:
-        write_summary(args.summary, hbm, tf, kind, lin, cmp_)
+        write_summary(args.summary, hbm, tf, kind, lin, cmp_, results)
 
 
-def write_summary(path, hbm, tf, kind, lin, cmp_):
+def write_summary(path, hbm, tf, kind, lin, cmp_, results):
     med = statistics.median
     out = ["# Shape / sparsity sweep (%d linear points, %d compress points) -- summary" % (len(lin), len(cmp_)), "",
            "Command: `python bench_sweep.py --out bench_out/sweep.json --summary <this file>` (B200;",
@@ -136,6 +153,25 @@ def write_summary(path, hbm, tf, kind, lin, cmp_):
             % (med(r["gbs"] for r in cmp_), max(r["gbs"] for r in cmp_)),
             "are 1.2-8.4 MB, so a single launch lasts a few microseconds and is latency-bound; tables of weights go",
             "through `elsa_vit_compress`, one launch for all of them.", ""]
+    empty = [r for r in results if r["op"] == "empty_kernel"]
+    dense = [r for r in results if r["op"] == "library_dense"]
+    if empty and dense:
+        out += ["For scale, same timing method: an empty kernel reads %.1f us (the floor every point carries).  Microseconds,"
+                % (empty[0]["ms"] * 1e3),
+                "bf16: the library's dense product (torch.matmul) / this library at 2:8 / at 4:8, per shape and rows:", "",
+                "| K, O | " + " | ".join("rows %d" % R for R in synth.SWEEP_ROWS) + " |", "|---|" + "---|" * len(synth.SWEEP_ROWS)]
+        for K, O in synth.SWEEP_SHAPES:
+            row = ["%d, %d" % (K, O)]
+            for R in synth.SWEEP_ROWS:
+                d = [r["ms"] * 1e3 for r in dense if r["rows"] == R and r["in"] == K and r["out"] == O]
+                ours = []
+                for lv in ("2:8", "4:8"):
+                    v = [r["ms"] * 1e3 for r in lin if r["rows"] == R and r["in"] == K and r["out"] == O
+                         and r["level"] == lv and r["dtype"] == "bf16"]
+                    ours.append("%.1f" % v[0] if v else "-")
+                row.append("%s / %s / %s" % ("%.1f" % d[0] if d else "-", ours[0], ours[1]))
+            out.append("| " + " | ".join(row) + " |")
+        out.append("")
     with open(path, "w") as f:
         f.write("\n".join(out))
 
