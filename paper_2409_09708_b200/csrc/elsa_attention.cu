@@ -20,7 +20,8 @@
 // Persistent: one CTA per SM walks the items with the stride of the grid, with several items in flight: two for up
 // to 256 keys, four for up to 128 (Swin's windows), each with its own shared-memory stage (Q, K, V), its own share
 // of tensor memory (256 or 128 columns) and its own group of four softmax warps: item n uses stage, share and group
-// n % 2 (n % 4).  The producer warp loads ahead as stages come free; the MMA warp issues S of item n, then P V of the
+// n % 2 (n % 4).  The producer warp loads ahead as stages come free (Q and K of a stage after the scores of its
+// previous item, V after that item's second product); the MMA warp issues S of item n, then P V of the
 // oldest item whose probabilities are due, so one group's softmax runs under the others' products and epilogues.
 // Every wait is bounded as in the GEMM kernels.
 #include <atomic>
@@ -121,9 +122,9 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = smem_base + kBufs * kStageBytes;
-    // per buffer b: +0 qk_full, +8 v_full, +16 smem_empty, +24 s_full, +32 p_full, +40 o_full, +48 tmem_empty
+    // per buffer b: +0 qk_full, +8 v_full, +16 qk_empty, +24 s_full, +32 p_full, +40 o_full, +48 tmem_empty, +56 v_empty
     auto bar = [&](int which, int b) { return bars + (uint32_t)(64 * b + 8 * which); };
-    enum { kQkFull = 0, kVFull, kSmemEmpty, kSFull, kPFull, kOFull, kTmemEmpty };
+    enum { kQkFull = 0, kVFull, kQkEmpty, kSFull, kPFull, kOFull, kTmemEmpty, kVEmpty };
     const uint32_t tmem_holder_addr = bars + 64 * kBufs;
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(smem_raw + (tmem_holder_addr - smem_u32(smem_raw)));
     volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem_raw + (bars + 64 * kBufs + 8 - smem_u32(smem_raw)));
@@ -137,7 +138,8 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
             for (int b = 0; b < kBufs; ++b) {
                 mbar_init(bar(kQkFull, b), 1);
                 mbar_init(bar(kVFull, b), 1);
-                mbar_init(bar(kSmemEmpty, b), 1);
+                mbar_init(bar(kQkEmpty, b), 1);
+                mbar_init(bar(kVEmpty, b), 1);
                 mbar_init(bar(kSFull, b), 1);
                 mbar_init(bar(kPFull, b), kGroupWarps);
                 mbar_init(bar(kOFull, b), 1);
@@ -160,23 +162,42 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
         // ------------------------------------------------ TMA producer
         const bool elected = elect_one();
         bool ok = true;
-        for (int n = 0; ok && n < n_items; ++n) {
-            const int b = n % kBufs;
-            const uint32_t ph = (uint32_t)((n / kBufs) & 1);
-            ok = mbar_wait(bar(kSmemEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 20);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            const int item = first + n * stride;
-            const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
-            const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
-            if (elected) {
-                mbar_arrive_expect_tx(bar(kQkFull, b), (uint32_t)(kItemQBytes + p.tk * kHeadDim * 2));
-                tma_load_3d(q_smem, &p.map_q, bar(kQkFull, b), head * kHeadDim, mt * kQRows, img);
-                tma_load_3d(q_smem + kQBytes, &p.map_kv, bar(kQkFull, b), p.dim + head * kHeadDim, 0, img);
-                mbar_arrive_expect_tx(bar(kVFull, b), (uint32_t)(p.tk * kHeadDim * 2));
-                tma_load_3d(q_smem + kQBytes + kKvBytesMax, &p.map_kv, bar(kVFull, b), 2 * p.dim + head * kHeadDim, 0, img);
+        // Q and K of a stage are free as soon as the scores of its previous item are complete, V only after that item's
+        // second product.  The loop asks for Q and K of item n, then for V of item n - 1: the order in which the MMA
+        // warp frees them (S of item n - kBufs, then P V of item n - 1 - kBufs), so the next item's Q and K arrive under
+        // the softmax, off the chain of the buffer, and no wait holds back a load whose stage is free already.
+        for (int n = 0; ok && n <= n_items; ++n) {
+            if (n < n_items) {
+                const int b = n % kBufs;
+                const uint32_t ph = (uint32_t)((n / kBufs) & 1);
+                ok = mbar_wait(bar(kQkEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 20);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                const int item = first + n * stride;
+                const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
+                const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
+                if (elected) {
+                    mbar_arrive_expect_tx(bar(kQkFull, b), (uint32_t)(kItemQBytes + p.tk * kHeadDim * 2));
+                    tma_load_3d(q_smem, &p.map_q, bar(kQkFull, b), head * kHeadDim, mt * kQRows, img);
+                    tma_load_3d(q_smem + kQBytes, &p.map_kv, bar(kQkFull, b), p.dim + head * kHeadDim, 0, img);
+                }
+                __syncwarp();
             }
-            __syncwarp();
+            if (n >= 1) {
+                const int m = n - 1, b = m % kBufs;
+                const uint32_t ph = (uint32_t)((m / kBufs) & 1);
+                ok = mbar_wait(bar(kVEmpty, b), ph ^ 1u, abort_flag, p.dev_status, 27);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                const int item = first + m * stride;
+                const int head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
+                const uint32_t q_smem = smem_base + (uint32_t)(b * kStageBytes);
+                if (elected) {
+                    mbar_arrive_expect_tx(bar(kVFull, b), (uint32_t)(p.tk * kHeadDim * 2));
+                    tma_load_3d(q_smem + kQBytes + kKvBytesMax, &p.map_kv, bar(kVFull, b), 2 * p.dim + head * kHeadDim, 0, img);
+                }
+                __syncwarp();
+            }
         }
     } else if (warp == 1) {
         // ------------------------------------------------ MMA issuer: S of item n, then P V of item n - 1
@@ -203,6 +224,7 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
                     umma_f16_if(tmem_u + (uint32_t)(b * kBufCols), a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), p.idesc_s,
                                 (uint32_t)(k != 0), elected);
                 umma_commit_if(bar(kSFull, b), elected);
+                umma_commit_if(bar(kQkEmpty, b), elected);     // Q and K of the stage have been read
             }
             if (n >= kLag) {
                 const int m = n - kLag, b = m % kBufs;
@@ -223,7 +245,7 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
                     umma_f16_ts_if(t_buf + (uint32_t)p.o_col, t_buf + (uint32_t)(8 * k), v_desc + (uint64_t)(k * (16 * kD * 2 >> 4)),
                                    p.idesc_o, (uint32_t)(k != 0), elected);
                 umma_commit_if(bar(kOFull, b), elected);
-                umma_commit_if(bar(kSmemEmpty, b), elected);   // both products of the item have read its stage
+                umma_commit_if(bar(kVEmpty, b), elected);      // V of the stage has been read
             }
         }
         __syncwarp();
