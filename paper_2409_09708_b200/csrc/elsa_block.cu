@@ -1,8 +1,9 @@
 // Elementwise and row-wise kernels of the transformer block around the four N:M linears (ELSA, Sec. 3: the
 // pruned modules qkv, proj, fc1, fc2 sit in the standard pre-norm ViT block; Sec. 4.2 measures whole models):
 // LayerNorm, residual add (alone or followed by LayerNorm in the same pass), GELU in place, and the copy of a
-// column range.  All of them are HBM-bound streaming kernels: 16-byte loads and stores, one warp per token row
-// for the row-wise ones, fp32 arithmetic, one rounding to the 16-bit type per stored value.
+// column range.  All of them are HBM-bound streaming kernels: 16-byte loads and stores, fp32 arithmetic, one
+// rounding to the 16-bit type per stored value; the row-wise ones give a row to a warp, or, for the model widths
+// (128, 256, 512, 768, 1024), several rows at a time to groups of 16 or 32 lanes.
 #include "elsa_internal.h"
 
 #include <cuda_bf16.h>
@@ -179,6 +180,111 @@ layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint1
     }
 }
 
+// Rows of exactly kLanes * kVpl vectors of eight values (dim = 128, 256, 512, 768, 1024): a group of kLanes lanes owns a row and
+// takes kUnroll rows at a time, all of their loads requested before the first is used.  With one row per warp a
+// short row leaves (resident warps x row bytes) in flight per SM, a fraction of what the memory latency asks for.
+// Same arithmetic per row as layer_norm_kernel (sum, mean, squared deviations about it, one rounding).
+template <bool kBf16, bool kAdd, int kLanes, int kVpl, int kUnroll>
+__global__ void __launch_bounds__(kWarpsPerBlock * 32)
+layer_norm_rows_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* __restrict__ gain,
+                       const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, float eps, const RowMap map)
+{
+    constexpr int kGroups = 32 / kLanes;               // rows side by side in a warp
+    constexpr int kRowsPerStep = kGroups * kUnroll;
+    constexpr int kDim = kLanes * kVpl * 8;
+    pdl_wait_for_predecessors();
+    pdl_release_successors();
+    const int lane = threadIdx.x & 31;
+    const int sub = lane % kLanes, grp = lane / kLanes;
+    const float inv_dim = 1.0f / (float)kDim;
+    // this lane's vectors of a row are the same in every row: gain and bias stay in registers
+    uint4 g4[kVpl], b4[kVpl];
+    if (Yn != nullptr) {
+#pragma unroll
+        for (int c = 0; c < kVpl; ++c) {
+            g4[c] = __ldg(reinterpret_cast<const uint4*>(gain) + sub + kLanes * c);
+            b4[c] = __ldg(reinterpret_cast<const uint4*>(beta) + sub + kLanes * c);
+        }
+    }
+    auto group_sum = [&](float v) {
+#pragma unroll
+        for (int o = kLanes / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        return v;
+    };
+    const long long steps = ((long long)rows + kRowsPerStep - 1) / kRowsPerStep;
+    for (long long step = (long long)blockIdx.x * kWarpsPerBlock + (threadIdx.x >> 5); step < steps;
+         step += (long long)gridDim.x * kWarpsPerBlock) {
+        uint4 x[kUnroll][kVpl];
+        int mapped[kUnroll];
+        int row_of[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const long long r = step * kRowsPerStep + u * kGroups + grp;
+            row_of[u] = r < rows ? (int)r : -1;
+            mapped[u] = row_of[u] >= 0 ? window_row(map, row_of[u]) : 0;
+        }
+        // every load of the step first
+        uint4 w[kAdd ? kUnroll : 1][kVpl];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+#pragma unroll
+            for (int c = 0; c < kVpl; ++c) {
+                x[u][c] = make_uint4(0u, 0u, 0u, 0u);
+                if constexpr (kAdd) w[u][c] = make_uint4(0u, 0u, 0u, 0u);
+                if (row_of[u] >= 0) {
+                    const size_t src = (size_t)(map.on_input ? mapped[u] : row_of[u]) * (size_t)kDim;
+                    x[u][c] = reinterpret_cast<const uint4*>(A + src)[sub + kLanes * c];
+                    if constexpr (kAdd) w[u][c] = reinterpret_cast<const uint4*>(R + (size_t)row_of[u] * (size_t)kDim)[sub + kLanes * c];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < kVpl; ++c) {
+                float f[8];
+                unpack8<kBf16>(x[u][c], f);
+                if constexpr (kAdd) {
+                    float fr[8];
+                    unpack8<kBf16>(w[u][c], fr);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) f[e] += fr[e];
+                    x[u][c] = pack8<kBf16>(f);
+                    if (row_of[u] >= 0) reinterpret_cast<uint4*>(S + (size_t)row_of[u] * (size_t)kDim)[sub + kLanes * c] = x[u][c];
+                    unpack8<kBf16>(x[u][c], f);          // the statistics are those of the row as stored
+                }
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sum += f[e];
+            }
+            if (Yn == nullptr) continue;
+            const float mean = group_sum(sum) * inv_dim;
+            float sq = 0.f;
+#pragma unroll
+            for (int c = 0; c < kVpl; ++c) {
+                float f[8];
+                unpack8<kBf16>(x[u][c], f);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) sq += (f[e] - mean) * (f[e] - mean);
+            }
+            const float rstd = 1.0f / sqrtf(group_sum(sq) * inv_dim + eps);
+            if (row_of[u] >= 0) {
+                uint4* y4 = reinterpret_cast<uint4*>(Yn + (size_t)(map.on_output ? mapped[u] : row_of[u]) * (size_t)kDim);
+#pragma unroll
+                for (int c = 0; c < kVpl; ++c) {
+                    float f[8], g[8], b[8];
+                    unpack8<kBf16>(x[u][c], f);
+                    unpack8<kBf16>(g4[c], g);
+                    unpack8<kBf16>(b4[c], b);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) f[e] = (f[e] - mean) * rstd * g[e] + b[e];
+                    y4[sub + kLanes * c] = pack8<kBf16>(f);
+                }
+            }
+        }
+    }
+}
+
 // Y = act(Y) in place, eight values per thread and step.
 template <bool kBf16>
 __global__ void __launch_bounds__(256) act_inplace_kernel(uint16_t* Y, long long vecs, int act)
@@ -232,10 +338,30 @@ elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S,
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
     if (rows <= 0) return ELSA_OK;
-    const unsigned grid = streaming_grid(rows, kWarpsPerBlock, dev);
     const dim3 block(kWarpsPerBlock * 32);
     const bool add = R != nullptr;
     ProfileScope scope(ELSA_KERNEL_BLOCK_ROWWISE, stream);
+    // the model widths: several rows per warp in flight
+#define ELSA_LN_ROWS(LANES, VPL, UNROLL)                                                                                  \
+    do {                                                                                                                  \
+        const long long steps = ((long long)rows + (32 / LANES) * UNROLL - 1) / ((32 / LANES) * UNROLL);                  \
+        const unsigned g = streaming_grid(steps, kWarpsPerBlock, dev);                                                    \
+        if (dtype == ELSA_BF16) {                                                                                         \
+            if (add) launch_pdl(layer_norm_rows_kernel<true, true, LANES, VPL, UNROLL>, dim3(g), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, eps, map);   \
+            else launch_pdl(layer_norm_rows_kernel<true, false, LANES, VPL, UNROLL>, dim3(g), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, eps, map);     \
+        } else {                                                                                                          \
+            if (add) launch_pdl(layer_norm_rows_kernel<false, true, LANES, VPL, UNROLL>, dim3(g), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, eps, map);  \
+            else launch_pdl(layer_norm_rows_kernel<false, false, LANES, VPL, UNROLL>, dim3(g), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, eps, map);    \
+        }                                                                                                                 \
+        return launched(add ? "residual_add_layer_norm" : "layer_norm");                                                  \
+    } while (0)
+    if (dim == 128) ELSA_LN_ROWS(16, 1, 4);
+    if (dim == 256) ELSA_LN_ROWS(32, 1, 4);
+    if (dim == 512) ELSA_LN_ROWS(32, 2, 2);
+    if (dim == 1024) ELSA_LN_ROWS(32, 4, 2);
+    if (dim == 768) ELSA_LN_ROWS(32, 3, 2);
+#undef ELSA_LN_ROWS
+    const unsigned grid = streaming_grid(rows, kWarpsPerBlock, dev);
     if (dtype == ELSA_BF16) {
         if (add) launch_pdl(layer_norm_kernel<true, true>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);
         else launch_pdl(layer_norm_kernel<true, false>, dim3(grid), block, 0, stream, 1, A, R, S, gain, beta, Yn, rows, dim, eps, map);

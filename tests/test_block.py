@@ -220,6 +220,21 @@ def test_block_matches_oracle_on_every_kernel_family(lib, variant, levels, dtype
 
 
 @pytest.mark.gpu
+@pytest.mark.parametrize("levels", [SPARSE_LEVELS, MIXED_LEVELS], ids=["sparse", "mixed"])
+@pytest.mark.parametrize("dim", [128, 512, 768, 1024])
+def test_row_widths_of_the_row_wise_kernels(lib, dim, levels):
+    # 128, 256 (above), 512 and 1024 take the several-rows-per-warp LayerNorm, 768 the one-row-per-warp one; 77 rows
+    # leave a ragged last step for every rows-per-step (8, 4, 2); sparse proj / fc2 make the add-and-normalise form run
+    dtype = torch.bfloat16
+    rows, mlp = 77, 512
+    host, p = make_params(dim, mlp, levels, dtype, 310 + dim)
+    x = synth.randn((rows, dim), 9, 1.25, dtype)
+    x[3] = -0.5
+    got = run_block(lib, x, host, levels, mlp)
+    check_rows(got, x, p, dtype, np.arange(rows))
+
+
+@pytest.mark.gpu
 def test_rows_longer_than_the_register_cache(lib):
     # dim > 1024: LayerNorm re-reads the part of the row it does not keep in registers
     dtype = torch.bfloat16
