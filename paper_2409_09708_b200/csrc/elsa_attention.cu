@@ -261,10 +261,6 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
             const int mt = item % p.m_tiles, head = (item / p.m_tiles) % p.heads, img = item / (p.m_tiles * p.heads);
             const int row = mt * kQRows + quarter * 32 + lane;         // token index inside the image
             const uint32_t t_lane = tmem_base + (uint32_t)(g * kBufCols) + ((uint32_t)(quarter * 32) << 16);
-            ok = mbar_wait(bar(kSFull, g), ph, abort_flag, p.dev_status, 25);
-            ok = __all_sync(0xFFFFFFFFu, ok);
-            if (!ok) break;
-            tc_fence_after();
             float sum = 0.f;
             // biased form: what is exponentiated is s * scale + (bias + mask) * log2(e); the tables' rows of this lane
             const float* brow = nullptr;
@@ -293,6 +289,25 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
                     bb[4 * v + 2] = b4.z * 1.4426950408889634f; bb[4 * v + 3] = b4.w * 1.4426950408889634f;
                 }
             };
+            // The bias table's values of one unit, as loaded (no arithmetic on them here, so a request stays in flight
+            // until the values are used): the first unit is asked for before the scores are waited for, every other
+            // one while the unit before it is worked on, which takes most of the L2 latency out of the item's chain.
+            // The mask (shifted windows only) is read where it is used: a second array across the wait would spill.
+            constexpr int kReq = kBias ? Shape<kBufs>::kUnit : 1;
+            float bq[kReq];
+            auto request = [&](int col0) {
+#pragma unroll
+                for (int v = 0; v < kReq / 4; ++v) {
+                    float4 b4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (brow != nullptr && col0 + 4 * v < p.bias_pitch) b4 = __ldg(reinterpret_cast<const float4*>(brow + col0) + v);
+                    bq[4 * v] = b4.x; bq[4 * v + 1] = b4.y; bq[4 * v + 2] = b4.z; bq[4 * v + 3] = b4.w;
+                }
+            };
+            if constexpr (kBias) request(0);
+            ok = mbar_wait(bar(kSFull, g), ph, abort_flag, p.dev_status, 25);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after();
             {
                 // Tensor-memory reads are waited for all at once, so the loads of a pass are issued in batches: the
                 // row maximum from two units per round trip, the second pass with the next unit in flight while
@@ -311,7 +326,16 @@ __global__ void __launch_bounds__(Shape<kBufs>::kThreads, 1) attention_kernel(co
                         uint32_t r[U];
                         float bb[U];
                         ld_unit(t_lane + (uint32_t)(U * u), r);
-                        load_bias(bb, U * u, U);
+#pragma unroll
+                        for (int v = 0; v < U / 4; ++v) {
+                            float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (mrow != nullptr && U * u + 4 * v < p.bias_pitch) m4 = __ldg(reinterpret_cast<const float4*>(mrow + U * u) + v);
+                            bb[4 * v] = (bq[4 * v] + m4.x) * 1.4426950408889634f;
+                            bb[4 * v + 1] = (bq[4 * v + 1] + m4.y) * 1.4426950408889634f;
+                            bb[4 * v + 2] = (bq[4 * v + 2] + m4.z) * 1.4426950408889634f;
+                            bb[4 * v + 3] = (bq[4 * v + 3] + m4.w) * 1.4426950408889634f;
+                        }
+                        if (u + 1 < units) request(U * (u + 1));
                         tmem_wait_ld();
 #pragma unroll
                         for (int j = 0; j < U; ++j) {
