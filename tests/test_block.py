@@ -502,16 +502,32 @@ SWIN_CASES = [(2, 14, 14, 7, 0, 2, 32), (2, 14, 14, 7, 3, 2, 32), (1, 28, 28, 7,
 @pytest.mark.parametrize("dtype", [torch.bfloat16, torch.float16], ids=["bf16", "f16"])
 @pytest.mark.parametrize("case", SWIN_CASES, ids=["%dx%dx%d_w%d_s%d_h%d_d%d" % c for c in SWIN_CASES])
 def test_swin_block_matches_oracle(lib, case, dtype, pack):
+    run_swin_case(lib, case, dtype, pack, MIXED_LEVELS)
+
+
+# the grids, widths and head counts of Swin-B's stages 1, 3 and 4 (window 7; stage 4's grid is one window, so it is
+# never shifted), a few images each: 64 window positions with their own masks, rows of 128 / 512 / 1024 values
+SWIN_B_STAGE_CASES = [(4, 56, 56, 7, 3, 4, 32), (16, 14, 14, 7, 3, 16, 32), (32, 7, 7, 7, 0, 32, 32)]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("levels", [SPARSE_LEVELS, MIXED_LEVELS], ids=["sparse", "mixed"])
+@pytest.mark.parametrize("case", SWIN_B_STAGE_CASES, ids=["%dx%dx%d_w%d_s%d_h%d_d%d" % c for c in SWIN_B_STAGE_CASES])
+def test_swin_b_stage_shapes_match_oracle(lib, case, levels):
+    run_swin_case(lib, case, torch.bfloat16, 1, levels)
+
+
+def run_swin_case(lib, case, dtype, pack, levels):
     B, H, W, ws, shift, heads, d = case
     dim, T, mlp = heads * d, ws * ws, 4 * heads * d
     rows = B * H * W
-    host, p = make_params(dim, mlp, MIXED_LEVELS, dtype, 3100)
+    host, p = make_params(dim, mlp, levels, dtype, 3100)
     x = synth.randn((rows, dim), 14, 1.0, dtype)
     rel_bias = np.random.default_rng(9).standard_normal((heads, T, T)) * 0.5
     dev = {k: v.cuda() for k, v in host.items()}
     lin = {}
     for name in NAMES:
-        N, M = MIXED_LEVELS[name]
+        N, M = levels[name]
         vals, idx = lib.elsa_nm_compress(dev["W_" + name], N, M)
         lin[name] = (vals, idx, dev["b_" + name], N, M)
     w, keep = lib.make_block_weights(dev["ln1_g"], dev["ln1_b"], dev["ln2_g"], dev["ln2_b"], lin, eps=1e-6)
