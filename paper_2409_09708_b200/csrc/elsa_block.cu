@@ -75,17 +75,33 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// The row map as the kernels take it: the caller's fields plus what the host can work out once.  Inside an image
+// every quotient has a dividend below 2^16 (the host checks H * W), so a division by d is the high half of a product
+// with ceil(2^32 / d): exact while dividend * d < 2^32.  With one image's row per 16 or 32 lanes the map's integer
+// divisions were most of what a short row's LayerNorm executed.
+struct RowMapDev {
+    int H, W, ws, shift, on_input, on_output;
+    int hw, windows_per_row, ws2;
+    uint32_t magic_W, magic_ws;
+};
+
+__device__ __forceinline__ int small_div(int n, uint32_t magic, int d)
+{
+    return d == 1 ? n : (int)__umulhi((uint32_t)n, magic);
+}
+
 // Where a row of the token grid goes in window order (Swin): the H x W grid of an image rolled by -shift along both
 // axes and cut into ws x ws windows, windows row-major, tokens row-major inside a window.  H == 0: identity.
-__device__ __forceinline__ int window_row(const RowMap& m, int row)
+__device__ __forceinline__ int window_row(const RowMapDev& m, int row)
 {
     if (m.H == 0) return row;
-    const int hw = m.H * m.W;
-    const int b = row / hw, t = row - b * hw;
-    const int i = t / m.W, j = t - i * m.W;
-    const int ir = (i - m.shift + m.H) % m.H, jr = (j - m.shift + m.W) % m.W;      // position in the rolled grid
-    const int win = (ir / m.ws) * (m.W / m.ws) + jr / m.ws;
-    return b * hw + win * m.ws * m.ws + (ir % m.ws) * m.ws + jr % m.ws;
+    const int b = row / m.hw, t = row - b * m.hw;
+    const int i = small_div(t, m.magic_W, m.W), j = t - i * m.W;
+    int ir = i - m.shift, jr = j - m.shift;                       // position in the rolled grid (0 <= shift < H, W)
+    if (ir < 0) ir += m.H;
+    if (jr < 0) jr += m.W;
+    const int wi = small_div(ir, m.magic_ws, m.ws), wj = small_div(jr, m.magic_ws, m.ws);
+    return b * m.hw + (wi * m.windows_per_row + wj) * m.ws2 + (ir - wi * m.ws) * m.ws + (jr - wj * m.ws);
 }
 
 // One warp per row.  map.on_input: A's row r is read at window_row(r) (a tensor in window order brought back to the
@@ -96,7 +112,7 @@ __device__ __forceinline__ int window_row(const RowMap& m, int row)
 template <bool kBf16, bool kAdd>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* __restrict__ gain,
-                  const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, int dim, float eps, const RowMap map)
+                  const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, int dim, float eps, const RowMapDev map)
 {
     pdl_wait_for_predecessors();
     pdl_release_successors();
@@ -187,7 +203,7 @@ layer_norm_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint1
 template <bool kBf16, bool kAdd, int kLanes, int kVpl, int kUnroll>
 __global__ void __launch_bounds__(kWarpsPerBlock * 32)
 layer_norm_rows_kernel(const uint16_t* A, const uint16_t* R, uint16_t* S, const uint16_t* __restrict__ gain,
-                       const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, float eps, const RowMap map)
+                       const uint16_t* __restrict__ beta, uint16_t* Yn, int rows, float eps, const RowMapDev map)
 {
     constexpr int kGroups = 32 / kLanes;               // rows side by side in a warp
     constexpr int kRowsPerStep = kGroups * kUnroll;
@@ -332,8 +348,18 @@ elsa_status launch_layer_norm(const uint16_t* A, const uint16_t* R, uint16_t* S,
                               const uint16_t* beta, uint16_t* Yn, int rows, int dim, float eps, elsa_dtype dtype,
                               cudaStream_t stream, const RowMap* row_map)
 {
-    RowMap map = {0, 0, 0, 0, 0, 0};
-    if (row_map != nullptr) map = *row_map;
+    RowMapDev map = {};
+    if (row_map != nullptr && row_map->H != 0) {
+        const RowMap& r = *row_map;
+        if (r.H < 1 || r.W < 1 || r.ws < 1 || r.H % r.ws != 0 || r.W % r.ws != 0 || r.shift < 0 || r.shift >= r.H ||
+            r.shift >= r.W || (long long)r.H * r.W >= 65536)
+            return fail(ELSA_ERR_SHAPE, "row map: grid %d x %d, window %d, shift %d", r.H, r.W, r.ws, r.shift);
+        map.H = r.H; map.W = r.W; map.ws = r.ws; map.shift = r.shift;
+        map.hw = r.H * r.W; map.windows_per_row = r.W / r.ws; map.ws2 = r.ws * r.ws;
+        map.magic_W = (uint32_t)(((1ull << 32) + (uint32_t)r.W - 1) / (uint32_t)r.W);
+        map.magic_ws = (uint32_t)(((1ull << 32) + (uint32_t)r.ws - 1) / (uint32_t)r.ws);
+    }
+    if (row_map != nullptr) { map.on_input = row_map->on_input; map.on_output = row_map->on_output; }
     DeviceInfo dev;
     elsa_status st = device_info(&dev);
     if (st != ELSA_OK) return st;
